@@ -1,0 +1,210 @@
+/*
+ * lamp.h - C ABI of the B200 (sm_100a) 3-D U-Net convolution library.
+ *
+ * Scope: the dense 3-D convolutions of a large 3-D U-Net - forward, data
+ * gradient and weight gradient - and the U-Net passes around them: one forward
+ * pass, one forward+backward training step with a softmax-Dice loss, and
+ * whole-volume versus sliding-window inference.  This is the per-device work
+ * that the paper's model parallelism spreads over GPUs (Sec. 2.1, Eq. 1: each
+ * partition's forward F_k is a chain of such layers, its backward B_k their
+ * chain-rule derivative).  The network is the U-Net of Sec. 2.2 (Eq. 2).
+ *
+ * Conventions (all entry points):
+ *  - Every data pointer is a DEVICE pointer unless the comment says "host".
+ *    Descriptors (lamp_tensor_t, lamp_conv_desc_t, lamp_unet_spec_t) and the
+ *    opaque lamp_unet_t are host objects, read during the call only.
+ *  - The caller owns every buffer, including the workspace.  No entry point
+ *    allocates or frees device memory.  Outputs are overwritten, never
+ *    accumulated into, unless stated.
+ *  - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*; NULL
+ *    is the default stream) and return without synchronising.  Errors that
+ *    the host can detect return a status and launch nothing.  Conditions only
+ *    the device can detect (a bounded wait that ran out) are recorded in a
+ *    device-side status word read by lamp_get_async_status().
+ *  - Activations are NDHWC, channel-contiguous.  A lamp_tensor_t describes a
+ *    channel slice [c_offset, c_offset + c) of a buffer whose voxels are
+ *    c_pitch elements apart, so a layer can write straight into its slice of a
+ *    skip-concatenation buffer (Sec. 2.2: the skip s_i is a concatenation
+ *    along the channel dimension).
+ *  - Convolution is cross-correlation with zero padding.  Weights are bf16
+ *    w[tap][c_out][c_in] with tap = (kd*k + kh)*k + kw for every variant;
+ *    biases are fp32 [c_out].  Accumulation is fp32.  Weight and bias
+ *    gradients are fp32.
+ *  - Alignment: data pointers 16-byte aligned; for bf16 tensors c, c_pitch and
+ *    c_offset are multiples of 8 except where a function says otherwise.
+ */
+#ifndef LAMP_H_
+#define LAMP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LAMP_OK = 0,
+    LAMP_ERR_INVALID_ARG = 1,     /* null pointer, negative size, inconsistent shapes            */
+    LAMP_ERR_UNSUPPORTED = 2,     /* a combination this library has no kernel for                */
+    LAMP_ERR_WORKSPACE = 3,       /* workspace missing, misaligned or smaller than required      */
+    LAMP_ERR_CUDA = 4,            /* a CUDA runtime / driver call failed                         */
+    LAMP_ERR_TIMEOUT = 5,         /* a bounded device-side wait ran out (see async status)       */
+    LAMP_ERR_NOT_IMPLEMENTED = 6
+} lamp_status_t;
+
+typedef enum { LAMP_BF16 = 0, LAMP_F32 = 1 } lamp_dtype_t;
+
+/* A channel-slice view of an NDHWC device buffer.
+ * ptr points at voxel (0,0,0,0), channel 0 of the underlying buffer; the view
+ * covers channels [c_offset, c_offset + c) of each voxel; consecutive voxels
+ * are c_pitch elements apart (c_pitch >= c_offset + c). */
+typedef struct {
+    void   *ptr;
+    int32_t dtype;       /* lamp_dtype_t */
+    int32_t n, d, h, w, c;
+    int64_t c_pitch;
+    int32_t c_offset;
+} lamp_tensor_t;
+
+/* Supported (ksize, stride, pad, transposed): (3,1,1,0) (3,2,1,0) (1,1,0,0) (2,2,0,1). */
+typedef struct {
+    int32_t c_in, c_out, ksize, stride, pad, transposed;
+} lamp_conv_desc_t;
+
+enum { LAMP_PASS_FWD = 0, LAMP_PASS_DGRAD = 1, LAMP_PASS_WGRAD = 2 };
+
+/* ------------------------------------------------------------------------
+ * Single-layer convolution passes (the layer functions f_i of Sec. 2.1 and
+ * their derivatives).
+ * ---------------------------------------------------------------------- */
+
+/* Bytes of workspace the given pass needs for input x (for LAMP_PASS_DGRAD, x is
+ * the tensor that receives the gradient, i.e. the conv's input shape). */
+size_t lamp_conv3d_workspace_bytes(const lamp_conv_desc_t *desc, const lamp_tensor_t *x, int pass);
+
+/* y[n,od,oh,ow,co] = bias[co] + sum_{tap,ci} x[n, od*s+kd-p, oh*s+kh-p, ow*s+kw-p, ci] * w[tap][co][ci]
+ * (transposed: y[n, d*s+a, h*s+b, w*s+c, co] = bias[co] + sum_ci x[n,d,h,w,ci] * w[(a,b,c)][co][ci]).
+ * x: bf16.  y: bf16 or fp32, extents must equal the conv's output extents.
+ * bias: fp32 [c_out] or NULL.
+ * stats: NULL, or fp64 [n][c_out][2]; the kernel ADDS, per (n, co), the sum and
+ *   the sum of squares of the fp32 results (before any rounding to bf16) - the
+ *   caller zeroes it.  These are the InstanceNorm statistics of the layer.
+ * c_in may be any positive value (c_in == 1 is the network's first layer);
+ * when x is not a multiple of 8 channels wide, c_pitch/c_offset need no alignment. */
+lamp_status_t lamp_conv3d_fwd(const lamp_conv_desc_t *desc, const lamp_tensor_t *x, const void *w,
+                              const float *bias, lamp_tensor_t *y, double *stats,
+                              void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* dx = gradient of lamp_conv3d_fwd with respect to x, given dy (bf16); dx bf16 or fp32,
+ * its extents are the conv's input extents. */
+lamp_status_t lamp_conv3d_dgrad(const lamp_conv_desc_t *desc, const lamp_tensor_t *dy, const void *w,
+                                lamp_tensor_t *dx, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* dw[tap][c_out][c_in] (fp32) = gradient with respect to w; dbias[c_out] (fp32, may be NULL)
+ * = sum of dy over voxels.  x, dy bf16.  Both outputs are overwritten. */
+lamp_status_t lamp_conv3d_wgrad(const lamp_conv_desc_t *desc, const lamp_tensor_t *x, const lamp_tensor_t *dy,
+                                float *dw, float *dbias, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* ------------------------------------------------------------------------
+ * Normalisation steps of a block (exported so they can be checked alone).
+ * ---------------------------------------------------------------------- */
+
+/* z = max(0, (y - mu) * rstd) per (n, c), mu = S1/V, rstd = (S2/V - mu^2 + eps)^-1/2 with
+ * (S1, S2) = stats[n][c][0..1] (fp64, as accumulated by lamp_conv3d_fwd), V = d*h*w.
+ * y bf16, z bf16 (may be a channel slice of a concat buffer).  mu_rstd: fp32 [n][c][2] scratch
+ * that receives (mu, rstd) and is needed again by the backward call. */
+lamp_status_t lamp_instnorm_relu_fwd(const lamp_tensor_t *y, const double *stats, float eps,
+                                     float *mu_rstd, lamp_tensor_t *z, void *cuda_stream);
+
+/* dy = rstd * (g - mean(g) - xhat * mean(g * xhat)),  g = (dz_a + dz_b) * [xhat > 0],
+ * xhat = (y - mu) * rstd, means over d*h*w per (n, c).  dz_b may be NULL (the second
+ * gradient source exists where a block output feeds both the next level and a skip).
+ * sums: fp64 [n][c][2] scratch, zeroed by the call.  y, dz_*, dy bf16. */
+lamp_status_t lamp_instnorm_relu_bwd(const lamp_tensor_t *dz_a, const lamp_tensor_t *dz_b,
+                                     const lamp_tensor_t *y, const float *mu_rstd,
+                                     double *sums, lamp_tensor_t *dy, void *cuda_stream);
+
+/* ------------------------------------------------------------------------
+ * U-Net (Sec. 2.2, Eq. 2; widths per Sec. 3).
+ *   encoder level l: convs_per_level x [conv 3x3x3 s1 p1 -> InstanceNorm -> ReLU]; between
+ *   levels a conv 3x3x3 s2 p1 -> InstanceNorm -> ReLU; decoder level l: transposed conv 2x2x2 s2
+ *   (+bias), concat(skip, up), convs_per_level x [conv -> InstanceNorm -> ReLU]; head: conv 1x1x1
+ *   to num_classes, softmax.  InstanceNorm: biased variance, eps = in_eps, no affine parameters.
+ * Layer order (also parameter order): encoder levels top-down (convs, then the down conv),
+ * decoder levels bottom-up (up conv, then convs), head.
+ * ---------------------------------------------------------------------- */
+typedef struct {
+    int32_t levels;            /* 1..8                                     */
+    int32_t channels[8];       /* width of each level, multiples of 8      */
+    int32_t convs_per_level;   /* >= 1                                     */
+    int32_t in_channels;       /* 1, or a multiple of 8                    */
+    int32_t num_classes;       /* 2..16                                    */
+    float   in_eps;
+} lamp_unet_spec_t;
+
+typedef struct lamp_unet lamp_unet_t;          /* opaque, host-only plan */
+
+lamp_status_t lamp_unet_create(const lamp_unet_spec_t *spec, lamp_unet_t **out);
+void          lamp_unet_destroy(lamp_unet_t *net);
+int32_t       lamp_unet_num_layers(const lamp_unet_t *net);
+/* Elements of the flat bf16 weight buffer / of the flat fp32 bias buffer. */
+size_t        lamp_unet_weight_count(const lamp_unet_t *net);
+size_t        lamp_unet_bias_count(const lamp_unet_t *net);
+/* Offsets (in elements) of layer `layer` inside the two flat buffers, and its conv descriptor. */
+lamp_status_t lamp_unet_param_layout(const lamp_unet_t *net, int32_t layer, size_t *w_off, size_t *b_off,
+                                     lamp_conv_desc_t *desc);
+
+enum { LAMP_MODE_INFER = 0, LAMP_MODE_TRAIN = 1 };
+size_t lamp_unet_workspace_bytes(const lamp_unet_t *net, int32_t n, int32_t d, int32_t h, int32_t w, int32_t mode);
+
+/* One forward pass.  x: bf16 [n,d,h,w,in_channels] (d,h,w divisible by 2^(levels-1)).
+ * probs: fp32 [n*d*h*w][num_classes] softmax output, or NULL.  argmax: uint8 [n*d*h*w] class of
+ * largest probability (lowest index on ties), or NULL.  Stored intermediates are bf16. */
+lamp_status_t lamp_unet_forward(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                const lamp_tensor_t *x, float *probs, uint8_t *argmax,
+                                void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* One forward + backward pass with the softmax-Dice loss
+ *   L = mean_n [ 1 - (1/K) sum_k (2 I_k + e)/(P_k + G_k + e) ],  I = sum p g, P = sum p, G = sum g, e = 1e-5.
+ * labels: uint8 [n*d*h*w], values < num_classes.  loss: fp32 device scalar.
+ * grad_w: fp32, laid out like the weight buffer; grad_b: fp32, like the bias buffer.
+ * probs: fp32 [n*d*h*w][num_classes] or NULL (then taken from the workspace). */
+lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                   const lamp_tensor_t *x, const uint8_t *labels, float *loss,
+                                   float *grad_w, float *grad_b, float *probs,
+                                   void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Sliding-window inference (Sec. 3: patches versus the whole image).  Patch origins per axis are
+ * 0, s, 2s, ... with s = round(patch * (1 - overlap)) while the patch fits, plus one patch flush
+ * with the border if needed; patches are ordered by origin (d, h, w), w fastest; each patch is a
+ * separate network input (own InstanceNorm statistics).  Patch probabilities are blended with
+ * weight 1 (window = 0) or a Gaussian (window = 1: sigma = patch/8 per axis, normalised to
+ * maximum 1, floored at 1e-3): A[v,k] = sum_p w p / sum_p w.
+ * volume: bf16 [1,d,h,w,in_channels].  probs_planar: fp32 [num_classes][d][h][w] or NULL.
+ * argmax: uint8 [d*h*w].  sw_batch: patches per network pass (>= 1). */
+size_t lamp_sliding_window_workspace_bytes(const lamp_unet_t *net, int32_t d, int32_t h, int32_t w,
+                                           const int32_t patch[3], float overlap, int32_t sw_batch);
+lamp_status_t lamp_sliding_window_infer(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                        const lamp_tensor_t *volume, const int32_t patch[3], float overlap,
+                                        int32_t sw_batch, int32_t window, float *probs_planar, uint8_t *argmax,
+                                        void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Weighted overlap-add of per-patch probabilities on its own (the aggregation step of
+ * lamp_sliding_window_infer).  patch_probs: fp32 [n_patches][pd*ph*pw][k], patches in the order
+ * above for a d x h x w volume. */
+lamp_status_t lamp_overlap_add(const float *patch_probs, int32_t k, int32_t d, int32_t h, int32_t w,
+                               const int32_t patch[3], float overlap, int32_t window,
+                               float *probs_planar, uint8_t *argmax, void *cuda_stream);
+
+/* Synchronises `cuda_stream`, then returns and clears the device-side status word
+ * (LAMP_OK, or LAMP_ERR_TIMEOUT if a bounded wait inside a kernel ran out). */
+lamp_status_t lamp_get_async_status(void *cuda_stream);
+const char   *lamp_status_string(lamp_status_t s);
+/* Library build identifier: "lamp-b200 <sm arch>". */
+const char   *lamp_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAMP_H_ */

@@ -1,0 +1,224 @@
+// C ABI (include/lamp.h): argument checks, kernel selection, status word.
+#include "common.cuh"
+
+namespace lamp {
+
+__device__ int g_status_word = 0;
+
+int *status_word_ptr()
+{
+    int *p = nullptr;
+    if (cudaGetSymbolAddress((void **)&p, g_status_word) != cudaSuccess) return nullptr;
+    return p;
+}
+
+static bool aligned16(const void *p) { return ((uintptr_t)p & 15) == 0; }
+
+static lamp_status_t check_tensor(const lamp_tensor_t *t, bool allow_f32, bool any_channels)
+{
+    if (!t || !t->ptr) return LAMP_ERR_INVALID_ARG;
+    if (t->n < 0 || t->d < 0 || t->h < 0 || t->w < 0 || t->c <= 0 || t->c_offset < 0) return LAMP_ERR_INVALID_ARG;
+    if (t->c_pitch < (int64_t)t->c_offset + t->c) return LAMP_ERR_INVALID_ARG;
+    if (t->dtype != LAMP_BF16 && !(allow_f32 && t->dtype == LAMP_F32)) return LAMP_ERR_UNSUPPORTED;
+    if (!aligned16(t->ptr)) return LAMP_ERR_INVALID_ARG;
+    if (!any_channels && t->dtype == LAMP_BF16 && ((t->c & 7) || (t->c_pitch & 7) || (t->c_offset & 7)))
+        return LAMP_ERR_UNSUPPORTED;
+    if ((double)voxels(t) * (double)t->c_pitch * 4.0 > 1099511627776.0) return LAMP_ERR_UNSUPPORTED;   // 2^40 B
+    return LAMP_OK;
+}
+
+// `in` has the conv's input extents, `out` its output extents (either may be NULL to skip the check).
+lamp_status_t conv_geom(const lamp_conv_desc_t *d, const lamp_tensor_t *in, const lamp_tensor_t *out, ConvGeom *g)
+{
+    if (!d || !g) return LAMP_ERR_INVALID_ARG;
+    if (d->c_in <= 0 || d->c_out <= 0) return LAMP_ERR_INVALID_ARG;
+    const bool ok = (d->ksize == 3 && d->stride == 1 && d->pad == 1 && !d->transposed) ||
+                    (d->ksize == 3 && d->stride == 2 && d->pad == 1 && !d->transposed) ||
+                    (d->ksize == 1 && d->stride == 1 && d->pad == 0 && !d->transposed) ||
+                    (d->ksize == 2 && d->stride == 2 && d->pad == 0 && d->transposed == 1);
+    if (!ok) return LAMP_ERR_UNSUPPORTED;
+    g->ci = d->c_in; g->co = d->c_out; g->k = d->ksize; g->s = d->stride; g->p = d->pad; g->transposed = d->transposed;
+    const lamp_tensor_t *ref = in ? in : out;
+    if (!ref) return LAMP_ERR_INVALID_ARG;
+    if (in) {
+        g->n = in->n; g->d = in->d; g->h = in->h; g->w = in->w;
+        if (in->c != d->c_in) return LAMP_ERR_INVALID_ARG;
+        if (d->transposed) { g->od = in->d * 2; g->oh = in->h * 2; g->ow = in->w * 2; }
+        else {
+            g->od = in->d ? (in->d + 2 * d->pad - d->ksize) / d->stride + 1 : 0;
+            g->oh = in->h ? (in->h + 2 * d->pad - d->ksize) / d->stride + 1 : 0;
+            g->ow = in->w ? (in->w + 2 * d->pad - d->ksize) / d->stride + 1 : 0;
+        }
+    }
+    if (out) {
+        if (out->c != d->c_out) return LAMP_ERR_INVALID_ARG;
+        if (in) {
+            if (out->n != g->n || out->d != g->od || out->h != g->oh || out->w != g->ow) return LAMP_ERR_INVALID_ARG;
+        } else {
+            return LAMP_ERR_INVALID_ARG;
+        }
+    }
+    return LAMP_OK;
+}
+
+static bool dgrad_via_umma(const ConvGeom &g)
+{
+    // data gradient of the 3x3x3 s1 p1 conv = the same conv on dy with mirrored taps and swapped channels
+    if (!(g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed)) return false;
+    ConvGeom t = g;
+    t.ci = g.co; t.co = g.ci;
+    TView a{}, b{};
+    a.pitch = 8; b.pitch = 8;      // alignment of the real views is checked again at launch
+    return umma_conv_fwd_supported(t, a, b);
+}
+
+size_t conv_ws_bytes(const ConvGeom &g, int pass)
+{
+    if (pass == LAMP_PASS_DGRAD) return dgrad_via_umma(g) ? umma_dgrad_ws(g) : 0;
+    if (pass == LAMP_PASS_WGRAD) return simt_conv_wgrad_ws(g);
+    return 0;
+}
+
+lamp_status_t conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
+                       double *stats, cudaStream_t st)
+{
+    if (umma_conv_fwd_supported(g, x, y)) return umma_conv_fwd(g, x, w, bias, y, stats, 0, st);
+    return simt_conv_fwd(g, x, w, bias, y, stats, st);
+}
+
+lamp_status_t conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w, const TView &dx, void *ws, size_t ws_bytes,
+                         cudaStream_t st)
+{
+    if (dgrad_via_umma(g)) {
+        ConvGeom t = g;
+        t.ci = g.co; t.co = g.ci;
+        if (umma_conv_fwd_supported(t, dy, dx)) {
+            const size_t need = umma_dgrad_ws(g);
+            if (!ws || ws_bytes < need || !aligned16(ws)) return LAMP_ERR_WORKSPACE;
+            lamp_status_t s = umma_transpose_weights(w, (bf16 *)ws, 27, g.co, g.ci, st);
+            if (s != LAMP_OK) return s;
+            return umma_conv_fwd(t, dy, (const bf16 *)ws, nullptr, dx, nullptr, 1, st);
+        }
+    }
+    return simt_conv_dgrad(g, dy, w, dx, st);
+}
+
+lamp_status_t conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, float *db, void *ws,
+                         size_t ws_bytes, cudaStream_t st)
+{
+    return simt_conv_wgrad(g, x, dy, dw, db, ws, ws_bytes, st);
+}
+
+}  // namespace lamp
+
+using namespace lamp;
+
+extern "C" {
+
+size_t lamp_conv3d_workspace_bytes(const lamp_conv_desc_t *desc, const lamp_tensor_t *x, int pass)
+{
+    ConvGeom g;
+    if (!x || conv_geom(desc, x, nullptr, &g) != LAMP_OK) return 0;
+    return conv_ws_bytes(g, pass);
+}
+
+lamp_status_t lamp_conv3d_fwd(const lamp_conv_desc_t *desc, const lamp_tensor_t *x, const void *w,
+                              const float *bias, lamp_tensor_t *y, double *stats,
+                              void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    (void)ws; (void)ws_bytes;
+    if (!desc || !x || !w || !y) return LAMP_ERR_INVALID_ARG;
+    lamp_status_t s;
+    if ((s = check_tensor(x, false, true)) != LAMP_OK) return s;
+    if ((s = check_tensor(y, true, true)) != LAMP_OK) return s;
+    if (!aligned16(w)) return LAMP_ERR_INVALID_ARG;
+    ConvGeom g;
+    if ((s = conv_geom(desc, x, y, &g)) != LAMP_OK) return s;
+    return conv_fwd(g, make_view(x), (const bf16 *)w, bias, make_view(y), stats, (cudaStream_t)cuda_stream);
+}
+
+lamp_status_t lamp_conv3d_dgrad(const lamp_conv_desc_t *desc, const lamp_tensor_t *dy, const void *w,
+                                lamp_tensor_t *dx, void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!desc || !dy || !w || !dx) return LAMP_ERR_INVALID_ARG;
+    lamp_status_t s;
+    if ((s = check_tensor(dy, false, true)) != LAMP_OK) return s;
+    if ((s = check_tensor(dx, true, true)) != LAMP_OK) return s;
+    if (!aligned16(w)) return LAMP_ERR_INVALID_ARG;
+    ConvGeom g;
+    if ((s = conv_geom(desc, dx, dy, &g)) != LAMP_OK) return s;
+    return conv_dgrad(g, make_view(dy), (const bf16 *)w, make_view(dx), ws, ws_bytes, (cudaStream_t)cuda_stream);
+}
+
+lamp_status_t lamp_conv3d_wgrad(const lamp_conv_desc_t *desc, const lamp_tensor_t *x, const lamp_tensor_t *dy,
+                                float *dw, float *dbias, void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!desc || !x || !dy || !dw) return LAMP_ERR_INVALID_ARG;
+    lamp_status_t s;
+    if ((s = check_tensor(x, false, true)) != LAMP_OK) return s;
+    if ((s = check_tensor(dy, false, true)) != LAMP_OK) return s;
+    ConvGeom g;
+    if ((s = conv_geom(desc, x, dy, &g)) != LAMP_OK) return s;
+    if (conv_ws_bytes(g, LAMP_PASS_WGRAD) > 0 && (!ws || !aligned16(ws))) return LAMP_ERR_WORKSPACE;
+    return conv_wgrad(g, make_view(x), make_view(dy), dw, dbias, ws, ws_bytes, (cudaStream_t)cuda_stream);
+}
+
+lamp_status_t lamp_instnorm_relu_fwd(const lamp_tensor_t *y, const double *stats, float eps,
+                                     float *mu_rstd, lamp_tensor_t *z, void *cuda_stream)
+{
+    if (!y || !stats || !mu_rstd || !z) return LAMP_ERR_INVALID_ARG;
+    lamp_status_t s;
+    if ((s = check_tensor(y, false, false)) != LAMP_OK) return s;
+    if ((s = check_tensor(z, false, false)) != LAMP_OK) return s;
+    if (y->n != z->n || y->d != z->d || y->h != z->h || y->w != z->w || y->c != z->c) return LAMP_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int64_t Vn = (int64_t)y->d * y->h * y->w;
+    if ((s = k_finalize_stats(stats, mu_rstd, (int64_t)y->n * y->c, Vn ? 1.0 / (double)Vn : 0.0, eps, st)) != LAMP_OK) return s;
+    return k_instnorm_relu_fwd(make_view(y), mu_rstd, make_view(z), st);
+}
+
+lamp_status_t lamp_instnorm_relu_bwd(const lamp_tensor_t *dz_a, const lamp_tensor_t *dz_b,
+                                     const lamp_tensor_t *y, const float *mu_rstd,
+                                     double *sums, lamp_tensor_t *dy, void *cuda_stream)
+{
+    if (!dz_a || !y || !mu_rstd || !sums || !dy) return LAMP_ERR_INVALID_ARG;
+    lamp_status_t s;
+    const lamp_tensor_t *all[4] = {dz_a, dz_b, y, dy};
+    for (int i = 0; i < 4; ++i) {
+        if (!all[i]) continue;
+        if ((s = check_tensor(all[i], false, false)) != LAMP_OK) return s;
+        if (all[i]->n != y->n || all[i]->d != y->d || all[i]->h != y->h || all[i]->w != y->w || all[i]->c != y->c)
+            return LAMP_ERR_INVALID_ARG;
+    }
+    TView vb{};
+    if (dz_b) vb = make_view(dz_b);
+    return k_instnorm_relu_bwd(make_view(dz_a), dz_b ? &vb : nullptr, make_view(y), mu_rstd, sums, make_view(dy),
+                               (cudaStream_t)cuda_stream);
+}
+
+lamp_status_t lamp_get_async_status(void *cuda_stream)
+{
+    if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return LAMP_ERR_CUDA;
+    int v = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_status_word, sizeof(int)) != cudaSuccess) return LAMP_ERR_CUDA;
+    if (v != 0 && cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int)) != cudaSuccess) return LAMP_ERR_CUDA;
+    return (lamp_status_t)v;
+}
+
+const char *lamp_status_string(lamp_status_t s)
+{
+    switch (s) {
+    case LAMP_OK: return "ok";
+    case LAMP_ERR_INVALID_ARG: return "invalid argument";
+    case LAMP_ERR_UNSUPPORTED: return "unsupported configuration";
+    case LAMP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case LAMP_ERR_CUDA: return "CUDA call failed";
+    case LAMP_ERR_TIMEOUT: return "device-side wait timed out";
+    case LAMP_ERR_NOT_IMPLEMENTED: return "not implemented";
+    }
+    return "unknown status";
+}
+
+const char *lamp_version(void) { return "lamp-b200 sm_100a"; }
+
+}  // extern "C"

@@ -1,0 +1,128 @@
+// Shared device/host helpers of the library (not used by the CPU oracle).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "../../include/lamp.h"
+
+namespace lamp {
+
+typedef __nv_bfloat16 bf16;
+
+// Device view of a lamp_tensor_t: pointer already advanced to the slice's first channel.
+struct TView {
+    void   *p;
+    int32_t n, d, h, w, c;
+    int64_t pitch;     // elements between voxels
+    int32_t f32;       // 1: float elements, 0: bf16
+};
+
+static inline TView make_view(const lamp_tensor_t *t)
+{
+    TView v;
+    const size_t es = t->dtype == LAMP_F32 ? 4 : 2;
+    v.p = (char *)t->ptr + (size_t)t->c_offset * es;
+    v.n = t->n; v.d = t->d; v.h = t->h; v.w = t->w; v.c = t->c;
+    v.pitch = t->c_pitch;
+    v.f32 = t->dtype == LAMP_F32;
+    return v;
+}
+
+static inline int64_t voxels(const lamp_tensor_t *t) { return (int64_t)t->n * t->d * t->h * t->w; }
+
+__device__ __forceinline__ float bf2f(bf16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ bf16 f2bf(float v) { return __float2bfloat16_rn(v); }
+
+// 8 bf16 values in one 16-byte word.
+struct __align__(16) bf16x8 { bf16 v[8]; };
+
+__device__ __forceinline__ void unpack8(const uint4 &u, float (&f)[8])
+{
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        f[2 * i]     = __uint_as_float(w[i] << 16);
+        f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+}
+
+__device__ __forceinline__ uint4 pack8(const float (&f)[8])
+{
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+        w[i] = *reinterpret_cast<uint32_t *>(&h);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Device address of the status word (LAMP_OK or LAMP_ERR_TIMEOUT) on the current device
+// (api.cu); NULL if it cannot be resolved.
+int *status_word_ptr();
+
+#define LAMP_CUDA_OK(expr)                                   \
+    do {                                                     \
+        cudaError_t e__ = (expr);                            \
+        if (e__ != cudaSuccess) return LAMP_ERR_CUDA;        \
+    } while (0)
+
+static inline lamp_status_t launch_status()
+{
+    return cudaGetLastError() == cudaSuccess ? LAMP_OK : LAMP_ERR_CUDA;
+}
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---------------------------------------------------------------------------
+// Internal launchers (one per kernel family); all enqueue on `st`.
+// ---------------------------------------------------------------------------
+struct ConvGeom {
+    int32_t n, d, h, w;        // input extents (of x / dx)
+    int32_t od, oh, ow;        // output extents (of y / dy)
+    int32_t ci, co, k, s, p, transposed;
+};
+
+// conv_simt.cu
+lamp_status_t simt_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
+                            double *stats, cudaStream_t st);
+lamp_status_t simt_conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w, const TView &dx, cudaStream_t st);
+size_t        simt_conv_wgrad_ws(const ConvGeom &g);
+lamp_status_t simt_conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, float *db,
+                              void *ws, size_t ws_bytes, cudaStream_t st);
+
+// conv_umma.cu (tcgen05 implicit GEMM)
+bool          umma_conv_fwd_supported(const ConvGeom &g, const TView &x, const TView &y);
+lamp_status_t umma_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
+                            double *stats, int mirror_taps, cudaStream_t st);
+size_t        umma_dgrad_ws(const ConvGeom &g);
+lamp_status_t umma_transpose_weights(const bf16 *w, bf16 *wt, int taps, int co, int ci, cudaStream_t st);
+
+// elementwise.cu
+lamp_status_t k_finalize_stats(const double *stats, float *mu_rstd, int64_t nc, double inv_v, float eps, cudaStream_t st);
+lamp_status_t k_instnorm_relu_fwd(const TView &y, const float *mu_rstd, const TView &z, cudaStream_t st);
+lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TView &y, const float *mu_rstd,
+                                  double *sums, const TView &dy, cudaStream_t st);
+lamp_status_t k_head_softmax(const TView &z, const bf16 *w, const float *b, int K, float *probs, uint8_t *argmax,
+                             const uint8_t *labels, double *dice_sums, cudaStream_t st);
+lamp_status_t k_dice_loss(const double *dice_sums, int N, int K, float *loss, cudaStream_t st);
+lamp_status_t k_head_bwd(const TView &z, const bf16 *w, int K, const float *probs, const uint8_t *labels,
+                         const double *dice_sums, const TView &dz, float *dw, float *db, float *dlogits,
+                         cudaStream_t st);
+lamp_status_t k_gather_patches(const TView &vol, const TView &patches, int first_patch, const int32_t nst[3],
+                               const int32_t stride[3], cudaStream_t st);
+lamp_status_t k_overlap_add(const float *pp, int K, int D, int H, int W, const int32_t patch[3],
+                            const int32_t nst[3], const int32_t stride[3], int window, float *planar,
+                            uint8_t *argmax, cudaStream_t st);
+
+// api.cu: shape checks + kernel selection for one conv pass (used by the ABI and by the U-Net executor)
+lamp_status_t conv_geom(const lamp_conv_desc_t *desc, const lamp_tensor_t *in, const lamp_tensor_t *out, ConvGeom *g);
+size_t        conv_ws_bytes(const ConvGeom &g, int pass);
+lamp_status_t conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
+                       double *stats, cudaStream_t st);
+lamp_status_t conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w, const TView &dx, void *ws, size_t ws_bytes,
+                         cudaStream_t st);
+lamp_status_t conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, float *db, void *ws,
+                         size_t ws_bytes, cudaStream_t st);
+
+}  // namespace lamp

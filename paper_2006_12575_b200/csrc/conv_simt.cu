@@ -1,0 +1,303 @@
+// Direct (CUDA-core) convolution kernels for every variant of the layer
+//   y[n,o,co] = b[co] + sum_{tap,ci} x[n, o*s + k - p, ci] * w[tap][co][ci]        (and its transposed form)
+// and its two derivatives.  They serve the shapes the tensor-core path does not take: the
+// single-channel first layer, narrow networks, the stride-2 and 2x2x2 transposed variants.
+// bf16 operands, fp32 accumulation, one sequential sum per output element.
+#include "common.cuh"
+
+namespace lamp {
+
+namespace {
+
+__device__ __forceinline__ float dot_row(const bf16 *__restrict__ a, const bf16 *__restrict__ b, int n, bool vec)
+{
+    float acc = 0.f;
+    if (vec) {
+        for (int i = 0; i < n; i += 8) {
+            float fa[8], fb[8];
+            unpack8(__ldg(reinterpret_cast<const uint4 *>(a + i)), fa);
+            unpack8(__ldg(reinterpret_cast<const uint4 *>(b + i)), fb);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc = fmaf(fa[j], fb[j], acc);
+        }
+    } else {
+        for (int i = 0; i < n; ++i) acc = fmaf(bf2f(a[i]), bf2f(b[i]), acc);
+    }
+    return acc;
+}
+
+// One thread per (output voxel, output channel); blockDim.x = 256 = TV voxels x TC channels.
+template <bool TR>
+__global__ void __launch_bounds__(256)
+conv_fwd_kernel(ConvGeom g, const bf16 *__restrict__ x, int64_t xp, const bf16 *__restrict__ w,
+                const float *__restrict__ bias, void *__restrict__ y, int64_t yp, int y_f32,
+                double *__restrict__ stats, int TC, int iters, int vec)
+{
+    __shared__ float red[2][256];
+    const int TV = 256 / TC;
+    const int cl = threadIdx.x % TC, vl = threadIdx.x / TC;
+    const int n = blockIdx.y;
+    const int64_t Vn = (int64_t)g.od * g.oh * g.ow;
+    const int64_t v0 = (int64_t)blockIdx.x * TV * iters;
+    const int co_round = (g.co + TC - 1) / TC * TC;
+    const int K = g.k;
+    for (int c = cl; c < co_round; c += TC) {
+        const bool cvalid = c < g.co;
+        float s1 = 0.f, s2 = 0.f;
+        for (int it = 0; it < iters; ++it) {
+            const int64_t v = v0 + (int64_t)it * TV + vl;
+            if (v >= Vn || !cvalid) continue;
+            const int ow = (int)(v % g.ow);
+            const int oh = (int)((v / g.ow) % g.oh);
+            const int od = (int)(v / ((int64_t)g.ow * g.oh));
+            float acc = bias ? bias[c] : 0.f;
+            for (int kd = 0; kd < K; ++kd) {
+                int id;
+                if (TR) { const int t = od - kd; if (t < 0 || t % g.s) continue; id = t / g.s; }
+                else    { id = od * g.s + kd - g.p; }
+                if (id < 0 || id >= g.d) continue;
+                for (int kh = 0; kh < K; ++kh) {
+                    int ih;
+                    if (TR) { const int t = oh - kh; if (t < 0 || t % g.s) continue; ih = t / g.s; }
+                    else    { ih = oh * g.s + kh - g.p; }
+                    if (ih < 0 || ih >= g.h) continue;
+                    for (int kw = 0; kw < K; ++kw) {
+                        int iw;
+                        if (TR) { const int t = ow - kw; if (t < 0 || t % g.s) continue; iw = t / g.s; }
+                        else    { iw = ow * g.s + kw - g.p; }
+                        if (iw < 0 || iw >= g.w) continue;
+                        const int tap = (kd * K + kh) * K + kw;
+                        const bf16 *xr = x + ((((int64_t)n * g.d + id) * g.h + ih) * g.w + iw) * xp;
+                        const bf16 *wr = w + ((int64_t)tap * g.co + c) * g.ci;
+                        acc += dot_row(xr, wr, g.ci, vec);
+                    }
+                }
+            }
+            const int64_t o = ((int64_t)n * Vn + v) * yp + c;
+            if (y_f32) reinterpret_cast<float *>(y)[o] = acc;
+            else       reinterpret_cast<bf16 *>(y)[o] = f2bf(acc);
+            s1 += acc;
+            s2 += acc * acc;
+        }
+        if (stats) {
+            red[0][threadIdx.x] = s1;
+            red[1][threadIdx.x] = s2;
+            __syncthreads();
+            if (vl == 0 && cvalid) {
+                double a = 0.0, b = 0.0;
+                for (int j = 0; j < TV; ++j) { a += red[0][j * TC + cl]; b += red[1][j * TC + cl]; }
+                atomicAdd(&stats[((int64_t)n * g.co + c) * 2], a);
+                atomicAdd(&stats[((int64_t)n * g.co + c) * 2 + 1], b);
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// One thread per (input voxel, input channel).
+template <bool TR>
+__global__ void __launch_bounds__(256)
+conv_dgrad_kernel(ConvGeom g, const bf16 *__restrict__ dy, int64_t dyp, const bf16 *__restrict__ w,
+                  void *__restrict__ dx, int64_t dxp, int dx_f32, int vec)
+{
+    const int64_t Vn = (int64_t)g.d * g.h * g.w;
+    const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (e >= Vn * g.ci) return;
+    const int n = blockIdx.y;
+    const int c = (int)(e % g.ci);
+    const int64_t v = e / g.ci;
+    const int iw = (int)(v % g.w);
+    const int ih = (int)((v / g.w) % g.h);
+    const int id = (int)(v / ((int64_t)g.w * g.h));
+    const int K = g.k;
+    float acc = 0.f;
+    for (int kd = 0; kd < K; ++kd) {
+        int od;
+        if (TR) { od = id * g.s + kd; }
+        else    { const int t = id + g.p - kd; if (t < 0 || t % g.s) continue; od = t / g.s; }
+        if (od < 0 || od >= g.od) continue;
+        for (int kh = 0; kh < K; ++kh) {
+            int oh;
+            if (TR) { oh = ih * g.s + kh; }
+            else    { const int t = ih + g.p - kh; if (t < 0 || t % g.s) continue; oh = t / g.s; }
+            if (oh < 0 || oh >= g.oh) continue;
+            for (int kw = 0; kw < K; ++kw) {
+                int ow;
+                if (TR) { ow = iw * g.s + kw; }
+                else    { const int t = iw + g.p - kw; if (t < 0 || t % g.s) continue; ow = t / g.s; }
+                if (ow < 0 || ow >= g.ow) continue;
+                const int tap = (kd * K + kh) * K + kw;
+                const bf16 *gr = dy + ((((int64_t)n * g.od + od) * g.oh + oh) * g.ow + ow) * dyp;
+                const bf16 *wr = w + (int64_t)tap * g.co * g.ci + c;
+                if (vec) {
+                    for (int co = 0; co < g.co; co += 8) {
+                        float f[8];
+                        unpack8(__ldg(reinterpret_cast<const uint4 *>(gr + co)), f);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) acc = fmaf(f[j], bf2f(wr[(int64_t)(co + j) * g.ci]), acc);
+                    }
+                } else {
+                    for (int co = 0; co < g.co; ++co) acc = fmaf(bf2f(gr[co]), bf2f(wr[(int64_t)co * g.ci]), acc);
+                }
+            }
+        }
+    }
+    const int64_t o = ((int64_t)n * Vn + v) * dxp + c;
+    if (dx_f32) reinterpret_cast<float *>(dx)[o] = acc;
+    else        reinterpret_cast<bf16 *>(dx)[o] = f2bf(acc);
+}
+
+// One thread per (tap, co, ci) entry and per split of the row range; a "row" is one (n, d, h)
+// line of the tensor the sum runs over (the conv output, or the input for the transposed form).
+template <bool TR>
+__global__ void __launch_bounds__(256)
+conv_wgrad_kernel(ConvGeom g, const bf16 *__restrict__ x, int64_t xp, const bf16 *__restrict__ dy, int64_t dyp,
+                  float *__restrict__ part, int64_t entries, int64_t rows, int64_t rows_per_split)
+{
+    const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (e >= entries) return;
+    const int ci = (int)(e % g.ci);
+    const int co = (int)((e / g.ci) % g.co);
+    const int tap = (int)(e / ((int64_t)g.ci * g.co));
+    const int K = g.k;
+    const int kd = tap / (K * K), kh = (tap / K) % K, kw = tap % K;
+    const int64_t r0 = (int64_t)blockIdx.y * rows_per_split;
+    const int64_t r1 = min(rows, r0 + rows_per_split);
+    // loop extents: conv -> output lines; transposed -> input lines
+    const int LH = TR ? g.h : g.oh, LD = TR ? g.d : g.od, LW = TR ? g.w : g.ow;
+    float acc = 0.f;
+    for (int64_t r = r0; r < r1; ++r) {
+        const int lh = (int)(r % LH);
+        const int ld = (int)((r / LH) % LD);
+        const int n = (int)(r / ((int64_t)LH * LD));
+        if (TR) {
+            const bf16 *xr = x + (((int64_t)n * g.d + ld) * g.h + lh) * (int64_t)g.w * xp + ci;
+            const bf16 *gr = dy + ((((int64_t)n * g.od + ld * g.s + kd) * g.oh + lh * g.s + kh) * (int64_t)g.ow + kw) * dyp + co;
+            for (int lw = 0; lw < LW; ++lw)
+                acc = fmaf(bf2f(gr[(int64_t)lw * g.s * dyp]), bf2f(xr[(int64_t)lw * xp]), acc);
+        } else {
+            const int id = ld * g.s + kd - g.p, ih = lh * g.s + kh - g.p;
+            if (id < 0 || id >= g.d || ih < 0 || ih >= g.h) continue;
+            const bf16 *xr = x + (((int64_t)n * g.d + id) * g.h + ih) * (int64_t)g.w * xp + ci;
+            const bf16 *gr = dy + (((int64_t)n * g.od + ld) * g.oh + lh) * (int64_t)g.ow * dyp + co;
+            for (int lw = 0; lw < LW; ++lw) {
+                const int iw = lw * g.s + kw - g.p;
+                if (iw < 0 || iw >= g.w) continue;
+                acc = fmaf(bf2f(gr[(int64_t)lw * dyp]), bf2f(xr[(int64_t)iw * xp]), acc);
+            }
+        }
+    }
+    part[(int64_t)blockIdx.y * entries + e] = acc;
+}
+
+// Column sums of dy over a chunk of voxels: part[chunk][co].
+__global__ void __launch_bounds__(256)
+colsum_kernel(const bf16 *__restrict__ dy, int64_t dyp, int co, int64_t V, int64_t v_per_block, float *__restrict__ part)
+{
+    const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = min(V, v0 + v_per_block);
+    for (int c = threadIdx.x; c < co; c += 256) {
+        float acc = 0.f;
+        for (int64_t v = v0; v < v1; ++v) acc += bf2f(dy[v * dyp + c]);
+        part[(int64_t)blockIdx.x * co + c] = acc;
+    }
+}
+
+// out[e] = sum_s part[s][e], fixed order.
+__global__ void __launch_bounds__(256)
+reduce_parts_kernel(const float *__restrict__ part, int64_t entries, int splits, float *__restrict__ out)
+{
+    const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (e >= entries) return;
+    float acc = 0.f;
+    for (int s = 0; s < splits; ++s) acc += part[(int64_t)s * entries + e];
+    out[e] = acc;
+}
+
+inline int pick_tc(int co)
+{
+    int tc = 8;
+    while (tc < co && tc < 64) tc <<= 1;
+    return tc;
+}
+
+struct WgradPlan { int64_t entries, rows, rows_per_split; int splits; int64_t V; int cs_blocks; int64_t v_per_block; };
+
+inline WgradPlan wgrad_plan(const ConvGeom &g)
+{
+    WgradPlan p;
+    p.entries = (int64_t)g.k * g.k * g.k * g.co * g.ci;
+    p.rows = g.transposed ? (int64_t)g.n * g.d * g.h : (int64_t)g.n * g.od * g.oh;
+    int64_t want = (600000 + p.entries - 1) / p.entries;
+    if (want < 1) want = 1;
+    if (want > p.rows) want = p.rows;
+    if (want > 4096) want = 4096;
+    p.rows_per_split = (p.rows + want - 1) / want;
+    p.splits = (int)((p.rows + p.rows_per_split - 1) / p.rows_per_split);
+    p.V = (int64_t)g.n * g.od * g.oh * g.ow;
+    p.cs_blocks = (int)(((p.V + 255) / 256) < 1024 ? ((p.V + 255) / 256) : 1024); if (p.cs_blocks < 1) p.cs_blocks = 1;
+    p.v_per_block = (p.V + p.cs_blocks - 1) / p.cs_blocks;
+    return p;
+}
+
+}  // namespace
+
+lamp_status_t simt_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
+                            double *stats, cudaStream_t st)
+{
+    const int TC = pick_tc(g.co), TV = 256 / TC, iters = 16;
+    const int64_t Vn = (int64_t)g.od * g.oh * g.ow;
+    if (Vn == 0 || g.n == 0) return LAMP_OK;
+    const int vec = (g.ci % 8 == 0) && (x.pitch % 8 == 0) && ((uintptr_t)x.p % 16 == 0) && ((uintptr_t)w % 16 == 0);
+    dim3 grid((unsigned)((Vn + (int64_t)TV * iters - 1) / ((int64_t)TV * iters)), g.n);
+    if (g.transposed)
+        conv_fwd_kernel<true><<<grid, 256, 0, st>>>(g, (const bf16 *)x.p, x.pitch, w, bias, y.p, y.pitch, y.f32, stats, TC, iters, vec);
+    else
+        conv_fwd_kernel<false><<<grid, 256, 0, st>>>(g, (const bf16 *)x.p, x.pitch, w, bias, y.p, y.pitch, y.f32, stats, TC, iters, vec);
+    return launch_status();
+}
+
+lamp_status_t simt_conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w, const TView &dx, cudaStream_t st)
+{
+    const int64_t Vn = (int64_t)g.d * g.h * g.w;
+    if (Vn == 0 || g.n == 0) return LAMP_OK;
+    const int vec = (g.co % 8 == 0) && (dy.pitch % 8 == 0) && ((uintptr_t)dy.p % 16 == 0);
+    dim3 grid((unsigned)((Vn * g.ci + 255) / 256), g.n);
+    if (g.transposed)
+        conv_dgrad_kernel<true><<<grid, 256, 0, st>>>(g, (const bf16 *)dy.p, dy.pitch, w, dx.p, dx.pitch, dx.f32, vec);
+    else
+        conv_dgrad_kernel<false><<<grid, 256, 0, st>>>(g, (const bf16 *)dy.p, dy.pitch, w, dx.p, dx.pitch, dx.f32, vec);
+    return launch_status();
+}
+
+size_t simt_conv_wgrad_ws(const ConvGeom &g)
+{
+    const WgradPlan p = wgrad_plan(g);
+    return align_up((size_t)p.splits * p.entries * 4, 256) + align_up((size_t)p.cs_blocks * g.co * 4, 256);
+}
+
+lamp_status_t simt_conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, float *db,
+                              void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    const WgradPlan p = wgrad_plan(g);
+    if (ws_bytes < simt_conv_wgrad_ws(g) || !ws) return LAMP_ERR_WORKSPACE;
+    float *part = (float *)ws;
+    float *cpart = (float *)((char *)ws + align_up((size_t)p.splits * p.entries * 4, 256));
+    if (p.V == 0) {
+        LAMP_CUDA_OK(cudaMemsetAsync(dw, 0, p.entries * 4, st));
+        if (db) LAMP_CUDA_OK(cudaMemsetAsync(db, 0, (size_t)g.co * 4, st));
+        return LAMP_OK;
+    }
+    dim3 grid((unsigned)((p.entries + 255) / 256), p.splits);
+    if (g.transposed)
+        conv_wgrad_kernel<true><<<grid, 256, 0, st>>>(g, (const bf16 *)x.p, x.pitch, (const bf16 *)dy.p, dy.pitch, part, p.entries, p.rows, p.rows_per_split);
+    else
+        conv_wgrad_kernel<false><<<grid, 256, 0, st>>>(g, (const bf16 *)x.p, x.pitch, (const bf16 *)dy.p, dy.pitch, part, p.entries, p.rows, p.rows_per_split);
+    reduce_parts_kernel<<<(unsigned)((p.entries + 255) / 256), 256, 0, st>>>(part, p.entries, p.splits, dw);
+    if (db) {
+        colsum_kernel<<<p.cs_blocks, 256, 0, st>>>((const bf16 *)dy.p, dy.pitch, g.co, p.V, p.v_per_block, cpart);
+        reduce_parts_kernel<<<(g.co + 255) / 256, 256, 0, st>>>(cpart, g.co, p.cs_blocks, db);
+    }
+    return launch_status();
+}
+
+}  // namespace lamp

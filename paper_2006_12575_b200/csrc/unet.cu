@@ -1,0 +1,469 @@
+// U-Net executor: layer plan, workspace arena, forward pass, training step, sliding window.
+//
+// Network (Sec. 2.2, Eq. 2): encoder blocks e_1..e_L, decoder blocks d_{L-1}..d_1 with
+// d_i = s_i(e_i, d_{i+1}), s_i = channel concatenation, softmax at the end; widths per level
+// are given by the spec (Sec. 3: doubled per encoder block, decoder symmetric).  The output of
+// encoder block l is used twice (Eq. 3 writes it as e_{l,0}, e_{l,1}): it is stored once, in
+// channels [0, C_l) of level l's concat buffer, read by the down conv and by the decoder; its
+// gradient is the sum of the two consumers' gradients, formed inside the norm-backward kernel.
+#include <vector>
+#include <new>
+#include "common.cuh"
+
+using namespace lamp;
+
+enum { K_CONV = 0, K_DOWN = 1, K_UP = 2, K_HEAD = 3 };
+
+struct Layer {
+    int kind, level;            // level of the layer's OUTPUT
+    int c_in, c_out, taps;
+    size_t w_off, b_off;
+    bool to_cat;                // output is E_l, written to the concat buffer slice [0, C_l)
+    bool from_cat;              // input is the full concat buffer (2 C_l channels)
+};
+
+struct lamp_unet {
+    lamp_unet_spec_t spec;
+    std::vector<Layer> layers;
+    size_t n_w, n_b;
+};
+
+namespace {
+
+struct Arena {
+    char *base;
+    size_t off;
+    void *take(size_t bytes)
+    {
+        off = align_up(off, 256);
+        void *p = base ? base + off : nullptr;
+        off += bytes;
+        return p;
+    }
+};
+
+struct LayerBuf {
+    TView in, out;              // activation views (out: normalised z / up output / unused for head)
+    TView y;                    // raw conv output (norm layers)
+    double *stats;              // [n][c_out][2]
+    float *mr;                  // [n][c_out][2]
+    ConvGeom g;
+    lamp_conv_desc_t desc;
+};
+
+struct Plan {
+    std::vector<LayerBuf> lb;
+    std::vector<TView> cat, dcat;       // per level (levels - 1 entries)
+    float *probs;                       // [V][K] when the caller gave none
+    double *dice;                       // [n][K][3]
+    double *bwd_sums;                   // [n][cmax][2]
+    bf16 *dybuf;                        // gradient w.r.t. a raw conv output, max size
+    bf16 *gbuf[2];                      // ping-pong gradient w.r.t. a layer input
+    void *scratch;                      // conv workspace (wgrad partials / transposed weights)
+    size_t scratch_bytes;
+    size_t total;
+};
+
+TView view(void *p, int n, int d, int h, int w, int c, int64_t pitch, int c_off)
+{
+    TView v;
+    v.p = p ? (char *)p + (size_t)c_off * 2 : nullptr;
+    v.n = n; v.d = d; v.h = h; v.w = w; v.c = c; v.pitch = pitch; v.f32 = 0;
+    return v;
+}
+
+lamp_conv_desc_t layer_desc(const Layer &L)
+{
+    lamp_conv_desc_t d;
+    d.c_in = L.c_in; d.c_out = L.c_out;
+    switch (L.kind) {
+    case K_CONV: d.ksize = 3; d.stride = 1; d.pad = 1; d.transposed = 0; break;
+    case K_DOWN: d.ksize = 3; d.stride = 2; d.pad = 1; d.transposed = 0; break;
+    case K_UP:   d.ksize = 2; d.stride = 2; d.pad = 0; d.transposed = 1; break;
+    default:     d.ksize = 1; d.stride = 1; d.pad = 0; d.transposed = 0; break;
+    }
+    return d;
+}
+
+// Lays every buffer of one pass out in the workspace (base may be NULL: sizing only).
+void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pitch, int n, int d, int h, int w,
+               int mode, bool need_probs, Plan *P)
+{
+    const lamp_unet_spec_t &S = net->spec;
+    Arena A{(char *)base, 0};
+    const int L = S.levels;
+    auto dd = [&](int l) { return d >> l; };
+    auto hh = [&](int l) { return h >> l; };
+    auto ww = [&](int l) { return w >> l; };
+    auto vox = [&](int l) { return (size_t)n * dd(l) * hh(l) * ww(l); };
+    P->cat.resize(L > 1 ? L - 1 : 0);
+    P->dcat.resize(L > 1 ? L - 1 : 0);
+    for (int l = 0; l + 1 < L; ++l) {
+        void *p = A.take(vox(l) * 2 * S.channels[l] * sizeof(bf16));
+        P->cat[l] = view(p, n, dd(l), hh(l), ww(l), 2 * S.channels[l], 2 * S.channels[l], 0);
+    }
+    size_t ymax = 0, cmax = 0, inmax = 0;
+    for (const Layer &Ly : net->layers) {
+        if (Ly.kind == K_CONV || Ly.kind == K_DOWN) ymax = ymax > vox(Ly.level) * Ly.c_out ? ymax : vox(Ly.level) * Ly.c_out;
+        cmax = cmax > (size_t)Ly.c_out ? cmax : (size_t)Ly.c_out;
+    }
+    bf16 *yshared = (mode == LAMP_MODE_INFER) ? (bf16 *)A.take(ymax * sizeof(bf16)) : nullptr;
+    P->lb.resize(net->layers.size());
+    TView cur = view((void *)x_ptr, n, d, h, w, S.in_channels, x_pitch, 0);
+    size_t scratch = 0;
+    for (size_t i = 0; i < net->layers.size(); ++i) {
+        const Layer &Ly = net->layers[i];
+        LayerBuf &B = P->lb[i];
+        const int l = Ly.level;
+        B.in = cur;
+        B.desc = layer_desc(Ly);
+        B.stats = nullptr; B.mr = nullptr;
+        B.y = TView{};
+        {
+            ConvGeom g;
+            g.n = n; g.d = cur.d; g.h = cur.h; g.w = cur.w;
+            g.od = dd(l); g.oh = hh(l); g.ow = ww(l);
+            g.ci = Ly.c_in; g.co = Ly.c_out; g.k = B.desc.ksize; g.s = B.desc.stride; g.p = B.desc.pad;
+            g.transposed = B.desc.transposed;
+            B.g = g;
+        }
+        const size_t in_elems = (size_t)cur.n * cur.d * cur.h * cur.w * Ly.c_in;
+        inmax = inmax > in_elems ? inmax : in_elems;
+        if (mode == LAMP_MODE_TRAIN) {
+            size_t s1 = conv_ws_bytes(B.g, LAMP_PASS_WGRAD), s2 = conv_ws_bytes(B.g, LAMP_PASS_DGRAD);
+            scratch = scratch > s1 ? scratch : s1;
+            scratch = scratch > s2 ? scratch : s2;
+        }
+        if (Ly.kind == K_CONV || Ly.kind == K_DOWN) {
+            void *yp = yshared ? (void *)yshared : A.take(vox(l) * Ly.c_out * sizeof(bf16));
+            B.y = view(yp, n, dd(l), hh(l), ww(l), Ly.c_out, Ly.c_out, 0);
+            B.stats = (double *)A.take((size_t)n * Ly.c_out * 2 * sizeof(double));
+            B.mr = (float *)A.take((size_t)n * Ly.c_out * 2 * sizeof(float));
+            if (Ly.to_cat) {
+                B.out = P->cat[l];
+                B.out.c = Ly.c_out;                      // slice [0, C_l)
+            } else {
+                void *zp = A.take(vox(l) * Ly.c_out * sizeof(bf16));
+                B.out = view(zp, n, dd(l), hh(l), ww(l), Ly.c_out, Ly.c_out, 0);
+            }
+            cur = B.out;
+        } else if (Ly.kind == K_UP) {
+            B.out = P->cat[l];
+            B.out.p = B.out.p ? (char *)B.out.p + (size_t)Ly.c_out * 2 : nullptr;   // slice [C_l, 2 C_l)
+            B.out.c = Ly.c_out;
+            cur = P->cat[l];                             // the next conv reads all 2 C_l channels
+        } else {
+            B.out = TView{};
+        }
+    }
+    const size_t V0 = vox(0);
+    P->probs = need_probs ? (float *)A.take(V0 * S.num_classes * sizeof(float)) : nullptr;
+    P->dice = nullptr; P->bwd_sums = nullptr; P->dybuf = nullptr; P->gbuf[0] = P->gbuf[1] = nullptr;
+    P->scratch = nullptr; P->scratch_bytes = 0;
+    if (mode == LAMP_MODE_TRAIN) {
+        P->dice = (double *)A.take((size_t)n * S.num_classes * 3 * sizeof(double));
+        P->bwd_sums = (double *)A.take((size_t)n * cmax * 2 * sizeof(double));
+        P->dybuf = (bf16 *)A.take(ymax * sizeof(bf16));
+        P->gbuf[0] = (bf16 *)A.take(inmax * sizeof(bf16));
+        P->gbuf[1] = (bf16 *)A.take(inmax * sizeof(bf16));
+        for (int l = 0; l + 1 < L; ++l) {
+            void *p = A.take(vox(l) * 2 * S.channels[l] * sizeof(bf16));
+            P->dcat[l] = view(p, n, dd(l), hh(l), ww(l), 2 * S.channels[l], 2 * S.channels[l], 0);
+        }
+        P->scratch = A.take(scratch);
+        P->scratch_bytes = scratch;
+    }
+    P->total = align_up(A.off, 256);
+}
+
+lamp_status_t check_input(const lamp_unet *net, const lamp_tensor_t *x)
+{
+    if (!net || !x || !x->ptr) return LAMP_ERR_INVALID_ARG;
+    const lamp_unet_spec_t &S = net->spec;
+    if (x->dtype != LAMP_BF16) return LAMP_ERR_UNSUPPORTED;
+    if (x->c != S.in_channels || x->c_offset != 0 || x->c_pitch < x->c) return LAMP_ERR_INVALID_ARG;
+    if (x->n <= 0 || x->d <= 0 || x->h <= 0 || x->w <= 0) return LAMP_ERR_INVALID_ARG;
+    const int m = 1 << (S.levels - 1);
+    if (x->d % m || x->h % m || x->w % m) return LAMP_ERR_UNSUPPORTED;
+    if (((uintptr_t)x->ptr & 15) != 0) return LAMP_ERR_INVALID_ARG;
+    return LAMP_OK;
+}
+
+#define TRY(expr)                                   \
+    do {                                            \
+        lamp_status_t s__ = (expr);                 \
+        if (s__ != LAMP_OK) return s__;             \
+    } while (0)
+
+lamp_status_t run_forward(const lamp_unet *net, const Plan &P, const bf16 *W, const float *Bv, float *probs,
+                          uint8_t *argmax, const uint8_t *labels, double *dice, cudaStream_t st)
+{
+    const lamp_unet_spec_t &S = net->spec;
+    for (size_t i = 0; i < net->layers.size(); ++i) {
+        const Layer &Ly = net->layers[i];
+        const LayerBuf &B = P.lb[i];
+        const bf16 *w = W + Ly.w_off;
+        const float *b = Bv + Ly.b_off;
+        if (Ly.kind == K_CONV || Ly.kind == K_DOWN) {
+            const int64_t Vn = (int64_t)B.y.d * B.y.h * B.y.w;
+            LAMP_CUDA_OK(cudaMemsetAsync(B.stats, 0, (size_t)B.y.n * Ly.c_out * 2 * sizeof(double), st));
+            TRY(conv_fwd(B.g, B.in, w, b, B.y, B.stats, st));
+            TRY(k_finalize_stats(B.stats, B.mr, (int64_t)B.y.n * Ly.c_out, 1.0 / (double)Vn, S.in_eps, st));
+            TRY(k_instnorm_relu_fwd(B.y, B.mr, B.out, st));
+        } else if (Ly.kind == K_UP) {
+            TRY(conv_fwd(B.g, B.in, w, b, B.out, nullptr, st));
+        } else {
+            TRY(k_head_softmax(B.in, w, b, S.num_classes, probs, argmax, labels, dice, st));
+        }
+    }
+    return LAMP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+lamp_status_t lamp_unet_create(const lamp_unet_spec_t *spec, lamp_unet_t **out)
+{
+    if (!spec || !out) return LAMP_ERR_INVALID_ARG;
+    if (spec->levels < 1 || spec->levels > 8 || spec->convs_per_level < 1) return LAMP_ERR_INVALID_ARG;
+    if (spec->num_classes < 2 || spec->num_classes > 16) return LAMP_ERR_UNSUPPORTED;
+    if (spec->in_channels != 1 && (spec->in_channels <= 0 || spec->in_channels % 8)) return LAMP_ERR_UNSUPPORTED;
+    for (int l = 0; l < spec->levels; ++l)
+        if (spec->channels[l] <= 0 || spec->channels[l] % 8 || spec->channels[l] > 2048) return LAMP_ERR_UNSUPPORTED;
+    if (spec->channels[0] > 64) return LAMP_ERR_UNSUPPORTED;           // head kernel limit
+    if (!(spec->in_eps > 0.f)) return LAMP_ERR_INVALID_ARG;
+    lamp_unet *net = new (std::nothrow) lamp_unet;
+    if (!net) return LAMP_ERR_INVALID_ARG;
+    net->spec = *spec;
+    const int L = spec->levels;
+    const int32_t *ch = spec->channels;
+    size_t wo = 0, bo = 0;
+    auto add = [&](int kind, int level, int ci, int co, int taps, bool to_cat, bool from_cat) {
+        Layer y{kind, level, ci, co, taps, wo, bo, to_cat, from_cat};
+        net->layers.push_back(y);
+        wo += (size_t)taps * ci * co;
+        wo = (wo + 7) / 8 * 8;                  // keep every layer's weights 16-byte aligned
+        bo += (size_t)co;
+    };
+    int c = spec->in_channels;
+    for (int l = 0; l < L; ++l) {
+        for (int j = 0; j < spec->convs_per_level; ++j) {
+            add(K_CONV, l, c, ch[l], 27, j == spec->convs_per_level - 1 && l < L - 1, false);
+            c = ch[l];
+        }
+        if (l < L - 1) { add(K_DOWN, l + 1, ch[l], ch[l + 1], 27, false, false); c = ch[l + 1]; }
+    }
+    for (int l = L - 2; l >= 0; --l) {
+        add(K_UP, l, ch[l + 1], ch[l], 8, false, false);
+        c = 2 * ch[l];
+        for (int j = 0; j < spec->convs_per_level; ++j) { add(K_CONV, l, c, ch[l], 27, false, j == 0); c = ch[l]; }
+    }
+    add(K_HEAD, 0, ch[0], spec->num_classes, 1, false, false);
+    net->n_w = wo;
+    net->n_b = bo;
+    *out = net;
+    return LAMP_OK;
+}
+
+void lamp_unet_destroy(lamp_unet_t *net) { delete net; }
+int32_t lamp_unet_num_layers(const lamp_unet_t *net) { return net ? (int32_t)net->layers.size() : 0; }
+size_t lamp_unet_weight_count(const lamp_unet_t *net) { return net ? net->n_w : 0; }
+size_t lamp_unet_bias_count(const lamp_unet_t *net) { return net ? net->n_b : 0; }
+
+lamp_status_t lamp_unet_param_layout(const lamp_unet_t *net, int32_t layer, size_t *w_off, size_t *b_off,
+                                     lamp_conv_desc_t *desc)
+{
+    if (!net || layer < 0 || layer >= (int32_t)net->layers.size()) return LAMP_ERR_INVALID_ARG;
+    const Layer &L = net->layers[layer];
+    if (w_off) *w_off = L.w_off;
+    if (b_off) *b_off = L.b_off;
+    if (desc) *desc = layer_desc(L);
+    return LAMP_OK;
+}
+
+size_t lamp_unet_workspace_bytes(const lamp_unet_t *net, int32_t n, int32_t d, int32_t h, int32_t w, int32_t mode)
+{
+    if (!net || n <= 0 || d <= 0 || h <= 0 || w <= 0) return 0;
+    Plan P;
+    make_plan(net, nullptr, nullptr, net->spec.in_channels, n, d, h, w, mode, true, &P);
+    return P.total;
+}
+
+lamp_status_t lamp_unet_forward(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                const lamp_tensor_t *x, float *probs, uint8_t *argmax,
+                                void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!weights_bf16 || !biases_f32) return LAMP_ERR_INVALID_ARG;
+    TRY(check_input(net, x));
+    if (!ws || ((uintptr_t)ws & 255)) return LAMP_ERR_WORKSPACE;
+    Plan P;
+    make_plan(net, ws, x->ptr, x->c_pitch, x->n, x->d, x->h, x->w, LAMP_MODE_INFER, false, &P);
+    if (P.total > ws_bytes) return LAMP_ERR_WORKSPACE;
+    return run_forward(net, P, (const bf16 *)weights_bf16, biases_f32, probs, argmax, nullptr, nullptr,
+                       (cudaStream_t)cuda_stream);
+}
+
+lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                   const lamp_tensor_t *x, const uint8_t *labels, float *loss,
+                                   float *grad_w, float *grad_b, float *probs,
+                                   void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!weights_bf16 || !biases_f32 || !labels || !loss || !grad_w || !grad_b) return LAMP_ERR_INVALID_ARG;
+    TRY(check_input(net, x));
+    if (!ws || ((uintptr_t)ws & 255)) return LAMP_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const lamp_unet_spec_t &S = net->spec;
+    Plan P;
+    make_plan(net, ws, x->ptr, x->c_pitch, x->n, x->d, x->h, x->w, LAMP_MODE_TRAIN, probs == nullptr, &P);
+    if (P.total > ws_bytes) return LAMP_ERR_WORKSPACE;
+    const bf16 *W = (const bf16 *)weights_bf16;
+    if (!probs) probs = P.probs;
+    TRY(run_forward(net, P, W, biases_f32, probs, nullptr, labels, P.dice, st));
+    TRY(k_dice_loss(P.dice, x->n, S.num_classes, loss, st));
+
+    // backward, last layer first.  `g` = gradient w.r.t. the current layer's output.
+    TView g{};
+    int pp = 0;
+    for (int i = (int)net->layers.size() - 1; i >= 0; --i) {
+        const Layer &Ly = net->layers[i];
+        const LayerBuf &B = P.lb[i];
+        const bf16 *w = W + Ly.w_off;
+        float *dw = grad_w + Ly.w_off, *db = grad_b + Ly.b_off;
+        if (Ly.kind == K_HEAD) {
+            TView dz = view(P.gbuf[pp], B.in.n, B.in.d, B.in.h, B.in.w, Ly.c_in, Ly.c_in, 0);
+            TRY(k_head_bwd(B.in, w, S.num_classes, probs, labels, P.dice, dz, dw, db, nullptr, st));
+            g = dz;
+            pp ^= 1;
+            continue;
+        }
+        TView dy;
+        if (Ly.kind == K_UP) {
+            dy = g;                                     // no norm / activation after the up conv
+        } else {
+            dy = view(P.dybuf, B.y.n, B.y.d, B.y.h, B.y.w, Ly.c_out, Ly.c_out, 0);
+            TView skip{};
+            if (Ly.to_cat) {                            // E_l also fed the skip: add that gradient
+                skip = P.dcat[Ly.level];
+                skip.c = Ly.c_out;                      // slice [0, C_l)
+            }
+            TRY(k_instnorm_relu_bwd(g, Ly.to_cat ? &skip : nullptr, B.y, B.mr, P.bwd_sums, dy, st));
+        }
+        TRY(conv_wgrad(B.g, B.in, dy, dw, db, P.scratch, P.scratch_bytes, st));
+        if (i == 0) break;                              // the network input needs no gradient
+        TView dx;
+        if (Ly.from_cat) {
+            dx = P.dcat[Ly.level];                      // all 2 C_l channels, kept for the encoder
+        } else {
+            dx = view(P.gbuf[pp], B.in.n, B.in.d, B.in.h, B.in.w, Ly.c_in, Ly.c_in, 0);
+            pp ^= 1;
+        }
+        TRY(conv_dgrad(B.g, dy, w, dx, P.scratch, P.scratch_bytes, st));
+        if (Ly.from_cat) {
+            g = dx;                                     // the up conv's output gradient: slice [C_l, 2 C_l)
+            g.p = (char *)g.p + (size_t)(Ly.c_in / 2) * 2;
+            g.c = Ly.c_in / 2;
+        } else {
+            g = dx;
+        }
+    }
+    return LAMP_OK;
+}
+
+static void window_grid(int len, int patch, float overlap, int32_t *nst, int32_t *stride)
+{
+    int s = (int)lrintf(patch * (1.0f - overlap));
+    if (s < 1) s = 1;
+    const int last = len > patch ? len - patch : 0;
+    int n = last / s + 1;
+    if ((n - 1) * s != last) ++n;
+    *nst = n;
+    *stride = s;
+}
+
+static lamp_status_t sw_check(const lamp_unet_t *net, int d, int h, int w, const int32_t patch[3], float overlap,
+                              int sw_batch)
+{
+    if (!net || !patch || sw_batch < 1 || !(overlap >= 0.f && overlap < 1.f)) return LAMP_ERR_INVALID_ARG;
+    const int dims[3] = {d, h, w};
+    const int m = 1 << (net->spec.levels - 1);
+    for (int a = 0; a < 3; ++a) {
+        if (patch[a] <= 0 || patch[a] > dims[a]) return LAMP_ERR_INVALID_ARG;
+        if (patch[a] % m) return LAMP_ERR_UNSUPPORTED;
+        if (patch[a] > 1024) return LAMP_ERR_UNSUPPORTED;
+    }
+    return LAMP_OK;
+}
+
+size_t lamp_sliding_window_workspace_bytes(const lamp_unet_t *net, int32_t d, int32_t h, int32_t w,
+                                           const int32_t patch[3], float overlap, int32_t sw_batch)
+{
+    if (sw_check(net, d, h, w, patch, overlap, sw_batch) != LAMP_OK) return 0;
+    int32_t nst[3], str[3];
+    window_grid(d, patch[0], overlap, &nst[0], &str[0]);
+    window_grid(h, patch[1], overlap, &nst[1], &str[1]);
+    window_grid(w, patch[2], overlap, &nst[2], &str[2]);
+    const size_t np = (size_t)nst[0] * nst[1] * nst[2];
+    const size_t pv = (size_t)patch[0] * patch[1] * patch[2];
+    size_t total = align_up(np * pv * net->spec.num_classes * sizeof(float), 256);
+    total += align_up((size_t)sw_batch * pv * net->spec.in_channels * sizeof(bf16), 256);
+    total += lamp_unet_workspace_bytes(net, sw_batch, patch[0], patch[1], patch[2], LAMP_MODE_INFER);
+    return total;
+}
+
+lamp_status_t lamp_sliding_window_infer(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                        const lamp_tensor_t *volume, const int32_t patch[3], float overlap,
+                                        int32_t sw_batch, int32_t window, float *probs_planar, uint8_t *argmax,
+                                        void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!weights_bf16 || !biases_f32 || !volume || !volume->ptr || (!argmax && !probs_planar)) return LAMP_ERR_INVALID_ARG;
+    if (volume->n != 1 || volume->dtype != LAMP_BF16 || volume->c != (net ? net->spec.in_channels : 0)) return LAMP_ERR_INVALID_ARG;
+    TRY(sw_check(net, volume->d, volume->h, volume->w, patch, overlap, sw_batch));
+    if (!ws || ((uintptr_t)ws & 255)) return LAMP_ERR_WORKSPACE;
+    if (ws_bytes < lamp_sliding_window_workspace_bytes(net, volume->d, volume->h, volume->w, patch, overlap, sw_batch))
+        return LAMP_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const lamp_unet_spec_t &S = net->spec;
+    int32_t nst[3], str[3];
+    window_grid(volume->d, patch[0], overlap, &nst[0], &str[0]);
+    window_grid(volume->h, patch[1], overlap, &nst[1], &str[1]);
+    window_grid(volume->w, patch[2], overlap, &nst[2], &str[2]);
+    const int np = nst[0] * nst[1] * nst[2];
+    const size_t pv = (size_t)patch[0] * patch[1] * patch[2];
+    char *p = (char *)ws;
+    float *pprobs = (float *)p;
+    p += align_up((size_t)np * pv * S.num_classes * sizeof(float), 256);
+    bf16 *pin = (bf16 *)p;
+    p += align_up((size_t)sw_batch * pv * S.in_channels * sizeof(bf16), 256);
+    void *nws = p;
+    TView vol = make_view(volume);
+    for (int first = 0; first < np; first += sw_batch) {
+        const int b = np - first < sw_batch ? np - first : sw_batch;
+        TView pt = view(pin, b, patch[0], patch[1], patch[2], S.in_channels, S.in_channels, 0);
+        TRY(k_gather_patches(vol, pt, first, nst, str, st));
+        Plan P;
+        make_plan(net, nws, pin, S.in_channels, b, patch[0], patch[1], patch[2], LAMP_MODE_INFER, false, &P);
+        TRY(run_forward(net, P, (const bf16 *)weights_bf16, biases_f32, pprobs + (size_t)first * pv * S.num_classes,
+                        nullptr, nullptr, nullptr, st));
+    }
+    return k_overlap_add(pprobs, S.num_classes, volume->d, volume->h, volume->w, patch, nst, str, window,
+                         probs_planar, argmax, st);
+}
+
+lamp_status_t lamp_overlap_add(const float *patch_probs, int32_t k, int32_t d, int32_t h, int32_t w,
+                               const int32_t patch[3], float overlap, int32_t window,
+                               float *probs_planar, uint8_t *argmax, void *cuda_stream)
+{
+    if (!patch_probs || !patch || d <= 0 || h <= 0 || w <= 0 || (!probs_planar && !argmax)) return LAMP_ERR_INVALID_ARG;
+    if (!(overlap >= 0.f && overlap < 1.f)) return LAMP_ERR_INVALID_ARG;
+    const int dims[3] = {d, h, w};
+    int32_t nst[3], str[3];
+    for (int a = 0; a < 3; ++a) {
+        if (patch[a] <= 0 || patch[a] > dims[a] || patch[a] > 1024) return LAMP_ERR_INVALID_ARG;
+        window_grid(dims[a], patch[a], overlap, &nst[a], &str[a]);
+    }
+    return k_overlap_add(patch_probs, k, d, h, w, patch, nst, str, window, probs_planar, argmax,
+                         (cudaStream_t)cuda_stream);
+}
+
+}  // extern "C"

@@ -24,3 +24,12 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Compile the CUDA library and the oracle's C file if they are missing or stale."""
+    from oracle import ops
+    from paper_2006_12575_b200 import build as lamp_build
+    ops.build()
+    lamp_build.build()

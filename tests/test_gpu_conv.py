@@ -1,0 +1,133 @@
+"""GPU parity of the single-layer convolution passes against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ops
+from paper_2006_12575_b200 import binding as B
+from paper_2006_12575_b200 import synth
+
+from _util import assert_close, dev_bf16, host_f64
+
+pytestmark = pytest.mark.gpu
+
+# (name, N, D, H, W, Ci, Co, k, s, p, transposed)
+CASES = [
+    ("first_layer_c1", 1, 9, 7, 10, 1, 8, 3, 1, 1, 0),
+    ("narrow_16_24", 2, 6, 5, 9, 16, 24, 3, 1, 1, 0),
+    ("down_8_16", 1, 8, 6, 10, 8, 16, 3, 2, 1, 0),
+    ("down_32_64", 1, 16, 8, 12, 32, 64, 3, 2, 1, 0),
+    ("up_16_8", 2, 3, 4, 5, 16, 8, 2, 2, 0, 1),
+    ("up_64_32", 1, 6, 4, 8, 64, 32, 2, 2, 0, 1),
+    ("head_8_4", 1, 5, 4, 6, 8, 4, 1, 1, 0, 0),
+    ("c32_ragged", 1, 9, 17, 33, 32, 32, 3, 1, 1, 0),
+    ("c64_ragged", 1, 33, 17, 9, 64, 64, 3, 1, 1, 0),
+    ("c64_cube16", 2, 16, 16, 16, 64, 64, 3, 1, 1, 0),
+    ("c64_to_32", 1, 8, 12, 20, 64, 32, 3, 1, 1, 0),
+    ("c128_64", 1, 8, 8, 24, 128, 64, 3, 1, 1, 0),
+    ("c32_to_128", 1, 4, 8, 16, 32, 128, 3, 1, 1, 0),
+    ("c256", 1, 4, 6, 8, 256, 256, 3, 1, 1, 0),
+    ("tiny_volume", 1, 2, 2, 2, 64, 64, 3, 1, 1, 0),
+    ("single_voxel", 1, 1, 1, 1, 32, 32, 3, 1, 1, 0),
+]
+
+
+def _oracle_shapes(N, D, H, W, k, s, p, tr):
+    if tr:
+        return (N, D * 2, H * 2, W * 2)
+    o = lambda n: (n + 2 * p - k) // s + 1
+    return (N, o(D), o(H), o(W))
+
+
+def _inputs(case, seed):
+    name, N, D, H, W, Ci, Co, k, s, p, tr = case
+    x = synth.normal_bf16((N, D, H, W, Ci), seed)
+    w = synth.kaiming_bf16(k ** 3, Co, Ci, (1 if tr else k ** 3) * Ci, seed + 1)
+    b = synth.rng(seed + 2).standard_normal(Co).astype(np.float32)
+    oshape = _oracle_shapes(N, D, H, W, k, s, p, tr) + (Co,)
+    dy = synth.normal_bf16(oshape, seed + 3)
+    return x, w, b, dy, oshape
+
+
+@pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
+def test_conv_fwd_matches_oracle(case):
+    name, N, D, H, W, Ci, Co, k, s, p, tr = case
+    x, w, b, dy, oshape = _inputs(case, 100)
+    ref = ops.convT3d_fwd(x, w, b, k, s) if tr else ops.conv3d_fwd(x, w, b, k, s, p)
+    desc = B.conv_desc(Ci, Co, k, s, p, tr)
+    xd, wd, bd = dev_bf16(x), dev_bf16(w), torch.from_numpy(b).cuda()
+    # fp32 output + statistics
+    y32 = torch.full(oshape, float("nan"), dtype=torch.float32, device="cuda")
+    stats = torch.zeros((N, Co, 2), dtype=torch.float64, device="cuda")
+    B.lamp_conv3d_fwd(desc, xd, wd, bd, y32, stats)
+    assert B.lamp_get_async_status() == 0
+    assert_close(host_f64(y32), ref, f"{name} fwd f32", rel=2e-5, mx=2e-5)
+    s_ref = np.stack([ref.sum(axis=(1, 2, 3)), (ref ** 2).sum(axis=(1, 2, 3))], axis=-1)
+    assert_close(host_f64(stats), s_ref, f"{name} stats", rel=1e-5, mx=1e-4)
+    # bf16 output into a channel slice of a wider buffer, no bias
+    pitch, off = Co + 16, 8
+    ybuf = torch.full(oshape[:4] + (pitch,), 7.0, dtype=torch.bfloat16, device="cuda")
+    B.lamp_conv3d_fwd(desc, xd, wd, None, B.tensor(ybuf, Co, off))
+    refnb = ref - b
+    assert_close(host_f64(ybuf[..., off:off + Co]), ops.bf16_round(refnb), f"{name} fwd bf16 slice")
+    assert (ybuf[..., :off] == 7.0).all() and (ybuf[..., off + Co:] == 7.0).all()
+    # twice the same call -> bit-identical output
+    y2 = torch.empty_like(y32)
+    B.lamp_conv3d_fwd(desc, xd, wd, bd, y2)
+    assert torch.equal(y2, y32)
+
+
+@pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
+def test_conv_dgrad_matches_oracle(case):
+    name, N, D, H, W, Ci, Co, k, s, p, tr = case
+    x, w, b, dy, oshape = _inputs(case, 200)
+    ref = ops.convT3d_dgrad(dy, w, (D, H, W), k, s) if tr else ops.conv3d_dgrad(dy, w, (D, H, W), k, s, p)
+    desc = B.conv_desc(Ci, Co, k, s, p, tr)
+    dyd, wd = dev_bf16(dy), dev_bf16(w)
+    dx = torch.full((N, D, H, W, Ci), float("nan"), dtype=torch.float32, device="cuda")
+    nbytes = B.lamp_conv3d_workspace_bytes(desc, dx, B.PASS_DGRAD)
+    ws = torch.empty(max(nbytes, 16), dtype=torch.uint8, device="cuda")
+    B.lamp_conv3d_dgrad(desc, dyd, wd, dx, ws)
+    assert B.lamp_get_async_status() == 0
+    assert_close(host_f64(dx), ref, f"{name} dgrad f32", rel=2e-5, mx=2e-5)
+    if Ci % 8 == 0:
+        pitch, off = Ci + 8, 8
+        dxb = torch.full((N, D, H, W, pitch), 3.0, dtype=torch.bfloat16, device="cuda")
+        # dy read from a channel slice as well
+        dyp = torch.zeros(oshape[:4] + (Co + 8,), dtype=torch.bfloat16, device="cuda")
+        dyp[..., 8:] = dyd
+        B.lamp_conv3d_dgrad(desc, B.tensor(dyp, Co, 8), wd, B.tensor(dxb, Ci, off), ws)
+        assert_close(host_f64(dxb[..., off:]), ops.bf16_round(ref), f"{name} dgrad bf16 slice")
+        assert (dxb[..., :off] == 3.0).all()
+
+
+@pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
+def test_conv_wgrad_matches_oracle(case):
+    name, N, D, H, W, Ci, Co, k, s, p, tr = case
+    x, w, b, dy, oshape = _inputs(case, 300)
+    dw_ref, db_ref = ops.convT3d_wgrad(x, dy, k, s) if tr else ops.conv3d_wgrad(x, dy, k, s, p)
+    desc = B.conv_desc(Ci, Co, k, s, p, tr)
+    xd, dyd = dev_bf16(x), dev_bf16(dy)
+    dw = torch.full((k ** 3, Co, Ci), float("nan"), dtype=torch.float32, device="cuda")
+    db = torch.full((Co,), float("nan"), dtype=torch.float32, device="cuda")
+    nbytes = B.lamp_conv3d_workspace_bytes(desc, xd, B.PASS_WGRAD)
+    ws = torch.empty(max(nbytes, 16), dtype=torch.uint8, device="cuda")
+    B.lamp_conv3d_wgrad(desc, xd, dyd, dw, db, ws)
+    assert B.lamp_get_async_status() == 0
+    assert_close(host_f64(dw), dw_ref, f"{name} wgrad", rel=2e-5, mx=2e-5)
+    assert_close(host_f64(db), db_ref, f"{name} dbias", rel=2e-5, mx=2e-5)
+    # too small a workspace is refused
+    if nbytes > 256:
+        with pytest.raises(B.LampError) as e:
+            B.lamp_conv3d_wgrad(desc, xd, dyd, dw, db, ws[:256])
+        assert e.value.status == 3
+
+
+def test_empty_volume_is_a_no_op():
+    desc = B.conv_desc(8, 8)
+    x = torch.empty((1, 0, 4, 4, 8), dtype=torch.bfloat16, device="cuda")
+    y = torch.empty((1, 0, 4, 4, 8), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((27, 8, 8), dtype=torch.bfloat16, device="cuda")
+    B.lamp_conv3d_fwd(desc, B.Tensor(w.data_ptr(), 0, 1, 0, 4, 4, 8, 8, 0), w, None,
+                      B.Tensor(w.data_ptr(), 0, 1, 0, 4, 4, 8, 8, 0))
+    assert B.lamp_get_async_status() == 0
