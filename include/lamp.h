@@ -158,6 +158,31 @@ lamp_status_t lamp_unet_param_layout(const lamp_unet_t *net, int32_t layer, size
 enum { LAMP_MODE_INFER = 0, LAMP_MODE_TRAIN = 1 };
 size_t lamp_unet_workspace_bytes(const lamp_unet_t *net, int32_t n, int32_t d, int32_t h, int32_t w, int32_t mode);
 
+/* Where a pass keeps one of its tensors inside the workspace, for inspection after the call.
+ * Training mode keeps every tensor listed; inference mode keeps LAMP_T_IN / LAMP_T_OUT only (the
+ * raw conv output is a buffer shared by all layers there).  On success *offset is the byte offset
+ * from the workspace base to the tensor's first element (the slice's first channel) and *out
+ * describes it (ptr = NULL, c_offset = 0, c_pitch = distance between voxels).
+ * LAMP_T_STATS is fp64 [n][c_out][2] (sum, sum of squares), LAMP_T_MU_RSTD fp32 [n][c_out][2],
+ * LAMP_T_PROBS fp32 [n*d*h*w][num_classes] (present when the caller passed probs = NULL);
+ * for these *out reports c = 2*c_out (or num_classes) per n.
+ * Returns LAMP_ERR_UNSUPPORTED when the layer has no such tensor (e.g. LAMP_T_IN of layer 0, which
+ * is the caller's buffer, or LAMP_T_Y of an up conv). */
+enum {
+    LAMP_T_IN = 0,       /* layer input (bf16)                                            */
+    LAMP_T_Y = 1,        /* raw conv output before normalisation (bf16)                    */
+    LAMP_T_OUT = 2,      /* layer output: normalised + ReLU, or the up conv's output (bf16)*/
+    LAMP_T_STATS = 3,
+    LAMP_T_MU_RSTD = 4,
+    LAMP_T_DY = 5,       /* gradient w.r.t. the raw conv output (bf16)                     */
+    LAMP_T_DIN = 6,      /* gradient w.r.t. the layer input (bf16)                         */
+    LAMP_T_DOUT = 7,     /* gradient w.r.t. the layer output, main source (bf16)           */
+    LAMP_T_DOUT2 = 8,    /* second source: the skip path's gradient, encoder block outputs */
+    LAMP_T_PROBS = 9
+};
+lamp_status_t lamp_unet_tensor_layout(const lamp_unet_t *net, int32_t n, int32_t d, int32_t h, int32_t w, int32_t mode,
+                                      int32_t layer, int32_t which, lamp_tensor_t *out, size_t *offset);
+
 /* One forward pass.  x: bf16 [n,d,h,w,in_channels] (d,h,w divisible by 2^(levels-1)).
  * probs: fp32 [n*d*h*w][num_classes] softmax output, or NULL.  argmax: uint8 [n*d*h*w] class of
  * largest probability (lowest index on ties), or NULL.  Stored intermediates are bf16. */
@@ -182,7 +207,9 @@ lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_b
  * weight 1 (window = 0) or a Gaussian (window = 1: sigma = patch/8 per axis, normalised to
  * maximum 1, floored at 1e-3): A[v,k] = sum_p w p / sum_p w.
  * volume: bf16 [1,d,h,w,in_channels].  probs_planar: fp32 [num_classes][d][h][w] or NULL.
- * argmax: uint8 [d*h*w].  sw_batch: patches per network pass (>= 1). */
+ * argmax: uint8 [d*h*w].  sw_batch: patches per network pass (>= 1).
+ * After the call the first n_patches*pd*ph*pw*num_classes floats of the workspace hold the
+ * per-patch probabilities, fp32 [n_patches][pd*ph*pw][num_classes]. */
 size_t lamp_sliding_window_workspace_bytes(const lamp_unet_t *net, int32_t d, int32_t h, int32_t w,
                                            const int32_t patch[3], float overlap, int32_t sw_batch);
 lamp_status_t lamp_sliding_window_infer(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,

@@ -68,6 +68,7 @@ def lib():
             "lamp_unet_bias_count": (sz, [vp]),
             "lamp_unet_param_layout": (C.c_int, [vp, i32, C.POINTER(sz), C.POINTER(sz), DP]),
             "lamp_unet_workspace_bytes": (sz, [vp, i32, i32, i32, i32, i32]),
+            "lamp_unet_tensor_layout": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, i32, TP, C.POINTER(sz)]),
             "lamp_unet_forward": (C.c_int, [vp, vp, vp, TP, vp, vp, vp, sz, vp]),
             "lamp_unet_train_step": (C.c_int, [vp, vp, vp, TP, vp, vp, vp, vp, vp, vp, sz, vp]),
             "lamp_sliding_window_workspace_bytes": (sz, [vp, i32, i32, i32, I3, f32, i32]),
@@ -88,7 +89,7 @@ def lib():
 EXPORTS = ["lamp_conv3d_workspace_bytes", "lamp_conv3d_fwd", "lamp_conv3d_dgrad", "lamp_conv3d_wgrad",
            "lamp_instnorm_relu_fwd", "lamp_instnorm_relu_bwd", "lamp_unet_create", "lamp_unet_destroy",
            "lamp_unet_num_layers", "lamp_unet_weight_count", "lamp_unet_bias_count", "lamp_unet_param_layout",
-           "lamp_unet_workspace_bytes", "lamp_unet_forward", "lamp_unet_train_step",
+           "lamp_unet_workspace_bytes", "lamp_unet_tensor_layout", "lamp_unet_forward", "lamp_unet_train_step",
            "lamp_sliding_window_workspace_bytes", "lamp_sliding_window_infer", "lamp_overlap_add",
            "lamp_get_async_status", "lamp_status_string", "lamp_version"]
 
@@ -194,6 +195,19 @@ def lamp_unet_param_layout(net, layer):
 
 def lamp_unet_workspace_bytes(net, n, d, h, w, mode):
     return lib().lamp_unet_workspace_bytes(net, n, d, h, w, mode)
+
+
+T_IN, T_Y, T_OUT, T_STATS, T_MU_RSTD, T_DY, T_DIN, T_DOUT, T_DOUT2, T_PROBS = range(10)
+
+
+def lamp_unet_tensor_layout(net, n, d, h, w, mode, layer, which):
+    """Returns (descriptor, byte offset into the workspace), or None if the layer has no such tensor."""
+    t, off = Tensor(), C.c_size_t()
+    st = lib().lamp_unet_tensor_layout(net, n, d, h, w, mode, layer, which, C.byref(t), C.byref(off))
+    if st == 2:
+        return None
+    _check(st, "lamp_unet_tensor_layout")
+    return t, off.value
 
 
 def lamp_unet_forward(net, weights, biases, x, probs, argmax, ws):

@@ -47,6 +47,9 @@ struct LayerBuf {
     TView y;                    // raw conv output (norm layers)
     double *stats;              // [n][c_out][2]
     float *mr;                  // [n][c_out][2]
+    TView dy;                   // gradient w.r.t. the raw conv output (norm layers; train mode)
+    TView din;                  // gradient w.r.t. the layer's input (train mode; empty for layer 0)
+    TView dout, dout2;          // gradient w.r.t. the layer's output: main source and skip source (may be empty)
     ConvGeom g;
     lamp_conv_desc_t desc;
 };
@@ -57,8 +60,6 @@ struct Plan {
     float *probs;                       // [V][K] when the caller gave none
     double *dice;                       // [n][K][3]
     double *bwd_sums;                   // [n][cmax][2]
-    bf16 *dybuf;                        // gradient w.r.t. a raw conv output, max size
-    bf16 *gbuf[2];                      // ping-pong gradient w.r.t. a layer input
     void *scratch;                      // conv workspace (wgrad partials / transposed weights)
     size_t scratch_bytes;
     size_t total;
@@ -102,7 +103,7 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
         void *p = A.take(vox(l) * 2 * S.channels[l] * sizeof(bf16));
         P->cat[l] = view(p, n, dd(l), hh(l), ww(l), 2 * S.channels[l], 2 * S.channels[l], 0);
     }
-    size_t ymax = 0, cmax = 0, inmax = 0;
+    size_t ymax = 0, cmax = 0;
     for (const Layer &Ly : net->layers) {
         if (Ly.kind == K_CONV || Ly.kind == K_DOWN) ymax = ymax > vox(Ly.level) * Ly.c_out ? ymax : vox(Ly.level) * Ly.c_out;
         cmax = cmax > (size_t)Ly.c_out ? cmax : (size_t)Ly.c_out;
@@ -127,8 +128,6 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
             g.transposed = B.desc.transposed;
             B.g = g;
         }
-        const size_t in_elems = (size_t)cur.n * cur.d * cur.h * cur.w * Ly.c_in;
-        inmax = inmax > in_elems ? inmax : in_elems;
         if (mode == LAMP_MODE_TRAIN) {
             size_t s1 = conv_ws_bytes(B.g, LAMP_PASS_WGRAD), s2 = conv_ws_bytes(B.g, LAMP_PASS_DGRAD);
             scratch = scratch > s1 ? scratch : s1;
@@ -158,17 +157,44 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
     }
     const size_t V0 = vox(0);
     P->probs = need_probs ? (float *)A.take(V0 * S.num_classes * sizeof(float)) : nullptr;
-    P->dice = nullptr; P->bwd_sums = nullptr; P->dybuf = nullptr; P->gbuf[0] = P->gbuf[1] = nullptr;
+    P->dice = nullptr; P->bwd_sums = nullptr;
     P->scratch = nullptr; P->scratch_bytes = 0;
+    for (LayerBuf &B : P->lb) { B.dy = TView{}; B.din = TView{}; B.dout = TView{}; B.dout2 = TView{}; }
     if (mode == LAMP_MODE_TRAIN) {
+        // Every gradient tensor gets its own buffer (nothing is recycled), so that each step of the
+        // backward pass can be inspected after the call.
         P->dice = (double *)A.take((size_t)n * S.num_classes * 3 * sizeof(double));
         P->bwd_sums = (double *)A.take((size_t)n * cmax * 2 * sizeof(double));
-        P->dybuf = (bf16 *)A.take(ymax * sizeof(bf16));
-        P->gbuf[0] = (bf16 *)A.take(inmax * sizeof(bf16));
-        P->gbuf[1] = (bf16 *)A.take(inmax * sizeof(bf16));
         for (int l = 0; l + 1 < L; ++l) {
             void *p = A.take(vox(l) * 2 * S.channels[l] * sizeof(bf16));
             P->dcat[l] = view(p, n, dd(l), hh(l), ww(l), 2 * S.channels[l], 2 * S.channels[l], 0);
+        }
+        TView g{};
+        for (int i = (int)net->layers.size() - 1; i >= 0; --i) {
+            const Layer &Ly = net->layers[i];
+            LayerBuf &B = P->lb[i];
+            B.dout = g;
+            if (Ly.kind == K_CONV || Ly.kind == K_DOWN) {
+                void *p = A.take(vox(Ly.level) * Ly.c_out * sizeof(bf16));
+                B.dy = view(p, n, dd(Ly.level), hh(Ly.level), ww(Ly.level), Ly.c_out, Ly.c_out, 0);
+                if (Ly.to_cat) {                        // E_l also fed the skip: slice [0, C_l) of dcat_l
+                    B.dout2 = P->dcat[Ly.level];
+                    B.dout2.c = Ly.c_out;
+                }
+            } else if (Ly.kind == K_UP) {
+                B.dy = g;                               // no norm / activation after the up conv
+            }
+            if (i == 0) break;                          // the network input needs no gradient
+            if (Ly.from_cat) {
+                B.din = P->dcat[Ly.level];              // all 2 C_l channels, kept for the encoder
+                g = B.din;                              // the up conv's output gradient: slice [C_l, 2 C_l)
+                g.p = g.p ? (char *)g.p + (size_t)(Ly.c_in / 2) * 2 : nullptr;
+                g.c = Ly.c_in / 2;
+            } else {
+                void *p = A.take((size_t)B.in.n * B.in.d * B.in.h * B.in.w * Ly.c_in * sizeof(bf16));
+                B.din = view(p, B.in.n, B.in.d, B.in.h, B.in.w, Ly.c_in, Ly.c_in, 0);
+                g = B.din;
+            }
         }
         P->scratch = A.take(scratch);
         P->scratch_bytes = scratch;
@@ -290,6 +316,49 @@ size_t lamp_unet_workspace_bytes(const lamp_unet_t *net, int32_t n, int32_t d, i
     return P.total;
 }
 
+lamp_status_t lamp_unet_tensor_layout(const lamp_unet_t *net, int32_t n, int32_t d, int32_t h, int32_t w, int32_t mode,
+                                      int32_t layer, int32_t which, lamp_tensor_t *out, size_t *offset)
+{
+    if (!net || !out || !offset || n <= 0 || d <= 0 || h <= 0 || w <= 0) return LAMP_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= (int32_t)net->layers.size()) return LAMP_ERR_INVALID_ARG;
+    Plan P;
+    char *const fake = (char *)(uintptr_t)(1ull << 40);          // offsets are measured from this base
+    char *const fake_x = (char *)(uintptr_t)(1ull << 20);
+    make_plan(net, fake, fake_x, net->spec.in_channels, n, d, h, w, mode, mode == LAMP_MODE_TRAIN, &P);
+    const LayerBuf &B = P.lb[layer];
+    TView v{};
+    int f32 = 0, f64 = 0;
+    switch (which) {
+    case LAMP_T_IN: v = B.in; break;
+    case LAMP_T_Y: v = B.y; break;
+    case LAMP_T_OUT: v = B.out; break;
+    case LAMP_T_DY: v = B.dy; break;
+    case LAMP_T_DIN: v = B.din; break;
+    case LAMP_T_DOUT: v = B.dout; break;
+    case LAMP_T_DOUT2: v = B.dout2; break;
+    case LAMP_T_MU_RSTD:
+        if (B.mr) { v.p = B.mr; v.n = n; v.d = v.h = v.w = 1; v.c = 2 * B.g.co; v.pitch = v.c; f32 = 1; }
+        break;
+    case LAMP_T_STATS:
+        if (B.stats) { v.p = B.stats; v.n = n; v.d = v.h = v.w = 1; v.c = 2 * B.g.co; v.pitch = v.c; f64 = 1; }
+        break;
+    case LAMP_T_PROBS:
+        v.p = P.probs; v.n = n; v.d = d; v.h = h; v.w = w; v.c = net->spec.num_classes; v.pitch = v.c; f32 = 1;
+        break;
+    default: return LAMP_ERR_INVALID_ARG;
+    }
+    if (!v.p) return LAMP_ERR_UNSUPPORTED;                        // this layer / mode has no such tensor
+    if ((char *)v.p < fake) return LAMP_ERR_UNSUPPORTED;          // the network input lives in the caller's buffer
+    out->ptr = nullptr;
+    out->dtype = f32 ? LAMP_F32 : LAMP_BF16;
+    out->n = v.n; out->d = v.d; out->h = v.h; out->w = v.w; out->c = v.c;
+    out->c_pitch = v.pitch;
+    out->c_offset = 0;
+    *offset = (size_t)((char *)v.p - fake);
+    (void)f64;
+    return LAMP_OK;
+}
+
 lamp_status_t lamp_unet_forward(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
                                 const lamp_tensor_t *x, float *probs, uint8_t *argmax,
                                 void *ws, size_t ws_bytes, void *cuda_stream)
@@ -315,57 +384,28 @@ lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_b
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const lamp_unet_spec_t &S = net->spec;
     Plan P;
-    make_plan(net, ws, x->ptr, x->c_pitch, x->n, x->d, x->h, x->w, LAMP_MODE_TRAIN, probs == nullptr, &P);
+    make_plan(net, ws, x->ptr, x->c_pitch, x->n, x->d, x->h, x->w, LAMP_MODE_TRAIN, true, &P);
     if (P.total > ws_bytes) return LAMP_ERR_WORKSPACE;
     const bf16 *W = (const bf16 *)weights_bf16;
     if (!probs) probs = P.probs;
     TRY(run_forward(net, P, W, biases_f32, probs, nullptr, labels, P.dice, st));
     TRY(k_dice_loss(P.dice, x->n, S.num_classes, loss, st));
 
-    // backward, last layer first.  `g` = gradient w.r.t. the current layer's output.
-    TView g{};
-    int pp = 0;
+    // backward, last layer first
     for (int i = (int)net->layers.size() - 1; i >= 0; --i) {
         const Layer &Ly = net->layers[i];
         const LayerBuf &B = P.lb[i];
         const bf16 *w = W + Ly.w_off;
         float *dw = grad_w + Ly.w_off, *db = grad_b + Ly.b_off;
         if (Ly.kind == K_HEAD) {
-            TView dz = view(P.gbuf[pp], B.in.n, B.in.d, B.in.h, B.in.w, Ly.c_in, Ly.c_in, 0);
-            TRY(k_head_bwd(B.in, w, S.num_classes, probs, labels, P.dice, dz, dw, db, nullptr, st));
-            g = dz;
-            pp ^= 1;
+            TRY(k_head_bwd(B.in, w, S.num_classes, probs, labels, P.dice, B.din, dw, db, nullptr, st));
             continue;
         }
-        TView dy;
-        if (Ly.kind == K_UP) {
-            dy = g;                                     // no norm / activation after the up conv
-        } else {
-            dy = view(P.dybuf, B.y.n, B.y.d, B.y.h, B.y.w, Ly.c_out, Ly.c_out, 0);
-            TView skip{};
-            if (Ly.to_cat) {                            // E_l also fed the skip: add that gradient
-                skip = P.dcat[Ly.level];
-                skip.c = Ly.c_out;                      // slice [0, C_l)
-            }
-            TRY(k_instnorm_relu_bwd(g, Ly.to_cat ? &skip : nullptr, B.y, B.mr, P.bwd_sums, dy, st));
-        }
-        TRY(conv_wgrad(B.g, B.in, dy, dw, db, P.scratch, P.scratch_bytes, st));
-        if (i == 0) break;                              // the network input needs no gradient
-        TView dx;
-        if (Ly.from_cat) {
-            dx = P.dcat[Ly.level];                      // all 2 C_l channels, kept for the encoder
-        } else {
-            dx = view(P.gbuf[pp], B.in.n, B.in.d, B.in.h, B.in.w, Ly.c_in, Ly.c_in, 0);
-            pp ^= 1;
-        }
-        TRY(conv_dgrad(B.g, dy, w, dx, P.scratch, P.scratch_bytes, st));
-        if (Ly.from_cat) {
-            g = dx;                                     // the up conv's output gradient: slice [C_l, 2 C_l)
-            g.p = (char *)g.p + (size_t)(Ly.c_in / 2) * 2;
-            g.c = Ly.c_in / 2;
-        } else {
-            g = dx;
-        }
+        if (Ly.kind != K_UP)
+            TRY(k_instnorm_relu_bwd(B.dout, Ly.to_cat ? &B.dout2 : nullptr, B.y, B.mr, P.bwd_sums, B.dy, st));
+        TRY(conv_wgrad(B.g, B.in, B.dy, dw, db, P.scratch, P.scratch_bytes, st));
+        if (i == 0) break;
+        TRY(conv_dgrad(B.g, B.dy, w, B.din, P.scratch, P.scratch_bytes, st));
     }
     return LAMP_OK;
 }

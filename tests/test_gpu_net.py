@@ -75,6 +75,123 @@ def test_instnorm_relu_fwd_bwd_match_oracle(shape, pitch, off):
         assert_close(host_f64(dy), ref, "instnorm bwd")
 
 
+def ws_read(wsb, layout):
+    """Copies a tensor kept in the workspace to the host as float64 [n,d,h,w,c]."""
+    t, off = layout
+    es = {B.LAMP_BF16: 2, B.LAMP_F32: 4}[t.dtype]
+    dt = {B.LAMP_BF16: torch.bfloat16, B.LAMP_F32: torch.float32}[t.dtype]
+    V = t.n * t.d * t.h * t.w
+    count = (V - 1) * t.c_pitch + t.c
+    flat = wsb[off:off + count * es].view(dt)
+    return host_f64(torch.as_strided(flat, (V, t.c), (t.c_pitch, 1))).reshape(t.n, t.d, t.h, t.w, t.c)
+
+
+def ws_read_f64(wsb, layout):
+    t, off = layout
+    return wsb[off:off + t.n * t.c * 8].view(torch.float64).cpu().numpy().reshape(t.n, t.c // 2, 2)
+
+
+def check_network_layer_by_layer(levels, ch, cpl, K, dhw, seed, x, lab, tight=2e-5):
+    """Runs lamp_unet_train_step once, then checks EVERY step of the forward and backward pass on
+    its own: the oracle recomputes each step in fp64 from the tensors the GPU actually stored as
+    that step's inputs, and the GPU's stored output must match (bf16-rounded where the path stores
+    bf16).  This isolates each kernel's arithmetic from the chaotic growth of rounding differences
+    along a deep bf16 chain, which the end-to-end comparison below then bounds separately."""
+    net, spec, lay, ws, bs, wd, bd, offs = make_net(levels, ch, cpl, K, seed=seed)
+    D, H, W = dhw
+    N = x.shape[0]
+    V = N * D * H * W
+    loss = torch.zeros((1,), dtype=torch.float32, device="cuda")
+    gw = torch.full((B.lamp_unet_weight_count(net),), float("nan"), dtype=torch.float32, device="cuda")
+    gb = torch.full((B.lamp_unet_bias_count(net),), float("nan"), dtype=torch.float32, device="cuda")
+    probs = torch.empty((V, K), dtype=torch.float32, device="cuda")
+    wsb = torch.empty(B.lamp_unet_workspace_bytes(net, N, D, H, W, B.MODE_TRAIN), dtype=torch.uint8, device="cuda")
+    B.lamp_unet_train_step(net, wd, bd, dev_bf16(x), torch.from_numpy(lab).cuda(), loss, gw, gb, probs, wsb)
+    assert B.lamp_get_async_status() == 0
+    gw_h, gb_h = host_f64(gw), host_f64(gb)
+    p_gpu = host_f64(probs).reshape(N, D, H, W, K)
+    lay_of = lambda i, which: B.lamp_unet_tensor_layout(net, N, D, H, W, B.MODE_TRAIN, i, which)
+    eps = spec.eps
+    for i, l in enumerate(lay):
+        w64, b64 = ws[i].astype(np.float64), bs[i].astype(np.float64)
+        x_in = x.astype(np.float64) if i == 0 else ws_read(wsb, lay_of(i, B.T_IN))
+        wo, bo = offs[i]
+        dW = gw_h[wo:wo + ws[i].size].reshape(ws[i].shape)
+        dB = gb_h[bo:bo + l.c_out]
+        what = f"{l.name}"
+        if l.kind in ("conv", "down"):
+            s = 2 if l.kind == "down" else 1
+            y_ref = ops.conv3d_fwd(x_in, w64, b64, 3, s, 1)
+            y_gpu = ws_read(wsb, lay_of(i, B.T_Y))
+            assert_close(y_gpu, ops.bf16_round(y_ref), what + " y")
+            st = ws_read_f64(wsb, lay_of(i, B.T_STATS))
+            st_ref = np.stack([y_ref.sum(axis=(1, 2, 3)), (y_ref ** 2).sum(axis=(1, 2, 3))], -1)
+            assert_close(st, st_ref, what + " stats", rel=1e-5, mx=1e-4)
+            mu, var, rstd = ops.instnorm_stats(y_ref, eps)
+            t, off = lay_of(i, B.T_MU_RSTD)
+            mr = wsb[off:off + N * l.c_out * 8].view(torch.float32).cpu().numpy().reshape(N, l.c_out, 2).astype(np.float64)
+            assert_close(mr[..., 0], mu[:, 0, 0, 0, :], what + " mu", rel=1e-4, mx=1e-4)
+            assert_close(mr[..., 1], rstd[:, 0, 0, 0, :], what + " rstd", rel=1e-4, mx=1e-4)
+            mu_g, rs_g = mr[..., 0][:, None, None, None, :], mr[..., 1][:, None, None, None, :]
+            z_gpu = ws_read(wsb, lay_of(i, B.T_OUT))
+            assert_close(z_gpu, ops.bf16_round(ops.instnorm_relu_fwd(y_gpu, mu_g, rs_g)), what + " z", rel=2e-4, mx=4e-3)
+            # backward
+            g = ws_read(wsb, lay_of(i, B.T_DOUT))
+            l2 = lay_of(i, B.T_DOUT2)
+            assert (l2 is not None) == (l.name.startswith("enc") and lay[i + 1].kind == "down")
+            if l2 is not None:
+                g = g + ws_read(wsb, l2)
+            dy_gpu = ws_read(wsb, lay_of(i, B.T_DY))
+            assert_close(dy_gpu, ops.bf16_round(ops.instnorm_relu_bwd(g, y_gpu, mu_g, rs_g)), what + " dy")
+            dw_ref, db_ref = ops.conv3d_wgrad(x_in, dy_gpu, 3, s, 1)
+            assert_close(dW, dw_ref, what + " dw", rel=tight, mx=tight)
+            assert_close(dB, db_ref, what + " db", rel=1e-4, mx=1e-4)
+            if i > 0:
+                din = ws_read(wsb, lay_of(i, B.T_DIN))
+                assert_close(din, ops.bf16_round(ops.conv3d_dgrad(dy_gpu, w64, x_in.shape[1:4], 3, s, 1)), what + " din")
+            else:
+                assert lay_of(i, B.T_DIN) is None
+        elif l.kind == "up":
+            u_gpu = ws_read(wsb, lay_of(i, B.T_OUT))
+            assert_close(u_gpu, ops.bf16_round(ops.convT3d_fwd(x_in, w64, b64, 2, 2)), what + " out")
+            dy_gpu = ws_read(wsb, lay_of(i, B.T_DY))
+            dw_ref, db_ref = ops.convT3d_wgrad(x_in, dy_gpu, 2, 2)
+            assert_close(dW, dw_ref, what + " dw", rel=tight, mx=tight)
+            assert_close(dB, db_ref, what + " db", rel=1e-4, mx=1e-4)
+            din = ws_read(wsb, lay_of(i, B.T_DIN))
+            assert_close(din, ops.bf16_round(ops.convT3d_dgrad(dy_gpu, w64, x_in.shape[1:4], 2, 2)), what + " din")
+        else:
+            p_ref = ops.softmax(ops.conv3d_fwd(x_in, w64, b64, 1, 1, 0))
+            assert_close(p_gpu, p_ref, what + " probs", rel=1e-5, mx=1e-5)
+            assert abs(float(loss.item()) - ops.dice_loss(p_gpu, lab)) < 1e-5
+            dl = ops.dice_loss_grad_logits(p_gpu, lab)
+            dw_ref, db_ref = ops.conv3d_wgrad(x_in, dl, 1, 1, 0)
+            assert_close(dW, dw_ref, what + " dw", rel=1e-4, mx=1e-4)
+            assert_close(dB, db_ref, what + " db", rel=1e-4, mx=1e-4)
+            din = ws_read(wsb, lay_of(i, B.T_DIN))
+            assert_close(din, ops.bf16_round(ops.conv3d_dgrad(dl, w64, x_in.shape[1:4], 1, 1, 0)), what + " din")
+    # End to end against the storage-mirrored oracle.  Two correct bf16 evaluations differ by rounding
+    # decisions that flip on fp32-level differences and then spread; their distance is bounded by the
+    # bf16 storage error itself, measured here as |mirrored oracle - unrounded oracle|.
+    ws64 = [a.astype(np.float64) for a in ws]
+    bs64 = [a.astype(np.float64) for a in bs]
+    loss_q, dWq, dBq, p_q = O.train_step(spec, ws64, bs64, x.astype(np.float64), lab, quantise=True)
+    loss_f, dWf, dBf, p_f = O.train_step(spec, ws64, bs64, x.astype(np.float64), lab, quantise=False)
+    budget = np.linalg.norm(p_q - p_f) / np.linalg.norm(p_f)
+    e2e = np.linalg.norm(p_gpu - p_q) / np.linalg.norm(p_q)
+    assert e2e <= max(1e-3, 2.0 * budget), (e2e, budget)
+    assert abs(float(loss.item()) - loss_q) <= max(1e-3, 2.0 * abs(loss_q - loss_f) / abs(loss_f)) * abs(loss_q)
+    for i, l in enumerate(lay):
+        wo, _ = offs[i]
+        got = gw_h[wo:wo + ws[i].size].reshape(ws[i].shape)
+        bud = np.linalg.norm(dWq[i] - dWf[i]) / np.linalg.norm(dWf[i])
+        err = np.linalg.norm(got - dWq[i]) / np.linalg.norm(dWq[i])
+        assert err <= max(1e-3, 2.0 * bud), (l.name, err, bud)
+    agree, strict, near = tie_aware_agreement(np.argmax(p_gpu, -1), p_q)
+    B.lamp_unet_destroy(net)
+    return dict(e2e=e2e, budget=budget, argmax_e2e=agree)
+
+
 CFG0 = dict(levels=3, ch=[8, 16, 32], cpl=2, K=4)
 
 
@@ -84,50 +201,55 @@ def _cfg0_inputs():
     return x, lab
 
 
-def test_unet_forward_tiny_matches_oracle():
+def test_train_step_tiny_unet_every_step_matches_oracle():
+    x, lab = _cfg0_inputs()
+    r = check_network_layer_by_layer(CFG0["levels"], CFG0["ch"], CFG0["cpl"], CFG0["K"], (32, 32, 32), 1, x, lab)
+    print("tiny U-Net:", r)
+
+
+def test_train_step_wide_unet_every_step_matches_oracle():
+    # widths that take the tensor-core path, a ragged non-cubic volume, batch of 2
+    D, H, W = 8, 12, 20
+    x = synth.bf16_round(np.stack([synth.blurred_noise((D, H, W), 1.5, s) for s in (3, 4)]))[..., None]
+    lab = np.stack([synth.labels_blobs((D, H, W), 5 + s, 5, 1.5) for s in (0, 1)])
+    r = check_network_layer_by_layer(2, [32, 64], 2, 5, (D, H, W), 2, x, lab)
+    print("wide U-Net:", r)
+
+
+def test_unet_forward_head_argmax_matches_oracle_on_stored_input():
     net, spec, lay, ws, bs, wd, bd, _ = make_net(CFG0["levels"], CFG0["ch"], CFG0["cpl"], CFG0["K"], seed=1)
     x, _ = _cfg0_inputs()
-    ref = O.forward(spec, ws, bs, x.astype(np.float64), quantise=True)
     V = 32 ** 3
     probs = torch.empty((V, 4), dtype=torch.float32, device="cuda")
     seg = torch.empty((V,), dtype=torch.uint8, device="cuda")
     wsb = torch.empty(B.lamp_unet_workspace_bytes(net, 1, 32, 32, 32, B.MODE_INFER), dtype=torch.uint8, device="cuda")
     B.lamp_unet_forward(net, wd, bd, dev_bf16(x), probs, seg, wsb)
     assert B.lamp_get_async_status() == 0
-    assert_close(host_f64(probs), ref.reshape(V, 4), "unet forward probs")
-    agree, strict, near = tie_aware_agreement(seg.cpu().numpy(), ref.reshape(V, 4))
+    # the head on its own: oracle applied to the input the GPU stored for it
+    hi = len(lay) - 1
+    z = ws_read(wsb, B.lamp_unet_tensor_layout(net, 1, 32, 32, 32, B.MODE_INFER, hi, B.T_IN))
+    p_ref = ops.softmax(ops.conv3d_fwd(z, ws[hi].astype(np.float64), bs[hi].astype(np.float64), 1, 1, 0)).reshape(V, 4)
+    assert_close(host_f64(probs), p_ref, "head probs", rel=1e-5, mx=1e-5)
+    agree, strict, near = tie_aware_agreement(seg.cpu().numpy(), p_ref)
     assert agree >= 0.9999, (agree, strict, near)
-    B.lamp_unet_destroy(net)
-
-
-def test_unet_train_step_tiny_matches_oracle():
-    net, spec, lay, ws, bs, wd, bd, offs = make_net(CFG0["levels"], CFG0["ch"], CFG0["cpl"], CFG0["K"], seed=1,
-                                                    bias_scale=0.0)
-    x, lab = _cfg0_inputs()
-    loss_ref, dW, dB, p_ref = O.train_step(spec, ws, bs, x.astype(np.float64), lab, quantise=True)
-    V = 32 ** 3
+    assert (seg.cpu().numpy() == np.argmax(host_f64(probs), -1)).all()
+    # inference and training forward passes give the same probabilities
     loss = torch.zeros((1,), dtype=torch.float32, device="cuda")
-    gw = torch.full((B.lamp_unet_weight_count(net),), float("nan"), dtype=torch.float32, device="cuda")
-    gb = torch.full((B.lamp_unet_bias_count(net),), float("nan"), dtype=torch.float32, device="cuda")
-    probs = torch.empty((V, 4), dtype=torch.float32, device="cuda")
-    wsb = torch.empty(B.lamp_unet_workspace_bytes(net, 1, 32, 32, 32, B.MODE_TRAIN), dtype=torch.uint8, device="cuda")
-    B.lamp_unet_train_step(net, wd, bd, dev_bf16(x), torch.from_numpy(lab).cuda(), loss, gw, gb, probs, wsb)
-    assert B.lamp_get_async_status() == 0
-    assert abs(float(loss.item()) - loss_ref) <= 1e-3 * abs(loss_ref)
-    assert_close(host_f64(probs), p_ref.reshape(V, 4), "train probs")
-    gw_h, gb_h = host_f64(gw), host_f64(gb)
-    gnorm = np.sqrt(sum((d ** 2).sum() for d in dW))
-    for i, l in enumerate(lay):
-        wo, bo = offs[i]
-        got = gw_h[wo:wo + dW[i].size].reshape(dW[i].shape)
-        assert_close(got, dW[i], f"grad_w {l.name}", rel=3e-3, mx=2e-2)
-        gotb = gb_h[bo:bo + l.c_out]
-        if l.kind in ("conv", "down"):
-            # InstanceNorm makes the preceding bias inert: both sides must give (numerically) zero
-            assert np.abs(gotb).max() <= 2e-2 * np.abs(dW[i]).max() * 27
-        else:
-            assert_close(gotb, dB[i], f"grad_b {l.name}", rel=3e-3, mx=2e-2)
-    assert gnorm > 0
+    gw = torch.empty((B.lamp_unet_weight_count(net),), dtype=torch.float32, device="cuda")
+    gb = torch.empty((B.lamp_unet_bias_count(net),), dtype=torch.float32, device="cuda")
+    p2 = torch.empty_like(probs)
+    wst = torch.empty(B.lamp_unet_workspace_bytes(net, 1, 32, 32, 32, B.MODE_TRAIN), dtype=torch.uint8, device="cuda")
+    lab = torch.zeros((V,), dtype=torch.uint8, device="cuda")
+    B.lamp_unet_train_step(net, wd, bd, dev_bf16(x), lab, loss, gw, gb, p2, wst)
+    assert torch.equal(p2, probs)
+    # end to end against the mirrored oracle, within the bf16 storage budget
+    ws64 = [a.astype(np.float64) for a in ws]
+    bs64 = [a.astype(np.float64) for a in bs]
+    p_q = O.forward(spec, ws64, bs64, x.astype(np.float64), quantise=True).reshape(V, 4)
+    p_f = O.forward(spec, ws64, bs64, x.astype(np.float64), quantise=False).reshape(V, 4)
+    budget = np.linalg.norm(p_q - p_f) / np.linalg.norm(p_f)
+    e2e = np.linalg.norm(host_f64(probs) - p_q) / np.linalg.norm(p_q)
+    assert e2e <= max(1e-3, 2 * budget), (e2e, budget)
     B.lamp_unet_destroy(net)
 
 
@@ -139,7 +261,9 @@ def test_unet_forward_batch_and_noncubic():
     probs = torch.empty((V, 3), dtype=torch.float32, device="cuda")
     wsb = torch.empty(B.lamp_unet_workspace_bytes(net, 2, 6, 8, 12, B.MODE_INFER), dtype=torch.uint8, device="cuda")
     B.lamp_unet_forward(net, wd, bd, dev_bf16(x), probs, None, wsb)
-    assert_close(host_f64(probs), ref.reshape(V, 3), "batched forward")
+    full = O.forward(spec, ws, bs, x.astype(np.float64), quantise=False)
+    budget = np.linalg.norm(ref - full) / np.linalg.norm(full)
+    assert_close(host_f64(probs), ref.reshape(V, 3), "batched forward", rel=max(1e-3, 2 * budget), mx=0.2)
     B.lamp_unet_destroy(net)
 
 
@@ -177,7 +301,11 @@ def test_sliding_window_matches_oracle_and_whole_patch_equals_forward():
     D, H, W, P = 12, 8, 10, (8, 8, 8)
     vol = synth.bf16_round(synth.ct_volume((D, H, W), 21))[None, ..., None]
     A, seg_ref, n_p = O.sliding_window(spec, ws, bs, vol.astype(np.float64), P, 0.25, gaussian=True, quantise=True)
+    A_full, _, _ = O.sliding_window(spec, ws, bs, vol.astype(np.float64), P, 0.25, gaussian=True, quantise=False)
+    budget = np.linalg.norm(A - A_full) / np.linalg.norm(A_full)
     assert n_p == 2 * 1 * 2
+    sd, sh, sw = (O.window_starts(n, p, 0.25) for n, p in zip((D, H, W), P))
+    origins = [(a, b, c) for a in sd for b in sh for c in sw]
     for sw_batch in (1, 3):
         planar = torch.empty((3, D, H, W), dtype=torch.float32, device="cuda")
         am = torch.empty((D * H * W,), dtype=torch.uint8, device="cuda")
@@ -185,9 +313,24 @@ def test_sliding_window_matches_oracle_and_whole_patch_equals_forward():
         wsb = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
         B.lamp_sliding_window_infer(net, wd, bd, dev_bf16(vol), P, 0.25, sw_batch, 1, planar, am, wsb)
         assert B.lamp_get_async_status() == 0
-        assert_close(host_f64(planar), A.transpose(3, 0, 1, 2), "sliding window probs")
-        agree, strict, near = tie_aware_agreement(am.cpu().numpy().reshape(D, H, W), A)
+        # step by step: (1) each patch's probabilities (kept at the start of the workspace) equal a
+        # plain forward pass on that patch cut out on the host, bit for bit
+        pp = wsb[:n_p * 512 * 3 * 4].view(torch.float32).reshape(n_p, 8, 8, 8, 3)
+        for i, (a, b, c) in enumerate(origins):
+            cut = np.ascontiguousarray(vol[:, a:a + 8, b:b + 8, c:c + 8, :])
+            pr = torch.empty((512, 3), dtype=torch.float32, device="cuda")
+            wsf = torch.empty(B.lamp_unet_workspace_bytes(net, 1, 8, 8, 8, B.MODE_INFER), dtype=torch.uint8, device="cuda")
+            B.lamp_unet_forward(net, wd, bd, dev_bf16(cut), pr, None, wsf)
+            assert torch.equal(pr.reshape(8, 8, 8, 3), pp[i])
+        # (2) the blend of exactly those probabilities equals the oracle's blend of them
+        pp_h = host_f64(pp)
+        A_loc, seg_loc, _ = O.sliding_window(spec, None, None, vol.astype(np.float64), P, 0.25, gaussian=True,
+                                             patch_probs=lambda i, pa: pp_h[i][None])
+        assert_close(host_f64(planar), A_loc.transpose(3, 0, 1, 2), "sliding window blend", rel=1e-5, mx=1e-5)
+        agree, strict, near = tie_aware_agreement(am.cpu().numpy().reshape(D, H, W), A_loc)
         assert agree >= 0.9999
+        # (3) end to end against the mirrored oracle, within the bf16 storage budget
+        assert_close(host_f64(planar), A.transpose(3, 0, 1, 2), "sliding window end to end", rel=max(1e-3, 2 * budget), mx=0.2)
     # patch = whole volume: identical to one forward pass
     probs = torch.empty((D * H * W, 3), dtype=torch.float32, device="cuda")
     wsf = torch.empty(B.lamp_unet_workspace_bytes(net, 1, D, H, W, B.MODE_INFER), dtype=torch.uint8, device="cuda")
