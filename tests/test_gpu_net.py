@@ -145,7 +145,9 @@ def check_network_layer_by_layer(levels, ch, cpl, K, dhw, seed, x, lab, tight=2e
             assert_close(dy_gpu, ops.bf16_round(ops.instnorm_relu_bwd(g, y_gpu, mu_g, rs_g)), what + " dy")
             dw_ref, db_ref = ops.conv3d_wgrad(x_in, dy_gpu, 3, s, 1)
             assert_close(dW, dw_ref, what + " dw", rel=tight, mx=tight)
-            assert_close(dB, db_ref, what + " db", rel=1e-4, mx=1e-4)
+            # dy sums to (nearly) zero per channel after InstanceNorm: the bias gradient is a
+            # cancellation, so its error is measured against sum |dy|
+            assert np.abs(dB - db_ref).max() <= 1e-5 * np.abs(dy_gpu).sum(axis=(0, 1, 2, 3)).max(), what + " db"
             if i > 0:
                 din = ws_read(wsb, lay_of(i, B.T_DIN))
                 assert_close(din, ops.bf16_round(ops.conv3d_dgrad(dy_gpu, w64, x_in.shape[1:4], 3, s, 1)), what + " din")
