@@ -1,0 +1,354 @@
+#!/usr/bin/env python
+"""Benchmark of the dense 3x3x3 conv3d passes (forward, data gradient, weight gradient).
+
+Workload: the single-layer sweep - NDHWC bf16, batch 1, 128x128x128 volume, 3x3x3 stride 1
+pad 1, C_in = C_out in {32, 64, 128, 256}, activations and upstream gradients N(0,1), Kaiming
+weights, seed 2.  One step = forward + dgrad + wgrad for every channel count.  The metric is
+dense FLOP/s: 2 * 27 * C^2 * voxels per pass (padded taps counted).
+
+    python bench.py --gpus 1 --steps 5 --warmup 3
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N   (independent replicas)
+    python bench.py --impl reference     (the CPU oracle on a bounded sample, same metric)
+
+Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+CHANNELS = (32, 64, 128, 256)
+VOL = (128, 128, 128)
+SEED = 2
+NOMINAL_BF16_TFLOPS = 2250.0
+
+
+def pass_flops(C, vol=VOL):
+    return 2.0 * 27 * C * C * vol[0] * vol[1] * vol[2]
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return dict(hbm_gbs=float(d["hbm_gbs"]), bf16=float(d["bf16_tflops"]),
+                        bf16_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+        except Exception:
+            pass
+    return dict(hbm_gbs=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# --------------------------------------------------------------------------------------------
+# CPU oracle legs (cpu_baseline of the GPU arm, and the whole of --impl reference)
+# --------------------------------------------------------------------------------------------
+ORACLE_SAMPLE = dict(C=64, slab=(16, 64, 64))
+
+
+def oracle_sample_once():
+    """fwd + dgrad + wgrad of the oracle on a slab of the workload.  Returns (seconds, flops)."""
+    from oracle import ops
+    from paper_2006_12575_b200 import synth
+    C = ORACLE_SAMPLE["C"]
+    D, H, W = ORACLE_SAMPLE["slab"]
+    x = synth.normal_bf16((1, D, H, W, C), SEED).astype(np.float64)
+    dy = synth.normal_bf16((1, D, H, W, C), SEED + 1).astype(np.float64)
+    w = synth.kaiming_bf16(27, C, C, 27 * C, SEED + 2).astype(np.float64)
+    t0 = time.perf_counter()
+    ops.conv3d_fwd(x, w, None, 3, 1, 1)
+    ops.conv3d_dgrad(dy, w, (D, H, W), 3, 1, 1)
+    ops.conv3d_wgrad(x, dy, 3, 1, 1)
+    return time.perf_counter() - t0, 3 * pass_flops(C, (D, H, W))
+
+
+def oracle_description():
+    from oracle import ops
+    D, H, W = ORACLE_SAMPLE["slab"]
+    return dict(kind="oracle", cores=ops.n_threads(), unit="TFLOP/s",
+                sample=f"fwd+dgrad+wgrad, C={ORACLE_SAMPLE['C']}, 1x{D}x{H}x{W} slab of the 128^3 volume, fp64 direct loops")
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import ops
+    ops.build()
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_once()
+    secs, flops = 0.0, 0.0
+    steps = max(1, min(args.steps, 3))
+    for _ in range(steps):
+        s, f = oracle_sample_once()
+        secs += s
+        flops += f
+    val = flops / secs / 1e12
+    desc = oracle_description()
+    desc["value"] = val
+    out = dict(impl="reference", metric="conv3d_tflops", value=val, unit="TFLOP/s", n_gpus=args.gpus, steps=steps,
+               warmup=min(args.warmup, 1), ms_per_step=1e3 * secs / steps, higher_is_better=True, scaling="weak",
+               vs_baseline=None, dtype="f64", data="synthetic",
+               config=dict(workload="conv3d sweep 128^3, C=32/64/128/256, fwd+dgrad+wgrad (bounded sample per step)"),
+               cpu_baseline=desc, e2e=dict(value=val, unit="TFLOP/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(out), flush=True)
+
+
+# --------------------------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        self.path = f"/tmp/lamp_bench_clocks_{os.getpid()}.csv"
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        res = dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
+        if not self.proc:
+            return res
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        try:
+            os.remove(self.path)
+        except OSError:
+            pass
+        if sm:
+            res = dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return res
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2006_12575_b200 import binding as B
+    from paper_2006_12575_b200 import build as lamp_build
+    from paper_2006_12575_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        lamp_build.build()
+    if world > 1:
+        dist.barrier()
+    B.lib()
+    chans = tuple(int(c) for c in args.channels.split(","))
+    D, H, W = VOL
+    dev = torch.device("cuda", local)
+
+    # host (pinned) copies of every input, device buffers for inputs and outputs
+    host, devb = {}, {}
+    for C in chans:
+        g = torch.Generator().manual_seed(SEED * 1000 + C + 7919 * rank)
+        hx = torch.randn((1, D, H, W, C), generator=g, dtype=torch.float32).to(torch.bfloat16).pin_memory()
+        hdy = torch.randn((1, D, H, W, C), generator=g, dtype=torch.float32).to(torch.bfloat16).pin_memory()
+        hw = torch.from_numpy(synth.kaiming_bf16(27, C, C, 27 * C, SEED * 1000 + C)).to(torch.bfloat16).pin_memory()
+        host[C] = (hx, hdy, hw)
+        desc = B.conv_desc(C, C)
+        x = hx.to(dev)
+        wsz = max(B.lamp_conv3d_workspace_bytes(desc, x, B.PASS_DGRAD), B.lamp_conv3d_workspace_bytes(desc, x, B.PASS_WGRAD), 256)
+        devb[C] = dict(desc=desc, x=x, dy=hdy.to(dev), w=hw.to(dev), y=torch.empty_like(x), dx=torch.empty_like(x),
+                       dw=torch.empty((27, C, C), dtype=torch.float32, device=dev),
+                       ws=torch.empty(wsz, dtype=torch.uint8, device=dev))
+    hout = {C: (torch.empty((1, D, H, W, C), dtype=torch.bfloat16).pin_memory(),
+                torch.empty((1, D, H, W, C), dtype=torch.bfloat16).pin_memory(),
+                torch.empty((27, C, C), dtype=torch.float32).pin_memory()) for C in chans}
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    pass_events = []
+
+    def step(record):
+        for C in chans:
+            b = devb[C]
+            marks = [ev() for _ in range(4)] if record else None
+            if record:
+                marks[0].record()
+            B.lamp_conv3d_fwd(b["desc"], b["x"], b["w"], None, b["y"])
+            if record:
+                marks[1].record()
+            B.lamp_conv3d_dgrad(b["desc"], b["dy"], b["w"], b["dx"], b["ws"])
+            if record:
+                marks[2].record()
+            B.lamp_conv3d_wgrad(b["desc"], b["x"], b["dy"], b["dw"], None, b["ws"])
+            if record:
+                marks[3].record()
+                pass_events.append((C, marks))
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step(False)
+    sync_all()
+    sampler = ClockSampler(local) if rank == 0 else None
+    t0, t1 = ev(), ev()
+    t0.record()
+    for _ in range(args.steps):
+        step(True)
+    t1.record()
+    sync_all()
+    ms = t0.elapsed_time(t1)
+    clocks = sampler.stop() if sampler else None
+    status = B.lamp_get_async_status()
+    if status != 0:
+        raise SystemExit(f"bench.py: device status {status}")
+
+    # end to end through the same calls with host buffers: H2D of x, dy, w and D2H of y, dx, dw every step
+    def e2e_step():
+        for C in chans:
+            b = devb[C]
+            hx, hdy, hw = host[C]
+            b["x"].copy_(hx, non_blocking=True)
+            b["dy"].copy_(hdy, non_blocking=True)
+            b["w"].copy_(hw, non_blocking=True)
+            B.lamp_conv3d_fwd(b["desc"], b["x"], b["w"], None, b["y"])
+            B.lamp_conv3d_dgrad(b["desc"], b["dy"], b["w"], b["dx"], b["ws"])
+            B.lamp_conv3d_wgrad(b["desc"], b["x"], b["dy"], b["dw"], None, b["ws"])
+            hout[C][0].copy_(b["y"], non_blocking=True)
+            hout[C][1].copy_(b["dx"], non_blocking=True)
+            hout[C][2].copy_(b["dw"], non_blocking=True)
+
+    e2e_step()
+    sync_all()
+    e0, e1 = ev(), ev()
+    e2e_steps = max(1, min(args.steps, 3))
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    sync_all()
+    e2e_ms = e0.elapsed_time(e1)
+
+    if world > 1:
+        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+
+    flops_step = sum(3 * pass_flops(C) for C in chans)
+    value = world * flops_step * args.steps / (ms * 1e-3) / 1e12
+    e2e_val = world * flops_step * e2e_steps / (e2e_ms * 1e-3) / 1e12
+    h2d = sum(2 * D * H * W * C * 2 + 27 * C * C * 2 for C in chans)
+    d2h = sum(2 * D * H * W * C * 2 + 27 * C * C * 4 for C in chans)
+
+    # per-pass times (this rank), and the roofline of the kernel with the largest share
+    per = {}
+    for C, m in pass_events:
+        for name, a, b_ in (("fwd", m[0], m[1]), ("dgrad", m[1], m[2]), ("wgrad", m[2], m[3])):
+            per.setdefault((C, name), []).append(a.elapsed_time(b_))
+    peaks = measured_peaks()
+    passes = {}
+    for (C, name), v in per.items():
+        mean = sum(v) / len(v)
+        tf = pass_flops(C) / (mean * 1e-3) / 1e12
+        passes[f"C{C}.{name}"] = dict(ms=round(mean, 4), tflops=round(tf, 1), pct_nominal=round(100 * tf / NOMINAL_BF16_TFLOPS, 1),
+                                      pct_measured=round(100 * tf / peaks["bf16"], 1))
+    # kernel families: tcgen05 implicit GEMM (fwd + dgrad) and the wgrad kernel
+    fam = {"conv3_umma_kernel (fwd+dgrad)": [k for k in per if k[1] in ("fwd", "dgrad")],
+           "conv_wgrad_kernel (wgrad)": [k for k in per if k[1] == "wgrad"]}
+    fam_time = {f: sum(sum(per[k]) for k in ks) for f, ks in fam.items()}
+    dom = max(fam_time, key=fam_time.get)
+    dom_flops = sum(pass_flops(k[0]) * len(per[k]) for k in fam[dom])
+    dom_launches = sum(len(per[k]) for k in fam[dom])
+    achieved = dom_flops / (fam_time[dom] * 1e-3) / 1e12
+    roofline = dict(bound="tensor", kernel=dom, achieved=round(achieved, 2), peak=peaks["bf16"], unit="TFLOP/s",
+                    frac=round(achieved / peaks["bf16"], 4), traffic=None, peak_source=peaks["source"] + " bf16 burst",
+                    avg_launch_ms=round(fam_time[dom] / dom_launches, 4), share_of_step=round(fam_time[dom] / sum(fam_time.values()), 3))
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu = oracle_description()
+    try:
+        from oracle import ops
+        ops.build()
+        secs, fl = oracle_sample_once()
+        cpu["value"] = fl / secs / 1e12
+        cpu["seconds"] = round(secs, 2)
+    except Exception as e:       # the baseline leg must not take the GPU numbers down with it
+        cpu["value"] = None
+        cpu["error"] = str(e)[:200]
+
+    launches_per_C = 1 + 2 + 4     # fwd; dgrad = weight transpose + conv; wgrad = partials + reduce (+ none for bias)
+    out = dict(metric="conv3d_tflops", value=round(value, 3), unit="TFLOP/s", n_gpus=world, steps=args.steps,
+               warmup=args.warmup, ms_per_step=round(ms / args.steps, 4), higher_is_better=True, scaling="weak",
+               vs_baseline=None, dtype="bf16", data="synthetic",
+               config=dict(workload="configs[1]: conv3d 3x3x3 s1 p1 sweep, NDHWC bf16, 1x128x128x128, C_in=C_out in "
+                                    + "/".join(str(c) for c in chans) + ", fwd+dgrad+wgrad per C",
+                           l2="inputs larger than L2: a step streams several GB through distinct buffers",
+                           flops_convention="2*27*C^2*voxels per pass", replicas=world),
+               clocks=clocks,
+               e2e=dict(value=round(e2e_val, 3), unit="TFLOP/s", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                        steps=e2e_steps),
+               gpu_launches=args.steps * len(chans) * launches_per_C,
+               roofline=roofline, cpu_baseline=cpu, passes=passes,
+               pct_of_nominal_bf16=round(100 * value / world / NOMINAL_BF16_TFLOPS, 2))
+    print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="lamp", choices=["lamp", "reference"])
+    ap.add_argument("--channels", default=",".join(str(c) for c in CHANNELS))
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

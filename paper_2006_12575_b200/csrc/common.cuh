@@ -91,6 +91,17 @@ size_t        simt_conv_wgrad_ws(const ConvGeom &g);
 lamp_status_t simt_conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, float *db,
                               void *ws, size_t ws_bytes, cudaStream_t st);
 
+// out[e] = sum_s part[s][e] in a fixed order; dbias[co] = sum_v dy[v][co] (ws: bias_grad_ws bytes)
+lamp_status_t reduce_partials(const float *part, int64_t entries, int splits, float *out, cudaStream_t st);
+size_t        bias_grad_ws(int64_t voxels, int co);
+lamp_status_t bias_grad(const TView &dy, float *db, void *ws, cudaStream_t st);
+
+// wgrad_umma.cu (tcgen05 weight gradient)
+bool          umma_wgrad_supported(const ConvGeom &g, const TView &x, const TView &dy);
+size_t        umma_wgrad_ws(const ConvGeom &g);
+lamp_status_t umma_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, void *ws, size_t ws_bytes,
+                         cudaStream_t st);
+
 // conv_umma.cu (tcgen05 implicit GEMM)
 bool          umma_conv_fwd_supported(const ConvGeom &g, const TView &x, const TView &y);
 lamp_status_t umma_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,

@@ -269,6 +269,39 @@ lamp_status_t simt_conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w,
     return launch_status();
 }
 
+lamp_status_t reduce_partials(const float *part, int64_t entries, int splits, float *out, cudaStream_t st)
+{
+    if (entries == 0) return LAMP_OK;
+    reduce_parts_kernel<<<(unsigned)((entries + 255) / 256), 256, 0, st>>>(part, entries, splits, out);
+    return launch_status();
+}
+
+static void bias_plan(int64_t V, int *blocks, int64_t *vpb)
+{
+    int b = (int)(((V + 255) / 256) < 1024 ? ((V + 255) / 256) : 1024);
+    if (b < 1) b = 1;
+    *blocks = b;
+    *vpb = (V + b - 1) / b;
+}
+
+size_t bias_grad_ws(int64_t voxels, int co)
+{
+    int b; int64_t vpb;
+    bias_plan(voxels, &b, &vpb);
+    return align_up((size_t)b * co * 4, 256);
+}
+
+lamp_status_t bias_grad(const TView &dy, float *db, void *ws, cudaStream_t st)
+{
+    const int64_t V = (int64_t)dy.n * dy.d * dy.h * dy.w;
+    if (V == 0) { LAMP_CUDA_OK(cudaMemsetAsync(db, 0, (size_t)dy.c * 4, st)); return LAMP_OK; }
+    int b; int64_t vpb;
+    bias_plan(V, &b, &vpb);
+    colsum_kernel<<<b, 256, 0, st>>>((const bf16 *)dy.p, dy.pitch, dy.c, V, vpb, (float *)ws);
+    reduce_parts_kernel<<<(dy.c + 255) / 256, 256, 0, st>>>((const float *)ws, dy.c, b, db);
+    return launch_status();
+}
+
 size_t simt_conv_wgrad_ws(const ConvGeom &g)
 {
     const WgradPlan p = wgrad_plan(g);
