@@ -50,7 +50,8 @@ typedef enum {
     LAMP_ERR_WORKSPACE = 3,       /* workspace missing, misaligned or smaller than required      */
     LAMP_ERR_CUDA = 4,            /* a CUDA runtime / driver call failed                         */
     LAMP_ERR_TIMEOUT = 5,         /* a bounded device-side wait ran out (see async status)       */
-    LAMP_ERR_NOT_IMPLEMENTED = 6
+    LAMP_ERR_NOT_IMPLEMENTED = 6,
+    LAMP_ERR_SCRATCH_LIMIT = 7    /* the problem needs more than the built-in static scratch     */
 } lamp_status_t;
 
 typedef enum { LAMP_BF16 = 0, LAMP_F32 = 1 } lamp_dtype_t;
@@ -100,6 +101,29 @@ lamp_status_t lamp_conv3d_fwd(const lamp_conv_desc_t *desc, const lamp_tensor_t 
  * its extents are the conv's input extents. */
 lamp_status_t lamp_conv3d_dgrad(const lamp_conv_desc_t *desc, const lamp_tensor_t *dy, const void *w,
                                 lamp_tensor_t *dx, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* The same data gradient for callers that cannot allocate device memory when they call - e.g. a
+ * layer running inside an engine that handed out all device memory at start-up, or a latency-
+ * critical loop where cudaMalloc (it synchronises the device and can fail under memory pressure)
+ * is ruled out - and so have no workspace to pass.  (The paper has no counterpart of this call:
+ * it is a packaging variant of lamp_conv3d_dgrad, with identical arithmetic and results.)
+ * The scratch this pass needs, a transposed copy of the weights, sits in a fixed array of
+ * LAMP_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads the library holds it
+ * until the process exits.  The call itself allocates and frees nothing.
+ *  - Limit: lamp_conv3d_workspace_bytes(desc, dx, LAMP_PASS_DGRAD) must not exceed
+ *    LAMP_STATIC_SCRATCH_BYTES (27 * c_in * c_out * 2 bytes for the 3x3x3 s1 p1 conv, i.e. up to
+ *    c_in * c_out = 77672, e.g. 256 x 256); otherwise LAMP_ERR_SCRATCH_LIMIT is returned and
+ *    nothing is launched.  Variants that need no scratch are accepted at any size.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current) and keeps it; make that first call before starting any stream capture.
+ *  - All calls on a device share the one array, which keeps whatever the last call left in it.
+ *    Nothing in it has to be zero beforehand (each call overwrites the part it reads), but two
+ *    calls that overlap in time on the same GPU - different streams or threads - race on it:
+ *    issue them on one stream, or order them yourself.
+ * Arguments and errors are otherwise those of lamp_conv3d_dgrad. */
+#define LAMP_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+lamp_status_t lamp_conv3d_dgrad_static_scratch(const lamp_conv_desc_t *desc, const lamp_tensor_t *dy, const void *w,
+                                               lamp_tensor_t *dx, void *cuda_stream);
 
 /* dw[tap][c_out][c_in] (fp32) = gradient with respect to w; dbias[c_out] (fp32, may be NULL)
  * = sum of dy over voxels.  x, dy bf16.  Both outputs are overwritten. */

@@ -58,6 +58,7 @@ def lib():
             "lamp_conv3d_workspace_bytes": (sz, [DP, TP, C.c_int]),
             "lamp_conv3d_fwd": (C.c_int, [DP, TP, vp, vp, TP, vp, vp, sz, vp]),
             "lamp_conv3d_dgrad": (C.c_int, [DP, TP, vp, TP, vp, sz, vp]),
+            "lamp_conv3d_dgrad_static_scratch": (C.c_int, [DP, TP, vp, TP, vp]),
             "lamp_conv3d_wgrad": (C.c_int, [DP, TP, TP, vp, vp, vp, sz, vp]),
             "lamp_instnorm_relu_fwd": (C.c_int, [TP, vp, f32, vp, TP, vp]),
             "lamp_instnorm_relu_bwd": (C.c_int, [TP, TP, TP, vp, vp, TP, vp]),
@@ -86,7 +87,8 @@ def lib():
     return _lib
 
 
-EXPORTS = ["lamp_conv3d_workspace_bytes", "lamp_conv3d_fwd", "lamp_conv3d_dgrad", "lamp_conv3d_wgrad",
+EXPORTS = ["lamp_conv3d_workspace_bytes", "lamp_conv3d_fwd", "lamp_conv3d_dgrad", "lamp_conv3d_dgrad_static_scratch",
+           "lamp_conv3d_wgrad",
            "lamp_instnorm_relu_fwd", "lamp_instnorm_relu_bwd", "lamp_unet_create", "lamp_unet_destroy",
            "lamp_unet_num_layers", "lamp_unet_weight_count", "lamp_unet_bias_count", "lamp_unet_param_layout",
            "lamp_unet_workspace_bytes", "lamp_unet_tensor_layout", "lamp_unet_forward", "lamp_unet_train_step",
@@ -141,6 +143,17 @@ def lamp_conv3d_dgrad(desc, dy, w, dx, ws=None):
     p, nbytes = _ws(ws)
     _check(lib().lamp_conv3d_dgrad(C.byref(desc), C.byref(_td(dy)), _ptr(w), C.byref(_td(dx)), p, nbytes, _stream()),
            "lamp_conv3d_dgrad")
+
+
+STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
+
+
+def lamp_conv3d_dgrad_static_scratch(desc, dy, w, dx):
+    """lamp_conv3d_dgrad without a caller workspace: the scratch is a fixed array inside the library
+    (for callers that cannot allocate device memory at call time).  Raises LampError with status 7
+    when the layer needs more than STATIC_SCRATCH_BYTES."""
+    _check(lib().lamp_conv3d_dgrad_static_scratch(C.byref(desc), C.byref(_td(dy)), _ptr(w), C.byref(_td(dx)), _stream()),
+           "lamp_conv3d_dgrad_static_scratch")
 
 
 def lamp_conv3d_wgrad(desc, x, dy, dw, dbias=None, ws=None):

@@ -227,6 +227,7 @@ const char *lamp_status_string(lamp_status_t s)
     case LAMP_ERR_CUDA: return "CUDA call failed";
     case LAMP_ERR_TIMEOUT: return "device-side wait timed out";
     case LAMP_ERR_NOT_IMPLEMENTED: return "not implemented";
+    case LAMP_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the library's built-in static array";
     }
     return "unknown status";
 }
