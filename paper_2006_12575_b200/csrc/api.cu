@@ -87,6 +87,7 @@ size_t conv_ws_bytes(const ConvGeom &g, int pass)
 lamp_status_t conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
                        double *stats, cudaStream_t st)
 {
+    if (ct_conv_fwd_supported(g, x, y)) return ct_conv_fwd(g, x, w, bias, y, stats, 0, st);
     if (umma_conv_fwd_supported(g, x, y)) return umma_conv_fwd(g, x, w, bias, y, stats, 0, st);
     return simt_conv_fwd(g, x, w, bias, y, stats, st);
 }
@@ -102,6 +103,7 @@ lamp_status_t conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w, cons
             if (!ws || ws_bytes < need || !aligned16(ws)) return LAMP_ERR_WORKSPACE;
             lamp_status_t s = umma_transpose_weights(w, (bf16 *)ws, 27, g.co, g.ci, st);
             if (s != LAMP_OK) return s;
+            if (ct_conv_fwd_supported(t, dy, dx)) return ct_conv_fwd(t, dy, (const bf16 *)ws, nullptr, dx, nullptr, 1, st);
             return umma_conv_fwd(t, dy, (const bf16 *)ws, nullptr, dx, nullptr, 1, st);
         }
     }

@@ -109,6 +109,11 @@ lamp_status_t umma_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, co
 size_t        umma_dgrad_ws(const ConvGeom &g);
 lamp_status_t umma_transpose_weights(const bf16 *w, bf16 *wt, int taps, int co, int ci, cudaStream_t st);
 
+// conv_t.cu (tcgen05 "weights x voxels" implicit GEMM over shared-memory-resident planes, c_out <= 128)
+bool          ct_conv_fwd_supported(const ConvGeom &g, const TView &x, const TView &y);
+lamp_status_t ct_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
+                          double *stats, int mirror_taps, cudaStream_t st);
+
 // elementwise.cu
 lamp_status_t k_finalize_stats(const double *stats, float *mu_rstd, int64_t nc, double inv_v, float eps, cudaStream_t st);
 lamp_status_t k_instnorm_relu_fwd(const TView &y, const float *mu_rstd, const TView &z, cudaStream_t st);

@@ -1,0 +1,432 @@
+// 3x3x3 stride-1 pad-1 convolution for c_out blocks of at most 128 channels: "weights x voxels"
+// implicit GEMM with the activation planes resident in shared memory.
+//
+// Why this shape.  One tcgen05.mma (M = 128, K = 16, bf16) occupies the tensor pipe for max(76, N/2)
+// cycles (measured): only N = 256 reaches the full rate.  With output channels on N, a 64-channel layer
+// would run at 42 % of it.  So here the OUTPUT CHANNELS are the M rows (A operand = weight tile
+// [128 x 64], K-major) and 256 OUTPUT VOXELS are the N columns (B operand = an 8 (w) x 32 (h) window of
+// an activation plane, K-major): D^T[co, voxel] += W[co, ci] * X[voxel + tap, ci].
+//
+//  * Activation planes.  For (input plane p, 64-channel chunk) one TMA load brings a halo box of
+//    34 x 10 voxels (out-of-volume voxels zero-filled = the conv's zero padding) with 128-byte swizzled
+//    rows.  The nine in-plane taps are shifted windows of that box: the shared-memory descriptor starts
+//    (kh*10 + kw) rows in and steps 10 rows between 8-voxel groups.  The swizzle is a function of the
+//    shared-memory address bits, so such a window reads exactly what TMA wrote.
+//  * Narrow layers.  With c_out = 64 (32) the 128 rows hold the weights of 2 (4) CONSECUTIVE OUTPUT
+//    PLANES: input plane p is tap kd = p - o + 1 of output plane o, so row block j carries the weights
+//    of tap (kd = p - (o0 + j) + 1, kh, kw); where that kd falls outside 0..2 the TMA coordinate is out
+//    of range and the block is zero-filled.  2 planes cost 4 input planes of MMAs instead of 2 x 3 at
+//    half-empty M: 75 % (50 % for c_out = 32) of the full rate instead of 50 % (25 %).
+//  * Accumulators: 128 lanes x 256 fp32 columns, two of them in TMEM, so the epilogue of one tile
+//    overlaps the MMAs of the next.  The epilogue owns one output channel per thread: bias and the
+//    InstanceNorm sums are per-thread scalars; a 32 x 32 shared-memory transpose per warp turns
+//    TMEM rows into 64-byte (bf16) or 128-byte (fp32) channel runs per voxel for the NDHWC store.
+//
+// Warps: 0 = activation-plane TMA producer, 1 = MMA issuer (+ TMEM owner), 2 = weight-tile TMA
+// producer, 3..6 = epilogue.  All waits are bounded (LAMP_ERR_TIMEOUT on expiry).
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include "common.cuh"
+#include "umma_ptx.cuh"
+
+namespace lamp {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int CT_THREADS = 224;
+constexpr int TW = 8, TH = 32;          // output window: 8 (w) x 32 (h) = 256 voxels = N
+constexpr int HALO_W = TW + 2, HALO_H = TH + 2;
+constexpr int MAX_NP = 4, MAX_NW = 8;
+
+struct CtParams {
+    int32_t N, D, H, W;
+    int32_t nwt, nht, ngr, nct;         // tiles along w, h; plane groups; c_out blocks of 128
+    int32_t chunks;                     // c_in / KC
+    int32_t total_items;
+    int32_t co, mirror, y_f32;
+    int32_t np, nw;                     // ring depths: activation planes, weight tiles
+    int32_t plane_bytes;                // 1024-aligned bytes of one plane box
+    int64_t y_pitch;
+    void   *y;
+    const float *bias;
+    double *stats;
+    int    *status;
+};
+
+struct Item { int n, o0, h0, w0, ct; };
+
+template <int S>
+__device__ __forceinline__ Item decode_item(const CtParams &P, int item)
+{
+    Item it;
+    it.ct = item % P.nct; item /= P.nct;
+    it.w0 = (item % P.nwt) * TW; item /= P.nwt;
+    it.h0 = (item % P.nht) * TH; item /= P.nht;
+    it.o0 = (item % P.ngr) * S;
+    it.n = item / P.ngr;
+    return it;
+}
+
+// KC: channels per chunk (64: 128-byte swizzle, 32: 64-byte swizzle).  COB: output channels per plane
+// inside the 128 rows (128, 64 or 32); S = 128 / COB output planes are stacked.
+template <int KC, int COB>
+__global__ void __launch_bounds__(CT_THREADS, 1)
+conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const CtParams P)
+{
+    constexpr int S = 128 / COB;
+    constexpr int ROWB = KC * 2;
+    constexpr uint32_t SWZ = KC == 64 ? 2u : 4u;
+    constexpr uint32_t PLANE_BOX_BYTES = HALO_W * HALO_H * ROWB;
+    constexpr uint32_t W_BYTES = 128 * ROWB;
+    constexpr uint32_t IDESC = make_idesc(256);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *p_base = smem;
+    uint8_t *w_base = p_base + (size_t)P.np * P.plane_bytes;
+    float *epi = (float *)(w_base + (size_t)P.nw * W_BYTES);
+    uint64_t *bars = (uint64_t *)((uint8_t *)epi + 4 * 32 * 33 * 4);
+    const uint32_t pfull0 = smem_u32(bars), pempty0 = smem_u32(bars + MAX_NP);
+    const uint32_t wfull0 = smem_u32(bars + 2 * MAX_NP), wempty0 = smem_u32(bars + 2 * MAX_NP + MAX_NW);
+    const uint32_t tfull0 = smem_u32(bars + 2 * MAX_NP + 2 * MAX_NW), tempty0 = tfull0 + 16;
+    uint32_t *tmem_slot = (uint32_t *)(bars + 2 * MAX_NP + 2 * MAX_NW + 4);
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MAX_NP; ++s) { mbar_init(pfull0 + 8 * s, 1); mbar_init(pempty0 + 8 * s, 1); }
+        for (int s = 0; s < MAX_NW; ++s) { mbar_init(wfull0 + 8 * s, 1); mbar_init(wempty0 + 8 * s, 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 4); }
+        *abort_flag = 0;
+        mbar_init_fence();
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---------------------------------------------------------------- activation planes
+            int ps = 0;
+            uint32_t pph = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
+                const Item it = decode_item<S>(P, item);
+                for (int pi = 0; pi < S + 2 && ok; ++pi) {
+                    const int p = it.o0 - 1 + pi;
+                    if (p < 0 || p >= P.D) continue;
+                    for (int c = 0; c < P.chunks; ++c) {
+                        if (!mbar_wait(pempty0 + 8 * ps, pph ^ 1, abort_flag)) { ok = false; break; }
+                        mbar_expect_tx(pfull0 + 8 * ps, PLANE_BOX_BYTES);
+                        tma_load_5d(smem_u32(p_base + (size_t)ps * P.plane_bytes), &map_x, pfull0 + 8 * ps, c * KC, it.w0 - 1,
+                                    it.h0 - 1, p, it.n);
+                        if (++ps == P.np) { ps = 0; pph ^= 1; }
+                    }
+                }
+            }
+        }
+    } else if (warp == 2) {
+        if (lane == 0) {
+            // ---------------------------------------------------------------- weight tiles
+            int ws = 0;
+            uint32_t wph = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
+                const Item it = decode_item<S>(P, item);
+                for (int pi = 0; pi < S + 2 && ok; ++pi) {
+                    const int p = it.o0 - 1 + pi;
+                    if (p < 0 || p >= P.D) continue;
+                    for (int c = 0; c < P.chunks && ok; ++c) {
+                        for (int t9 = 0; t9 < 9; ++t9) {
+                            if (!mbar_wait(wempty0 + 8 * ws, wph ^ 1, abort_flag)) { ok = false; break; }
+                            mbar_expect_tx(wfull0 + 8 * ws, W_BYTES);
+                            const uint32_t dst = smem_u32(w_base + (size_t)ws * W_BYTES);
+#pragma unroll
+                            for (int j = 0; j < S; ++j) {
+                                const int kd = pi - j;                      // tap of output plane o0 + j fed by input plane p
+                                int tap = kd * 9 + t9;
+                                if (kd < 0 || kd > 2) tap = 27;             // out of range: TMA fills the block with zeros
+                                else if (P.mirror) tap = 26 - tap;
+                                tma_load_3d(dst + j * COB * ROWB, &map_w, wfull0 + 8 * ws, c * KC, it.ct * 128, tap);
+                            }
+                            if (++ws == P.nw) { ws = 0; wph ^= 1; }
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---------------------------------------------------------------- MMA issuer
+            int ps = 0, ws = 0;
+            uint32_t pph = 0, wph = 0, acc = 0, acc_phase = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
+                const Item it = decode_item<S>(P, item);
+                if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * 256;
+                uint32_t accumulate = 0;
+                for (int pi = 0; pi < S + 2 && ok; ++pi) {
+                    const int p = it.o0 - 1 + pi;
+                    if (p < 0 || p >= P.D) continue;
+                    for (int c = 0; c < P.chunks && ok; ++c) {
+                        if (!mbar_wait(pfull0 + 8 * ps, pph, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t plane = smem_u32(p_base + (size_t)ps * P.plane_bytes);
+                        for (int t9 = 0; t9 < 9; ++t9) {
+                            const int kh = t9 / 3, kw = t9 - kh * 3;
+                            if (!mbar_wait(wfull0 + 8 * ws, wph, abort_flag)) { ok = false; break; }
+                            tc_fence_after();
+                            const uint64_t da = make_desc(smem_u32(w_base + (size_t)ws * W_BYTES), 0, 8 * ROWB, SWZ);
+                            const uint64_t db = make_desc(plane + (kh * HALO_W + kw) * ROWB, 0, HALO_W * ROWB, SWZ);
+#pragma unroll
+                            for (int k = 0; k < KC / 16; ++k) {
+                                umma_bf16(d_tmem, da + 2 * k, db + 2 * k, IDESC, accumulate);
+                                accumulate = 1;
+                            }
+                            umma_commit(wempty0 + 8 * ws);
+                            if (++ws == P.nw) { ws = 0; wph ^= 1; }
+                        }
+                        if (!ok) break;
+                        umma_commit(pempty0 + 8 * ps);
+                        if (++ps == P.np) { ps = 0; pph ^= 1; }
+                    }
+                }
+                if (!ok) break;
+                umma_commit(tfull0 + 8 * acc);
+                acc ^= 1;
+                if (acc == 0) acc_phase ^= 1;
+            }
+        }
+    } else {
+        // -------------------------------------------------------------------- epilogue (warps 3..6)
+        const int q = warp & 3;                                 // TMEM lane quarter of this warp
+        float *tr = epi + (warp - 3) * 32 * 33;
+        const int jplane = (q * 32) / COB;                      // which stacked output plane these 32 lanes belong to
+        const int co_in_blk = (q * 32) % COB;                   // first of this warp's 32 channels inside the block
+        uint32_t acc = 0, acc_phase = 0;
+        float s1 = 0.f, s2 = 0.f;                               // sums of this thread's channel
+        int stat_n = -1, stat_ct = 0;
+        bool ok = true;
+        auto flush = [&]() {
+            if (P.stats && stat_n >= 0) {
+                double *dst = P.stats + ((int64_t)stat_n * P.co + stat_ct * 128 + co_in_blk + lane) * 2;
+                atomicAdd(dst, (double)s1);
+                atomicAdd(dst + 1, (double)s2);
+            }
+            s1 = 0.f; s2 = 0.f;
+        };
+        for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
+            const Item it = decode_item<S>(P, item);
+            if (it.n != stat_n || it.ct != stat_ct) { flush(); stat_n = it.n; stat_ct = it.ct; }
+            const int o = it.o0 + jplane;
+            const bool plane_ok = o < P.D;
+            const int cbase = it.ct * 128 + co_in_blk;          // first of this warp's channels in the tensor
+            const float bias = P.bias ? __ldg(P.bias + cbase + lane) : 0.f;
+            ok = __all_sync(0xffffffffu, mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256;
+#pragma unroll 1
+            for (int c0 = 0; c0 < 256; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(trow + c0, r);
+                tmem_ld_wait();
+                if (plane_ok) {
+                    // r[j] = channel (cbase + lane) at voxel column c0 + j: column = hl * 8 + wx
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int col = c0 + j;
+                        const bool valid = (it.w0 + (col & 7) < P.W) && (it.h0 + (col >> 3) < P.H);
+                        const float f = valid ? __uint_as_float(r[j]) + bias : 0.f;
+                        s1 += f;
+                        s2 = fmaf(f, f, s2);
+                        tr[j * 33 + lane] = f;
+                    }
+                    __syncwarp();
+                    // this lane now stores voxel column c0 + lane: 32 consecutive channels
+                    const int col = c0 + lane;
+                    const int w = it.w0 + (col & 7), h = it.h0 + (col >> 3);
+                    if (w < P.W && h < P.H) {
+                        const int64_t vox = (((int64_t)it.n * P.D + o) * P.H + h) * P.W + w;
+                        if (P.y_f32) {
+                            float4 *dst = reinterpret_cast<float4 *>((float *)P.y + vox * P.y_pitch + cbase);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                dst[e] = make_float4(tr[lane * 33 + 4 * e], tr[lane * 33 + 4 * e + 1], tr[lane * 33 + 4 * e + 2],
+                                                     tr[lane * 33 + 4 * e + 3]);
+                        } else {
+                            uint4 *dst = reinterpret_cast<uint4 *>((bf16 *)P.y + vox * P.y_pitch + cbase);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                float f8[8];
+#pragma unroll
+                                for (int u = 0; u < 8; ++u) f8[u] = tr[lane * 33 + 8 * e + u];
+                                dst[e] = pack8(f8);
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+            acc ^= 1;
+            if (acc == 0) acc_phase ^= 1;
+        }
+        flush();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0 && P.status) atomicExch(P.status, (int)LAMP_ERR_TIMEOUT);
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) { }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 get_encode()
+{
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (PFN_cuTensorMapEncodeTiled_v12000)p;
+    }
+    return fn;
+}
+
+struct CtPlan { CtParams P; int KC, COB; size_t smem; int grid; };
+
+constexpr int EPI_BYTES = 4 * 32 * 33 * 4;
+constexpr int CTRL_BYTES = 1024;
+constexpr int SMEM_LIMIT = 227 * 1024;
+
+bool make_ct_plan(const ConvGeom &g, CtPlan *out)
+{
+    if (!(g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed)) return false;
+    if (g.ci % 32) return false;
+    int COB;
+    if (g.co == 32 || g.co == 64) COB = g.co;
+    else if (g.co % 128 == 0) COB = 128;
+    else return false;
+    const int KC = g.ci % 64 == 0 ? 64 : 32;
+    const int S = 128 / COB;
+    CtParams &P = out->P;
+    P.N = g.n; P.D = g.d; P.H = g.h; P.W = g.w;
+    P.chunks = g.ci / KC;
+    const int rowb = KC * 2;
+    P.plane_bytes = (int)align_up((size_t)HALO_W * HALO_H * rowb, 1024);
+    const int w_bytes = 128 * rowb;
+    const int budget = SMEM_LIMIT - 1024 - EPI_BYTES - CTRL_BYTES;
+    int np = KC == 64 ? 3 : 4;
+    int nw = (budget - np * P.plane_bytes) / w_bytes;
+    if (nw > MAX_NW) nw = MAX_NW;
+    if (nw < 3) return false;
+    P.np = np; P.nw = nw;
+    P.nwt = (g.w + TW - 1) / TW;
+    P.nht = (g.h + TH - 1) / TH;
+    P.ngr = (g.d + S - 1) / S;
+    P.nct = g.co / (COB == 128 ? 128 : COB);
+    const int64_t items = (int64_t)g.n * P.ngr * P.nht * P.nwt * P.nct;
+    if (items > 0x7FFFFFFF || items <= 0) return false;
+    P.total_items = (int32_t)items;
+    P.co = g.co;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    out->KC = KC; out->COB = COB;
+    out->smem = 1024 + (size_t)np * P.plane_bytes + (size_t)nw * w_bytes + EPI_BYTES + CTRL_BYTES;
+    out->grid = (int)(items < sms ? items : sms);
+    return true;
+}
+
+template <int KC, int COB>
+lamp_status_t launch_ct(const CUtensorMap &mx, const CUtensorMap &mw, const CtPlan &pl, cudaStream_t st)
+{
+    static bool attr = false;
+    if (!attr) {
+        LAMP_CUDA_OK(cudaFuncSetAttribute(conv3_t_kernel<KC, COB>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT));
+        attr = true;
+    }
+    conv3_t_kernel<KC, COB><<<pl.grid, CT_THREADS, pl.smem, st>>>(mx, mw, pl.P);
+    return launch_status();
+}
+
+}  // namespace
+
+bool ct_conv_fwd_supported(const ConvGeom &g, const TView &x, const TView &y)
+{
+    CtPlan pl;
+    if ((int64_t)g.n * g.d * g.h * g.w == 0) return false;
+    if (g.co > 128) return false;                              // wide layers: N = c_out already fills the tensor pipe
+    if (!make_ct_plan(g, &pl)) return false;
+    // the 8 x 32 window must not be mostly padding
+    const double used = (double)g.h * g.w / ((double)pl.P.nht * TH * pl.P.nwt * TW);
+    if (used < 0.55) return false;
+    if (x.pitch % 8 || ((uintptr_t)x.p & 15)) return false;
+    if (y.f32 ? (y.pitch % 4 != 0) : (y.pitch % 8 != 0)) return false;
+    if ((uintptr_t)y.p & 15) return false;
+    return true;
+}
+
+lamp_status_t ct_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
+                          double *stats, int mirror_taps, cudaStream_t st)
+{
+    CtPlan pl;
+    if (!make_ct_plan(g, &pl)) return LAMP_ERR_UNSUPPORTED;
+    PFN_cuTensorMapEncodeTiled_v12000 encode = get_encode();
+    if (!encode) return LAMP_ERR_CUDA;
+    CtParams &P = pl.P;
+    P.mirror = mirror_taps; P.y_f32 = y.f32; P.y_pitch = y.pitch; P.y = y.p;
+    P.bias = bias; P.stats = stats; P.status = status_word_ptr();
+    const CUtensorMapSwizzle swz = pl.KC == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+    CUtensorMap mx, mw;
+    {
+        const cuuint64_t dims[5] = {(cuuint64_t)g.ci, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.d, (cuuint64_t)g.n};
+        const cuuint64_t strides[4] = {(cuuint64_t)x.pitch * 2, (cuuint64_t)x.pitch * 2 * g.w,
+                                       (cuuint64_t)x.pitch * 2 * g.w * g.h, (cuuint64_t)x.pitch * 2 * g.w * g.h * g.d};
+        const cuuint32_t box[5] = {(cuuint32_t)pl.KC, (cuuint32_t)HALO_W, (cuuint32_t)HALO_H, 1, 1};
+        const cuuint32_t es[5] = {1, 1, 1, 1, 1};
+        if (encode(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, x.p, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return LAMP_ERR_CUDA;
+    }
+    {
+        const cuuint64_t dims[3] = {(cuuint64_t)g.ci, (cuuint64_t)g.co, 27};
+        const cuuint64_t strides[2] = {(cuuint64_t)g.ci * 2, (cuuint64_t)g.ci * 2 * g.co};
+        const cuuint32_t box[3] = {(cuuint32_t)pl.KC, (cuuint32_t)pl.COB, 1};
+        const cuuint32_t es[3] = {1, 1, 1};
+        if (encode(&mw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void *)w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return LAMP_ERR_CUDA;
+    }
+    const int key = pl.KC * 1000 + pl.COB;
+    switch (key) {
+    case 64 * 1000 + 32:  return launch_ct<64, 32>(mx, mw, pl, st);
+    case 64 * 1000 + 64:  return launch_ct<64, 64>(mx, mw, pl, st);
+    case 64 * 1000 + 128: return launch_ct<64, 128>(mx, mw, pl, st);
+    case 32 * 1000 + 32:  return launch_ct<32, 32>(mx, mw, pl, st);
+    case 32 * 1000 + 64:  return launch_ct<32, 64>(mx, mw, pl, st);
+    case 32 * 1000 + 128: return launch_ct<32, 128>(mx, mw, pl, st);
+    }
+    return LAMP_ERR_UNSUPPORTED;
+}
+
+}  // namespace lamp

@@ -27,6 +27,13 @@ CASES = [
     ("c128_64", 1, 8, 8, 24, 128, 64, 3, 1, 1, 0),
     ("c32_to_128", 1, 4, 8, 16, 32, 128, 3, 1, 1, 0),
     ("c256", 1, 4, 6, 8, 256, 256, 3, 1, 1, 0),
+    ("t_c64_h40", 1, 5, 40, 24, 64, 64, 3, 1, 1, 0),
+    ("t_c32_h33", 2, 6, 33, 15, 32, 32, 3, 1, 1, 0),
+    ("t_c128_h64", 1, 3, 64, 16, 128, 128, 3, 1, 1, 0),
+    ("t_c64_to_32", 1, 7, 32, 8, 64, 32, 3, 1, 1, 0),
+    ("t_c128_to_64", 1, 3, 36, 10, 128, 64, 3, 1, 1, 0),
+    ("t_c32_to_128", 1, 4, 34, 9, 32, 128, 3, 1, 1, 0),
+    ("t_single_plane", 1, 1, 32, 8, 64, 64, 3, 1, 1, 0),
     ("tiny_volume", 1, 2, 2, 2, 64, 64, 3, 1, 1, 0),
     ("single_voxel", 1, 1, 1, 1, 32, 32, 3, 1, 1, 0),
 ]
