@@ -336,6 +336,122 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+# --------------------------------------------------------------------------------------------
+# Secondary workloads: the U-Net passes (one JSON line each; the headline stays the conv sweep)
+# --------------------------------------------------------------------------------------------
+UNET_CFGS = {
+    0: dict(levels=3, ch=[8, 16, 32], cpl=2, K=4, vol=(32, 32, 32)),
+    2: dict(levels=5, ch=[32, 64, 128, 256, 512], cpl=2, K=10, vol=(128, 128, 128)),
+    3: dict(levels=5, ch=[64, 128, 256, 512, 1024], cpl=3, K=10, vol=(192, 192, 64)),
+    4: dict(levels=5, ch=[32, 64, 128, 256, 512], cpl=2, K=10, vol=(512, 512, 128)),
+}
+
+
+def unet_fwd_flops(cfg):
+    D, H, W = cfg["vol"]
+    ch, L = cfg["ch"], cfg["levels"]
+    vox = [(D >> l) * (H >> l) * (W >> l) for l in range(L)]
+    fl, c = 0.0, 1
+    for l in range(L):
+        for _ in range(cfg["cpl"]):
+            fl += 2.0 * 27 * c * ch[l] * vox[l]
+            c = ch[l]
+        if l < L - 1:
+            fl += 2.0 * 27 * ch[l] * ch[l + 1] * vox[l + 1]
+            c = ch[l + 1]
+    for l in range(L - 2, -1, -1):
+        fl += 2.0 * ch[l + 1] * ch[l] * vox[l]
+        c = 2 * ch[l]
+        for _ in range(cfg["cpl"]):
+            fl += 2.0 * 27 * c * ch[l] * vox[l]
+            c = ch[l]
+    return fl + 2.0 * ch[0] * cfg["K"] * vox[0]
+
+
+def run_unet(args):
+    import torch
+    from paper_2006_12575_b200 import binding as B
+    from paper_2006_12575_b200 import build as lamp_build
+    from paper_2006_12575_b200 import synth
+    lamp_build.build()
+    torch.cuda.set_device(0)
+    cfg = UNET_CFGS[args.cfg]
+    D, H, W = cfg["vol"]
+    V = D * H * W
+    net = B.lamp_unet_create(B.unet_spec(cfg["levels"], cfg["ch"], cfg["cpl"], 1, cfg["K"]))
+    nl = B.lamp_unet_num_layers(net)
+    g = torch.Generator().manual_seed(10 * args.cfg + 1)
+    wflat = torch.zeros(B.lamp_unet_weight_count(net), dtype=torch.float32)
+    for i in range(nl):
+        wo, bo, d = B.lamp_unet_param_layout(net, i)
+        taps = d.ksize ** 3
+        fan = (1 if d.transposed else taps) * d.c_in
+        n = taps * d.c_in * d.c_out
+        wflat[wo:wo + n] = torch.randn(n, generator=g) * (2.0 / fan) ** 0.5
+    wd = wflat.cuda().to(torch.bfloat16)
+    bd = torch.zeros(B.lamp_unet_bias_count(net), dtype=torch.float32, device="cuda")
+    if args.cfg == 4:
+        vol = synth.ct_volume((D, H, W), 40)
+    else:
+        vol = synth.blurred_noise((D, H, W), 2.0, 10 * args.cfg)
+    hx = torch.from_numpy(vol).to(torch.bfloat16).reshape(1, D, H, W, 1).pin_memory()
+    x = hx.cuda()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    out = dict(n_gpus=1, steps=args.steps, warmup=args.warmup, higher_is_better=True, scaling="weak", vs_baseline=None,
+               dtype="bf16", data="synthetic", unit="voxels/s")
+    if args.workload == "unet_train":
+        lab = torch.from_numpy(synth.labels_quartiles((D, H, W), 10 * args.cfg + 2, cfg["K"], 4.0)).reshape(-1).cuda()
+        loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+        gw = torch.empty(B.lamp_unet_weight_count(net), dtype=torch.float32, device="cuda")
+        gb = torch.empty(B.lamp_unet_bias_count(net), dtype=torch.float32, device="cuda")
+        nbytes = B.lamp_unet_workspace_bytes(net, 1, D, H, W, B.MODE_TRAIN)
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        fn = lambda: B.lamp_unet_train_step(net, wd, bd, x, lab, loss, gw, gb, None, ws)
+        flops = 3 * unet_fwd_flops(cfg)
+        out.update(metric="unet_train_step_voxels_per_s", config=dict(workload=f"configs[{args.cfg}] U-Net forward+backward",
+                                                                         workspace_bytes=nbytes))
+    elif args.workload == "unet_infer":
+        probs = torch.empty((V, cfg["K"]), dtype=torch.float32, device="cuda")
+        seg = torch.empty(V, dtype=torch.uint8, device="cuda")
+        nbytes = B.lamp_unet_workspace_bytes(net, 1, D, H, W, B.MODE_INFER)
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        fn = lambda: B.lamp_unet_forward(net, wd, bd, x, probs, seg, ws)
+        flops = unet_fwd_flops(cfg)
+        out.update(metric="unet_whole_volume_infer_voxels_per_s",
+                   config=dict(workload=f"configs[{args.cfg}] whole-volume forward", workspace_bytes=nbytes))
+    else:
+        patch = (64, 64, 64)
+        seg = torch.empty(V, dtype=torch.uint8, device="cuda")
+        nbytes = B.lamp_sliding_window_workspace_bytes(net, D, H, W, patch, 0.25, args.sw_batch)
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        fn = lambda: B.lamp_sliding_window_infer(net, wd, bd, x, patch, 0.25, args.sw_batch, 1, None, seg, ws)
+        pc = dict(cfg, vol=patch)
+        npatch = 1
+        for n_, p_ in zip((D, H, W), patch):
+            s_ = 48
+            k = (n_ - p_) // s_ + 1
+            npatch *= k + (1 if (k - 1) * s_ != n_ - p_ else 0)
+        flops = npatch * unet_fwd_flops(pc)
+        out.update(metric="unet_sliding_window_infer_voxels_per_s",
+                   config=dict(workload=f"configs[{args.cfg}] sliding window 64^3, overlap 0.25, gaussian", patches=npatch,
+                               sw_batch=args.sw_batch, workspace_bytes=nbytes))
+    for _ in range(args.warmup):
+        fn()
+    torch.cuda.synchronize()
+    t0, t1 = ev(), ev()
+    t0.record()
+    for _ in range(args.steps):
+        fn()
+    t1.record()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / args.steps
+    if B.lamp_get_async_status() != 0:
+        raise SystemExit("device status not ok")
+    out.update(value=round(V / (ms * 1e-3), 1), ms_per_step=round(ms, 3), tflops=round(flops / (ms * 1e-3) / 1e12, 2),
+               seconds_per_volume=round(ms * 1e-3, 5))
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -343,7 +459,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="lamp", choices=["lamp", "reference"])
     ap.add_argument("--channels", default=",".join(str(c) for c in CHANNELS))
+    ap.add_argument("--workload", default="conv_sweep", choices=["conv_sweep", "unet_train", "unet_infer", "sliding"])
+    ap.add_argument("--cfg", type=int, default=2)
+    ap.add_argument("--sw-batch", type=int, default=8)
     args = ap.parse_args()
+    if args.workload != "conv_sweep":
+        run_unet(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -61,20 +61,34 @@ lamp_status_t conv_geom(const lamp_conv_desc_t *d, const lamp_tensor_t *in, cons
     return LAMP_OK;
 }
 
-static bool dgrad_via_umma(const ConvGeom &g)
+static int fwd_kind(const ConvGeom &g)
 {
-    // data gradient of the 3x3x3 s1 p1 conv = the same conv on dy with mirrored taps and swapped channels
-    if (!(g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed)) return false;
-    ConvGeom t = g;
-    t.ci = g.co; t.co = g.ci;
+    if (g.transposed) return UK_T_FWD;
+    if (g.k == 3 && g.s == 2) return UK_S2_FWD;
+    if (g.k == 3 && g.s == 1) return UK_S1_FWD;
+    return -1;
+}
+
+static int dgrad_kind(const ConvGeom &g)
+{
+    if (g.transposed) return UK_T_DGRAD;
+    if (g.k == 3 && g.s == 2) return UK_S2_DGRAD;
+    if (g.k == 3 && g.s == 1) return UK_S1_DGRAD;
+    return -1;
+}
+
+static bool dgrad_on_tensor_cores(const ConvGeom &g)
+{
+    // channel counts only; the alignment of the real views is checked again at launch
     TView a{}, b{};
-    a.pitch = 8; b.pitch = 8;      // alignment of the real views is checked again at launch
-    return umma_conv_fwd_supported(t, a, b);
+    a.pitch = 8; b.pitch = 8;
+    const int kind = dgrad_kind(g);
+    return kind >= 0 && umma_conv_supported(kind, g, a, b);
 }
 
 size_t conv_ws_bytes(const ConvGeom &g, int pass)
 {
-    if (pass == LAMP_PASS_DGRAD) return dgrad_via_umma(g) ? umma_dgrad_ws(g) : 0;
+    if (pass == LAMP_PASS_DGRAD) return dgrad_on_tensor_cores(g) ? umma_dgrad_ws(g) : 0;
     if (pass == LAMP_PASS_WGRAD) {
         const size_t u = umma_wgrad_ws(g);       // 0 when the tensor-core kernel does not take this shape
         const size_t tc = u ? u + bias_grad_ws((int64_t)g.n * g.od * g.oh * g.ow, g.co) : 0;
@@ -88,24 +102,27 @@ lamp_status_t conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const f
                        double *stats, cudaStream_t st)
 {
     if (ct_conv_fwd_supported(g, x, y)) return ct_conv_fwd(g, x, w, bias, y, stats, 0, st);
-    if (umma_conv_fwd_supported(g, x, y)) return umma_conv_fwd(g, x, w, bias, y, stats, 0, st);
+    const int kind = fwd_kind(g);
+    if (kind >= 0 && umma_conv_supported(kind, g, x, y)) return umma_conv(kind, g, x, w, bias, y, stats, st);
     return simt_conv_fwd(g, x, w, bias, y, stats, st);
 }
 
 lamp_status_t conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w, const TView &dx, void *ws, size_t ws_bytes,
                          cudaStream_t st)
 {
-    if (dgrad_via_umma(g)) {
-        ConvGeom t = g;
-        t.ci = g.co; t.co = g.ci;
-        if (umma_conv_fwd_supported(t, dy, dx)) {
-            const size_t need = umma_dgrad_ws(g);
-            if (!ws || ws_bytes < need || !aligned16(ws)) return LAMP_ERR_WORKSPACE;
-            lamp_status_t s = umma_transpose_weights(w, (bf16 *)ws, 27, g.co, g.ci, st);
-            if (s != LAMP_OK) return s;
+    const int kind = dgrad_kind(g);
+    if (kind >= 0 && umma_conv_supported(kind, g, dy, dx)) {
+        // every tensor-core data gradient reads the weights as [tap][c_in][c_out]
+        const size_t need = umma_dgrad_ws(g);
+        if (!ws || ws_bytes < need || !aligned16(ws)) return LAMP_ERR_WORKSPACE;
+        lamp_status_t s = umma_transpose_weights(w, (bf16 *)ws, g.k * g.k * g.k, g.co, g.ci, st);
+        if (s != LAMP_OK) return s;
+        if (kind == UK_S1_DGRAD) {
+            ConvGeom t = g;
+            t.ci = g.co; t.co = g.ci;
             if (ct_conv_fwd_supported(t, dy, dx)) return ct_conv_fwd(t, dy, (const bf16 *)ws, nullptr, dx, nullptr, 1, st);
-            return umma_conv_fwd(t, dy, (const bf16 *)ws, nullptr, dx, nullptr, 1, st);
         }
+        return umma_conv(kind, g, dy, (const bf16 *)ws, nullptr, dx, nullptr, st);
     }
     return simt_conv_dgrad(g, dy, w, dx, st);
 }

@@ -102,10 +102,11 @@ size_t        umma_wgrad_ws(const ConvGeom &g);
 lamp_status_t umma_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, void *ws, size_t ws_bytes,
                          cudaStream_t st);
 
-// conv_umma.cu (tcgen05 implicit GEMM)
-bool          umma_conv_fwd_supported(const ConvGeom &g, const TView &x, const TView &y);
-lamp_status_t umma_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
-                            double *stats, int mirror_taps, cudaStream_t st);
+// conv_umma.cu (tcgen05 implicit GEMM, voxels x channels form; see the file header for the kinds)
+enum { UK_S1_FWD = 0, UK_S1_DGRAD = 1, UK_S2_FWD = 2, UK_S2_DGRAD = 3, UK_T_FWD = 4, UK_T_DGRAD = 5 };
+bool          umma_conv_supported(int kind, const ConvGeom &g, const TView &a, const TView &y);
+lamp_status_t umma_conv(int kind, const ConvGeom &g, const TView &a, const bf16 *w, const float *bias, const TView &y,
+                        double *stats, cudaStream_t st);
 size_t        umma_dgrad_ws(const ConvGeom &g);
 lamp_status_t umma_transpose_weights(const bf16 *w, bf16 *wt, int taps, int co, int ci, cudaStream_t st);
 

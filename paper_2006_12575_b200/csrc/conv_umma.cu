@@ -1,24 +1,32 @@
-// 3x3x3 stride-1 pad-1 convolution as an implicit GEMM on the sm_100a tensor cores.
+// Convolution passes as an implicit GEMM on the sm_100a tensor cores, "voxels x channels" form:
+//   M = 128 output points (a tw x th x td box), N = output-channel tile (<= 256), K = taps x input channels.
 //
-//   y[v, co] = b[co] + sum_{tap, ci} x[v + off(tap), ci] * w[tap][co][ci]
-//   GEMM view: M = output voxels (tiles of 128 = tw x th x td), N = c_out (tile BN), K = 27 * c_in.
+// One kernel serves every pass whose result at a point j is a sum over taps of a [c_in]-vector read at
+// (in_scale * j + shift(tap)) times a [c_out x c_in] weight tile:
+//   3x3x3 s1 p1 forward            27 taps, shift k-1                      (c_out >= 256; narrower: conv_t.cu)
+//   3x3x3 s1 p1 data gradient      the same on dy with taps mirrored, weights transposed
+//   3x3x3 s2 p1 forward            27 taps, in_scale 2: the TMA box walks the input with element stride 2
+//   3x3x3 s2 p1 data gradient      8 parity classes of dx (i = 2j + parity), 1..8 taps each, written with stride 2
+//   2x2x2 s2 transposed forward    8 parity classes of y, one tap each
+//   2x2x2 s2 transposed data grad. 8 taps, in_scale 2
+// Which taps, shifts and weight tiles a class uses comes from a small table built on the host.
 //
 // Per CTA (persistent over tiles), warp-specialised:
-//   warp 0   : TMA producer.  For each (tap, channel chunk) it loads the A tile - a tw x th x td box of
-//              the NDHWC activation shifted by the tap offset, out-of-volume voxels zero-filled by the
-//              TMA unit, which is exactly the zero padding - and the matching [BN x KC] weight tile,
-//              both with the 128-byte (KC = 64) or 64-byte (KC = 32) shared-memory swizzle.
+//   warp 0   : TMA producer.  For each (tap, channel chunk) it loads the A tile - the tw x th x td box of
+//              the NDHWC tensor at the tap's shift, out-of-volume voxels zero-filled by the TMA unit,
+//              which is exactly the zero padding - and the matching [BN x KC] weight tile, both with
+//              the 128-byte (KC = 64) or 64-byte (KC = 32) shared-memory swizzle.
 //   warp 1   : allocates TMEM and issues tcgen05.mma (M = 128, N = BN, K = 16 per instruction) from one
 //              thread; fp32 accumulators live in TMEM, double-buffered so that the epilogue of tile i
 //              overlaps the MMAs of tile i + 1.
-//   warps 2-5: epilogue.  tcgen05.ld the accumulator rows (one voxel per thread), add the bias, reduce
+//   warps 2-5: epilogue.  tcgen05.ld the accumulator rows (one point per thread), add the bias, reduce
 //              the per-channel sum and sum of squares (InstanceNorm statistics), convert and store the
 //              row into the output's channel slice.
-// The data-gradient pass runs the same kernel on dy with the taps mirrored and the weights transposed.
 // Every mbarrier wait is bounded; on expiry the CTA records LAMP_ERR_TIMEOUT and winds down.
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include "common.cuh"
+#include <string.h>
 #include "umma_ptx.cuh"
 
 namespace lamp {
@@ -27,22 +35,45 @@ namespace {
 
 using namespace ptx;
 
+struct TapTable {                  // per parity class: the taps that contribute, their weight tile and input shift
+    int8_t ntaps[8];
+    int8_t wtap[8][27];
+    int8_t sd[8][27], sh[8][27], sw[8][27];
+};
+
 struct UmmaParams {
-    int32_t N, D, H, W;            // volume
+    int32_t N, D, H, W;            // batch; extents of the point grid j the tiles cover
+    int32_t OD, OH, OW;            // extents of the output tensor
+    int32_t in_scale, out_scale;   // input voxel = in_scale * j + shift; output voxel = out_scale * j + class parity
+    int32_t nclass;                // 1, or 8 parity classes
     int32_t tw, th, td;            // voxel tile, tw * th * td = 128
     int32_t ntw, nth, ntd;         // tiles per axis
     int32_t nct;                   // c_out tiles
     int32_t chunks;                // c_in / KC
     int32_t total_tiles;
     int32_t co;                    // c_out
-    int32_t mirror;                // 1: weight tap index = 26 - tap
     int32_t y_f32;
     int64_t y_pitch;
     void   *y;
     const float *bias;
     double *stats;                 // [N][co][2] or NULL
     int    *status;
+    TapTable taps;
 };
+
+struct Tile { int ct, w0, h0, d0, cls, n; };
+
+__device__ __forceinline__ Tile decode_tile(const UmmaParams &P, int t)
+{
+    Tile r;
+    r.ct = t % P.nct; t /= P.nct;
+    r.w0 = (t % P.ntw) * P.tw; t /= P.ntw;
+    r.h0 = (t % P.nth) * P.th; t /= P.nth;
+    r.d0 = (t % P.ntd) * P.td; t /= P.ntd;
+    r.cls = t % P.nclass;
+    r.n = t / P.nclass;
+    return r;
+}
 
 constexpr int NUM_THREADS = 192;
 constexpr int MAX_STAGES = 8;
@@ -95,8 +126,6 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int kiters = 27 * P.chunks;
-
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -104,23 +133,22 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             uint32_t phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
-                int t = tile;
-                const int ct = t % P.nct; t /= P.nct;
-                const int wt = t % P.ntw; t /= P.ntw;
-                const int ht = t % P.nth; t /= P.nth;
-                const int dt = t % P.ntd;
-                const int n = t / P.ntd;
-                const int w0 = wt * P.tw, h0 = ht * P.th, d0 = dt * P.td;
-                for (int ki = 0; ki < kiters; ++ki) {
-                    const int tap = ki / P.chunks, ch = ki - tap * P.chunks;
-                    const int kd = tap / 9, kh = (tap / 3) % 3, kw = tap % 3;
-                    if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
-                    const uint32_t fb = full0 + 8 * stage;
-                    mbar_expect_tx(fb, L::STAGE_BYTES);
-                    const uint32_t sa = smem_u32(stage_base + stage * L::STAGE_BYTES);
-                    tma_load_5d(sa, &map_x, fb, ch * KC, w0 + kw - 1, h0 + kh - 1, d0 + kd - 1, n);
-                    tma_load_3d(sa + L::A_BYTES, &map_w, fb, ch * KC, ct * BN, P.mirror ? 26 - tap : tap);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                const Tile T = decode_tile(P, tile);
+                const int ntaps = P.taps.ntaps[T.cls];
+                for (int tp = 0; tp < ntaps && ok; ++tp) {
+                    const int cw = P.in_scale * T.w0 + P.taps.sw[T.cls][tp];
+                    const int chh = P.in_scale * T.h0 + P.taps.sh[T.cls][tp];
+                    const int cd = P.in_scale * T.d0 + P.taps.sd[T.cls][tp];
+                    const int wt = P.taps.wtap[T.cls][tp];
+                    for (int ch = 0; ch < P.chunks; ++ch) {
+                        if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                        const uint32_t fb = full0 + 8 * stage;
+                        mbar_expect_tx(fb, L::STAGE_BYTES);
+                        const uint32_t sa = smem_u32(stage_base + stage * L::STAGE_BYTES);
+                        tma_load_5d(sa, &map_x, fb, ch * KC, cw, chh, cd, T.n);
+                        tma_load_3d(sa + L::A_BYTES, &map_w, fb, ch * KC, T.ct * BN, wt);
+                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    }
                 }
             }
         }
@@ -131,6 +159,7 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             uint32_t phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
+                const int kiters = P.taps.ntaps[decode_tile(P, tile).cls] * P.chunks;
                 if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
@@ -176,18 +205,16 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             }
         };
         for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
-            int t = tile;
-            const int ct = t % P.nct; t /= P.nct;
-            const int wt = t % P.ntw; t /= P.ntw;
-            const int ht = t % P.nth; t /= P.nth;
-            const int dt = t % P.ntd;
-            const int n = t / P.ntd;
+            const Tile T = decode_tile(P, tile);
+            const int ct = T.ct, n = T.n;
             if (n != stat_n || ct != stat_ct) { flush(); stat_n = n; stat_ct = ct; }
             const int m = q * 32 + lane;
             const int wx = m % P.tw, hy = (m / P.tw) % P.th, dz = m / (P.tw * P.th);
-            const int w = wt * P.tw + wx, h = ht * P.th + hy, d = dt * P.td + dz;
-            const bool valid = (w < P.W) && (h < P.H) && (d < P.D);
-            const int64_t vox = (((int64_t)n * P.D + d) * P.H + h) * P.W + w;
+            const int jw = T.w0 + wx, jh = T.h0 + hy, jd = T.d0 + dz;
+            const int w = P.out_scale * jw + (T.cls & 1), h = P.out_scale * jh + ((T.cls >> 1) & 1),
+                      d = P.out_scale * jd + ((T.cls >> 2) & 1);
+            const bool valid = (jw < P.W) && (jh < P.H) && (jd < P.D) && (w < P.OW) && (h < P.OH) && (d < P.OD);
+            const int64_t vox = (((int64_t)n * P.OD + d) * P.OH + h) * P.OW + w;
             // the whole warp takes the same decision, so no lane is left behind at a __syncwarp
             ok = __all_sync(0xffffffffu, mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag));
             if (!ok) break;
@@ -346,20 +373,100 @@ lamp_status_t launch_bn(int bn, const CUtensorMap &mx, const CUtensorMap &mw, co
     return LAMP_ERR_UNSUPPORTED;
 }
 
+struct KindInfo {
+    int a_c, n_rows, taps;               // channels of the A tensor (GEMM K per tap), weight rows (GEMM N), taps in the weight tensor
+    int ad, ah, aw;                      // extents of the A tensor
+    int jd, jh, jw;                      // point grid
+    int od, oh, ow;                      // output tensor extents
+    int in_scale, out_scale, nclass;
+};
+
+bool kind_info(int kind, const ConvGeom &g, KindInfo *k)
+{
+    const bool s1 = g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed;
+    const bool s2 = g.k == 3 && g.s == 2 && g.p == 1 && !g.transposed;
+    const bool tr = g.k == 2 && g.s == 2 && g.p == 0 && g.transposed;
+    k->in_scale = 1; k->out_scale = 1; k->nclass = 1;
+    switch (kind) {
+    case UK_S1_FWD:
+        if (!s1) return false;
+        *k = KindInfo{g.ci, g.co, 27, g.d, g.h, g.w, g.d, g.h, g.w, g.d, g.h, g.w, 1, 1, 1};
+        return true;
+    case UK_S1_DGRAD:
+        if (!s1) return false;
+        *k = KindInfo{g.co, g.ci, 27, g.d, g.h, g.w, g.d, g.h, g.w, g.d, g.h, g.w, 1, 1, 1};
+        return true;
+    case UK_S2_FWD:
+        if (!s2) return false;
+        *k = KindInfo{g.ci, g.co, 27, g.d, g.h, g.w, g.od, g.oh, g.ow, g.od, g.oh, g.ow, 2, 1, 1};
+        return true;
+    case UK_S2_DGRAD:
+        if (!s2) return false;
+        *k = KindInfo{g.co, g.ci, 27, g.od, g.oh, g.ow, g.od, g.oh, g.ow, g.d, g.h, g.w, 1, 2, 8};
+        return true;
+    case UK_T_FWD:
+        if (!tr) return false;
+        *k = KindInfo{g.ci, g.co, 8, g.d, g.h, g.w, g.d, g.h, g.w, g.od, g.oh, g.ow, 1, 2, 8};
+        return true;
+    case UK_T_DGRAD:
+        if (!tr) return false;
+        *k = KindInfo{g.co, g.ci, 8, g.od, g.oh, g.ow, g.d, g.h, g.w, g.d, g.h, g.w, 2, 1, 1};
+        return true;
+    }
+    return false;
+}
+
+void fill_taps(int kind, TapTable *T)
+{
+    memset(T, 0, sizeof(*T));
+    auto set = [&](int cls, int wtap, int sd, int sh, int sw) {
+        const int i = T->ntaps[cls]++;
+        T->wtap[cls][i] = (int8_t)wtap; T->sd[cls][i] = (int8_t)sd; T->sh[cls][i] = (int8_t)sh; T->sw[cls][i] = (int8_t)sw;
+    };
+    if (kind == UK_S1_FWD || kind == UK_S2_FWD || kind == UK_S1_DGRAD) {
+        // tap (kd,kh,kw) reads the input at shift k - 1; the data gradient uses the mirrored weight tap
+        for (int t = 0; t < 27; ++t)
+            set(0, kind == UK_S1_DGRAD ? 26 - t : t, t / 9 - 1, (t / 3) % 3 - 1, t % 3 - 1);
+    } else if (kind == UK_T_DGRAD) {
+        for (int t = 0; t < 8; ++t) set(0, t, t >> 2, (t >> 1) & 1, t & 1);
+    } else if (kind == UK_T_FWD) {
+        for (int c = 0; c < 8; ++c) set(c, c, 0, 0, 0);           // output parity (pd,ph,pw) = tap (a,b,c)
+    } else {
+        // stride-2 data gradient: dx[2j + parity] collects taps k with (parity + 1 - k) even, from dy[j + (parity + 1 - k) / 2]
+        for (int c = 0; c < 8; ++c) {
+            const int par[3] = {(c >> 2) & 1, (c >> 1) & 1, c & 1};
+            for (int kd = 0; kd < 3; ++kd) {
+                if ((par[0] + 1 - kd) & 1) continue;
+                for (int kh = 0; kh < 3; ++kh) {
+                    if ((par[1] + 1 - kh) & 1) continue;
+                    for (int kw = 0; kw < 3; ++kw) {
+                        if ((par[2] + 1 - kw) & 1) continue;
+                        set(c, (kd * 3 + kh) * 3 + kw, (par[0] + 1 - kd) / 2, (par[1] + 1 - kh) / 2, (par[2] + 1 - kw) / 2);
+                    }
+                }
+            }
+        }
+    }
+}
+
 }  // namespace
 
-bool umma_conv_fwd_supported(const ConvGeom &g, const TView &x, const TView &y)
+bool umma_conv_supported(int kind, const ConvGeom &g, const TView &a, const TView &y)
 {
-    if (!(g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed)) return false;
-    if (g.ci % 32 || g.co % 16) return false;
-    if (!bn_instantiated(pick_bn(g.co))) return false;
-    if (x.pitch % 8 || ((uintptr_t)x.p & 15)) return false;
+    KindInfo k;
+    if (!kind_info(kind, g, &k)) return false;
+    if (k.a_c % 32 || k.n_rows % 16) return false;
+    if (!bn_instantiated(pick_bn(k.n_rows))) return false;
+    if (a.pitch % 8 || ((uintptr_t)a.p & 15)) return false;
     if (y.f32 ? (y.pitch % 4 != 0) : (y.pitch % 8 != 0)) return false;
     if ((uintptr_t)y.p & 15) return false;
     return true;
 }
 
-size_t umma_dgrad_ws(const ConvGeom &g) { return align_up((size_t)27 * g.co * g.ci * sizeof(bf16), 256); }
+size_t umma_dgrad_ws(const ConvGeom &g)
+{
+    return align_up((size_t)g.k * g.k * g.k * g.co * g.ci * sizeof(bf16), 256);
+}
 
 lamp_status_t umma_transpose_weights(const bf16 *w, bf16 *wt, int taps, int co, int ci, cudaStream_t st)
 {
@@ -368,41 +475,50 @@ lamp_status_t umma_transpose_weights(const bf16 *w, bf16 *wt, int taps, int co, 
     return launch_status();
 }
 
-lamp_status_t umma_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
-                            double *stats, int mirror_taps, cudaStream_t st)
+// a: the tensor the taps read (x for forward kinds, dy for data-gradient kinds); w: [taps][n_rows][a_c] bf16
+// (the layer's weights for forward kinds, their per-tap transpose for data-gradient kinds).
+lamp_status_t umma_conv(int kind, const ConvGeom &g, const TView &a, const bf16 *w, const float *bias, const TView &y,
+                        double *stats, cudaStream_t st)
 {
-    if ((int64_t)g.n * g.d * g.h * g.w == 0) return LAMP_OK;
+    KindInfo k;
+    if (!kind_info(kind, g, &k)) return LAMP_ERR_UNSUPPORTED;
+    if ((int64_t)g.n * k.jd * k.jh * k.jw == 0) return LAMP_OK;
     PFN_cuTensorMapEncodeTiled_v12000 encode = get_encode();
     if (!encode) return LAMP_ERR_CUDA;
-    const int KC = (g.ci % 64 == 0) ? 64 : 32;
-    const int BN = pick_bn(g.co);
+    const int KC = (k.a_c % 64 == 0) ? 64 : 32;
+    const int BN = pick_bn(k.n_rows);
     UmmaParams P;
-    P.N = g.n; P.D = g.d; P.H = g.h; P.W = g.w;
-    pick_tile(g.d, g.h, g.w, &P.tw, &P.th, &P.td);
-    P.ntw = (g.w + P.tw - 1) / P.tw; P.nth = (g.h + P.th - 1) / P.th; P.ntd = (g.d + P.td - 1) / P.td;
-    P.nct = g.co / BN;
-    P.chunks = g.ci / KC;
-    const int64_t tiles = (int64_t)g.n * P.ntd * P.nth * P.ntw * P.nct;
+    P.N = g.n; P.D = k.jd; P.H = k.jh; P.W = k.jw;
+    P.OD = k.od; P.OH = k.oh; P.OW = k.ow;
+    P.in_scale = k.in_scale; P.out_scale = k.out_scale; P.nclass = k.nclass;
+    pick_tile(k.jd, k.jh, k.jw, &P.tw, &P.th, &P.td);
+    P.ntw = (k.jw + P.tw - 1) / P.tw; P.nth = (k.jh + P.th - 1) / P.th; P.ntd = (k.jd + P.td - 1) / P.td;
+    P.nct = k.n_rows / BN;
+    P.chunks = k.a_c / KC;
+    const int64_t tiles = (int64_t)g.n * k.nclass * P.ntd * P.nth * P.ntw * P.nct;
     if (tiles > 0x7FFFFFFF) return LAMP_ERR_UNSUPPORTED;
     P.total_tiles = (int32_t)tiles;
-    P.co = g.co; P.mirror = mirror_taps; P.y_f32 = y.f32; P.y_pitch = y.pitch; P.y = y.p;
+    P.co = k.n_rows; P.y_f32 = y.f32; P.y_pitch = y.pitch; P.y = y.p;
     P.bias = bias; P.stats = stats; P.status = status_word_ptr();
+    fill_taps(kind, &P.taps);
 
     CUtensorMap mx, mw;
     {
-        const cuuint64_t dims[5] = {(cuuint64_t)g.ci, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.d, (cuuint64_t)g.n};
-        const cuuint64_t strides[4] = {(cuuint64_t)x.pitch * 2, (cuuint64_t)x.pitch * 2 * g.w,
-                                       (cuuint64_t)x.pitch * 2 * g.w * g.h, (cuuint64_t)x.pitch * 2 * g.w * g.h * g.d};
-        const cuuint32_t box[5] = {(cuuint32_t)KC, (cuuint32_t)P.tw, (cuuint32_t)P.th, (cuuint32_t)P.td, 1};
-        const cuuint32_t es[5] = {1, 1, 1, 1, 1};
-        if (encode(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, x.p, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        const cuuint32_t s = (cuuint32_t)k.in_scale;
+        const cuuint64_t dims[5] = {(cuuint64_t)k.a_c, (cuuint64_t)k.aw, (cuuint64_t)k.ah, (cuuint64_t)k.ad, (cuuint64_t)g.n};
+        const cuuint64_t strides[4] = {(cuuint64_t)a.pitch * 2, (cuuint64_t)a.pitch * 2 * k.aw,
+                                       (cuuint64_t)a.pitch * 2 * k.aw * k.ah, (cuuint64_t)a.pitch * 2 * k.aw * k.ah * k.ad};
+        // with an element stride s the box spans s times the number of voxels it delivers
+        const cuuint32_t box[5] = {(cuuint32_t)KC, (cuuint32_t)P.tw * s, (cuuint32_t)P.th * s, (cuuint32_t)P.td * s, 1};
+        const cuuint32_t es[5] = {1, s, s, s, 1};
+        if (encode(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, a.p, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                    KC == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return LAMP_ERR_CUDA;
     }
     {
-        const cuuint64_t dims[3] = {(cuuint64_t)g.ci, (cuuint64_t)g.co, 27};
-        const cuuint64_t strides[2] = {(cuuint64_t)g.ci * 2, (cuuint64_t)g.ci * 2 * g.co};
+        const cuuint64_t dims[3] = {(cuuint64_t)k.a_c, (cuuint64_t)k.n_rows, (cuuint64_t)k.taps};
+        const cuuint64_t strides[2] = {(cuuint64_t)k.a_c * 2, (cuuint64_t)k.a_c * 2 * k.n_rows};
         const cuuint32_t box[3] = {(cuuint32_t)KC, (cuuint32_t)BN, 1};
         const cuuint32_t es[3] = {1, 1, 1};
         if (encode(&mw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void *)w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,

@@ -17,6 +17,12 @@ CASES = [
     ("narrow_16_24", 2, 6, 5, 9, 16, 24, 3, 1, 1, 0),
     ("down_8_16", 1, 8, 6, 10, 8, 16, 3, 2, 1, 0),
     ("down_32_64", 1, 16, 8, 12, 32, 64, 3, 2, 1, 0),
+    ("down_64_128_odd", 1, 9, 10, 14, 64, 128, 3, 2, 1, 0),
+    ("down_256_512", 2, 4, 4, 8, 256, 512, 3, 2, 1, 0),
+    ("down_32_32_big", 1, 20, 34, 18, 32, 32, 3, 2, 1, 0),
+    ("up_128_64", 1, 4, 5, 6, 128, 64, 2, 2, 0, 1),
+    ("up_512_256", 1, 2, 2, 4, 512, 256, 2, 2, 0, 1),
+    ("up_32_32_big", 2, 9, 10, 7, 32, 32, 2, 2, 0, 1),
     ("up_16_8", 2, 3, 4, 5, 16, 8, 2, 2, 0, 1),
     ("up_64_32", 1, 6, 4, 8, 64, 32, 2, 2, 0, 1),
     ("head_8_4", 1, 5, 4, 6, 8, 4, 1, 1, 0, 0),

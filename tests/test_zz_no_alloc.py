@@ -55,8 +55,8 @@ def test_static_scratch_dgrad_rejects_layers_beyond_the_limit_and_takes_scratch_
         B.lamp_conv3d_dgrad_static_scratch(desc, dy, w, dx)
     assert e.value.status == 7 and "scratch" in str(e.value)
     assert (dx == 0).all()                                   # nothing was launched
-    # the stride-2 conv's data gradient needs no scratch at all
-    desc, dy, w, shape = _layer(16, 32, (8, 6, 10), 41, s=2)
+    # the 1x1x1 conv's data gradient needs no scratch at all
+    desc, dy, w, shape = _layer(16, 32, (8, 6, 10), 41, k=1, s=1, p=0)
     ref, nbytes = _reference(desc, dy, w, shape)
     assert nbytes == 0
     dx = torch.full(shape, float("nan"), dtype=torch.bfloat16, device="cuda")
