@@ -190,7 +190,7 @@ conv_wgrad_kernel(ConvGeom g, const bf16 *__restrict__ x, int64_t xp, const bf16
     part[(int64_t)blockIdx.y * entries + e] = acc;
 }
 
-// Column sums of dy over a chunk of voxels: part[chunk][co].
+// Column sums of dy over a chunk of voxels: part[chunk][co].  Generic (any co, any alignment).
 __global__ void __launch_bounds__(256)
 colsum_kernel(const bf16 *__restrict__ dy, int64_t dyp, int co, int64_t V, int64_t v_per_block, float *__restrict__ part)
 {
@@ -199,6 +199,178 @@ colsum_kernel(const bf16 *__restrict__ dy, int64_t dyp, int co, int64_t V, int64
         float acc = 0.f;
         for (int64_t v = v0; v < v1; ++v) acc += bf2f(dy[v * dyp + c]);
         part[(int64_t)blockIdx.x * co + c] = acc;
+    }
+}
+
+// The same for co % 8 == 0 and 16-byte aligned rows: thread = (voxel row in the block, group of 8 channels).
+__global__ void __launch_bounds__(256)
+colsum_vec_kernel(const bf16 *__restrict__ dy, int64_t dyp, int co, int64_t V, int64_t v_per_block, float *__restrict__ part)
+{
+    extern __shared__ float red[];          // [RB][G][8]
+    const int G = co >> 3, RB = 256 / G;
+    const int g = threadIdx.x % G, r = threadIdx.x / G;
+    const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = min(V, v0 + v_per_block);
+    float s[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) s[j] = 0.f;
+    if (r < RB) {
+        for (int64_t v = v0 + r; v < v1; v += RB) {
+            float f[8];
+            unpack8(__ldg(reinterpret_cast<const uint4 *>(dy + v * dyp + g * 8)), f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s[j] += f[j];
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) red[(r * G + g) * 8 + j] = s[j];
+    }
+    __syncthreads();
+    for (int t = threadIdx.x; t < co; t += 256) {
+        float acc = 0.f;
+        for (int rr = 0; rr < RB; ++rr) acc += red[rr * co + t];
+        part[(int64_t)blockIdx.x * co + t] = acc;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// First layer of the network: one input channel, 3x3x3 s1 p1, c_out <= 64 (HBM-bound: the output
+// is 2 * c_out bytes per voxel against 2 bytes read).  One thread per output voxel, all channels.
+// ---------------------------------------------------------------------------------------------
+template <int CO>
+__global__ void __launch_bounds__(128)
+conv_c1_fwd_kernel(ConvGeom g, const bf16 *__restrict__ x, int64_t xp, const bf16 *__restrict__ w,
+                   const float *__restrict__ bias, void *__restrict__ y, int64_t yp, int y_f32, double *__restrict__ stats)
+{
+    __shared__ float sw[27 * CO];
+    __shared__ float sb[CO];
+    __shared__ float tr[4][32 * (CO + 1)];
+    __shared__ float bs1[CO], bs2[CO];
+    for (int i = threadIdx.x; i < 27 * CO; i += 128) sw[i] = bf2f(w[i]);          // w[t][co][0]
+    for (int i = threadIdx.x; i < CO; i += 128) { sb[i] = bias ? bias[i] : 0.f; bs1[i] = 0.f; bs2[i] = 0.f; }
+    __syncthreads();
+    const int n = blockIdx.y;
+    const int64_t Vn = (int64_t)g.d * g.h * g.w;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float cs1[(CO + 31) / 32], cs2[(CO + 31) / 32];
+#pragma unroll
+    for (int i = 0; i < (CO + 31) / 32; ++i) { cs1[i] = 0.f; cs2[i] = 0.f; }
+    for (int64_t v0 = (int64_t)blockIdx.x * 128; v0 < Vn; v0 += (int64_t)gridDim.x * 128) {
+        const int64_t v = v0 + threadIdx.x;
+        const bool live = v < Vn;
+        float acc[CO];
+#pragma unroll
+        for (int c = 0; c < CO; ++c) acc[c] = sb[c];
+        if (live) {
+            const int iw = (int)(v % g.w), ih = (int)((v / g.w) % g.h), id = (int)(v / ((int64_t)g.w * g.h));
+            for (int kd = 0; kd < 3; ++kd) {
+                const int zd = id + kd - 1;
+                if (zd < 0 || zd >= g.d) continue;
+                for (int kh = 0; kh < 3; ++kh) {
+                    const int zh = ih + kh - 1;
+                    if (zh < 0 || zh >= g.h) continue;
+#pragma unroll
+                    for (int kw = 0; kw < 3; ++kw) {
+                        const int zw = iw + kw - 1;
+                        if (zw < 0 || zw >= g.w) continue;
+                        const float xv = bf2f(x[((((int64_t)n * g.d + zd) * g.h + zh) * g.w + zw) * xp]);
+                        const float *wt = sw + ((kd * 3 + kh) * 3 + kw) * CO;
+#pragma unroll
+                        for (int c = 0; c < CO; ++c) acc[c] = fmaf(xv, wt[c], acc[c]);
+                    }
+                }
+            }
+            const int64_t o = ((int64_t)n * Vn + v) * yp;
+            if (y_f32) {
+                float4 *dst = reinterpret_cast<float4 *>((float *)y + o);
+#pragma unroll
+                for (int c = 0; c < CO; c += 4) dst[c / 4] = make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]);
+            } else {
+                uint4 *dst = reinterpret_cast<uint4 *>((bf16 *)y + o);
+#pragma unroll
+                for (int c = 0; c < CO; c += 8) {
+                    float f8[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) f8[u] = acc[c + u];
+                    dst[c / 8] = pack8(f8);
+                }
+            }
+        }
+        if (stats) {
+            // per-warp transpose: lane c then sums channel c (and c + 32) over the warp's 32 voxels
+            float *t = tr[warp];
+#pragma unroll
+            for (int c = 0; c < CO; ++c) t[lane * (CO + 1) + c] = live ? acc[c] : 0.f;
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < (CO + 31) / 32; ++i) {
+                const int c = i * 32 + lane;
+                if (c < CO) {
+                    float a = 0.f, b = 0.f;
+                    for (int r = 0; r < 32; ++r) { const float f = t[r * (CO + 1) + c]; a += f; b = fmaf(f, f, b); }
+                    cs1[i] += a;
+                    cs2[i] += b;
+                }
+            }
+            __syncwarp();
+        }
+    }
+    if (stats) {
+#pragma unroll
+        for (int i = 0; i < (CO + 31) / 32; ++i) {
+            const int c = i * 32 + lane;
+            if (c < CO) { atomicAdd(&bs1[c], cs1[i]); atomicAdd(&bs2[c], cs2[i]); }
+        }
+        __syncthreads();
+        for (int c = threadIdx.x; c < CO; c += 128) {
+            atomicAdd(&stats[((int64_t)n * CO + c) * 2], (double)bs1[c]);
+            atomicAdd(&stats[((int64_t)n * CO + c) * 2 + 1], (double)bs2[c]);
+        }
+    }
+}
+
+// Weight gradient of the same layer: dw[t][co] = sum_v dy[v][co] * x[v + off_t].  A warp owns a stripe of
+// voxels; lane = output channel (plus 32 for c_out = 64); 27 accumulators per lane; part[block][27 * co].
+template <int CO>
+__global__ void __launch_bounds__(256)
+conv_c1_wgrad_kernel(ConvGeom g, const bf16 *__restrict__ x, int64_t xp, const bf16 *__restrict__ dy, int64_t dyp,
+                     float *__restrict__ part, int64_t v_per_block)
+{
+    constexpr int CPL = (CO + 31) / 32;          // channels per lane
+    constexpr int NWARP = CO > 32 ? 4 : 8;       // blockDim.x = 32 * NWARP (static shared memory stays under 48 KB)
+    __shared__ float red[NWARP][27 * CO];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t V = (int64_t)g.n * g.d * g.h * g.w;
+    const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = min(V, v0 + v_per_block);
+    float acc[CPL][27];
+#pragma unroll
+    for (int i = 0; i < CPL; ++i)
+#pragma unroll
+        for (int t = 0; t < 27; ++t) acc[i][t] = 0.f;
+    for (int64_t v = v0 + warp; v < v1; v += NWARP) {
+        const int iw = (int)(v % g.w), ih = (int)((v / g.w) % g.h), id = (int)((v / ((int64_t)g.w * g.h)) % g.d);
+        const int64_t nb = v - (((int64_t)id * g.h + ih) * g.w + iw);      // voxel index of (n, 0, 0, 0)
+        float gy[CPL];
+#pragma unroll
+        for (int i = 0; i < CPL; ++i) gy[i] = (i * 32 + lane < CO) ? bf2f(dy[v * dyp + i * 32 + lane]) : 0.f;
+#pragma unroll
+        for (int t = 0; t < 27; ++t) {
+            const int zd = id + t / 9 - 1, zh = ih + (t / 3) % 3 - 1, zw = iw + t % 3 - 1;
+            float xv = 0.f;
+            if (zd >= 0 && zd < g.d && zh >= 0 && zh < g.h && zw >= 0 && zw < g.w)
+                xv = bf2f(x[(nb + ((int64_t)zd * g.h + zh) * g.w + zw) * xp]);
+#pragma unroll
+            for (int i = 0; i < CPL; ++i) acc[i][t] = fmaf(gy[i], xv, acc[i][t]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < CPL; ++i)
+#pragma unroll
+        for (int t = 0; t < 27; ++t)
+            if (i * 32 + lane < CO) red[warp][t * CO + i * 32 + lane] = acc[i][t];
+    __syncthreads();
+    for (int e = threadIdx.x; e < 27 * CO; e += 32 * NWARP) {
+        float a = 0.f;
+        for (int wv = 0; wv < NWARP; ++wv) a += red[wv][e];
+        part[(int64_t)blockIdx.x * 27 * CO + e] = a;
     }
 }
 
@@ -244,9 +416,23 @@ inline WgradPlan wgrad_plan(const ConvGeom &g)
 lamp_status_t simt_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
                             double *stats, cudaStream_t st)
 {
-    const int TC = pick_tc(g.co), TV = 256 / TC, iters = 16;
     const int64_t Vn = (int64_t)g.od * g.oh * g.ow;
     if (Vn == 0 || g.n == 0) return LAMP_OK;
+    if (g.ci == 1 && g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed && (g.co == 32 || g.co == 64) &&
+        ((uintptr_t)y.p & 15) == 0 && (y.f32 ? y.pitch % 4 == 0 : y.pitch % 8 == 0)) {
+        int blocks = (int)((Vn + 127) / 128);
+        const int cap = 148 * 16 / (g.n > 0 ? g.n : 1) + 1;
+        if (blocks > cap) blocks = cap;
+        dim3 grid(blocks, g.n);
+        if (g.co == 32)
+            conv_c1_fwd_kernel<32><<<grid, 128, 0, st>>>(g, (const bf16 *)x.p, x.pitch, w, bias, y.p, y.pitch, y.f32, stats);
+        else
+            conv_c1_fwd_kernel<64><<<grid, 128, 0, st>>>(g, (const bf16 *)x.p, x.pitch, w, bias, y.p, y.pitch, y.f32, stats);
+        return launch_status();
+    }
+    const int TC = pick_tc(g.co), TV = 256 / TC;
+    // few voxels (deep levels): one voxel group per block so that the grid still fills the machine
+    const int iters = Vn >= 65536 ? 16 : (Vn >= 8192 ? 4 : 1);
     const int vec = (g.ci % 8 == 0) && (x.pitch % 8 == 0) && ((uintptr_t)x.p % 16 == 0) && ((uintptr_t)w % 16 == 0);
     dim3 grid((unsigned)((Vn + (int64_t)TV * iters - 1) / ((int64_t)TV * iters)), g.n);
     if (g.transposed)
@@ -297,9 +483,29 @@ lamp_status_t bias_grad(const TView &dy, float *db, void *ws, cudaStream_t st)
     if (V == 0) { LAMP_CUDA_OK(cudaMemsetAsync(db, 0, (size_t)dy.c * 4, st)); return LAMP_OK; }
     int b; int64_t vpb;
     bias_plan(V, &b, &vpb);
-    colsum_kernel<<<b, 256, 0, st>>>((const bf16 *)dy.p, dy.pitch, dy.c, V, vpb, (float *)ws);
+    if (dy.c % 8 == 0 && dy.c <= 2048 && dy.pitch % 8 == 0 && ((uintptr_t)dy.p & 15) == 0) {
+        const int G = dy.c / 8, RB = 256 / G;
+        colsum_vec_kernel<<<b, 256, (size_t)RB * dy.c * sizeof(float), st>>>((const bf16 *)dy.p, dy.pitch, dy.c, V, vpb, (float *)ws);
+    } else {
+        colsum_kernel<<<b, 256, 0, st>>>((const bf16 *)dy.p, dy.pitch, dy.c, V, vpb, (float *)ws);
+    }
     reduce_parts_kernel<<<(dy.c + 255) / 256, 256, 0, st>>>((const float *)ws, dy.c, b, db);
     return launch_status();
+}
+
+static bool c1_wgrad_shape(const ConvGeom &g)
+{
+    return g.ci == 1 && g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed && (g.co == 32 || g.co == 64);
+}
+
+static void c1_wgrad_plan(const ConvGeom &g, int *blocks, int64_t *vpb)
+{
+    const int64_t V = (int64_t)g.n * g.d * g.h * g.w;
+    int b = (int)((V + 2047) / 2048);
+    if (b > 148 * 8) b = 148 * 8;
+    if (b < 1) b = 1;
+    *blocks = b;
+    *vpb = (V + b - 1) / b;
 }
 
 size_t simt_conv_wgrad_ws(const ConvGeom &g)
@@ -313,6 +519,24 @@ lamp_status_t simt_conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy
 {
     const WgradPlan p = wgrad_plan(g);
     if (ws_bytes < simt_conv_wgrad_ws(g) || !ws) return LAMP_ERR_WORKSPACE;
+    if (c1_wgrad_shape(g) && p.V > 0) {
+        // partials [blocks][27 * co] fit the generic plan's workspace (blocks <= 1184 <= its split count bound)
+        int blocks; int64_t vpb;
+        c1_wgrad_plan(g, &blocks, &vpb);
+        if ((size_t)blocks * p.entries * 4 <= align_up((size_t)p.splits * p.entries * 4, 256)) {
+            float *part1 = (float *)ws;
+            if (g.co == 32)
+                conv_c1_wgrad_kernel<32><<<blocks, 256, 0, st>>>(g, (const bf16 *)x.p, x.pitch, (const bf16 *)dy.p, dy.pitch, part1, vpb);
+            else
+                conv_c1_wgrad_kernel<64><<<blocks, 128, 0, st>>>(g, (const bf16 *)x.p, x.pitch, (const bf16 *)dy.p, dy.pitch, part1, vpb);
+            reduce_parts_kernel<<<(unsigned)((p.entries + 255) / 256), 256, 0, st>>>(part1, p.entries, blocks, dw);
+            if (db) {
+                lamp_status_t sb = bias_grad(dy, db, (char *)ws + align_up((size_t)p.splits * p.entries * 4, 256), st);
+                if (sb != LAMP_OK) return sb;
+            }
+            return launch_status();
+        }
+    }
     float *part = (float *)ws;
     float *cpart = (float *)((char *)ws + align_up((size_t)p.splits * p.entries * 4, 256));
     if (p.V == 0) {

@@ -1,18 +1,22 @@
-// Weight gradient of the 3x3x3 stride-1 pad-1 convolution on the sm_100a tensor cores.
+// Weight gradients on the sm_100a tensor cores.
 //
-//   dw[tap][co][ci] = sum_v dy[v][co] * x[v + off(tap)][ci] = sum_u dy[u - off(tap)][co] * x[u][ci]
+//   3x3x3 s1 p1 :  dw[tap][co][ci] = sum_u dy[u - off(tap)][co] * x[u][ci]
+//   3x3x3 s2 p1 :  dw[tap][co][ci] = sum_o dy[o][co] * x[2 o + off(tap)][ci]
+//   2x2x2 s2 T  :  dw[tap][co][ci] = sum_j dy[2 j + tap][co] * x[j][ci]
 //
-// GEMM view per tap: D[co x ci] = dy_shifted^T * x with the reduction over voxels.  Both operands are
-// read straight from the NDHWC tensors, i.e. with the reduction (voxel) index as the smem row and the
-// channels contiguous: "MN-major" operands of tcgen05.mma.  A voxel tile (tw x th x td = 128 voxels)
-// is one K = 128 slab: the x tile is loaded once, the dy tile once per tap, shifted by -off(tap), with
-// out-of-volume voxels zero-filled by TMA (the conv's zero padding).
+// In each case one tensor is read at the tile's own voxels ("fixed", F) and the other at per-tap shifted
+// (and possibly stride-2) voxels ("moving", G).  GEMM view per tap: D[G channels x F channels] = G_tap^T * F with
+// the reduction over voxels.  Both operands are read straight from the NDHWC tensors, i.e. with the
+// reduction (voxel) index as the shared-memory row and the channels contiguous: "MN-major" operands of
+// tcgen05.mma.  A voxel tile (tw x th x td = 128 voxels) is one K = 128 slab: the F tile is loaded once,
+// the G tile once per tap, at scale * j + shift(tap), out-of-volume voxels zero-filled by TMA (the
+// conv's zero padding); a stride-2 G tile is fetched by a TMA box with element stride 2.
 //
-// M = 128 accumulator rows hold 128 output channels of one tap (c_out >= 128), two taps x 64 channels
-// (c_out = 64) or four taps x 32 channels (c_out = 32); N = min(c_in, 256) columns.  The fp32
-// accumulators of up to 512 / N such blocks stay in TMEM while the CTA sweeps its share of the voxel
-// tiles (split-K over CTAs); each CTA then writes its partial sums and a second kernel adds the
-// partials in a fixed order, so the result does not depend on scheduling.
+// M = 128 accumulator rows hold 128 G channels of one tap, two taps x 64 channels or four taps x 32
+// channels; N = min(F channels, 256) columns.  The fp32 accumulators of up to 512 / N such blocks stay in
+// TMEM while the CTA sweeps its share of the voxel tiles (split-K over CTAs); each CTA then writes its
+// partial sums and a second kernel adds the partials in a fixed order (transposing where G is x), so
+// the result does not depend on scheduling.
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include "common.cuh"
@@ -27,16 +31,19 @@ using namespace ptx;
 struct WgParams {
     int32_t N, D, H, W;
     int32_t tw, th, td, ntw, nth, ntd, ntiles;
-    int32_t co, ci;
-    int32_t co_blk;          // output channels per tap inside an M block: min(co, 128)
+    int32_t co, ci;          // channels of the moving tensor G (M side) and of the fixed tensor F (N side)
+    int32_t ntaps;           // 27 or 8
+    int32_t g_scale;         // G voxel = g_scale * j + shift(tap)
+    int8_t  sd[27], sh[27], sw[27];
+    int32_t co_blk;          // G channels per tap inside an M block: min(co, 128)
     int32_t tpm;             // taps per M block: 128 / co_blk
     int32_t co_chunks;       // co / co_blk
-    int32_t MB;              // M blocks: ceil(27 / tpm) * co_chunks
+    int32_t MB;              // M blocks: ceil(ntaps / tpm) * co_chunks
     int32_t nchunks;         // ci / NC
     int32_t sps;             // accumulator slots per set (512 / NC, at most MB)
     int32_t sets_per_chunk;  // ceil(MB / sps)
     int32_t nsets, nsplit, nunits;
-    int64_t entries;         // 27 * co * ci
+    int64_t entries;         // ntaps * co * ci
     float  *part;            // [nsplit][entries]
     int    *status;
 };
@@ -126,18 +133,16 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                         int nvalid = 0;
 #pragma unroll
                         for (int b = 0; b < ABOXES; ++b)
-                            nvalid += (tg * P.tpm + (b * BOXA) / P.co_blk) < 27;
+                            nvalid += (tg * P.tpm + (b * BOXA) / P.co_blk) < P.ntaps;
                         mbar_expect_tx(afull0 + 8 * as, nvalid * BOXA_BYTES);
                         const uint32_t asm_ = smem_u32(as_base + as * A_STAGE_BYTES);
 #pragma unroll
                         for (int b = 0; b < ABOXES; ++b) {
                             const int m0 = b * BOXA;
                             const int tap = tg * P.tpm + m0 / P.co_blk;
-                            if (tap < 27) {
-                                const int kd = tap / 9, kh = (tap / 3) % 3, kw = tap % 3;
+                            if (tap < P.ntaps)
                                 tma_load_5d(asm_ + b * BOXA_BYTES, &map_dy, afull0 + 8 * as, cc * P.co_blk + m0 % P.co_blk,
-                                            w0 - (kw - 1), h0 - (kh - 1), d0 - (kd - 1), n);
-                            }
+                                            P.g_scale * w0 + P.sw[tap], P.g_scale * h0 + P.sh[tap], P.g_scale * d0 + P.sd[tap], n);
                         }
                         if (++as == NA) { as = 0; aph ^= 1; }
                     }
@@ -208,7 +213,7 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     uint32_t r[32];
                     tmem_ld32(trow + c0, r);
                     tmem_ld_wait();
-                    if (tap < 27) {
+                    if (tap < P.ntaps) {
                         float4 *d4 = reinterpret_cast<float4 *>(dst + c0);
 #pragma unroll
                         for (int j = 0; j < 8; ++j)
@@ -264,41 +269,74 @@ void pick_tile128(int D, int H, int W, int *tw, int *th, int *td)
         }
 }
 
-bool encode_act(PFN_cuTensorMapEncodeTiled_v12000 encode, CUtensorMap *m, const TView &t, int box_c, int tw, int th, int td)
+bool encode_act(PFN_cuTensorMapEncodeTiled_v12000 encode, CUtensorMap *m, const TView &t, int box_c, int tw, int th, int td, int scale)
 {
+    const cuuint32_t s = (cuuint32_t)scale;
     const cuuint64_t dims[5] = {(cuuint64_t)t.c, (cuuint64_t)t.w, (cuuint64_t)t.h, (cuuint64_t)t.d, (cuuint64_t)t.n};
     const cuuint64_t strides[4] = {(cuuint64_t)t.pitch * 2, (cuuint64_t)t.pitch * 2 * t.w, (cuuint64_t)t.pitch * 2 * t.w * t.h,
                                    (cuuint64_t)t.pitch * 2 * t.w * t.h * t.d};
-    const cuuint32_t box[5] = {(cuuint32_t)box_c, (cuuint32_t)tw, (cuuint32_t)th, (cuuint32_t)td, 1};
-    const cuuint32_t es[5] = {1, 1, 1, 1, 1};
+    const cuuint32_t box[5] = {(cuuint32_t)box_c, (cuuint32_t)tw * s, (cuuint32_t)th * s, (cuuint32_t)td * s, 1};
+    const cuuint32_t es[5] = {1, s, s, s, 1};
     return encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, t.p, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                   box_c == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-struct WgPlan { WgParams P; int NC, BOXA, BOXB; int grid; };
+// out[t][b][a] = sum_s part[s][t][a][b]   (partials were accumulated as [tap][G channel][F channel] with G = x)
+__global__ void __launch_bounds__(256)
+reduce_transposed_kernel(const float *__restrict__ part, int64_t entries, int splits, int A, int Bc, float *__restrict__ out)
+{
+    const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;      // index into out: (t * Bc + b) * A + a
+    if (e >= entries) return;
+    const int a = (int)(e % A);
+    const int b = (int)((e / A) % Bc);
+    const int64_t t = e / ((int64_t)A * Bc);
+    const int64_t src = (t * A + a) * Bc + b;
+    float acc = 0.f;
+    for (int s = 0; s < splits; ++s) acc += part[(int64_t)s * entries + src];
+    out[e] = acc;
+}
 
+struct WgPlan { WgParams P; int NC, BOXA, BOXB; int grid; bool g_is_x; };
+
+// Which tensor moves: s1 and transposed convs shift dy (G = dy, F = x); the stride-2 conv shifts x (G = x, F = dy).
 bool make_wg_plan(const ConvGeom &g, WgPlan *out)
 {
-    if (!(g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed)) return false;
-    if (!(g.co == 32 || g.co == 64 || g.co % 128 == 0)) return false;
+    const bool s1 = g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed;
+    const bool s2 = g.k == 3 && g.s == 2 && g.p == 1 && !g.transposed;
+    const bool tr = g.k == 2 && g.s == 2 && g.p == 0 && g.transposed;
+    if (!s1 && !s2 && !tr) return false;
+    out->g_is_x = s2;
+    const int gc = s2 ? g.ci : g.co;                 // channels of G (M side)
+    const int fc = s2 ? g.co : g.ci;                 // channels of F (N side)
+    if (!(gc == 32 || gc == 64 || gc % 128 == 0)) return false;
     int NC;
-    if (g.ci == 32 || g.ci == 64 || g.ci == 128) NC = g.ci;
-    else if (g.ci % 256 == 0) NC = 256;
+    if (fc == 32 || fc == 64 || fc == 128) NC = fc;
+    else if (fc % 256 == 0) NC = 256;
     else return false;
     WgParams &P = out->P;
-    P.N = g.n; P.D = g.d; P.H = g.h; P.W = g.w;
-    pick_tile128(g.d, g.h, g.w, &P.tw, &P.th, &P.td);
-    P.ntw = (g.w + P.tw - 1) / P.tw; P.nth = (g.h + P.th - 1) / P.th; P.ntd = (g.d + P.td - 1) / P.td;
+    // the tile grid is F's voxel grid: x for s1 / transposed, dy for the stride-2 conv
+    const int fd = s2 ? g.od : g.d, fh = s2 ? g.oh : g.h, fw = s2 ? g.ow : g.w;
+    P.N = g.n; P.D = fd; P.H = fh; P.W = fw;
+    pick_tile128(fd, fh, fw, &P.tw, &P.th, &P.td);
+    P.ntw = (fw + P.tw - 1) / P.tw; P.nth = (fh + P.th - 1) / P.th; P.ntd = (fd + P.td - 1) / P.td;
     const int64_t nt = (int64_t)g.n * P.ntd * P.nth * P.ntw;
     if (nt > 0x7FFFFFFF || nt <= 0) return false;
     P.ntiles = (int32_t)nt;
-    P.co = g.co; P.ci = g.ci;
-    P.co_blk = g.co < 128 ? g.co : 128;
+    P.co = gc; P.ci = fc;
+    P.ntaps = g.k * g.k * g.k;
+    P.g_scale = s1 ? 1 : 2;
+    for (int t = 0; t < P.ntaps; ++t) {
+        const int kd = t / (g.k * g.k), kh = (t / g.k) % g.k, kw = t % g.k;
+        if (s1)      { P.sd[t] = (int8_t)(1 - kd); P.sh[t] = (int8_t)(1 - kh); P.sw[t] = (int8_t)(1 - kw); }   // dy[u - (k - 1)]
+        else if (s2) { P.sd[t] = (int8_t)(kd - 1); P.sh[t] = (int8_t)(kh - 1); P.sw[t] = (int8_t)(kw - 1); }   // x[2 o + k - 1]
+        else         { P.sd[t] = (int8_t)kd; P.sh[t] = (int8_t)kh; P.sw[t] = (int8_t)kw; }                     // dy[2 j + tap]
+    }
+    P.co_blk = gc < 128 ? gc : 128;
     P.tpm = 128 / P.co_blk;
-    P.co_chunks = g.co / P.co_blk;
-    P.MB = (27 + P.tpm - 1) / P.tpm * P.co_chunks;
-    P.nchunks = g.ci / NC;
+    P.co_chunks = gc / P.co_blk;
+    P.MB = (P.ntaps + P.tpm - 1) / P.tpm * P.co_chunks;
+    P.nchunks = fc / NC;
     P.sps = 512 / NC < P.MB ? 512 / NC : P.MB;
     P.sets_per_chunk = (P.MB + P.sps - 1) / P.sps;
     P.nsets = P.nchunks * P.sets_per_chunk;
@@ -310,10 +348,10 @@ bool make_wg_plan(const ConvGeom &g, WgPlan *out)
     if (nsplit > P.ntiles) nsplit = P.ntiles;
     P.nsplit = nsplit;
     P.nunits = P.nsets * nsplit;
-    P.entries = (int64_t)27 * g.co * g.ci;
+    P.entries = (int64_t)P.ntaps * g.co * g.ci;
     out->NC = NC;
-    out->BOXA = g.co == 32 ? 32 : 64;
-    out->BOXB = g.ci == 32 ? 32 : 64;
+    out->BOXA = gc == 32 ? 32 : 64;
+    out->BOXB = fc == 32 ? 32 : 64;
     out->grid = P.nunits < sms ? P.nunits : sms;
     return true;
 }
@@ -336,7 +374,7 @@ lamp_status_t launch_wg(const CUtensorMap &mx, const CUtensorMap &mdy, const WgP
 bool umma_wgrad_supported(const ConvGeom &g, const TView &x, const TView &dy)
 {
     WgPlan pl;
-    if ((int64_t)g.n * g.d * g.h * g.w == 0) return false;
+    if ((int64_t)g.n * g.d * g.h * g.w == 0 || (int64_t)g.od * g.oh * g.ow == 0) return false;
     if (!make_wg_plan(g, &pl)) return false;
     if (x.pitch % 8 || dy.pitch % 8 || ((uintptr_t)x.p & 15) || ((uintptr_t)dy.p & 15)) return false;
     return true;
@@ -360,8 +398,10 @@ lamp_status_t umma_wgrad(const ConvGeom &g, const TView &x, const TView &dy, flo
     pl.P.part = (float *)ws;
     pl.P.status = status_word_ptr();
     CUtensorMap mx, mdy;
-    if (!encode_act(encode, &mx, x, pl.BOXB, pl.P.tw, pl.P.th, pl.P.td)) return LAMP_ERR_CUDA;
-    if (!encode_act(encode, &mdy, dy, pl.BOXA, pl.P.tw, pl.P.th, pl.P.td)) return LAMP_ERR_CUDA;
+    // first map = fixed tensor F (N side), second = moving tensor G (M side)
+    const TView &F = pl.g_is_x ? dy : x, &G = pl.g_is_x ? x : dy;
+    if (!encode_act(encode, &mx, F, pl.BOXB, pl.P.tw, pl.P.th, pl.P.td, 1)) return LAMP_ERR_CUDA;
+    if (!encode_act(encode, &mdy, G, pl.BOXA, pl.P.tw, pl.P.th, pl.P.td, pl.P.g_scale)) return LAMP_ERR_CUDA;
     lamp_status_t s = LAMP_ERR_UNSUPPORTED;
     const int key = pl.NC * 10000 + pl.BOXA * 100 + pl.BOXB;
     switch (key) {
@@ -375,7 +415,9 @@ lamp_status_t umma_wgrad(const ConvGeom &g, const TView &x, const TView &dy, flo
     case 256 * 10000 + 64 * 100 + 64: s = launch_wg<256, 64, 64>(mx, mdy, pl, st); break;
     }
     if (s != LAMP_OK) return s;
-    return reduce_partials(pl.P.part, pl.P.entries, pl.P.nsplit, dw, st);
+    if (!pl.g_is_x) return reduce_partials(pl.P.part, pl.P.entries, pl.P.nsplit, dw, st);
+    reduce_transposed_kernel<<<(unsigned)((pl.P.entries + 255) / 256), 256, 0, st>>>(pl.P.part, pl.P.entries, pl.P.nsplit, g.ci, g.co, dw);
+    return launch_status();
 }
 
 }  // namespace lamp

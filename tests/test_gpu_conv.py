@@ -14,6 +14,8 @@ pytestmark = pytest.mark.gpu
 # (name, N, D, H, W, Ci, Co, k, s, p, transposed)
 CASES = [
     ("first_layer_c1", 1, 9, 7, 10, 1, 8, 3, 1, 1, 0),
+    ("first_layer_c1_32", 2, 9, 17, 12, 1, 32, 3, 1, 1, 0),
+    ("first_layer_c1_64", 1, 6, 5, 21, 1, 64, 3, 1, 1, 0),
     ("narrow_16_24", 2, 6, 5, 9, 16, 24, 3, 1, 1, 0),
     ("down_8_16", 1, 8, 6, 10, 8, 16, 3, 2, 1, 0),
     ("down_32_64", 1, 16, 8, 12, 32, 64, 3, 2, 1, 0),
