@@ -511,7 +511,14 @@ static void c1_wgrad_plan(const ConvGeom &g, int *blocks, int64_t *vpb)
 size_t simt_conv_wgrad_ws(const ConvGeom &g)
 {
     const WgradPlan p = wgrad_plan(g);
-    return align_up((size_t)p.splits * p.entries * 4, 256) + align_up((size_t)p.cs_blocks * g.co * 4, 256);
+    size_t main_part = (size_t)p.splits * p.entries * 4;
+    if (c1_wgrad_shape(g)) {
+        int blocks; int64_t vpb;
+        c1_wgrad_plan(g, &blocks, &vpb);
+        if ((size_t)blocks * p.entries * 4 > main_part) main_part = (size_t)blocks * p.entries * 4;
+    }
+    return align_up(main_part, 256) + align_up((size_t)p.cs_blocks * g.co * 4, 256) +
+           bias_grad_ws((int64_t)g.n * g.od * g.oh * g.ow, g.co);
 }
 
 lamp_status_t simt_conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, float *db,
@@ -523,7 +530,7 @@ lamp_status_t simt_conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy
         // partials [blocks][27 * co] fit the generic plan's workspace (blocks <= 1184 <= its split count bound)
         int blocks; int64_t vpb;
         c1_wgrad_plan(g, &blocks, &vpb);
-        if ((size_t)blocks * p.entries * 4 <= align_up((size_t)p.splits * p.entries * 4, 256)) {
+        {
             float *part1 = (float *)ws;
             if (g.co == 32)
                 conv_c1_wgrad_kernel<32><<<blocks, 256, 0, st>>>(g, (const bf16 *)x.p, x.pitch, (const bf16 *)dy.p, dy.pitch, part1, vpb);
@@ -531,7 +538,8 @@ lamp_status_t simt_conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy
                 conv_c1_wgrad_kernel<64><<<blocks, 128, 0, st>>>(g, (const bf16 *)x.p, x.pitch, (const bf16 *)dy.p, dy.pitch, part1, vpb);
             reduce_parts_kernel<<<(unsigned)((p.entries + 255) / 256), 256, 0, st>>>(part1, p.entries, blocks, dw);
             if (db) {
-                lamp_status_t sb = bias_grad(dy, db, (char *)ws + align_up((size_t)p.splits * p.entries * 4, 256), st);
+                const size_t off = simt_conv_wgrad_ws(g) - bias_grad_ws((int64_t)g.n * g.od * g.oh * g.ow, g.co);
+                lamp_status_t sb = bias_grad(dy, db, (char *)ws + off, st);
                 if (sb != LAMP_OK) return sb;
             }
             return launch_status();

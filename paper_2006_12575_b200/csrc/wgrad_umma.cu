@@ -395,7 +395,9 @@ lamp_status_t umma_wgrad(const ConvGeom &g, const TView &x, const TView &dy, flo
     if (!ws || ws_bytes < umma_wgrad_ws(g)) return LAMP_ERR_WORKSPACE;
     PFN_cuTensorMapEncodeTiled_v12000 encode = get_encode();
     if (!encode) return LAMP_ERR_CUDA;
-    pl.P.part = (float *)ws;
+    // a single split needs no second pass: the CTAs write the gradient itself
+    const bool direct = pl.P.nsplit == 1 && !pl.g_is_x;
+    pl.P.part = direct ? dw : (float *)ws;
     pl.P.status = status_word_ptr();
     CUtensorMap mx, mdy;
     // first map = fixed tensor F (N side), second = moving tensor G (M side)
@@ -414,7 +416,7 @@ lamp_status_t umma_wgrad(const ConvGeom &g, const TView &x, const TView &dy, flo
     case 256 * 10000 + 32 * 100 + 64: s = launch_wg<256, 32, 64>(mx, mdy, pl, st); break;
     case 256 * 10000 + 64 * 100 + 64: s = launch_wg<256, 64, 64>(mx, mdy, pl, st); break;
     }
-    if (s != LAMP_OK) return s;
+    if (s != LAMP_OK || direct) return s;
     if (!pl.g_is_x) return reduce_partials(pl.P.part, pl.P.entries, pl.P.nsplit, dw, st);
     reduce_transposed_kernel<<<(unsigned)((pl.P.entries + 255) / 256), 256, 0, st>>>(pl.P.part, pl.P.entries, pl.P.nsplit, g.ci, g.co, dw);
     return launch_status();

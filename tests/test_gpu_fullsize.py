@@ -1,0 +1,207 @@
+"""Full-size parity: the benchmark's own shapes and launch configuration, checked on sampled outputs
+that the CPU oracle evaluates one by one (a full fp64 pass over a 128^3 x 256-channel layer would take
+the oracle hours)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ops, unet as O
+from paper_2006_12575_b200 import binding as B
+from paper_2006_12575_b200 import synth
+
+from _util import assert_close, host_f64
+
+pytestmark = pytest.mark.gpu
+
+
+def _sample_points(rs, N, D, H, W, n_rand, n_edge):
+    """Random voxels plus voxels on faces / edges / corners of the volume."""
+    pts = np.stack([rs.integers(0, N, n_rand), rs.integers(0, D, n_rand), rs.integers(0, H, n_rand),
+                    rs.integers(0, W, n_rand)], axis=1)
+    edge = np.stack([rs.integers(0, N, n_edge)] + [rs.choice([0, 1, n // 2, n - 2, n - 1], n_edge) for n in (D, H, W)], axis=1)
+    return np.concatenate([pts, edge]).astype(np.int32)
+
+
+def _randn_bf16(shape, seed):
+    g = torch.Generator().manual_seed(seed)
+    return torch.randn(shape, generator=g, dtype=torch.float32).to(torch.bfloat16)
+
+
+@pytest.mark.parametrize("C", [32, 64, 128, 256])
+def test_conv_sweep_layer_at_benchmark_size(C):
+    D = H = W = 128
+    rs = np.random.default_rng(C)
+    hx, hdy = _randn_bf16((1, D, H, W, C), 2000 + C), _randn_bf16((1, D, H, W, C), 3000 + C)
+    w = synth.kaiming_bf16(27, C, C, 27 * C, 2000 + C)
+    xd, dyd, wd = hx.cuda(), hdy.cuda(), torch.from_numpy(w).cuda().to(torch.bfloat16)
+    desc = B.conv_desc(C, C)
+    y = torch.empty_like(xd)
+    dx = torch.empty_like(xd)
+    dw = torch.empty((27, C, C), dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(B.lamp_conv3d_workspace_bytes(desc, xd, B.PASS_DGRAD),
+                         B.lamp_conv3d_workspace_bytes(desc, xd, B.PASS_WGRAD), 256), dtype=torch.uint8, device="cuda")
+    B.lamp_conv3d_fwd(desc, xd, wd, None, y)
+    B.lamp_conv3d_dgrad(desc, dyd, wd, dx, ws)
+    B.lamp_conv3d_wgrad(desc, xd, dyd, dw, None, ws)
+    assert B.lamp_get_async_status() == 0
+    x64 = hx.to(torch.float64).numpy()
+    dy64 = hdy.to(torch.float64).numpy()
+    w64 = w.astype(np.float64)
+    n_pts = 1200 if C <= 128 else 500
+    pts = _sample_points(rs, 1, D, H, W, n_pts, n_pts // 3)
+    idx = (pts[:, 0], pts[:, 1], pts[:, 2], pts[:, 3])
+    ref = ops.conv3d_fwd_points(x64, w64, None, pts, 3, 1, 1)
+    assert_close(host_f64(y[idx]), ops.bf16_round(ref), f"C={C} fwd (sampled)")
+    # data gradient of the s1 p1 conv = the conv of dy with mirrored taps and swapped channels
+    wm = np.ascontiguousarray(w64[::-1].transpose(0, 2, 1))
+    ref = ops.conv3d_fwd_points(dy64, wm, None, pts, 3, 1, 1)
+    assert_close(host_f64(dx[idx]), ops.bf16_round(ref), f"C={C} dgrad (sampled)")
+    ent = np.stack([rs.integers(0, 27, 160), rs.integers(0, C, 160), rs.integers(0, C, 160)], axis=1).astype(np.int32)
+    ent[:27, 0] = np.arange(27)                      # every tap at least once
+    ref = ops.conv3d_wgrad_points(x64, dy64, ent, 3, 1, 1)
+    got = host_f64(dw[ent[:, 0], ent[:, 1], ent[:, 2]])
+    assert_close(got, ref, f"C={C} wgrad (sampled)", rel=1e-4, mx=1e-3)
+
+
+def _ws_view(wsb, layout):
+    t, off = layout
+    es = {B.LAMP_BF16: 2, B.LAMP_F32: 4}[t.dtype]
+    dt = {B.LAMP_BF16: torch.bfloat16, B.LAMP_F32: torch.float32}[t.dtype]
+    V = t.n * t.d * t.h * t.w
+    flat = wsb[off:off + ((V - 1) * t.c_pitch + t.c) * es].view(dt)
+    return torch.as_strided(flat, (t.n, t.d, t.h, t.w, t.c),
+                            (t.d * t.h * t.w * t.c_pitch, t.h * t.w * t.c_pitch, t.w * t.c_pitch, t.c_pitch, 1))
+
+
+def test_standard_unet_train_step_at_full_size_sampled():
+    """128^3 volume, widths 32..512, K = 10: one training step; every kind of layer is checked on sampled
+    outputs against the oracle evaluated on the tensors the GPU stored as that layer's input."""
+    levels, ch, cpl, K = 5, [32, 64, 128, 256, 512], 2, 10
+    D = H = W = 128
+    V = D * H * W
+    net = B.lamp_unet_create(B.unet_spec(levels, ch, cpl, 1, K))
+    spec = O.UNetSpec(levels, ch, cpl, 1, K)
+    lay = O.unet_layers(spec)
+    wl = synth.kaiming_for_layers([(l.taps, l.c_out, l.c_in, l.fan_in) for l in lay], 21)
+    wflat = np.zeros(B.lamp_unet_weight_count(net), dtype=np.float32)
+    offs = []
+    for i in range(len(lay)):
+        wo, bo, _ = B.lamp_unet_param_layout(net, i)
+        wflat[wo:wo + wl[i].size] = wl[i].ravel()
+        offs.append((wo, bo))
+    bflat = 0.05 * synth.rng(22).standard_normal(B.lamp_unet_bias_count(net)).astype(np.float32)
+    x = synth.bf16_round(synth.blurred_noise((D, H, W), 2.0, 20))[None, ..., None]
+    lab = synth.labels_blobs((D, H, W), 22, K, 4.0)[None]
+    wd = torch.from_numpy(wflat).cuda().to(torch.bfloat16)
+    bd = torch.from_numpy(bflat).cuda()
+    loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+    gw = torch.empty(B.lamp_unet_weight_count(net), dtype=torch.float32, device="cuda")
+    gb = torch.empty(B.lamp_unet_bias_count(net), dtype=torch.float32, device="cuda")
+    probs = torch.empty((V, K), dtype=torch.float32, device="cuda")
+    wsb = torch.empty(B.lamp_unet_workspace_bytes(net, 1, D, H, W, B.MODE_TRAIN), dtype=torch.uint8, device="cuda")
+    xd = torch.from_numpy(x).cuda().to(torch.bfloat16)
+    B.lamp_unet_train_step(net, wd, bd, xd, torch.from_numpy(lab).cuda().reshape(-1), loss, gw, gb, probs, wsb)
+    assert B.lamp_get_async_status() == 0
+    p_gpu = host_f64(probs).reshape(1, D, H, W, K)
+    assert np.isfinite(p_gpu).all() and np.allclose(p_gpu.sum(-1), 1, atol=1e-5)
+    assert abs(float(loss.item()) - ops.dice_loss(p_gpu, lab)) < 1e-5
+    lay_of = lambda i, which: B.lamp_unet_tensor_layout(net, 1, D, H, W, B.MODE_TRAIN, i, which)
+    rs = np.random.default_rng(5)
+    names = {l.name: i for i, l in enumerate(lay)}
+    gw_h = gw.cpu().numpy().astype(np.float64)
+    for name in ["enc0.conv0", "enc0.conv1", "down0", "enc1.conv1", "down2", "enc4.conv1", "up3", "dec1.conv0", "up0",
+                 "dec0.conv0", "dec0.conv1"]:
+        i = names[name]
+        l = lay[i]
+        w64 = wl[i].astype(np.float64)
+        bo = offs[i][1]
+        b64 = bflat[bo:bo + l.c_out].astype(np.float64)
+        x_in = x.astype(np.float64) if i == 0 else host_f64(_ws_view(wsb, lay_of(i, B.T_IN)))
+        if l.kind in ("conv", "down"):
+            s = 2 if l.kind == "down" else 1
+            y_gpu = _ws_view(wsb, lay_of(i, B.T_Y))
+            _, Do, Ho, Wo, _ = y_gpu.shape
+            pts = _sample_points(rs, 1, Do, Ho, Wo, 300, 100)
+            ref = ops.conv3d_fwd_points(x_in, w64, b64, pts, 3, s, 1)
+            idx = (pts[:, 0], pts[:, 1], pts[:, 2], pts[:, 3])
+            assert_close(host_f64(y_gpu[idx]), ops.bf16_round(ref), f"{name} y (sampled)")
+            # weight gradient on sampled entries, from the GPU's own stored dy
+            dy_gpu = host_f64(_ws_view(wsb, lay_of(i, B.T_DY)))
+            ent = np.stack([rs.integers(0, 27, 40), rs.integers(0, l.c_out, 40), rs.integers(0, l.c_in, 40)], 1).astype(np.int32)
+            ref = ops.conv3d_wgrad_points(x_in, dy_gpu, ent, 3, s, 1)
+            wo = offs[i][0]
+            got = gw_h[wo:wo + wl[i].size].reshape(wl[i].shape)[ent[:, 0], ent[:, 1], ent[:, 2]]
+            assert_close(got, ref, f"{name} dw (sampled)", rel=2e-4, mx=2e-3)
+        else:
+            u_gpu = _ws_view(wsb, lay_of(i, B.T_OUT))
+            _, Do, Ho, Wo, _ = u_gpu.shape
+            pts = _sample_points(rs, 1, Do, Ho, Wo, 300, 100)
+            tap = ((pts[:, 1] & 1) * 2 + (pts[:, 2] & 1)) * 2 + (pts[:, 3] & 1)
+            xi = x_in[pts[:, 0], pts[:, 1] // 2, pts[:, 2] // 2, pts[:, 3] // 2]          # [P, ci]
+            ref = np.einsum("pi,poi->po", xi, w64[tap]) + b64
+            idx = (pts[:, 0], pts[:, 1], pts[:, 2], pts[:, 3])
+            assert_close(host_f64(u_gpu[idx]), ops.bf16_round(ref), f"{name} out (sampled)")
+    # head: probabilities from the stored input, all voxels of a few planes
+    hi = len(lay) - 1
+    z = host_f64(_ws_view(wsb, lay_of(hi, B.T_IN))[:, 60:64])
+    bo = offs[hi][1]
+    p_ref = ops.softmax(ops.conv3d_fwd(z, wl[hi].astype(np.float64), bflat[bo:bo + K].astype(np.float64), 1, 1, 0))
+    assert_close(p_gpu[:, 60:64], p_ref, "head probs", rel=1e-5, mx=1e-5)
+    B.lamp_unet_destroy(net)
+
+
+def test_sliding_window_full_size_blend_sampled():
+    """512 x 512 x 128 CT-like volume, 64^3 patches at 25 % overlap: 363 patches.  The Gaussian blend and the
+    argmax are recomputed with the oracle's window on sampled voxels from the per-patch probabilities the GPU kept."""
+    levels, ch, cpl, K = 5, [32, 64, 128, 256, 512], 2, 10
+    D, H, W, P = 512, 512, 128, (64, 64, 64)
+    net = B.lamp_unet_create(B.unet_spec(levels, ch, cpl, 1, K))
+    g = torch.Generator().manual_seed(41)
+    wflat = torch.zeros(B.lamp_unet_weight_count(net), dtype=torch.float32)
+    for i in range(B.lamp_unet_num_layers(net)):
+        wo, bo, d = B.lamp_unet_param_layout(net, i)
+        n = d.ksize ** 3 * d.c_in * d.c_out
+        fan = (1 if d.transposed else d.ksize ** 3) * d.c_in
+        wflat[wo:wo + n] = torch.randn(n, generator=g) * (2.0 / fan) ** 0.5
+    wd = wflat.cuda().to(torch.bfloat16)
+    bd = torch.zeros(B.lamp_unet_bias_count(net), dtype=torch.float32, device="cuda")
+    vol = synth.ct_volume((D // 4, H // 4, W // 4), 40)                  # generated small and tiled: cheap, still structured
+    vol = np.tile(vol, (4, 4, 4))
+    xd = torch.from_numpy(synth.bf16_round(vol)).cuda().to(torch.bfloat16).reshape(1, D, H, W, 1)
+    seg = torch.empty(D * H * W, dtype=torch.uint8, device="cuda")
+    planar = torch.empty((K, D, H, W), dtype=torch.float32, device="cuda")
+    wsb = torch.empty(B.lamp_sliding_window_workspace_bytes(net, D, H, W, P, 0.25, 8), dtype=torch.uint8, device="cuda")
+    B.lamp_sliding_window_infer(net, wd, bd, xd, P, 0.25, 8, 1, planar, seg, wsb)
+    assert B.lamp_get_async_status() == 0
+    sd, sh, sw = (O.window_starts(n, p, 0.25) for n, p in zip((D, H, W), P))
+    assert len(sd) * len(sh) * len(sw) == 363
+    pp = wsb[:363 * 64 ** 3 * K * 4].view(torch.float32).reshape(363, 64, 64, 64, K)
+    win = O.gaussian_window(P)
+    rs = np.random.default_rng(9)
+    pts = _sample_points(rs, 1, D, H, W, 600, 200)[:, 1:]
+    pts[:100, 0] = 48 + rs.integers(0, 16, 100)        # inside the overlap band of two patches along d
+    got = host_f64(planar[:, pts[:, 0], pts[:, 1], pts[:, 2]]).T
+    segs = seg.reshape(D, H, W)[pts[:, 0], pts[:, 1], pts[:, 2]].cpu().numpy()
+    want = np.zeros((len(pts), K))
+    for n_, (d, h, w) in enumerate(pts):
+        acc, wsum = np.zeros(K), 0.0
+        for a, d0 in enumerate(sd):
+            if not d0 <= d < d0 + 64:
+                continue
+            for b, h0 in enumerate(sh):
+                if not h0 <= h < h0 + 64:
+                    continue
+                for c, w0 in enumerate(sw):
+                    if not w0 <= w < w0 + 64:
+                        continue
+                    wt = win[d - d0, h - h0, w - w0]
+                    acc += wt * pp[(a * len(sh) + b) * len(sw) + c, d - d0, h - h0, w - w0].double().cpu().numpy()
+                    wsum += wt
+        want[n_] = acc / wsum
+    assert_close(got, want, "sliding-window blend (sampled)", rel=1e-5, mx=1e-5)
+    order = np.argsort(-want, axis=1)
+    margin = want[np.arange(len(pts)), order[:, 0]] - want[np.arange(len(pts)), order[:, 1]]
+    ok = (segs == order[:, 0]) | ((margin < 1e-3) & (segs == order[:, 1]))
+    assert ok.mean() >= 0.9999
+    assert np.allclose(got.sum(1), 1, atol=1e-5)
+    B.lamp_unet_destroy(net)
