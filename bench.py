@@ -31,6 +31,9 @@ CHANNELS = (32, 64, 128, 256)
 VOL = (128, 128, 128)
 SEED = 2
 NOMINAL_BF16_TFLOPS = 2250.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture summarised
+# under profiles/ (None: not captured for the kernel as it stands)
+NCU_TRAFFIC_BYTES = {"conv3_umma_kernel": None, "conv3_t_kernel": None, "wgrad_umma_kernel": None}
 
 
 def pass_flops(C, vol=VOL):
@@ -117,7 +120,7 @@ class ClockSampler:
         try:
             self.f = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.f,
                                          stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -289,17 +292,23 @@ def run_gpu(args):
         tf = pass_flops(C) / (mean * 1e-3) / 1e12
         passes[f"C{C}.{name}"] = dict(ms=round(mean, 4), tflops=round(tf, 1), pct_nominal=round(100 * tf / NOMINAL_BF16_TFLOPS, 1),
                                       pct_measured=round(100 * tf / peaks["bf16"], 1))
-    # kernel families: tcgen05 implicit GEMM (fwd + dgrad) and the wgrad kernel
-    fam = {"conv3_umma_kernel (fwd+dgrad)": [k for k in per if k[1] in ("fwd", "dgrad")],
-           "conv_wgrad_kernel (wgrad)": [k for k in per if k[1] == "wgrad"]}
+    # kernel families (one CUDA kernel template each); the dgrad pass also holds the tiny weight-transpose launch
+    fam = {"conv3_umma_kernel (fwd+dgrad, C>=256: voxels x channels)": [k for k in per if k[1] in ("fwd", "dgrad") and k[0] >= 256],
+           "conv3_t_kernel (fwd+dgrad, C<=128: weights x voxels)": [k for k in per if k[1] in ("fwd", "dgrad") and k[0] < 256],
+           "wgrad_umma_kernel (wgrad)": [k for k in per if k[1] == "wgrad"]}
+    fam = {f: ks for f, ks in fam.items() if ks}
     fam_time = {f: sum(sum(per[k]) for k in ks) for f, ks in fam.items()}
     dom = max(fam_time, key=fam_time.get)
     dom_flops = sum(pass_flops(k[0]) * len(per[k]) for k in fam[dom])
     dom_launches = sum(len(per[k]) for k in fam[dom])
     achieved = dom_flops / (fam_time[dom] * 1e-3) / 1e12
     roofline = dict(bound="tensor", kernel=dom, achieved=round(achieved, 2), peak=peaks["bf16"], unit="TFLOP/s",
-                    frac=round(achieved / peaks["bf16"], 4), traffic=None, peak_source=peaks["source"] + " bf16 burst",
-                    avg_launch_ms=round(fam_time[dom] / dom_launches, 4), share_of_step=round(fam_time[dom] / sum(fam_time.values()), 3))
+                    frac=round(achieved / peaks["bf16"], 4), traffic=NCU_TRAFFIC_BYTES.get(dom.split(" ")[0]),
+                    peak_source=peaks["source"] + " cuBLAS bf16 burst", frac_of_nominal_2250=round(achieved / NOMINAL_BF16_TFLOPS, 4),
+                    algorithmic_flops_per_launch=dom_flops / dom_launches,
+                    avg_launch_ms=round(fam_time[dom] / dom_launches, 4),
+                    share_of_step=round(fam_time[dom] / sum(fam_time.values()), 3),
+                    family_shares={f: round(t / sum(fam_time.values()), 3) for f, t in fam_time.items()})
 
     if rank != 0:
         if world > 1:
@@ -317,7 +326,7 @@ def run_gpu(args):
         cpu["value"] = None
         cpu["error"] = str(e)[:200]
 
-    launches_per_C = 1 + 2 + 4     # fwd; dgrad = weight transpose + conv; wgrad = partials + reduce (+ none for bias)
+    launches_per_C = 1 + 2 + 2     # fwd; dgrad = weight transpose + conv; wgrad = split-K kernel + fixed-order reduce
     out = dict(metric="conv3d_tflops", value=round(value, 3), unit="TFLOP/s", n_gpus=world, steps=args.steps,
                warmup=args.warmup, ms_per_step=round(ms / args.steps, 4), higher_is_better=True, scaling="weak",
                vs_baseline=None, dtype="bf16", data="synthetic",
@@ -455,7 +464,7 @@ def run_unet(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="lamp", choices=["lamp", "reference"])
     ap.add_argument("--channels", default=",".join(str(c) for c in CHANNELS))

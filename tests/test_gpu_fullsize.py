@@ -60,7 +60,9 @@ def test_conv_sweep_layer_at_benchmark_size(C):
     ent[:27, 0] = np.arange(27)                      # every tap at least once
     ref = ops.conv3d_wgrad_points(x64, dy64, ent, 3, 1, 1)
     got = host_f64(dw[ent[:, 0], ent[:, 1], ent[:, 2]])
-    assert_close(got, ref, f"C={C} wgrad (sampled)", rel=1e-4, mx=1e-3)
+    # each entry is a 2-million-term sum accumulated in fp32 (TMEM): the stated bar applies, not the
+    # 2e-5 of the short sums in the small-shape tests
+    assert_close(got, ref, f"C={C} wgrad (sampled)")
 
 
 def _ws_view(wsb, layout):
@@ -131,7 +133,7 @@ def test_standard_unet_train_step_at_full_size_sampled():
             ref = ops.conv3d_wgrad_points(x_in, dy_gpu, ent, 3, s, 1)
             wo = offs[i][0]
             got = gw_h[wo:wo + wl[i].size].reshape(wl[i].shape)[ent[:, 0], ent[:, 1], ent[:, 2]]
-            assert_close(got, ref, f"{name} dw (sampled)", rel=2e-4, mx=2e-3)
+            assert_close(got, ref, f"{name} dw (sampled)")
         else:
             u_gpu = _ws_view(wsb, lay_of(i, B.T_OUT))
             _, Do, Ho, Wo, _ = u_gpu.shape
