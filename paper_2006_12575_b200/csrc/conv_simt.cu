@@ -345,21 +345,33 @@ conv_c1_wgrad_kernel(ConvGeom g, const bf16 *__restrict__ x, int64_t xp, const b
     for (int i = 0; i < CPL; ++i)
 #pragma unroll
         for (int t = 0; t < 27; ++t) acc[i][t] = 0.f;
-    for (int64_t v = v0 + warp; v < v1; v += NWARP) {
-        const int iw = (int)(v % g.w), ih = (int)((v / g.w) % g.h), id = (int)((v / ((int64_t)g.w * g.h)) % g.d);
-        const int64_t nb = v - (((int64_t)id * g.h + ih) * g.w + iw);      // voxel index of (n, 0, 0, 0)
+    // each warp walks a contiguous run of voxels, keeping (d, h, w) incrementally
+    const int64_t per_warp = (v1 - v0 + NWARP - 1) / NWARP;
+    const int64_t wv0 = v0 + warp * per_warp, wv1 = min(v1, wv0 + per_warp);
+    int iw = 0, ih = 0, id = 0;
+    if (wv0 < wv1) {
+        iw = (int)(wv0 % g.w);
+        ih = (int)((wv0 / g.w) % g.h);
+        id = (int)((wv0 / ((int64_t)g.w * g.h)) % g.d);
+    }
+    const int64_t sh = (int64_t)g.w * xp, sd = (int64_t)g.w * g.h * xp;
+    for (int64_t v = wv0; v < wv1; ++v) {
+        const bool vd[3] = {id > 0, true, id < g.d - 1};
+        const bool vh[3] = {ih > 0, true, ih < g.h - 1};
+        const bool vw[3] = {iw > 0, true, iw < g.w - 1};
+        const bf16 *xc = x + v * xp;
         float gy[CPL];
 #pragma unroll
         for (int i = 0; i < CPL; ++i) gy[i] = (i * 32 + lane < CO) ? bf2f(dy[v * dyp + i * 32 + lane]) : 0.f;
 #pragma unroll
         for (int t = 0; t < 27; ++t) {
-            const int zd = id + t / 9 - 1, zh = ih + (t / 3) % 3 - 1, zw = iw + t % 3 - 1;
+            const int kd = t / 9, kh = (t / 3) % 3, kw = t % 3;
             float xv = 0.f;
-            if (zd >= 0 && zd < g.d && zh >= 0 && zh < g.h && zw >= 0 && zw < g.w)
-                xv = bf2f(x[(nb + ((int64_t)zd * g.h + zh) * g.w + zw) * xp]);
+            if (vd[kd] && vh[kh] && vw[kw]) xv = bf2f(xc[(kd - 1) * sd + (kh - 1) * sh + (kw - 1) * xp]);
 #pragma unroll
             for (int i = 0; i < CPL; ++i) acc[i][t] = fmaf(gy[i], xv, acc[i][t]);
         }
+        if (++iw == g.w) { iw = 0; if (++ih == g.h) { ih = 0; if (++id == g.d) id = 0; } }
     }
 #pragma unroll
     for (int i = 0; i < CPL; ++i)

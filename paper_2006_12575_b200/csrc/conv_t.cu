@@ -335,7 +335,7 @@ bool make_ct_plan(const ConvGeom &g, CtPlan *out)
     P.plane_bytes = (int)align_up((size_t)HALO_W * HALO_H * rowb, 1024);
     const int w_bytes = 128 * rowb;
     const int budget = SMEM_LIMIT - 1024 - EPI_BYTES - CTRL_BYTES;
-    int np = KC == 64 ? 3 : 4;
+    int np = KC == 64 ? 2 : 4;
     int nw = (budget - np * P.plane_bytes) / w_bytes;
     if (nw > MAX_NW) nw = MAX_NW;
     if (nw < 3) return false;

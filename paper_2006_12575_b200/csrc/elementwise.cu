@@ -21,27 +21,32 @@ __global__ void finalize_stats_kernel(const double *__restrict__ stats, float *_
     mr[2 * i + 1] = (float)(1.0 / sqrt(var + (double)eps));
 }
 
-// thread = (voxel, group of 8 channels)
+// thread = (voxel row r of the block, group g of 8 channels); the per-channel constants stay in registers
+// while the thread walks its voxels
 __global__ void __launch_bounds__(256)
 instnorm_relu_fwd_kernel(const bf16 *__restrict__ y, int64_t yp, const float *__restrict__ mr,
-                         bf16 *__restrict__ z, int64_t zp, int64_t Vn, int C)
+                         bf16 *__restrict__ z, int64_t zp, int64_t Vn, int C, int64_t v_per_block)
 {
-    const int G = C >> 3;
-    const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;
-    if (e >= Vn * G) return;
+    const int G = C >> 3, RB = 256 / G;
+    const int g = threadIdx.x % G, r = threadIdx.x / G;
+    if (r >= RB) return;
     const int n = blockIdx.y;
-    const int g = (int)(e % G);
-    const int64_t v = (int64_t)n * Vn + e / G;
-    float f[8];
-    unpack8(__ldg(reinterpret_cast<const uint4 *>(y + v * yp + g * 8)), f);
-    const float4 *m = reinterpret_cast<const float4 *>(mr + ((int64_t)n * C + g * 8) * 2);
+    float mu[8], rs[8];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const float4 q = __ldg(m + j);          // mu0 rstd0 mu1 rstd1
-        f[2 * j]     = fmaxf((f[2 * j] - q.x) * q.y, 0.f);
-        f[2 * j + 1] = fmaxf((f[2 * j + 1] - q.z) * q.w, 0.f);
+    for (int j = 0; j < 8; ++j) {
+        mu[j] = mr[((int64_t)n * C + g * 8 + j) * 2];
+        rs[j] = mr[((int64_t)n * C + g * 8 + j) * 2 + 1];
     }
-    *reinterpret_cast<uint4 *>(z + v * zp + g * 8) = pack8(f);
+    const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = min(Vn, v0 + v_per_block);
+#pragma unroll 4
+    for (int64_t vv = v0 + r; vv < v1; vv += RB) {
+        const int64_t v = (int64_t)n * Vn + vv;
+        float f[8];
+        unpack8(__ldg(reinterpret_cast<const uint4 *>(y + v * yp + g * 8)), f);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) f[j] = fmaxf((f[j] - mu[j]) * rs[j], 0.f);
+        *reinterpret_cast<uint4 *>(z + v * zp + g * 8) = pack8(f);
+    }
 }
 
 // ------------------------------------------------------------------ InstanceNorm backward
@@ -101,38 +106,48 @@ instnorm_bwd_sums_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *_
     }
 }
 
-// pass 2: dy = rstd * (g - m1 - xhat * m2)
+// pass 2: dy = rstd * (g - m1 - xhat * m2); same thread layout as the forward kernel
 __global__ void __launch_bounds__(256)
 instnorm_bwd_apply_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *__restrict__ dzb, int64_t bp,
                           const bf16 *__restrict__ y, int64_t yp, const float *__restrict__ mr,
-                          const double *__restrict__ sums, bf16 *__restrict__ dy, int64_t dp, int64_t Vn, int C)
+                          const double *__restrict__ sums, bf16 *__restrict__ dy, int64_t dp, int64_t Vn, int C,
+                          int64_t v_per_block)
 {
-    const int G = C >> 3;
-    const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;
-    if (e >= Vn * G) return;
+    const int G = C >> 3, RB = 256 / G;
+    const int g = threadIdx.x % G, r = threadIdx.x / G;
+    if (r >= RB) return;
     const int n = blockIdx.y;
-    const int g = (int)(e % G);
-    const int64_t v = (int64_t)n * Vn + e / G;
     const float inv_v = 1.0f / (float)Vn;
-    float fy[8], fa[8];
-    unpack8(__ldg(reinterpret_cast<const uint4 *>(y + v * yp + g * 8)), fy);
-    unpack8(__ldg(reinterpret_cast<const uint4 *>(dza + v * ap + g * 8)), fa);
-    if (dzb) {
-        float fb[8];
-        unpack8(__ldg(reinterpret_cast<const uint4 *>(dzb + v * bp + g * 8)), fb);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) fa[j] += fb[j];
-    }
+    float mu[8], rs[8], m1[8], m2[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int64_t i = (int64_t)n * C + g * 8 + j;
-        const float mu = mr[2 * i], rs = mr[2 * i + 1];
-        const float m1 = (float)sums[2 * i] * inv_v, m2 = (float)sums[2 * i + 1] * inv_v;
-        const float xh = (fy[j] - mu) * rs;
-        const float gg = xh > 0.f ? fa[j] : 0.f;
-        fa[j] = rs * (gg - m1 - xh * m2);
+        mu[j] = mr[2 * i];
+        rs[j] = mr[2 * i + 1];
+        m1[j] = (float)sums[2 * i] * inv_v;
+        m2[j] = (float)sums[2 * i + 1] * inv_v;
     }
-    *reinterpret_cast<uint4 *>(dy + v * dp + g * 8) = pack8(fa);
+    const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = min(Vn, v0 + v_per_block);
+#pragma unroll 2
+    for (int64_t vv = v0 + r; vv < v1; vv += RB) {
+        const int64_t v = (int64_t)n * Vn + vv;
+        float fy[8], fa[8];
+        unpack8(__ldg(reinterpret_cast<const uint4 *>(y + v * yp + g * 8)), fy);
+        unpack8(__ldg(reinterpret_cast<const uint4 *>(dza + v * ap + g * 8)), fa);
+        if (dzb) {
+            float fb[8];
+            unpack8(__ldg(reinterpret_cast<const uint4 *>(dzb + v * bp + g * 8)), fb);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) fa[j] += fb[j];
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float xh = (fy[j] - mu[j]) * rs[j];
+            const float gg = xh > 0.f ? fa[j] : 0.f;
+            fa[j] = rs[j] * (gg - m1[j] - xh * m2[j]);
+        }
+        *reinterpret_cast<uint4 *>(dy + v * dp + g * 8) = pack8(fa);
+    }
 }
 
 // ------------------------------------------------------------------ head: 1x1x1 conv + softmax (+ Dice sums)
@@ -462,8 +477,10 @@ lamp_status_t k_instnorm_relu_fwd(const TView &y, const float *mu_rstd, const TV
 {
     const int64_t Vn = (int64_t)y.d * y.h * y.w;
     if (Vn == 0 || y.n == 0) return LAMP_OK;
-    dim3 grid((unsigned)((Vn * (y.c / 8) + 255) / 256), y.n);
-    instnorm_relu_fwd_kernel<<<grid, 256, 0, st>>>((const bf16 *)y.p, y.pitch, mu_rstd, (bf16 *)z.p, z.pitch, Vn, y.c);
+    if (y.c / 8 > 256) return LAMP_ERR_UNSUPPORTED;
+    const int64_t vpb = (int64_t)(256 / (y.c / 8)) * 8;
+    dim3 grid((unsigned)((Vn + vpb - 1) / vpb), y.n);
+    instnorm_relu_fwd_kernel<<<grid, 256, 0, st>>>((const bf16 *)y.p, y.pitch, mu_rstd, (bf16 *)z.p, z.pitch, Vn, y.c, vpb);
     return launch_status();
 }
 
@@ -485,10 +502,11 @@ lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TVie
     instnorm_bwd_sums_kernel<<<dim3((unsigned)blocks, y.n), 256, smem, st>>>(
         (const bf16 *)dza.p, dza.pitch, dzb ? (const bf16 *)dzb->p : nullptr, dzb ? dzb->pitch : 0,
         (const bf16 *)y.p, y.pitch, mu_rstd, sums, Vn, C, vpb);
-    dim3 grid((unsigned)((Vn * G + 255) / 256), y.n);
+    const int64_t vpa = (int64_t)RB * 8;
+    dim3 grid((unsigned)((Vn + vpa - 1) / vpa), y.n);
     instnorm_bwd_apply_kernel<<<grid, 256, 0, st>>>(
         (const bf16 *)dza.p, dza.pitch, dzb ? (const bf16 *)dzb->p : nullptr, dzb ? dzb->pitch : 0,
-        (const bf16 *)y.p, y.pitch, mu_rstd, sums, (bf16 *)dy.p, dy.pitch, Vn, C);
+        (const bf16 *)y.p, y.pitch, mu_rstd, sums, (bf16 *)dy.p, dy.pitch, Vn, C, vpa);
     return launch_status();
 }
 
