@@ -90,7 +90,9 @@ size_t conv_ws_bytes(const ConvGeom &g, int pass)
 {
     if (pass == LAMP_PASS_DGRAD) return dgrad_on_tensor_cores(g) ? umma_dgrad_ws(g) : 0;
     if (pass == LAMP_PASS_WGRAD) {
-        const size_t u = umma_wgrad_ws(g);       // 0 when the tensor-core kernel does not take this shape
+        size_t u = umma_wgrad_ws(g);             // 0 when the tensor-core kernels do not take this shape
+        const size_t u2 = win_wgrad_ws(g);
+        if (u2 > u) u = u2;
         const size_t tc = u ? u + bias_grad_ws((int64_t)g.n * g.od * g.oh * g.ow, g.co) : 0;
         const size_t sm = simt_conv_wgrad_ws(g);
         return tc > sm ? tc : sm;
@@ -130,6 +132,13 @@ lamp_status_t conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w, cons
 lamp_status_t conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, float *db, void *ws,
                          size_t ws_bytes, cudaStream_t st)
 {
+    if (win_wgrad_supported(g, x, dy)) {
+        const size_t u = win_wgrad_ws(g);
+        if (!ws || ws_bytes < u + (db ? bias_grad_ws((int64_t)g.n * g.od * g.oh * g.ow, g.co) : 0)) return LAMP_ERR_WORKSPACE;
+        lamp_status_t s = win_wgrad(g, x, dy, dw, ws, u, st);
+        if (s != LAMP_OK || !db) return s;
+        return bias_grad(dy, db, (char *)ws + u, st);
+    }
     if (umma_wgrad_supported(g, x, dy)) {
         const size_t u = umma_wgrad_ws(g);
         if (!ws || ws_bytes < u + (db ? bias_grad_ws((int64_t)g.n * g.od * g.oh * g.ow, g.co) : 0)) return LAMP_ERR_WORKSPACE;

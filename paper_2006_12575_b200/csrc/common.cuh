@@ -102,6 +102,12 @@ size_t        umma_wgrad_ws(const ConvGeom &g);
 lamp_status_t umma_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, void *ws, size_t ws_bytes,
                          cudaStream_t st);
 
+// wgrad_win.cu (tcgen05 weight gradient of the 3x3x3 s1 conv with the three kw taps on N; c_in < 256)
+bool          win_wgrad_supported(const ConvGeom &g, const TView &x, const TView &dy);
+size_t        win_wgrad_ws(const ConvGeom &g);
+lamp_status_t win_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, void *ws, size_t ws_bytes,
+                        cudaStream_t st);
+
 // conv_umma.cu (tcgen05 implicit GEMM, voxels x channels form; see the file header for the kinds)
 enum { UK_S1_FWD = 0, UK_S1_DGRAD = 1, UK_S2_FWD = 2, UK_S2_DGRAD = 3, UK_T_FWD = 4, UK_T_DGRAD = 5 };
 bool          umma_conv_supported(int kind, const ConvGeom &g, const TView &a, const TView &y);

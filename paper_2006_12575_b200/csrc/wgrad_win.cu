@@ -1,0 +1,378 @@
+// Weight gradient of the 3x3x3 stride-1 pad-1 convolution with N = 3 x 64 columns per MMA.
+//
+//   dw[kd,kh,kw][co][ci] = sum_u dy[u - (kd-1, kh-1, 0)][co] * x[u + (0, 0, kw-1)][ci]
+//
+// One tcgen05.mma (M = 128, K = 16) holds the tensor pipe for max(76, N/2) cycles, so the plain kernel
+// (wgrad_umma.cu, N = c_in) runs a 64-channel layer at 42 % of the full rate.  Here the three kw taps
+// sit side by side on N: the B operand is ONE x halo box (10 (w) x 16 (h) voxels x 64 channels, rows =
+// voxels, MN-major) read through a descriptor whose three 64-channel blocks are the windows starting
+// 0, 1 and 2 rows in (leading-dimension offset = one row, 8-voxel groups 10 rows apart).  N = 192 costs
+// 96 cycles: the full rate.  The A operand is a window of a dy halo box (8 (w) x 18 (h) voxels of plane
+// d + 1 - kd): it starts (2 - kh) lines in; for c_out = 64 (32) the 128 rows hold two (four) windows one
+// line apart, i.e. two (three) kh taps per MMA.  Out-of-volume voxels are zero-filled by TMA (the
+// conv's zero padding).  The swizzle is a function of the shared-memory address bits, so windows that
+// start off the swizzle-atom boundary read exactly what TMA wrote.
+//
+// A CTA keeps two accumulators (128 x 192 fp32 each) in TMEM while it sweeps its share of the
+// 8 x 16-voxel tiles (split-K over CTAs); partial sums go to scratch and are added in a fixed order.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include "common.cuh"
+#include "umma_ptx.cuh"
+
+namespace lamp {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int WW_THREADS = 192;
+constexpr int TWW = 8, THH = 16;                   // tile: 8 (w) x 16 (h) voxels of one plane = K = 128
+constexpr int XW = TWW + 2;                        // x box: w halo only
+constexpr int DYH = THH + 2;                       // dy box: h halo only
+constexpr int MAX_ST = 5;
+
+struct WwParams {
+    int32_t N, D, H, W;
+    int32_t nwt, nht, ntiles;
+    int32_t co, ci;
+    int32_t cob;             // c_out channels per window inside an M block: min(co, 128)
+    int32_t nmb;             // M blocks: 3 kd x (per-kd blocks) x (co / 128 or 1)
+    int32_t mb_per_kd;       // cob = 128: 3 * (co / 128); cob = 64: 2; cob = 32: 1
+    int32_t ncx;             // c_in chunks (of 64, or one of 32)
+    int32_t pair_cx;         // 1: a set = one M block x two c_in chunks; 0: a set = two M blocks x the one chunk
+    int32_t nsets, nsplit, nunits;
+    int32_t nst;             // pipeline stages
+    int32_t ndy;             // dy buffers per stage (2 where the two accumulators of a set can need different planes)
+    int32_t dy_bytes, x_bytes, stage_bytes;
+    int64_t entries;
+    float  *part;
+    int    *status;
+};
+
+struct Acc { int kd, ls0, nvalid, cc, cx; bool live; };
+
+// accumulator a (0 or 1) of a set
+__device__ __forceinline__ Acc decode_acc(const WwParams &P, int set, int a)
+{
+    Acc r;
+    int mb, cx;
+    if (P.pair_cx) { mb = set / (P.ncx / 2); cx = (set % (P.ncx / 2)) * 2 + a; }
+    else           { mb = set * 2 + a; cx = 0; }
+    r.live = mb < P.nmb;
+    if (!r.live) mb = P.nmb - 1;
+    r.cx = cx;
+    r.kd = mb / P.mb_per_kd;
+    const int j = mb % P.mb_per_kd;
+    if (P.cob >= 128)     { const int kh = j % 3; r.cc = j / 3; r.ls0 = 2 - kh; r.nvalid = 1; }
+    else if (P.cob == 64) { r.cc = 0; r.ls0 = j == 0 ? 1 : 0; r.nvalid = j == 0 ? 2 : 1; }
+    else                  { r.cc = 0; r.ls0 = 0; r.nvalid = 3; }
+    return r;
+}
+
+// CBA / CBB: channels per TMA box of dy / x (64: 128-byte swizzle, 32: 64-byte swizzle)
+template <int CBA, int CBB>
+__global__ void __launch_bounds__(WW_THREADS, 1)
+wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_dy, const WwParams P)
+{
+    constexpr uint32_t SWA = CBA == 64 ? 2u : 4u, SWB = CBB == 64 ? 2u : 4u;
+    constexpr uint32_t ROWA = CBA * 2, ROWB = CBB * 2;
+    constexpr uint32_t LINE_A = TWW * ROWA;                     // one h-line of the dy box = one 8-row group
+    constexpr uint32_t DYBOX = TWW * DYH * ROWA, XBOX = XW * THH * ROWB;
+    constexpr int NCOL = 3 * CBB;                               // 192 or 96
+    constexpr uint32_t IDESC = make_idesc(NCOL, 1, 1);
+    constexpr int ACC_COLS = 256;                               // TMEM column stride between the two accumulators
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = (uint64_t *)(smem + (size_t)P.nst * P.stage_bytes);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + MAX_ST);
+    const uint32_t done_bar = smem_u32(bars + 2 * MAX_ST), drained_bar = smem_u32(bars + 2 * MAX_ST + 1);
+    uint32_t *tmem_slot = (uint32_t *)(bars + 2 * MAX_ST + 2);
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MAX_ST; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        mbar_init(done_bar, 1);
+        mbar_init(drained_bar, 4);
+        *abort_flag = 0;
+        mbar_init_fence();
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const int aboxes = P.cob >= 128 ? 2 : 1;                    // dy boxes per plane (64 channels each, or one of 32)
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---------------------------------------------------------------- TMA producer
+            int st = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int unit = blockIdx.x; unit < P.nunits && ok; unit += gridDim.x) {
+                const int set = unit / P.nsplit, split = unit - set * P.nsplit;
+                const Acc a0 = decode_acc(P, set, 0), a1 = decode_acc(P, set, 1);
+                const bool two_dy = P.ndy == 2 && (a1.kd != a0.kd || a1.cc != a0.cc);
+                const bool two_x = P.pair_cx;
+                const uint32_t bytes = (two_dy ? 2 : 1) * aboxes * DYBOX + (two_x ? 2 : 1) * XBOX;
+                for (int tile = split; tile < P.ntiles && ok; tile += P.nsplit) {
+                    int t = tile;
+                    const int w0 = (t % P.nwt) * TWW; t /= P.nwt;
+                    const int h0 = (t % P.nht) * THH; t /= P.nht;
+                    const int d = t % P.D;
+                    const int n = t / P.D;
+                    if (!mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag)) { ok = false; break; }
+                    mbar_expect_tx(full0 + 8 * st, bytes);
+                    const uint32_t sb = smem_u32(smem + (size_t)st * P.stage_bytes);
+                    for (int q = 0; q < (two_dy ? 2 : 1); ++q) {
+                        const Acc &a = q ? a1 : a0;
+                        for (int b = 0; b < aboxes; ++b)
+                            tma_load_5d(sb + q * P.dy_bytes + b * DYBOX, &map_dy, full0 + 8 * st, a.cc * 128 + b * 64, w0, h0 - 1,
+                                        d + 1 - a.kd, n);
+                    }
+                    for (int q = 0; q < (two_x ? 2 : 1); ++q)
+                        tma_load_5d(sb + P.ndy * P.dy_bytes + q * P.x_bytes, &map_x, full0 + 8 * st, (q ? a1.cx : a0.cx) * CBB, w0 - 1, h0, d, n);
+                    if (++st == P.nst) { st = 0; ph ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---------------------------------------------------------------- MMA issuer
+            int st = 0;
+            uint32_t ph = 0, uph = 0;
+            bool ok = true;
+            for (int unit = blockIdx.x; unit < P.nunits && ok; unit += gridDim.x) {
+                const int set = unit / P.nsplit, split = unit - set * P.nsplit;
+                const Acc a0 = decode_acc(P, set, 0), a1 = decode_acc(P, set, 1);
+                const bool two_dy = P.ndy == 2 && (a1.kd != a0.kd || a1.cc != a0.cc);
+                if (!mbar_wait(drained_bar, uph ^ 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                uint32_t accumulate = 0;
+                for (int tile = split; tile < P.ntiles && ok; tile += P.nsplit) {
+                    if (!mbar_wait(full0 + 8 * st, ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sb = smem_u32(smem + (size_t)st * P.stage_bytes);
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        const Acc &a = q ? a1 : a0;
+                        if (!a.live) continue;
+                        const uint32_t dyb = sb + ((q && two_dy) ? P.dy_bytes : 0) + a.ls0 * LINE_A;
+                        const uint32_t xb = sb + P.ndy * P.dy_bytes + ((q && P.pair_cx) ? P.x_bytes : 0);
+                        // A: blocks of 64 (32) rows = c_out channels of one window; next block = next 64 channels of
+                        // the same window (cob = 128: next box) or the window one line further down (cob < 128)
+                        const uint64_t da = make_desc(dyb, P.cob >= 128 ? DYBOX : LINE_A, LINE_A, SWA);
+                        // B: three blocks = the windows kw = 0, 1, 2 (one row apart); 8-voxel groups 10 rows apart
+                        const uint64_t db = make_desc(xb, ROWB, XW * ROWB, SWB);
+                        const uint32_t d_tmem = tmem_base + q * ACC_COLS;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)     // 16 voxels = two h-lines per MMA
+                            umma_bf16(d_tmem, da + (uint64_t)(j * ((2 * LINE_A) >> 4)), db + (uint64_t)(j * ((2 * XW * ROWB) >> 4)), IDESC,
+                                      (accumulate | j) ? 1u : 0u);
+                    }
+                    umma_commit(empty0 + 8 * st);
+                    if (++st == P.nst) { st = 0; ph ^= 1; }
+                    accumulate = 1;
+                }
+                if (!ok) break;
+                umma_commit(done_bar);
+                uph ^= 1;
+            }
+        }
+    } else {
+        // -------------------------------------------------------------------- epilogue (warps 2..5)
+        const int q4 = warp & 3;
+        uint32_t uph = 0;
+        bool ok = true;
+        for (int unit = blockIdx.x; unit < P.nunits && ok; unit += gridDim.x) {
+            const int set = unit / P.nsplit, split = unit - set * P.nsplit;
+            ok = __all_sync(0xffffffffu, mbar_wait(done_bar, uph, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            const int m = q4 * 32 + lane;
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const Acc a = decode_acc(P, set, q);
+                const int rows_per_win = P.cob >= 128 ? 128 : P.cob;
+                const int b = m / rows_per_win;                     // window index inside the M block
+                const int kh = 2 - (a.ls0 + b);
+                const bool row_ok = a.live && b < a.nvalid;
+                const int co = a.cc * 128 + m % rows_per_win;
+                const uint32_t trow = tmem_base + ((uint32_t)(q4 * 32) << 16) + q * ACC_COLS;
+#pragma unroll
+                for (int c0 = 0; c0 < NCOL; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld32(trow + c0, r);
+                    tmem_ld_wait();
+                    if (row_ok) {
+                        const int kw = c0 / CBB, ci = a.cx * CBB + c0 % CBB;
+                        const int tap = (a.kd * 3 + kh) * 3 + kw;
+                        float4 *d4 = reinterpret_cast<float4 *>(P.part + (int64_t)split * P.entries +
+                                                                ((int64_t)tap * P.co + co) * P.ci + ci);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            d4[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                                __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(drained_bar);
+            uph ^= 1;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0 && P.status) atomicExch(P.status, (int)LAMP_ERR_TIMEOUT);
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) { }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 get_encode()
+{
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (PFN_cuTensorMapEncodeTiled_v12000)p;
+    }
+    return fn;
+}
+
+bool encode_box(PFN_cuTensorMapEncodeTiled_v12000 encode, CUtensorMap *m, const TView &t, int box_c, int bw, int bh)
+{
+    const cuuint64_t dims[5] = {(cuuint64_t)t.c, (cuuint64_t)t.w, (cuuint64_t)t.h, (cuuint64_t)t.d, (cuuint64_t)t.n};
+    const cuuint64_t strides[4] = {(cuuint64_t)t.pitch * 2, (cuuint64_t)t.pitch * 2 * t.w, (cuuint64_t)t.pitch * 2 * t.w * t.h,
+                                   (cuuint64_t)t.pitch * 2 * t.w * t.h * t.d};
+    const cuuint32_t box[5] = {(cuuint32_t)box_c, (cuuint32_t)bw, (cuuint32_t)bh, 1, 1};
+    const cuuint32_t es[5] = {1, 1, 1, 1, 1};
+    return encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, t.p, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  box_c == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct WwPlan { WwParams P; int CBA, CBB; size_t smem; int grid; };
+
+bool make_ww_plan(const ConvGeom &g, WwPlan *out)
+{
+    if (!(g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed)) return false;
+    if (!(g.co == 32 || g.co == 64 || g.co % 128 == 0)) return false;
+    int ncx, CBB;
+    if (g.ci == 32) { ncx = 1; CBB = 32; }
+    else if (g.ci == 64) { ncx = 1; CBB = 64; }
+    else if (g.ci % 128 == 0) { ncx = g.ci / 64; CBB = 64; }
+    else return false;
+    // the fixed 8 x 16 tile must not be mostly padding (small or thin volumes go to the plain kernel)
+    const int nwt = (g.w + TWW - 1) / TWW, nht = (g.h + THH - 1) / THH;
+    if ((double)g.h * g.w < 0.6 * (double)nwt * TWW * nht * THH) return false;
+    WwParams &P = out->P;
+    P.N = g.n; P.D = g.d; P.H = g.h; P.W = g.w;
+    P.nwt = nwt; P.nht = nht;
+    const int64_t nt = (int64_t)g.n * g.d * nht * nwt;
+    if (nt > 0x7FFFFFFF || nt <= 0) return false;
+    P.ntiles = (int32_t)nt;
+    P.co = g.co; P.ci = g.ci;
+    P.cob = g.co < 128 ? g.co : 128;
+    P.mb_per_kd = P.cob >= 128 ? 3 * (g.co / 128) : (P.cob == 64 ? 2 : 1);
+    P.nmb = 3 * P.mb_per_kd;
+    P.ncx = ncx;
+    P.pair_cx = ncx >= 2;
+    P.nsets = P.pair_cx ? P.nmb * (ncx / 2) : (P.nmb + 1) / 2;
+    const int CBA = g.co == 32 ? 32 : 64;
+    const int aboxes = P.cob >= 128 ? 2 : 1;
+    // one extra h-line behind the dy box: the fourth (unused) window of a 32-channel block reads it
+    P.dy_bytes = (int)align_up((size_t)aboxes * TWW * DYH * CBA * 2 + TWW * CBA * 2, 1024);
+    P.x_bytes = (int)align_up((size_t)XW * THH * CBB * 2, 1024);
+    P.ndy = (P.pair_cx || P.mb_per_kd % 2 == 0) ? 1 : 2;
+    P.stage_bytes = P.ndy * P.dy_bytes + (P.pair_cx ? 2 : 1) * P.x_bytes;
+    const int budget = 227 * 1024 - 1024 - 1024;
+    int nst = budget / P.stage_bytes;
+    if (nst > MAX_ST) nst = MAX_ST;
+    if (nst < 2) return false;
+    P.nst = nst;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int nsplit = sms / P.nsets;
+    if (nsplit < 1) nsplit = 1;
+    if (nsplit > P.ntiles) nsplit = P.ntiles;
+    P.nsplit = nsplit;
+    P.nunits = P.nsets * nsplit;
+    P.entries = (int64_t)27 * g.co * g.ci;
+    out->CBA = CBA; out->CBB = CBB;
+    out->smem = 1024 + (size_t)nst * P.stage_bytes + 1024;
+    out->grid = P.nunits < sms ? P.nunits : sms;
+    return true;
+}
+
+template <int CBA, int CBB>
+lamp_status_t launch_ww(const CUtensorMap &mx, const CUtensorMap &mdy, const WwPlan &pl, cudaStream_t st)
+{
+    static bool attr = false;
+    if (!attr) {
+        LAMP_CUDA_OK(cudaFuncSetAttribute(wgrad_win_kernel<CBA, CBB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr = true;
+    }
+    wgrad_win_kernel<CBA, CBB><<<pl.grid, WW_THREADS, pl.smem, st>>>(mx, mdy, pl.P);
+    return launch_status();
+}
+
+}  // namespace
+
+bool win_wgrad_supported(const ConvGeom &g, const TView &x, const TView &dy)
+{
+    WwPlan pl;
+    if ((int64_t)g.n * g.d * g.h * g.w == 0) return false;
+    if (g.ci >= 256) return false;                     // N = c_in = 256 already runs at the full rate in the plain kernel
+    if (!make_ww_plan(g, &pl)) return false;
+    if (x.pitch % 8 || dy.pitch % 8 || ((uintptr_t)x.p & 15) || ((uintptr_t)dy.p & 15)) return false;
+    return true;
+}
+
+size_t win_wgrad_ws(const ConvGeom &g)
+{
+    WwPlan pl;
+    if (g.ci >= 256 || !make_ww_plan(g, &pl)) return 0;
+    return align_up((size_t)pl.P.nsplit * pl.P.entries * sizeof(float), 256);
+}
+
+lamp_status_t win_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, void *ws, size_t ws_bytes,
+                        cudaStream_t st)
+{
+    WwPlan pl;
+    if (!make_ww_plan(g, &pl)) return LAMP_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < win_wgrad_ws(g)) return LAMP_ERR_WORKSPACE;
+    PFN_cuTensorMapEncodeTiled_v12000 encode = get_encode();
+    if (!encode) return LAMP_ERR_CUDA;
+    const bool direct = pl.P.nsplit == 1;
+    pl.P.part = direct ? dw : (float *)ws;
+    pl.P.status = status_word_ptr();
+    CUtensorMap mx, mdy;
+    if (!encode_box(encode, &mx, x, pl.CBB, XW, THH)) return LAMP_ERR_CUDA;
+    if (!encode_box(encode, &mdy, dy, pl.CBA, TWW, DYH)) return LAMP_ERR_CUDA;
+    lamp_status_t s;
+    if (pl.CBA == 64 && pl.CBB == 64) s = launch_ww<64, 64>(mx, mdy, pl, st);
+    else if (pl.CBA == 64 && pl.CBB == 32) s = launch_ww<64, 32>(mx, mdy, pl, st);
+    else if (pl.CBA == 32 && pl.CBB == 64) s = launch_ww<32, 64>(mx, mdy, pl, st);
+    else s = launch_ww<32, 32>(mx, mdy, pl, st);
+    if (s != LAMP_OK || direct) return s;
+    return reduce_partials(pl.P.part, pl.P.entries, pl.P.nsplit, dw, st);
+}
+
+}  // namespace lamp
