@@ -1,4 +1,4 @@
-// 3x3x3 stride-1 pad-1 convolution for c_out blocks of at most 128 channels: "weights x voxels"
+// 3x3x3 stride-1 pad-1 convolution, c_out in blocks of at most 128 channels: "weights x voxels"
 // implicit GEMM with the activation planes resident in shared memory.
 //
 // Why this shape.  One tcgen05.mma (M = 128, K = 16, bf16) occupies the tensor pipe for max(76, N/2)
@@ -375,7 +375,6 @@ bool ct_conv_fwd_supported(const ConvGeom &g, const TView &x, const TView &y)
 {
     CtPlan pl;
     if ((int64_t)g.n * g.d * g.h * g.w == 0) return false;
-    if (g.co > 128) return false;                              // wide layers: N = c_out already fills the tensor pipe
     if (!make_ct_plan(g, &pl)) return false;
     // the 8 x 32 window must not be mostly padding
     const double used = (double)g.h * g.w / ((double)pl.P.nht * TH * pl.P.nwt * TW);

@@ -339,7 +339,6 @@ bool win_wgrad_supported(const ConvGeom &g, const TView &x, const TView &dy)
 {
     WwPlan pl;
     if ((int64_t)g.n * g.d * g.h * g.w == 0) return false;
-    if (g.ci >= 256) return false;                     // N = c_in = 256 already runs at the full rate in the plain kernel
     if (!make_ww_plan(g, &pl)) return false;
     if (x.pitch % 8 || dy.pitch % 8 || ((uintptr_t)x.p & 15) || ((uintptr_t)dy.p & 15)) return false;
     return true;
@@ -348,7 +347,7 @@ bool win_wgrad_supported(const ConvGeom &g, const TView &x, const TView &dy)
 size_t win_wgrad_ws(const ConvGeom &g)
 {
     WwPlan pl;
-    if (g.ci >= 256 || !make_ww_plan(g, &pl)) return 0;
+    if (!make_ww_plan(g, &pl)) return 0;
     return align_up((size_t)pl.P.nsplit * pl.P.entries * sizeof(float), 256);
 }
 

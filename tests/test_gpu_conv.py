@@ -42,6 +42,9 @@ CASES = [
     ("t_c128_to_64", 1, 3, 36, 10, 128, 64, 3, 1, 1, 0),
     ("t_c32_to_128", 1, 4, 34, 9, 32, 128, 3, 1, 1, 0),
     ("t_single_plane", 1, 1, 32, 8, 64, 64, 3, 1, 1, 0),
+    ("t_c256_h32", 1, 3, 32, 8, 256, 256, 3, 1, 1, 0),
+    ("t_c512_to_256", 1, 2, 32, 8, 512, 256, 3, 1, 1, 0),
+    ("t_c128_to_384", 1, 2, 30, 16, 128, 384, 3, 1, 1, 0),
     ("tiny_volume", 1, 2, 2, 2, 64, 64, 3, 1, 1, 0),
     ("single_voxel", 1, 1, 1, 1, 32, 32, 3, 1, 1, 0),
 ]
