@@ -33,7 +33,8 @@ SEED = 2
 NOMINAL_BF16_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture summarised
 # under profiles/ (None: not captured for the kernel as it stands)
-NCU_TRAFFIC_BYTES = {"conv3_umma_kernel": None, "conv3_t_kernel": None, "wgrad_umma_kernel": None}
+NCU_TRAFFIC_BYTES = {"conv3_t_kernel (fwd+dgrad, C=256)": 2.199e9,     # profiles/conv3_t_c256_128cube.txt
+                     "wgrad_win_kernel (wgrad, C=256)": 2.153e9}      # profiles/wgrad_win_c256_128cube.txt
 
 
 def pass_flops(C, vol=VOL):
@@ -293,9 +294,11 @@ def run_gpu(args):
         passes[f"C{C}.{name}"] = dict(ms=round(mean, 4), tflops=round(tf, 1), pct_nominal=round(100 * tf / NOMINAL_BF16_TFLOPS, 1),
                                       pct_measured=round(100 * tf / peaks["bf16"], 1))
     # kernel families (one CUDA kernel template each); the dgrad pass also holds the tiny weight-transpose launch
-    fam = {"conv3_umma_kernel (fwd+dgrad, C>=256: voxels x channels)": [k for k in per if k[1] in ("fwd", "dgrad") and k[0] >= 256],
-           "conv3_t_kernel (fwd+dgrad, C<=128: weights x voxels)": [k for k in per if k[1] in ("fwd", "dgrad") and k[0] < 256],
-           "wgrad_umma_kernel (wgrad)": [k for k in per if k[1] == "wgrad"]}
+    cmax = max(chans)
+    fam = {f"conv3_t_kernel (fwd+dgrad, C={cmax})": [k for k in per if k[1] in ("fwd", "dgrad") and k[0] == cmax],
+           f"conv3_t_kernel (fwd+dgrad, C<{cmax})": [k for k in per if k[1] in ("fwd", "dgrad") and k[0] != cmax],
+           f"wgrad_win_kernel (wgrad, C={cmax})": [k for k in per if k[1] == "wgrad" and k[0] == cmax],
+           f"wgrad_win_kernel (wgrad, C<{cmax})": [k for k in per if k[1] == "wgrad" and k[0] != cmax]}
     fam = {f: ks for f, ks in fam.items() if ks}
     fam_time = {f: sum(sum(per[k]) for k in ks) for f, ks in fam.items()}
     dom = max(fam_time, key=fam_time.get)
@@ -303,7 +306,7 @@ def run_gpu(args):
     dom_launches = sum(len(per[k]) for k in fam[dom])
     achieved = dom_flops / (fam_time[dom] * 1e-3) / 1e12
     roofline = dict(bound="tensor", kernel=dom, achieved=round(achieved, 2), peak=peaks["bf16"], unit="TFLOP/s",
-                    frac=round(achieved / peaks["bf16"], 4), traffic=NCU_TRAFFIC_BYTES.get(dom.split(" ")[0]),
+                    frac=round(achieved / peaks["bf16"], 4), traffic=NCU_TRAFFIC_BYTES.get(dom),
                     peak_source=peaks["source"] + " cuBLAS bf16 burst", frac_of_nominal_2250=round(achieved / NOMINAL_BF16_TFLOPS, 4),
                     algorithmic_flops_per_launch=dom_flops / dom_launches,
                     avg_launch_ms=round(fam_time[dom] / dom_launches, 4),
