@@ -227,3 +227,34 @@ def test_sliding_window_aggregation_properties():
     p0, p1 = fields[0][0, 3, 0, 0], fields[nh * nw][0, 0, 0, 0]
     want = (w[3, 0, 0] * p0 + w[0, 0, 0] * p1) / (w[3, 0, 0] + w[0, 0, 0])
     np.testing.assert_allclose(A[3, 0, 0], want, rtol=1e-13)
+
+
+def test_bf16_storage_chain_amplifies_fp32_level_differences_beyond_1e3():
+    """Why network-level parity is checked step by step: perturb every conv output of the oracle by a
+    relative 1e-7 (the size of an fp32-vs-fp64 accumulation difference) before its bf16 storage rounding.
+    Roundings that flip are 2^-8 relative jumps that spread through 27 taps x all channels per layer, so
+    the oracle's OWN output moves by more than the 1e-3 bar, though far less than the bf16 storage error."""
+    spec = unet.UNetSpec(3, [8, 16, 32], 2, 1, 4)
+    lay = unet.unet_layers(spec)
+    ws = [w.astype(np.float64) for w in synth.kaiming_for_layers([(l.taps, l.c_out, l.c_in, l.fan_in) for l in lay], 1)]
+    bs = [np.zeros(l.c_out) for l in lay]
+    x = synth.bf16_round(synth.blurred_noise((32, 32, 32), 2.0, 0)).astype(np.float64)[None, ..., None]
+    ref = unet.forward(spec, ws, bs, x, quantise=True)
+    full = unet.forward(spec, ws, bs, x, quantise=False)
+    orig = ops.conv3d_fwd
+    rs = np.random.default_rng(0)
+    try:
+        ops.conv3d_fwd = lambda *a, **k: (lambda y: y * (1 + 1e-7 * rs.standard_normal(y.shape)))(orig(*a, **k))
+        pert = unet.forward(spec, ws, bs, x, quantise=True)
+    finally:
+        ops.conv3d_fwd = orig
+    moved = np.linalg.norm(pert - ref) / np.linalg.norm(ref)
+    budget = np.linalg.norm(ref - full) / np.linalg.norm(full)
+    assert 1e-3 < moved < 2 * budget, (moved, budget)
+    # without the storage rounding the same perturbation is harmless
+    try:
+        ops.conv3d_fwd = lambda *a, **k: (lambda y: y * (1 + 1e-7 * rs.standard_normal(y.shape)))(orig(*a, **k))
+        pert_f = unet.forward(spec, ws, bs, x, quantise=False)
+    finally:
+        ops.conv3d_fwd = orig
+    assert np.linalg.norm(pert_f - full) / np.linalg.norm(full) < 1e-5
