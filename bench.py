@@ -270,10 +270,8 @@ def run_gpu(args):
     sync_all()
     e2e_ms = e0.elapsed_time(e1)
 
-    if world > 1:
-        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = float(t[0]), float(t[1])
+    from paper_2006_12575_b200 import replicas
+    ms, e2e_ms = replicas.job_time_ms(ms, dev), replicas.job_time_ms(e2e_ms, dev)       # slowest rank
 
     flops_step = sum(3 * pass_flops(C) for C in chans)
     value = world * flops_step * args.steps / (ms * 1e-3) / 1e12
@@ -464,6 +462,66 @@ def run_unet(args):
     print(json.dumps(out), flush=True)
 
 
+def run_hbm(args):
+    """HBM-bound kernels of the path on their own, through the C ABI: achieved GB/s of algorithmic bytes
+    against the measured copy bandwidth."""
+    import torch
+    from paper_2006_12575_b200 import binding as B
+    from paper_2006_12575_b200 import build as lamp_build
+    lamp_build.build()
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, flush):
+        for _ in range(args.warmup):
+            fn()
+        tot = 0.0
+        for _ in range(args.steps):
+            flush.add_(1)                                # > L2: evicts the previous iteration's lines
+            a, b = ev(), ev()
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            tot += a.elapsed_time(b)
+        return tot / args.steps
+
+    flush = torch.zeros(256 << 20, dtype=torch.uint8, device="cuda")
+    res = {}
+    D = H = W = 128
+    for C in (32, 64):
+        shape = (1, D, H, W, C)
+        y = torch.randn(shape, device="cuda").to(torch.bfloat16)
+        dz = torch.randn(shape, device="cuda").to(torch.bfloat16)
+        z = torch.empty_like(y)
+        dy = torch.empty_like(y)
+        yf = y.float()
+        stats = torch.stack([yf.sum(dim=(1, 2, 3)), (yf * yf).sum(dim=(1, 2, 3))], dim=-1).double().contiguous()
+        mr = torch.empty((1, C, 2), dtype=torch.float32, device="cuda")
+        sums = torch.empty((1, C, 2), dtype=torch.float64, device="cuda")
+        n = y.numel()
+        ms = timed(lambda: B.lamp_instnorm_relu_fwd(y, stats, 1e-5, mr, z), flush)
+        res[f"instnorm_relu_fwd C={C}"] = dict(ms=round(ms, 4), bytes=4 * n, gbs=round(4 * n / ms / 1e6, 1))
+        ms = timed(lambda: B.lamp_instnorm_relu_bwd(dz, None, y, mr, sums, dy), flush)
+        res[f"instnorm_relu_bwd C={C}"] = dict(ms=round(ms, 4), bytes=10 * n, gbs=round(10 * n / ms / 1e6, 1))
+        del y, dz, z, dy, yf
+    # overlap-add on the 512 x 512 x 128 volume: 363 patches of 64^3, K = 10
+    K, P = 10, (64, 64, 64)
+    Dv, Hv, Wv = 512, 512, 128
+    pp = torch.rand((363, 64 ** 3, K), device="cuda")
+    planar = torch.empty((K, Dv, Hv, Wv), dtype=torch.float32, device="cuda")
+    seg = torch.empty(Dv * Hv * Wv, dtype=torch.uint8, device="cuda")
+    nbytes = pp.numel() * 4 + planar.numel() * 4 + seg.numel()
+    ms = timed(lambda: B.lamp_overlap_add(pp, K, Dv, Hv, Wv, P, 0.25, 1, planar, seg), flush)
+    res["overlap_add 512x512x128"] = dict(ms=round(ms, 4), bytes=nbytes, gbs=round(nbytes / ms / 1e6, 1))
+    for v in res.values():
+        v["frac_of_measured_copy"] = round(v["gbs"] / peaks["hbm_gbs"], 3)
+    print(json.dumps(dict(metric="hbm_bound_kernels_gbs", unit="GB/s", peak=peaks["hbm_gbs"], peak_source=peaks["source"],
+                          l2="a 256 MiB buffer is rewritten between timed calls", steps=args.steps, warmup=args.warmup,
+                          kernels=res)), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -471,10 +529,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="lamp", choices=["lamp", "reference"])
     ap.add_argument("--channels", default=",".join(str(c) for c in CHANNELS))
-    ap.add_argument("--workload", default="conv_sweep", choices=["conv_sweep", "unet_train", "unet_infer", "sliding"])
+    ap.add_argument("--workload", default="conv_sweep", choices=["conv_sweep", "unet_train", "unet_infer", "sliding", "hbm"])
     ap.add_argument("--cfg", type=int, default=2)
     ap.add_argument("--sw-batch", type=int, default=8)
     args = ap.parse_args()
+    if args.workload == "hbm":
+        run_hbm(args)
+        return
     if args.workload != "conv_sweep":
         run_unet(args)
         return
