@@ -73,6 +73,7 @@ instnorm_bwd_sums_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *_
         }
         const int64_t v0 = (int64_t)blockIdx.x * v_per_block;
         const int64_t v1 = min(Vn, v0 + v_per_block);
+#pragma unroll 4
         for (int64_t vv = v0 + r; vv < v1; vv += RB) {
             const int64_t v = (int64_t)n * Vn + vv;
             float fy[8], fa[8];
@@ -373,12 +374,15 @@ gather_patches_kernel(const bf16 *__restrict__ vol, int64_t vp, int D, int H, in
 
 // A[k][v] = sum_p w_p(v) p_p[v][k] / sum_p w_p(v) over the patches covering v, ascending patch
 // index; argmax over k (lowest index on ties).  One thread per 4 voxels along W.
-template <int VEC>
+// KT > 0: the class count is a compile-time constant and, where every patch origin and extent along W is a
+// multiple of 4 (aligned4), the 4 voxels x KT probabilities of a patch are read as KT 16-byte vectors.
+template <int VEC, int KT>
 __global__ void __launch_bounds__(256)
-overlap_add_kernel(const float *__restrict__ pp, int K, int D, int H, int W, int PD, int PH, int PW,
-                   int nd, int nh, int nw, int sd, int sh, int sw, int window,
+overlap_add_kernel(const float *__restrict__ pp, int Krt, int D, int H, int W, int PD, int PH, int PW,
+                   int nd, int nh, int nw, int sd, int sh, int sw, int window, int aligned4,
                    float *__restrict__ planar, uint8_t *__restrict__ amax)
 {
+    const int K = KT > 0 ? KT : Krt;
     extern __shared__ float tab[];          // 1-D window factors: [PD] [PH] [PW], each normalised to max 1
     float *td = tab, *th = tab + PD, *tw = th + PH;
     for (int i = threadIdx.x; i < PD + PH + PW; i += 256) {
@@ -419,6 +423,30 @@ overlap_add_kernel(const float *__restrict__ pp, int K, int D, int H, int W, int
                 if (w0 + VEC - 1 < ow || w0 >= ow + PW) continue;
                 const int64_t pi = ((int64_t)id * nh + ih) * nw + iw;
                 const float wdh = td[d - od] * th[h - oh];
+                if (VEC == 4 && KT > 0 && aligned4) {
+                    // origins and extents are multiples of 4: the four voxels lie inside the patch together
+                    float wt[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        wt[i] = wdh * tw[w0 + i - ow];
+                        if (window) wt[i] = fmaxf(wt[i], 1e-3f);
+                        wsum[i] += wt[i];
+                    }
+                    const float4 *src4 = reinterpret_cast<const float4 *>(
+                        pp + (pi * PV + ((int64_t)(d - od) * PH + (h - oh)) * PW + (w0 - ow)) * KT);
+#pragma unroll
+                    for (int j = 0; j < (KT > 0 ? KT : 1); ++j) {
+                        const float4 q = __ldg(src4 + j);
+                        const float qq[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                        for (int e2 = 0; e2 < 4; ++e2) {
+                            constexpr int KD = KT > 0 ? KT : 1;
+                            const int f = 4 * j + e2;
+                            acc[(f / KD) % VEC][f % KD] = fmaf(wt[(f / KD) % VEC], qq[e2], acc[(f / KD) % VEC][f % KD]);
+                        }
+                    }
+                    continue;
+                }
 #pragma unroll
                 for (int i = 0; i < VEC; ++i) {
                     const int w = w0 + i;
@@ -478,7 +506,9 @@ lamp_status_t k_instnorm_relu_fwd(const TView &y, const float *mu_rstd, const TV
     const int64_t Vn = (int64_t)y.d * y.h * y.w;
     if (Vn == 0 || y.n == 0) return LAMP_OK;
     if (y.c / 8 > 256) return LAMP_ERR_UNSUPPORTED;
-    const int64_t vpb = (int64_t)(256 / (y.c / 8)) * 8;
+    const int64_t rb = 256 / (y.c / 8);
+    int64_t vpb = (Vn / (148 * 16) + rb - 1) / rb * rb;
+    if (vpb < rb * 8) vpb = rb * 8;
     dim3 grid((unsigned)((Vn + vpb - 1) / vpb), y.n);
     instnorm_relu_fwd_kernel<<<grid, 256, 0, st>>>((const bf16 *)y.p, y.pitch, mu_rstd, (bf16 *)z.p, z.pitch, Vn, y.c, vpb);
     return launch_status();
@@ -502,7 +532,8 @@ lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TVie
     instnorm_bwd_sums_kernel<<<dim3((unsigned)blocks, y.n), 256, smem, st>>>(
         (const bf16 *)dza.p, dza.pitch, dzb ? (const bf16 *)dzb->p : nullptr, dzb ? dzb->pitch : 0,
         (const bf16 *)y.p, y.pitch, mu_rstd, sums, Vn, C, vpb);
-    const int64_t vpa = (int64_t)RB * 8;
+    int64_t vpa = (Vn / (148 * 16) + RB - 1) / RB * RB;
+    if (vpa < (int64_t)RB * 8) vpa = (int64_t)RB * 8;
     dim3 grid((unsigned)((Vn + vpa - 1) / vpa), y.n);
     instnorm_bwd_apply_kernel<<<grid, 256, 0, st>>>(
         (const bf16 *)dza.p, dza.pitch, dzb ? (const bf16 *)dzb->p : nullptr, dzb ? dzb->pitch : 0,
@@ -585,17 +616,29 @@ lamp_status_t k_overlap_add(const float *pp, int K, int D, int H, int W, const i
     if ((int64_t)D * H * W == 0) return LAMP_OK;
     const size_t smem = (size_t)(patch[0] + patch[1] + patch[2]) * sizeof(float);
     const bool vec = (W % 4 == 0) && ((uintptr_t)planar % 16 == 0) && ((uintptr_t)argmax % 4 == 0);
+    const int aligned4 = vec && patch[2] % 4 == 0 && (nst[2] == 1 || stride[2] % 4 == 0) && (W - patch[2]) % 4 == 0 &&
+                         ((uintptr_t)pp % 16 == 0);
+#define LAMP_OA(VECN, KTN)                                                                                              \
+    overlap_add_kernel<VECN, KTN><<<(unsigned)((total + 255) / 256), 256, smem, st>>>(                                \
+        pp, K, D, H, W, patch[0], patch[1], patch[2], nst[0], nst[1], nst[2], stride[0], stride[1], stride[2], window, \
+        aligned4, planar, argmax)
     if (vec) {
         const int64_t total = (int64_t)D * H * (W / 4);
-        overlap_add_kernel<4><<<(unsigned)((total + 255) / 256), 256, smem, st>>>(
-            pp, K, D, H, W, patch[0], patch[1], patch[2], nst[0], nst[1], nst[2], stride[0], stride[1], stride[2],
-            window, planar, argmax);
+        switch (aligned4 ? K : 0) {
+        case 2:  LAMP_OA(4, 2); break;
+        case 3:  LAMP_OA(4, 3); break;
+        case 4:  LAMP_OA(4, 4); break;
+        case 5:  LAMP_OA(4, 5); break;
+        case 8:  LAMP_OA(4, 8); break;
+        case 10: LAMP_OA(4, 10); break;
+        case 16: LAMP_OA(4, 16); break;
+        default: LAMP_OA(4, 0); break;
+        }
     } else {
         const int64_t total = (int64_t)D * H * W;
-        overlap_add_kernel<1><<<(unsigned)((total + 255) / 256), 256, smem, st>>>(
-            pp, K, D, H, W, patch[0], patch[1], patch[2], nst[0], nst[1], nst[2], stride[0], stride[1], stride[2],
-            window, planar, argmax);
+        LAMP_OA(1, 0);
     }
+#undef LAMP_OA
     return launch_status();
 }
 

@@ -343,3 +343,23 @@ def test_sliding_window_matches_oracle_and_whole_patch_equals_forward():
     B.lamp_sliding_window_infer(net, wd, bd, dev_bf16(vol), (D, H, W), 0.25, 1, 1, planar, am, wsb)
     assert torch.allclose(planar.permute(1, 2, 3, 0).reshape(-1, 3), probs, rtol=1e-6, atol=1e-7)
     B.lamp_unet_destroy(net)
+
+
+@pytest.mark.parametrize("K", [4, 10, 7])
+def test_overlap_add_vector_path_matches_oracle(K):
+    # every patch origin and extent along W is a multiple of 4: the 16-byte vector path (K = 7: generic path)
+    D, H, W, P, ov = 10, 12, 24, (8, 8, 8), 0.5
+    spec = O.UNetSpec(1, [8], 1, 1, K)
+    sd, sh, sw = (O.window_starts(n, p, ov) for n, p in zip((D, H, W), P))
+    assert all(s % 4 == 0 for s in sw)
+    n_p = len(sd) * len(sh) * len(sw)
+    fields = ops.softmax(synth.rng(13 + K).standard_normal((n_p, 8, 8, 8, K))).astype(np.float32)
+    for window in (1, 0):
+        A, seg, cnt = O.sliding_window(spec, None, None, np.zeros((1, D, H, W, 1)), P, ov, gaussian=bool(window),
+                                       patch_probs=lambda i, pa: fields[i][None].astype(np.float64))
+        planar = torch.empty((K, D, H, W), dtype=torch.float32, device="cuda")
+        am = torch.empty((D * H * W,), dtype=torch.uint8, device="cuda")
+        B.lamp_overlap_add(torch.from_numpy(fields).cuda(), K, D, H, W, P, ov, window, planar, am)
+        assert_close(host_f64(planar), A.transpose(3, 0, 1, 2), "overlap-add vector path", rel=1e-5, mx=1e-5)
+        agree, strict, near = tie_aware_agreement(am.cpu().numpy().reshape(D, H, W), A)
+        assert agree == 1.0
