@@ -86,6 +86,8 @@ static bool dgrad_on_tensor_cores(const ConvGeom &g)
     return kind >= 0 && umma_conv_supported(kind, g, a, b);
 }
 
+static size_t c1_padded_ws(const ConvGeom &g, size_t *xpad_bytes, size_t *dw32_bytes);
+
 size_t conv_ws_bytes(const ConvGeom &g, int pass)
 {
     if (pass == LAMP_PASS_DGRAD) return dgrad_on_tensor_cores(g) ? umma_dgrad_ws(g) : 0;
@@ -94,7 +96,10 @@ size_t conv_ws_bytes(const ConvGeom &g, int pass)
         const size_t u2 = win_wgrad_ws(g);
         if (u2 > u) u = u2;
         const size_t tc = u ? u + bias_grad_ws((int64_t)g.n * g.od * g.oh * g.ow, g.co) : 0;
-        const size_t sm = simt_conv_wgrad_ws(g);
+        size_t sm = simt_conv_wgrad_ws(g);
+        size_t xb = 0, wb = 0;
+        const size_t c1 = c1_padded_ws(g, &xb, &wb);
+        if (c1 > sm) sm = c1;
         return tc > sm ? tc : sm;
     }
     return 0;
@@ -129,9 +134,47 @@ lamp_status_t conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w, cons
     return simt_conv_dgrad(g, dy, w, dx, st);
 }
 
+// The one-channel first layer borrows the windowed tensor-core kernel: x is widened to 32 channels (zeros)
+// in scratch, the 27 x c_out x 32 gradient is formed, and its first input-channel column is the answer.
+static bool c1_padded_geom(const ConvGeom &g, ConvGeom *p)
+{
+    if (!(g.ci == 1 && g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed && (g.co == 32 || g.co == 64))) return false;
+    *p = g;
+    p->ci = 32;
+    return win_wgrad_ws(*p) > 0;
+}
+
+static size_t c1_padded_ws(const ConvGeom &g, size_t *xpad_bytes, size_t *dw32_bytes)
+{
+    ConvGeom p;
+    if (!c1_padded_geom(g, &p)) return 0;
+    *xpad_bytes = align_up((size_t)g.n * g.d * g.h * g.w * 32 * sizeof(bf16), 256);
+    *dw32_bytes = align_up((size_t)27 * g.co * 32 * sizeof(float), 256);
+    return *xpad_bytes + *dw32_bytes + win_wgrad_ws(p) + bias_grad_ws((int64_t)g.n * g.od * g.oh * g.ow, g.co);
+}
+
 lamp_status_t conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, float *db, void *ws,
                          size_t ws_bytes, cudaStream_t st)
 {
+    {
+        ConvGeom p;
+        size_t xb = 0, wb = 0;
+        const size_t need = c1_padded_ws(g, &xb, &wb);
+        if (need && c1_padded_geom(g, &p) && dy.pitch % 8 == 0 && ((uintptr_t)dy.p & 15) == 0) {
+            if (!ws || ws_bytes < need || !aligned16(ws)) return LAMP_ERR_WORKSPACE;
+            char *base = (char *)ws;
+            TView xp = x;
+            xp.p = base; xp.c = 32; xp.pitch = 32;
+            lamp_status_t s = pad_c1(x, (bf16 *)base, st);
+            if (s != LAMP_OK) return s;
+            const size_t u = win_wgrad_ws(p);
+            s = win_wgrad(p, xp, dy, (float *)(base + xb), base + xb + wb, u, st);
+            if (s != LAMP_OK) return s;
+            s = take_c0((const float *)(base + xb), dw, 27 * g.co, st);
+            if (s != LAMP_OK || !db) return s;
+            return bias_grad(dy, db, base + xb + wb + u, st);
+        }
+    }
     if (win_wgrad_supported(g, x, dy)) {
         const size_t u = win_wgrad_ws(g);
         if (!ws || ws_bytes < u + (db ? bias_grad_ws((int64_t)g.n * g.od * g.oh * g.ow, g.co) : 0)) return LAMP_ERR_WORKSPACE;

@@ -96,6 +96,10 @@ lamp_status_t reduce_partials(const float *part, int64_t entries, int splits, fl
 size_t        bias_grad_ws(int64_t voxels, int co);
 lamp_status_t bias_grad(const TView &dy, float *db, void *ws, cudaStream_t st);
 
+// first layer (c_in = 1) on the tensor-core wgrad path: widen x to 32 channels, keep column 0 of the result
+lamp_status_t pad_c1(const TView &x, bf16 *xpad, cudaStream_t st);
+lamp_status_t take_c0(const float *dw32, float *dw, int n, cudaStream_t st);
+
 // wgrad_umma.cu (tcgen05 weight gradient)
 bool          umma_wgrad_supported(const ConvGeom &g, const TView &x, const TView &dy);
 size_t        umma_wgrad_ws(const ConvGeom &g);

@@ -386,15 +386,45 @@ conv_c1_wgrad_kernel(ConvGeom g, const bf16 *__restrict__ x, int64_t xp, const b
     }
 }
 
-// out[e] = sum_s part[s][e], fixed order.
+// out[e] = sum_s part[s][e], fixed order: 32 entries x 8 split slices per block; slice j adds splits j, j + 8, ...
+// and the eight slice sums are then added in slice order.
 __global__ void __launch_bounds__(256)
 reduce_parts_kernel(const float *__restrict__ part, int64_t entries, int splits, float *__restrict__ out)
 {
-    const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;
-    if (e >= entries) return;
+    __shared__ float red[8][32];
+    const int el = threadIdx.x & 31, sl = threadIdx.x >> 5;
+    const int64_t e = (int64_t)blockIdx.x * 32 + el;
     float acc = 0.f;
-    for (int s = 0; s < splits; ++s) acc += part[(int64_t)s * entries + e];
-    out[e] = acc;
+    if (e < entries)
+        for (int s = sl; s < splits; s += 8) acc += part[(int64_t)s * entries + e];
+    red[sl][el] = acc;
+    __syncthreads();
+    if (sl == 0 && e < entries) {
+        float a = red[0][el];
+#pragma unroll
+        for (int j = 1; j < 8; ++j) a += red[j][el];
+        out[e] = a;
+    }
+}
+
+// xpad[v][0] = x[v], xpad[v][1..31] = 0 (the 1-channel input widened to one 32-channel chunk)
+__global__ void __launch_bounds__(256)
+pad_c1_kernel(const bf16 *__restrict__ x, int64_t xp, bf16 *__restrict__ xpad, int64_t V)
+{
+    const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;      // one 16-byte group of 8 channels
+    if (e >= V * 4) return;
+    const int64_t v = e >> 2;
+    uint4 q = make_uint4(0, 0, 0, 0);
+    if ((e & 3) == 0) q.x = (uint32_t)__bfloat16_as_ushort(x[v * xp]);
+    reinterpret_cast<uint4 *>(xpad)[e] = q;
+}
+
+// dw[t][co] = dw32[t][co][0]
+__global__ void __launch_bounds__(256)
+take_c0_kernel(const float *__restrict__ dw32, float *__restrict__ dw, int n)
+{
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i < n) dw[i] = dw32[(int64_t)i * 32];
 }
 
 inline int pick_tc(int co)
@@ -470,7 +500,7 @@ lamp_status_t simt_conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w,
 lamp_status_t reduce_partials(const float *part, int64_t entries, int splits, float *out, cudaStream_t st)
 {
     if (entries == 0) return LAMP_OK;
-    reduce_parts_kernel<<<(unsigned)((entries + 255) / 256), 256, 0, st>>>(part, entries, splits, out);
+    reduce_parts_kernel<<<(unsigned)((entries + 31) / 32), 256, 0, st>>>(part, entries, splits, out);
     return launch_status();
 }
 
@@ -501,7 +531,7 @@ lamp_status_t bias_grad(const TView &dy, float *db, void *ws, cudaStream_t st)
     } else {
         colsum_kernel<<<b, 256, 0, st>>>((const bf16 *)dy.p, dy.pitch, dy.c, V, vpb, (float *)ws);
     }
-    reduce_parts_kernel<<<(dy.c + 255) / 256, 256, 0, st>>>((const float *)ws, dy.c, b, db);
+    reduce_parts_kernel<<<(dy.c + 31) / 32, 256, 0, st>>>((const float *)ws, dy.c, b, db);
     return launch_status();
 }
 
@@ -518,6 +548,20 @@ static void c1_wgrad_plan(const ConvGeom &g, int *blocks, int64_t *vpb)
     if (b < 1) b = 1;
     *blocks = b;
     *vpb = (V + b - 1) / b;
+}
+
+lamp_status_t pad_c1(const TView &x, bf16 *xpad, cudaStream_t st)
+{
+    const int64_t V = (int64_t)x.n * x.d * x.h * x.w;
+    if (V == 0) return LAMP_OK;
+    pad_c1_kernel<<<(unsigned)((V * 4 + 255) / 256), 256, 0, st>>>((const bf16 *)x.p, x.pitch, xpad, V);
+    return launch_status();
+}
+
+lamp_status_t take_c0(const float *dw32, float *dw, int n, cudaStream_t st)
+{
+    take_c0_kernel<<<(n + 255) / 256, 256, 0, st>>>(dw32, dw, n);
+    return launch_status();
 }
 
 size_t simt_conv_wgrad_ws(const ConvGeom &g)
@@ -548,7 +592,7 @@ lamp_status_t simt_conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy
                 conv_c1_wgrad_kernel<32><<<blocks, 256, 0, st>>>(g, (const bf16 *)x.p, x.pitch, (const bf16 *)dy.p, dy.pitch, part1, vpb);
             else
                 conv_c1_wgrad_kernel<64><<<blocks, 128, 0, st>>>(g, (const bf16 *)x.p, x.pitch, (const bf16 *)dy.p, dy.pitch, part1, vpb);
-            reduce_parts_kernel<<<(unsigned)((p.entries + 255) / 256), 256, 0, st>>>(part1, p.entries, blocks, dw);
+            reduce_parts_kernel<<<(unsigned)((p.entries + 31) / 32), 256, 0, st>>>(part1, p.entries, blocks, dw);
             if (db) {
                 const size_t off = simt_conv_wgrad_ws(g) - bias_grad_ws((int64_t)g.n * g.od * g.oh * g.ow, g.co);
                 lamp_status_t sb = bias_grad(dy, db, (char *)ws + off, st);
@@ -569,10 +613,10 @@ lamp_status_t simt_conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy
         conv_wgrad_kernel<true><<<grid, 256, 0, st>>>(g, (const bf16 *)x.p, x.pitch, (const bf16 *)dy.p, dy.pitch, part, p.entries, p.rows, p.rows_per_split);
     else
         conv_wgrad_kernel<false><<<grid, 256, 0, st>>>(g, (const bf16 *)x.p, x.pitch, (const bf16 *)dy.p, dy.pitch, part, p.entries, p.rows, p.rows_per_split);
-    reduce_parts_kernel<<<(unsigned)((p.entries + 255) / 256), 256, 0, st>>>(part, p.entries, p.splits, dw);
+    reduce_parts_kernel<<<(unsigned)((p.entries + 31) / 32), 256, 0, st>>>(part, p.entries, p.splits, dw);
     if (db) {
         colsum_kernel<<<p.cs_blocks, 256, 0, st>>>((const bf16 *)dy.p, dy.pitch, g.co, p.V, p.v_per_block, cpart);
-        reduce_parts_kernel<<<(g.co + 255) / 256, 256, 0, st>>>(cpart, g.co, p.cs_blocks, db);
+        reduce_parts_kernel<<<(g.co + 31) / 32, 256, 0, st>>>(cpart, g.co, p.cs_blocks, db);
     }
     return launch_status();
 }
