@@ -252,6 +252,12 @@ lamp_status_t lamp_overlap_add(const float *patch_probs, int32_t k, int32_t d, i
  * (LAMP_OK, or LAMP_ERR_TIMEOUT if a bounded wait inside a kernel ran out). */
 lamp_status_t lamp_get_async_status(void *cuda_stream);
 const char   *lamp_status_string(lamp_status_t s);
+/* Self-test of the failure path every tensor-core kernel of this library shares: all device-side waits
+ * (on TMA completions, on tensor-pipe completions) are bounded, and a wait that runs out records
+ * LAMP_ERR_TIMEOUT and lets the kernel finish normally instead of hanging.  This call launches one
+ * small kernel whose wait can never be satisfied (limit about 10 ms); afterwards
+ * lamp_get_async_status() must return LAMP_ERR_TIMEOUT once and the context must remain usable. */
+lamp_status_t lamp_selftest_wait_timeout(void *cuda_stream);
 /* Library build identifier: "lamp-b200 <sm arch>". */
 const char   *lamp_version(void);
 

@@ -76,6 +76,7 @@ def lib():
             "lamp_sliding_window_infer": (C.c_int, [vp, vp, vp, TP, I3, f32, i32, i32, vp, vp, vp, sz, vp]),
             "lamp_overlap_add": (C.c_int, [vp, i32, i32, i32, i32, I3, f32, i32, vp, vp, vp]),
             "lamp_get_async_status": (C.c_int, [vp]),
+            "lamp_selftest_wait_timeout": (C.c_int, [vp]),
             "lamp_status_string": (C.c_char_p, [C.c_int]),
             "lamp_version": (C.c_char_p, []),
         }
@@ -93,7 +94,7 @@ EXPORTS = ["lamp_conv3d_workspace_bytes", "lamp_conv3d_fwd", "lamp_conv3d_dgrad"
            "lamp_unet_num_layers", "lamp_unet_weight_count", "lamp_unet_bias_count", "lamp_unet_param_layout",
            "lamp_unet_workspace_bytes", "lamp_unet_tensor_layout", "lamp_unet_forward", "lamp_unet_train_step",
            "lamp_sliding_window_workspace_bytes", "lamp_sliding_window_infer", "lamp_overlap_add",
-           "lamp_get_async_status", "lamp_status_string", "lamp_version"]
+           "lamp_get_async_status", "lamp_selftest_wait_timeout", "lamp_status_string", "lamp_version"]
 
 
 def _check(st, what):
@@ -258,6 +259,10 @@ def lamp_overlap_add(patch_probs, k, d, h, w, patch, overlap, window, probs_plan
 
 def lamp_get_async_status():
     return lib().lamp_get_async_status(_stream())
+
+
+def lamp_selftest_wait_timeout():
+    _check(lib().lamp_selftest_wait_timeout(_stream()), "lamp_selftest_wait_timeout")
 
 
 def lamp_version():

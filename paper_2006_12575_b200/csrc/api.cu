@@ -1,5 +1,6 @@
 // C ABI (include/lamp.h): argument checks, kernel selection, status word.
 #include "common.cuh"
+#include "umma_ptx.cuh"
 
 namespace lamp {
 
@@ -301,6 +302,30 @@ const char *lamp_status_string(lamp_status_t s)
     case LAMP_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the library's built-in static array";
     }
     return "unknown status";
+}
+
+// One CTA waits, with the kernels' own bounded wait, on an mbarrier that nothing ever arrives on.
+__global__ void wait_timeout_selftest_kernel(int *status, long long limit_clocks)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        ptx::mbar_init(ptx::smem_u32(&bar), 1);
+        ptx::mbar_init_fence();
+    }
+    __syncthreads();
+    const bool ok = ptx::mbar_wait(ptx::smem_u32(&bar), 0, &abort_flag, limit_clocks);
+    __syncthreads();
+    if (threadIdx.x == 0 && !ok && status) atomicExch(status, (int)LAMP_ERR_TIMEOUT);
+}
+
+lamp_status_t lamp_selftest_wait_timeout(void *cuda_stream)
+{
+    int *st = status_word_ptr();
+    if (!st) return LAMP_ERR_CUDA;
+    wait_timeout_selftest_kernel<<<1, 32, 0, (cudaStream_t)cuda_stream>>>(st, 20000000ll);      // about 10 ms
+    return launch_status();
 }
 
 const char *lamp_version(void) { return "lamp-b200 sm_100a"; }

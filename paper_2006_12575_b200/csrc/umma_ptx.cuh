@@ -38,7 +38,8 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 constexpr long long WAIT_LIMIT_CLOCKS = 4000000000ll;      // about two seconds
 
 // Bounded wait: false if the limit ran out or another role of the CTA already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          long long limit_clocks = WAIT_LIMIT_CLOCKS)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
@@ -46,7 +47,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CLOCKS) { *abort_flag = 1; return false; }
+        if (clock64() - t0 > limit_clocks) { *abort_flag = 1; return false; }
     }
 }
 

@@ -151,3 +151,18 @@ def test_empty_volume_is_a_no_op():
     B.lamp_conv3d_fwd(desc, B.Tensor(w.data_ptr(), 0, 1, 0, 4, 4, 8, 8, 0), w, None,
                       B.Tensor(w.data_ptr(), 0, 1, 0, 4, 4, 8, 8, 0))
     assert B.lamp_get_async_status() == 0
+
+
+def test_bounded_wait_reports_timeout_and_context_stays_usable():
+    # a wait that nothing satisfies runs out, the status word says so once, and later calls work
+    assert B.lamp_get_async_status() == 0
+    B.lamp_selftest_wait_timeout()
+    assert B.lamp_get_async_status() == 5
+    assert B.lamp_get_async_status() == 0
+    desc = B.conv_desc(64, 64)
+    x = dev_bf16(synth.normal_bf16((1, 4, 32, 8, 64), 1))
+    w = dev_bf16(synth.kaiming_bf16(27, 64, 64, 27 * 64, 2))
+    y = torch.empty((1, 4, 32, 8, 64), dtype=torch.float32, device="cuda")
+    B.lamp_conv3d_fwd(desc, x, w, None, y)
+    assert B.lamp_get_async_status() == 0
+    assert torch.isfinite(y).all()
