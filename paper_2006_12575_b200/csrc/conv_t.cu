@@ -144,15 +144,12 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         for (int t9 = 0; t9 < 9; ++t9) {
                             if (!mbar_wait(wempty0 + 8 * ws, wph ^ 1, abort_flag)) { ok = false; break; }
                             mbar_expect_tx(wfull0 + 8 * ws, W_BYTES);
+                            // one box over the kd axis of the weights fetches the S stacked blocks: block b holds tap
+                            // kd = pi - (S - 1) + b (forward) or, with mirrored taps, kd' = 2 - pi + b; kd outside 0..2 is
+                            // outside the tensor and arrives as zeros
                             const uint32_t dst = smem_u32(w_base + (size_t)ws * W_BYTES);
-#pragma unroll
-                            for (int j = 0; j < S; ++j) {
-                                const int kd = pi - j;                      // tap of output plane o0 + j fed by input plane p
-                                int tap = kd * 9 + t9;
-                                if (kd < 0 || kd > 2) tap = 27;             // out of range: TMA fills the block with zeros
-                                else if (P.mirror) tap = 26 - tap;
-                                tma_load_3d(dst + j * COB * ROWB, &map_w, wfull0 + 8 * ws, c * KC, it.ct * 128, tap);
-                            }
+                            if (P.mirror) tma_load_4d(dst, &map_w, wfull0 + 8 * ws, c * KC, it.ct * 128, 8 - t9, 2 - pi);
+                            else          tma_load_4d(dst, &map_w, wfull0 + 8 * ws, c * KC, it.ct * 128, t9, pi - (S - 1));
                             if (++ws == P.nw) { ws = 0; wph ^= 1; }
                         }
                     }
@@ -207,7 +204,9 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         // -------------------------------------------------------------------- epilogue (warps 3..6)
         const int q = warp & 3;                                 // TMEM lane quarter of this warp
         float *tr = epi + (warp - 3) * 32 * 33;
-        const int jplane = (q * 32) / COB;                      // which stacked output plane these 32 lanes belong to
+        // which stacked output plane these 32 lanes belong to: block b = (q * 32) / COB carries tap kd = pi - (S - 1) + b
+        // of output plane o0 + (S - 1 - b) in the forward pass, and of plane o0 + b with mirrored taps
+        const int jplane = P.mirror ? (q * 32) / COB : S - 1 - (q * 32) / COB;
         const int co_in_blk = (q * 32) % COB;                   // first of this warp's 32 channels inside the block
         uint32_t acc = 0, acc_phase = 0;
         float s1 = 0.f, s2 = 0.f;                               // sums of this thread's channel
@@ -408,11 +407,12 @@ lamp_status_t ct_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, cons
             return LAMP_ERR_CUDA;
     }
     {
-        const cuuint64_t dims[3] = {(cuuint64_t)g.ci, (cuuint64_t)g.co, 27};
-        const cuuint64_t strides[2] = {(cuuint64_t)g.ci * 2, (cuuint64_t)g.ci * 2 * g.co};
-        const cuuint32_t box[3] = {(cuuint32_t)pl.KC, (cuuint32_t)pl.COB, 1};
-        const cuuint32_t es[3] = {1, 1, 1};
-        if (encode(&mw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void *)w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+        // weights viewed as [kd][kh*3+kw][c_out][c_in]
+        const cuuint64_t dims[4] = {(cuuint64_t)g.ci, (cuuint64_t)g.co, 9, 3};
+        const cuuint64_t strides[3] = {(cuuint64_t)g.ci * 2, (cuuint64_t)g.ci * 2 * g.co, (cuuint64_t)g.ci * 2 * g.co * 9};
+        const cuuint32_t box[4] = {(cuuint32_t)pl.KC, (cuuint32_t)pl.COB, 1, (cuuint32_t)(128 / pl.COB)};
+        const cuuint32_t es[4] = {1, 1, 1, 1};
+        if (encode(&mw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void *)w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return LAMP_ERR_CUDA;
     }
