@@ -79,14 +79,17 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     constexpr int ROWB = KC * 2;
     constexpr uint32_t SWZ = KC == 64 ? 2u : 4u;
     constexpr uint32_t PLANE_BOX_BYTES = HALO_W * HALO_H * ROWB;
-    constexpr uint32_t W_BYTES = 128 * ROWB;
+    constexpr uint32_t W_BYTES = 128 * ROWB;                  // one tap's weight tile
+    constexpr int TPS = KC == 32 ? 3 : 1;                      // taps (one kh row) per weight stage: 32-channel chunks carry
+                                                               // too little work per tap to pay a barrier round trip each
+    constexpr uint32_t WST_BYTES = TPS * W_BYTES;
     constexpr uint32_t IDESC = make_idesc(256);
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *p_base = smem;
     uint8_t *w_base = p_base + (size_t)P.np * P.plane_bytes;
-    float *epi = (float *)(w_base + (size_t)P.nw * W_BYTES);
+    float *epi = (float *)(w_base + (size_t)P.nw * WST_BYTES);
     uint64_t *bars = (uint64_t *)((uint8_t *)epi + 4 * 32 * 33 * 4);
     const uint32_t pfull0 = smem_u32(bars), pempty0 = smem_u32(bars + MAX_NP);
     const uint32_t wfull0 = smem_u32(bars + 2 * MAX_NP), wempty0 = smem_u32(bars + 2 * MAX_NP + MAX_NW);
@@ -141,15 +144,15 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     const int p = it.o0 - 1 + pi;
                     if (p < 0 || p >= P.D) continue;
                     for (int c = 0; c < P.chunks && ok; ++c) {
-                        for (int t9 = 0; t9 < 9; ++t9) {
+                        for (int t9 = 0; t9 < 9; t9 += TPS) {
                             if (!mbar_wait(wempty0 + 8 * ws, wph ^ 1, abort_flag)) { ok = false; break; }
-                            mbar_expect_tx(wfull0 + 8 * ws, W_BYTES);
-                            // one box over the kd axis of the weights fetches the S stacked blocks: block b holds tap
-                            // kd = pi - (S - 1) + b (forward) or, with mirrored taps, kd' = 2 - pi + b; kd outside 0..2 is
-                            // outside the tensor and arrives as zeros
-                            const uint32_t dst = smem_u32(w_base + (size_t)ws * W_BYTES);
-                            if (P.mirror) tma_load_4d(dst, &map_w, wfull0 + 8 * ws, c * KC, it.ct * 128, 8 - t9, 2 - pi);
-                            else          tma_load_4d(dst, &map_w, wfull0 + 8 * ws, c * KC, it.ct * 128, t9, pi - (S - 1));
+                            mbar_expect_tx(wfull0 + 8 * ws, WST_BYTES);
+                            // one box fetches TPS taps x S stacked blocks: slot s, block b holds tap (kd, t9 + s) with
+                            // kd = pi - (S - 1) + b (forward) or, with mirrored taps, the weight tap (2 - pi + b, 8 - t9 - (TPS - 1) + s);
+                            // kd outside 0..2 is outside the tensor and arrives as zeros
+                            const uint32_t dst = smem_u32(w_base + (size_t)ws * WST_BYTES);
+                            if (P.mirror) tma_load_4d(dst, &map_w, wfull0 + 8 * ws, c * KC, it.ct * 128, 2 - pi, 8 - t9 - (TPS - 1));
+                            else          tma_load_4d(dst, &map_w, wfull0 + 8 * ws, c * KC, it.ct * 128, pi - (S - 1), t9);
                             if (++ws == P.nw) { ws = 0; wph ^= 1; }
                         }
                     }
@@ -175,16 +178,20 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         if (!mbar_wait(pfull0 + 8 * ps, pph, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t plane = smem_u32(p_base + (size_t)ps * P.plane_bytes);
-                        for (int t9 = 0; t9 < 9; ++t9) {
-                            const int kh = t9 / 3, kw = t9 - kh * 3;
+                        for (int t9 = 0; t9 < 9; t9 += TPS) {
                             if (!mbar_wait(wfull0 + 8 * ws, wph, abort_flag)) { ok = false; break; }
                             tc_fence_after();
-                            const uint64_t da = make_desc(smem_u32(w_base + (size_t)ws * W_BYTES), 0, 8 * ROWB, SWZ);
-                            const uint64_t db = make_desc(plane + (kh * HALO_W + kw) * ROWB, 0, HALO_W * ROWB, SWZ);
 #pragma unroll
-                            for (int k = 0; k < KC / 16; ++k) {
-                                umma_bf16(d_tmem, da + 2 * k, db + 2 * k, IDESC, accumulate);
-                                accumulate = 1;
+                            for (int sl = 0; sl < TPS; ++sl) {
+                                const int t = P.mirror ? t9 + TPS - 1 - sl : t9 + sl;        // conv tap whose weights sit in slot sl
+                                const int kh = t / 3, kw = t - kh * 3;
+                                const uint64_t da = make_desc(smem_u32(w_base + (size_t)ws * WST_BYTES + sl * W_BYTES), 0, 8 * ROWB, SWZ);
+                                const uint64_t db = make_desc(plane + (kh * HALO_W + kw) * ROWB, 0, HALO_W * ROWB, SWZ);
+#pragma unroll
+                                for (int k = 0; k < KC / 16; ++k) {
+                                    umma_bf16(d_tmem, da + 2 * k, db + 2 * k, IDESC, accumulate);
+                                    accumulate = 1;
+                                }
                             }
                             umma_commit(wempty0 + 8 * ws);
                             if (++ws == P.nw) { ws = 0; wph ^= 1; }
@@ -332,7 +339,7 @@ bool make_ct_plan(const ConvGeom &g, CtPlan *out)
     P.chunks = g.ci / KC;
     const int rowb = KC * 2;
     P.plane_bytes = (int)align_up((size_t)HALO_W * HALO_H * rowb, 1024);
-    const int w_bytes = 128 * rowb;
+    const int w_bytes = 128 * rowb * (KC == 32 ? 3 : 1);      // bytes of one weight stage
     const int budget = SMEM_LIMIT - 1024 - EPI_BYTES - CTRL_BYTES;
     int np = KC == 64 ? 2 : 4;
     int nw = (budget - np * P.plane_bytes) / w_bytes;
@@ -407,10 +414,10 @@ lamp_status_t ct_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, cons
             return LAMP_ERR_CUDA;
     }
     {
-        // weights viewed as [kd][kh*3+kw][c_out][c_in]
-        const cuuint64_t dims[4] = {(cuuint64_t)g.ci, (cuuint64_t)g.co, 9, 3};
-        const cuuint64_t strides[3] = {(cuuint64_t)g.ci * 2, (cuuint64_t)g.ci * 2 * g.co, (cuuint64_t)g.ci * 2 * g.co * 9};
-        const cuuint32_t box[4] = {(cuuint32_t)pl.KC, (cuuint32_t)pl.COB, 1, (cuuint32_t)(128 / pl.COB)};
+        // weights viewed as (c_in, c_out, kd, kh*3+kw): a box spans the stacked kd blocks, then the taps of a stage
+        const cuuint64_t dims[4] = {(cuuint64_t)g.ci, (cuuint64_t)g.co, 3, 9};
+        const cuuint64_t strides[3] = {(cuuint64_t)g.ci * 2, (cuuint64_t)g.ci * 2 * g.co * 9, (cuuint64_t)g.ci * 2 * g.co};
+        const cuuint32_t box[4] = {(cuuint32_t)pl.KC, (cuuint32_t)pl.COB, (cuuint32_t)(128 / pl.COB), (cuuint32_t)(pl.KC == 32 ? 3 : 1)};
         const cuuint32_t es[4] = {1, 1, 1, 1};
         if (encode(&mw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void *)w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
