@@ -80,9 +80,17 @@ enum { LAMP_PASS_FWD = 0, LAMP_PASS_DGRAD = 1, LAMP_PASS_WGRAD = 2 };
  * their derivatives).
  * ---------------------------------------------------------------------- */
 
-/* Bytes of workspace the given pass needs for input x (for LAMP_PASS_DGRAD, x is
- * the tensor that receives the gradient, i.e. the conv's input shape). */
+/* Bytes of workspace with which the given pass runs fastest for input x (for LAMP_PASS_DGRAD,
+ * x is the tensor that receives the gradient, i.e. the conv's input shape). */
 size_t lamp_conv3d_workspace_bytes(const lamp_conv_desc_t *desc, const lamp_tensor_t *x, int pass);
+
+/* The smallest workspace the pass accepts (a smaller one gives LAMP_ERR_WORKSPACE).  The
+ * two differ for forward and data-gradient passes over volumes so small that their tiles do
+ * not fill the GPU (the deep levels of the U-Net): given the larger workspace the kernels
+ * split the reduction over taps and input channels across several CTAs, keep fp32 partial
+ * results there and add them in a fixed order; given less they run unsplit.  Both are
+ * deterministic; they differ in the fp32 summation order only. */
+size_t lamp_conv3d_workspace_min_bytes(const lamp_conv_desc_t *desc, const lamp_tensor_t *x, int pass);
 
 /* y[n,od,oh,ow,co] = bias[co] + sum_{tap,ci} x[n, od*s+kd-p, oh*s+kh-p, ow*s+kw-p, ci] * w[tap][co][ci]
  * (transposed: y[n, d*s+a, h*s+b, w*s+c, co] = bias[co] + sum_ci x[n,d,h,w,ci] * w[(a,b,c)][co][ci]).
@@ -106,11 +114,12 @@ lamp_status_t lamp_conv3d_dgrad(const lamp_conv_desc_t *desc, const lamp_tensor_
  * layer running inside an engine that handed out all device memory at start-up, or a latency-
  * critical loop where cudaMalloc (it synchronises the device and can fail under memory pressure)
  * is ruled out - and so have no workspace to pass.  (The paper has no counterpart of this call:
- * it is a packaging variant of lamp_conv3d_dgrad, with identical arithmetic and results.)
+ * it is a packaging variant of lamp_conv3d_dgrad, with the arithmetic and results of that call
+ * given its smallest workspace.)
  * The scratch this pass needs, a transposed copy of the weights, sits in a fixed array of
  * LAMP_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads the library holds it
  * until the process exits.  The call itself allocates and frees nothing.
- *  - Limit: lamp_conv3d_workspace_bytes(desc, dx, LAMP_PASS_DGRAD) must not exceed
+ *  - Limit: lamp_conv3d_workspace_min_bytes(desc, dx, LAMP_PASS_DGRAD) must not exceed
  *    LAMP_STATIC_SCRATCH_BYTES (27 * c_in * c_out * 2 bytes for the 3x3x3 s1 p1 conv, i.e. up to
  *    c_in * c_out = 77672, e.g. 256 x 256); otherwise LAMP_ERR_SCRATCH_LIMIT is returned and
  *    nothing is launched.  Variants that need no scratch are accepted at any size.

@@ -56,6 +56,7 @@ def lib():
         I3 = C.POINTER(C.c_int32)
         sig = {
             "lamp_conv3d_workspace_bytes": (sz, [DP, TP, C.c_int]),
+            "lamp_conv3d_workspace_min_bytes": (sz, [DP, TP, C.c_int]),
             "lamp_conv3d_fwd": (C.c_int, [DP, TP, vp, vp, TP, vp, vp, sz, vp]),
             "lamp_conv3d_dgrad": (C.c_int, [DP, TP, vp, TP, vp, sz, vp]),
             "lamp_conv3d_dgrad_static_scratch": (C.c_int, [DP, TP, vp, TP, vp]),
@@ -88,7 +89,7 @@ def lib():
     return _lib
 
 
-EXPORTS = ["lamp_conv3d_workspace_bytes", "lamp_conv3d_fwd", "lamp_conv3d_dgrad", "lamp_conv3d_dgrad_static_scratch",
+EXPORTS = ["lamp_conv3d_workspace_bytes", "lamp_conv3d_workspace_min_bytes", "lamp_conv3d_fwd", "lamp_conv3d_dgrad", "lamp_conv3d_dgrad_static_scratch",
            "lamp_conv3d_wgrad",
            "lamp_instnorm_relu_fwd", "lamp_instnorm_relu_bwd", "lamp_unet_create", "lamp_unet_destroy",
            "lamp_unet_num_layers", "lamp_unet_weight_count", "lamp_unet_bias_count", "lamp_unet_param_layout",
@@ -128,6 +129,10 @@ def conv_desc(c_in, c_out, ksize=3, stride=1, pad=1, transposed=0) -> ConvDesc:
 
 def lamp_conv3d_workspace_bytes(desc, x, pass_):
     return lib().lamp_conv3d_workspace_bytes(C.byref(desc), C.byref(_td(x)), pass_)
+
+
+def lamp_conv3d_workspace_min_bytes(desc, x, pass_):
+    return lib().lamp_conv3d_workspace_min_bytes(C.byref(desc), C.byref(_td(x)), pass_)
 
 
 def _ws(ws):

@@ -89,9 +89,39 @@ static bool dgrad_on_tensor_cores(const ConvGeom &g)
 
 static size_t c1_padded_ws(const ConvGeom &g, size_t *xpad_bytes, size_t *dw32_bytes);
 
+// scratch for fp32 partial results when the tensor-core "voxels x channels" kernel would take the pass
+static size_t splitk_ws(const ConvGeom &g, int pass)
+{
+    TView a{}, b{};
+    a.pitch = 8; b.pitch = 8;
+    if (pass == LAMP_PASS_FWD) {
+        a.d = g.d; a.h = g.h; a.w = g.w; a.c = g.ci;
+        if (ct_conv_fwd_supported(g, a, b)) return 0;
+        const int kind = fwd_kind(g);
+        return kind >= 0 && umma_conv_supported(kind, g, a, b) ? umma_splitk_ws(kind, g) : 0;
+    }
+    const int kind = dgrad_kind(g);
+    if (kind < 0 || !umma_conv_supported(kind, g, a, b)) return 0;
+    if (kind == UK_S1_DGRAD) {
+        ConvGeom t = g;
+        t.ci = g.co; t.co = g.ci;
+        a.d = g.d; a.h = g.h; a.w = g.w; a.c = g.co;
+        if (ct_conv_fwd_supported(t, a, b)) return 0;
+    }
+    return umma_splitk_ws(kind, g);
+}
+
+size_t conv_ws_min_bytes(const ConvGeom &g, int pass)
+{
+    if (pass == LAMP_PASS_FWD) return 0;
+    if (pass == LAMP_PASS_DGRAD) return dgrad_on_tensor_cores(g) ? umma_dgrad_ws(g) : 0;
+    return conv_ws_bytes(g, pass);
+}
+
 size_t conv_ws_bytes(const ConvGeom &g, int pass)
 {
-    if (pass == LAMP_PASS_DGRAD) return dgrad_on_tensor_cores(g) ? umma_dgrad_ws(g) : 0;
+    if (pass == LAMP_PASS_FWD) return splitk_ws(g, pass);
+    if (pass == LAMP_PASS_DGRAD) return dgrad_on_tensor_cores(g) ? umma_dgrad_ws(g) + splitk_ws(g, pass) : 0;
     if (pass == LAMP_PASS_WGRAD) {
         size_t u = umma_wgrad_ws(g);             // 0 when the tensor-core kernels do not take this shape
         const size_t u2 = win_wgrad_ws(g);
@@ -107,11 +137,11 @@ size_t conv_ws_bytes(const ConvGeom &g, int pass)
 }
 
 lamp_status_t conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
-                       double *stats, cudaStream_t st)
+                       double *stats, void *ws, size_t ws_bytes, cudaStream_t st)
 {
     if (ct_conv_fwd_supported(g, x, y)) return ct_conv_fwd(g, x, w, bias, y, stats, 0, st);
     const int kind = fwd_kind(g);
-    if (kind >= 0 && umma_conv_supported(kind, g, x, y)) return umma_conv(kind, g, x, w, bias, y, stats, st);
+    if (kind >= 0 && umma_conv_supported(kind, g, x, y)) return umma_conv(kind, g, x, w, bias, y, stats, ws, ws_bytes, st);
     return simt_conv_fwd(g, x, w, bias, y, stats, st);
 }
 
@@ -130,7 +160,7 @@ lamp_status_t conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w, cons
             t.ci = g.co; t.co = g.ci;
             if (ct_conv_fwd_supported(t, dy, dx)) return ct_conv_fwd(t, dy, (const bf16 *)ws, nullptr, dx, nullptr, 1, st);
         }
-        return umma_conv(kind, g, dy, (const bf16 *)ws, nullptr, dx, nullptr, st);
+        return umma_conv(kind, g, dy, (const bf16 *)ws, nullptr, dx, nullptr, (char *)ws + need, ws_bytes - need, st);
     }
     return simt_conv_dgrad(g, dy, w, dx, st);
 }
@@ -206,11 +236,17 @@ size_t lamp_conv3d_workspace_bytes(const lamp_conv_desc_t *desc, const lamp_tens
     return conv_ws_bytes(g, pass);
 }
 
+size_t lamp_conv3d_workspace_min_bytes(const lamp_conv_desc_t *desc, const lamp_tensor_t *x, int pass)
+{
+    ConvGeom g;
+    if (!x || conv_geom(desc, x, nullptr, &g) != LAMP_OK) return 0;
+    return conv_ws_min_bytes(g, pass);
+}
+
 lamp_status_t lamp_conv3d_fwd(const lamp_conv_desc_t *desc, const lamp_tensor_t *x, const void *w,
                               const float *bias, lamp_tensor_t *y, double *stats,
                               void *ws, size_t ws_bytes, void *cuda_stream)
 {
-    (void)ws; (void)ws_bytes;
     if (!desc || !x || !w || !y) return LAMP_ERR_INVALID_ARG;
     lamp_status_t s;
     if ((s = check_tensor(x, false, true)) != LAMP_OK) return s;
@@ -218,7 +254,7 @@ lamp_status_t lamp_conv3d_fwd(const lamp_conv_desc_t *desc, const lamp_tensor_t 
     if (!aligned16(w)) return LAMP_ERR_INVALID_ARG;
     ConvGeom g;
     if ((s = conv_geom(desc, x, y, &g)) != LAMP_OK) return s;
-    return conv_fwd(g, make_view(x), (const bf16 *)w, bias, make_view(y), stats, (cudaStream_t)cuda_stream);
+    return conv_fwd(g, make_view(x), (const bf16 *)w, bias, make_view(y), stats, ws, ws_bytes, (cudaStream_t)cuda_stream);
 }
 
 lamp_status_t lamp_conv3d_dgrad(const lamp_conv_desc_t *desc, const lamp_tensor_t *dy, const void *w,
@@ -255,10 +291,7 @@ lamp_status_t lamp_instnorm_relu_fwd(const lamp_tensor_t *y, const double *stats
     if ((s = check_tensor(y, false, false)) != LAMP_OK) return s;
     if ((s = check_tensor(z, false, false)) != LAMP_OK) return s;
     if (y->n != z->n || y->d != z->d || y->h != z->h || y->w != z->w || y->c != z->c) return LAMP_ERR_INVALID_ARG;
-    cudaStream_t st = (cudaStream_t)cuda_stream;
-    const int64_t Vn = (int64_t)y->d * y->h * y->w;
-    if ((s = k_finalize_stats(stats, mu_rstd, (int64_t)y->n * y->c, Vn ? 1.0 / (double)Vn : 0.0, eps, st)) != LAMP_OK) return s;
-    return k_instnorm_relu_fwd(make_view(y), mu_rstd, make_view(z), st);
+    return k_instnorm_relu_fwd(make_view(y), stats, eps, mu_rstd, make_view(z), (cudaStream_t)cuda_stream);
 }
 
 lamp_status_t lamp_instnorm_relu_bwd(const lamp_tensor_t *dz_a, const lamp_tensor_t *dz_b,

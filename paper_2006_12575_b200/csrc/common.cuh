@@ -115,8 +115,11 @@ lamp_status_t win_wgrad(const ConvGeom &g, const TView &x, const TView &dy, floa
 // conv_umma.cu (tcgen05 implicit GEMM, voxels x channels form; see the file header for the kinds)
 enum { UK_S1_FWD = 0, UK_S1_DGRAD = 1, UK_S2_FWD = 2, UK_S2_DGRAD = 3, UK_T_FWD = 4, UK_T_DGRAD = 5 };
 bool          umma_conv_supported(int kind, const ConvGeom &g, const TView &a, const TView &y);
+// part / part_bytes: optional scratch of umma_splitk_ws bytes; with it a pass that has too few tiles to fill the
+// GPU splits its K range over several CTAs (fp32 partial results, added in a fixed order by a second kernel)
 lamp_status_t umma_conv(int kind, const ConvGeom &g, const TView &a, const bf16 *w, const float *bias, const TView &y,
-                        double *stats, cudaStream_t st);
+                        double *stats, void *part, size_t part_bytes, cudaStream_t st);
+size_t        umma_splitk_ws(int kind, const ConvGeom &g);
 size_t        umma_dgrad_ws(const ConvGeom &g);
 lamp_status_t umma_transpose_weights(const bf16 *w, bf16 *wt, int taps, int co, int ci, cudaStream_t st);
 
@@ -126,8 +129,9 @@ lamp_status_t ct_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, cons
                           double *stats, int mirror_taps, cudaStream_t st);
 
 // elementwise.cu
-lamp_status_t k_finalize_stats(const double *stats, float *mu_rstd, int64_t nc, double inv_v, float eps, cudaStream_t st);
-lamp_status_t k_instnorm_relu_fwd(const TView &y, const float *mu_rstd, const TView &z, cudaStream_t st);
+// z = relu((y - mu) * rstd) with (mu, rstd) derived from the fp64 sums; also stores (mu, rstd) to mu_rstd
+lamp_status_t k_instnorm_relu_fwd(const TView &y, const double *stats, float eps, float *mu_rstd, const TView &z,
+                                  cudaStream_t st);
 lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TView &y, const float *mu_rstd,
                                   double *sums, const TView &dy, cudaStream_t st);
 lamp_status_t k_head_softmax(const TView &z, const bf16 *w, const float *b, int K, float *probs, uint8_t *argmax,
@@ -144,9 +148,10 @@ lamp_status_t k_overlap_add(const float *pp, int K, int D, int H, int W, const i
 
 // api.cu: shape checks + kernel selection for one conv pass (used by the ABI and by the U-Net executor)
 lamp_status_t conv_geom(const lamp_conv_desc_t *desc, const lamp_tensor_t *in, const lamp_tensor_t *out, ConvGeom *g);
-size_t        conv_ws_bytes(const ConvGeom &g, int pass);
+size_t        conv_ws_bytes(const ConvGeom &g, int pass);       // scratch with which the pass runs fastest
+size_t        conv_ws_min_bytes(const ConvGeom &g, int pass);   // smallest scratch the pass accepts
 lamp_status_t conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
-                       double *stats, cudaStream_t st);
+                       double *stats, void *ws, size_t ws_bytes, cudaStream_t st);
 lamp_status_t conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w, const TView &dx, void *ws, size_t ws_bytes,
                          cudaStream_t st);
 lamp_status_t conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, float *db, void *ws,

@@ -49,6 +49,8 @@ struct UmmaParams {
     int32_t tw, th, td;            // voxel tile, tw * th * td = 128
     int32_t ntw, nth, ntd;         // tiles per axis
     int32_t nct;                   // c_out tiles
+    int32_t ksplit;                // CTAs that share the (tap, chunk) range of one tile; > 1: y is the fp32 partial buffer
+    int64_t part_stride;           // voxels between the partial results of consecutive splits
     int32_t chunks;                // c_in / KC
     int32_t total_tiles;
     int32_t co;                    // c_out
@@ -61,11 +63,12 @@ struct UmmaParams {
     TapTable taps;
 };
 
-struct Tile { int ct, w0, h0, d0, cls, n; };
+struct Tile { int ks, ct, w0, h0, d0, cls, n; };
 
 __device__ __forceinline__ Tile decode_tile(const UmmaParams &P, int t)
 {
     Tile r;
+    r.ks = t % P.ksplit; t /= P.ksplit;
     r.ct = t % P.nct; t /= P.nct;
     r.w0 = (t % P.ntw) * P.tw; t /= P.ntw;
     r.h0 = (t % P.nth) * P.th; t /= P.nth;
@@ -134,21 +137,21 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             bool ok = true;
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
                 const Tile T = decode_tile(P, tile);
-                const int ntaps = P.taps.ntaps[T.cls];
-                for (int tp = 0; tp < ntaps && ok; ++tp) {
+                const int kit = P.taps.ntaps[T.cls] * P.chunks;
+                const int k1 = kit * (T.ks + 1) / P.ksplit;
+                for (int ki = kit * T.ks / P.ksplit; ki < k1; ++ki) {
+                    const int tp = ki / P.chunks, ch = ki - tp * P.chunks;
                     const int cw = P.in_scale * T.w0 + P.taps.sw[T.cls][tp];
                     const int chh = P.in_scale * T.h0 + P.taps.sh[T.cls][tp];
                     const int cd = P.in_scale * T.d0 + P.taps.sd[T.cls][tp];
                     const int wt = P.taps.wtap[T.cls][tp];
-                    for (int ch = 0; ch < P.chunks; ++ch) {
-                        if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
-                        const uint32_t fb = full0 + 8 * stage;
-                        mbar_expect_tx(fb, L::STAGE_BYTES);
-                        const uint32_t sa = smem_u32(stage_base + stage * L::STAGE_BYTES);
-                        tma_load_5d(sa, &map_x, fb, ch * KC, cw, chh, cd, T.n);
-                        tma_load_3d(sa + L::A_BYTES, &map_w, fb, ch * KC, T.ct * BN, wt);
-                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
-                    }
+                    if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                    const uint32_t fb = full0 + 8 * stage;
+                    mbar_expect_tx(fb, L::STAGE_BYTES);
+                    const uint32_t sa = smem_u32(stage_base + stage * L::STAGE_BYTES);
+                    tma_load_5d(sa, &map_x, fb, ch * KC, cw, chh, cd, T.n);
+                    tma_load_3d(sa + L::A_BYTES, &map_w, fb, ch * KC, T.ct * BN, wt);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
             }
         }
@@ -159,7 +162,9 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             uint32_t phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
-                const int kiters = P.taps.ntaps[decode_tile(P, tile).cls] * P.chunks;
+                const Tile T = decode_tile(P, tile);
+                const int kit = P.taps.ntaps[T.cls] * P.chunks;
+                const int kiters = kit * (T.ks + 1) / P.ksplit - kit * T.ks / P.ksplit;   // >= 1: ksplit <= taps * chunks
                 if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
@@ -214,7 +219,7 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             const int w = P.out_scale * jw + (T.cls & 1), h = P.out_scale * jh + ((T.cls >> 1) & 1),
                       d = P.out_scale * jd + ((T.cls >> 2) & 1);
             const bool valid = (jw < P.W) && (jh < P.H) && (jd < P.D) && (w < P.OW) && (h < P.OH) && (d < P.OD);
-            const int64_t vox = (((int64_t)n * P.OD + d) * P.OH + h) * P.OW + w;
+            const int64_t vox = (((int64_t)n * P.OD + d) * P.OH + h) * P.OW + w + T.ks * P.part_stride;
             // the whole warp takes the same decision, so no lane is left behind at a __syncwarp
             ok = __all_sync(0xffffffffu, mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag));
             if (!ok) break;
@@ -292,6 +297,78 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     }
 }
 
+// Second step of a K-split pass: y = bias + sum over the splits (fixed order) of the fp32 partial results, plus the
+// InstanceNorm sums of the finished values.  A block covers FIN_VOX voxels x 128 channels of one sample: thread =
+// (4 channels, voxel lane), each voxel lane takes FIN_VOX / 8 voxels; the loads of one voxel are independent.
+constexpr int FIN_VOX = 16, FIN_THREADS = 256, FIN_CG = 32;
+
+__global__ void __launch_bounds__(FIN_THREADS)
+splitk_finish_kernel(const float *__restrict__ part, int64_t split_elems, int ksplit, int64_t vox_per_n, int co,
+                     const float *__restrict__ bias, void *__restrict__ y, int y_f32, int64_t y_pitch,
+                     double *__restrict__ stats)
+{
+    __shared__ float4 red[2][FIN_THREADS];
+    const int n = blockIdx.z;
+    const int cl = threadIdx.x % FIN_CG, vl = threadIdx.x / FIN_CG;
+    const int cg = blockIdx.y * FIN_CG + cl;                       // group of 4 channels
+    const bool cok = 4 * cg < co;
+    const int64_t v0 = (int64_t)blockIdx.x * FIN_VOX;
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    const float4 b = (bias && cok) ? __ldg(reinterpret_cast<const float4 *>(bias) + cg) : zero;
+    float4 s1 = zero, s2 = zero;
+    if (cok) {
+#pragma unroll
+        for (int i = 0; i < FIN_VOX / 8; ++i) {
+            const int64_t v = v0 + i * 8 + vl;
+            if (v >= vox_per_n) break;
+            const int64_t vox = (int64_t)n * vox_per_n + v;
+            const float4 *src = reinterpret_cast<const float4 *>(part + vox * co) + cg;
+            const size_t step = (size_t)(split_elems / 4);
+            float4 a = zero;
+            int s = 0;
+            for (; s + 6 <= ksplit; s += 6) {
+                float4 t[6];
+#pragma unroll
+                for (int u = 0; u < 6; ++u) t[u] = __ldcg(src + (size_t)(s + u) * step);
+#pragma unroll
+                for (int u = 0; u < 6; ++u) { a.x += t[u].x; a.y += t[u].y; a.z += t[u].z; a.w += t[u].w; }
+            }
+            for (; s < ksplit; ++s) {
+                const float4 t = __ldcg(src + (size_t)s * step);
+                a.x += t.x; a.y += t.y; a.z += t.z; a.w += t.w;
+            }
+            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+            if (y_f32) {
+                *reinterpret_cast<float4 *>((float *)y + vox * y_pitch + 4 * cg) = a;
+            } else {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
+                uint2 u;
+                u.x = *reinterpret_cast<uint32_t *>(&lo);
+                u.y = *reinterpret_cast<uint32_t *>(&hi);
+                *reinterpret_cast<uint2 *>((bf16 *)y + vox * y_pitch + 4 * cg) = u;
+            }
+            s1.x += a.x; s1.y += a.y; s1.z += a.z; s1.w += a.w;
+            s2.x = fmaf(a.x, a.x, s2.x); s2.y = fmaf(a.y, a.y, s2.y); s2.z = fmaf(a.z, a.z, s2.z); s2.w = fmaf(a.w, a.w, s2.w);
+        }
+    }
+    if (!stats) return;
+    red[0][threadIdx.x] = s1;
+    red[1][threadIdx.x] = s2;
+    __syncthreads();
+    if (vl == 0 && cok) {
+        for (int r = 1; r < FIN_THREADS / FIN_CG; ++r) {           // fixed order over the voxel lanes
+            const float4 p = red[0][r * FIN_CG + cl], q = red[1][r * FIN_CG + cl];
+            s1.x += p.x; s1.y += p.y; s1.z += p.z; s1.w += p.w;
+            s2.x += q.x; s2.y += q.y; s2.z += q.z; s2.w += q.w;
+        }
+        double *dst = stats + ((int64_t)n * co + 4 * cg) * 2;
+        atomicAdd(dst + 0, (double)s1.x); atomicAdd(dst + 1, (double)s2.x);
+        atomicAdd(dst + 2, (double)s1.y); atomicAdd(dst + 3, (double)s2.y);
+        atomicAdd(dst + 4, (double)s1.z); atomicAdd(dst + 5, (double)s2.z);
+        atomicAdd(dst + 6, (double)s1.w); atomicAdd(dst + 7, (double)s2.w);
+    }
+}
+
 __global__ void transpose_weights_kernel(const bf16 *__restrict__ w, bf16 *__restrict__ wt, int co, int ci, int64_t total)
 {
     // wt[t][ci][co] = w[t][co][ci]
@@ -306,6 +383,15 @@ __global__ void transpose_weights_kernel(const bf16 *__restrict__ w, bf16 *__res
 // ----------------------------------------------------------------------------------------------
 // host side
 // ----------------------------------------------------------------------------------------------
+int sm_count()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        sms <= 0)
+        sms = 148;
+    return sms;
+}
+
 PFN_cuTensorMapEncodeTiled_v12000 get_encode()
 {
     static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
@@ -352,9 +438,7 @@ lamp_status_t launch(const CUtensorMap &mx, const CUtensorMap &mw, const UmmaPar
         LAMP_CUDA_OK(cudaFuncSetAttribute(conv3_umma_kernel<KC, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
         attr = true;
     }
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     const int grid = P.total_tiles < sms ? P.total_tiles : sms;
     conv3_umma_kernel<KC, BN><<<grid, NUM_THREADS, L::TOTAL, st>>>(mx, mw, P);
     return launch_status();
@@ -449,7 +533,46 @@ void fill_taps(int kind, TapTable *T)
     }
 }
 
+struct TilePlan { int tw, th, td, ntw, nth, ntd, nct, chunks, KC, BN, ksplit; int64_t tiles; };
+
+// Tiling of a pass, and over how many CTAs the (tap, chunk) range of a tile is split: deep U-Net levels have so few
+// tiles that most SMs would idle, so their K range is shared out and a second small kernel adds the parts.
+TilePlan plan_tiles(int kind, const ConvGeom &g, const KindInfo &k)
+{
+    TilePlan T;
+    T.KC = (k.a_c % 64 == 0) ? 64 : 32;
+    T.BN = pick_bn(k.n_rows);
+    pick_tile(k.jd, k.jh, k.jw, &T.tw, &T.th, &T.td);
+    T.ntw = (k.jw + T.tw - 1) / T.tw; T.nth = (k.jh + T.th - 1) / T.th; T.ntd = (k.jd + T.td - 1) / T.td;
+    T.nct = T.BN ? k.n_rows / T.BN : 0;
+    T.chunks = k.a_c / T.KC;
+    T.tiles = (int64_t)g.n * k.nclass * T.ntd * T.nth * T.ntw * T.nct;
+    TapTable tt;
+    fill_taps(kind, &tt);
+    int min_taps = 27;
+    for (int c = 0; c < k.nclass; ++c) min_taps = tt.ntaps[c] < min_taps ? tt.ntaps[c] : min_taps;
+    const int sms = sm_count();
+    T.ksplit = 1;
+    if (T.tiles > 0 && T.tiles * 2 <= sms) {
+        int s = (int)(sms / T.tiles);
+        const int cap = min_taps * T.chunks / 4;          // at least four (tap, chunk) steps per CTA
+        if (s > cap) s = cap;
+        if (s >= 2) T.ksplit = s;
+    }
+    return T;
+}
+
 }  // namespace
+
+size_t umma_splitk_ws(int kind, const ConvGeom &g)
+{
+    KindInfo k;
+    if (!kind_info(kind, g, &k)) return 0;
+    if (k.a_c % 32 || k.n_rows % 16 || !bn_instantiated(pick_bn(k.n_rows))) return 0;
+    const TilePlan T = plan_tiles(kind, g, k);
+    if (T.ksplit < 2) return 0;
+    return align_up((size_t)T.ksplit * g.n * k.od * k.oh * k.ow * k.n_rows * sizeof(float), 256);
+}
 
 bool umma_conv_supported(int kind, const ConvGeom &g, const TView &a, const TView &y)
 {
@@ -478,28 +601,38 @@ lamp_status_t umma_transpose_weights(const bf16 *w, bf16 *wt, int taps, int co, 
 // a: the tensor the taps read (x for forward kinds, dy for data-gradient kinds); w: [taps][n_rows][a_c] bf16
 // (the layer's weights for forward kinds, their per-tap transpose for data-gradient kinds).
 lamp_status_t umma_conv(int kind, const ConvGeom &g, const TView &a, const bf16 *w, const float *bias, const TView &y,
-                        double *stats, cudaStream_t st)
+                        double *stats, void *part, size_t part_bytes, cudaStream_t st)
 {
     KindInfo k;
     if (!kind_info(kind, g, &k)) return LAMP_ERR_UNSUPPORTED;
     if ((int64_t)g.n * k.jd * k.jh * k.jw == 0) return LAMP_OK;
     PFN_cuTensorMapEncodeTiled_v12000 encode = get_encode();
     if (!encode) return LAMP_ERR_CUDA;
-    const int KC = (k.a_c % 64 == 0) ? 64 : 32;
-    const int BN = pick_bn(k.n_rows);
+    const TilePlan T = plan_tiles(kind, g, k);
+    const int KC = T.KC, BN = T.BN;
+    const int64_t out_vox = (int64_t)g.n * k.od * k.oh * k.ow;
+    // the K range is split only when the caller's scratch can hold the partial results
+    const bool split = T.ksplit > 1 && part && ((uintptr_t)part & 15) == 0 &&
+                       part_bytes >= (size_t)T.ksplit * out_vox * k.n_rows * sizeof(float);
     UmmaParams P;
     P.N = g.n; P.D = k.jd; P.H = k.jh; P.W = k.jw;
     P.OD = k.od; P.OH = k.oh; P.OW = k.ow;
     P.in_scale = k.in_scale; P.out_scale = k.out_scale; P.nclass = k.nclass;
-    pick_tile(k.jd, k.jh, k.jw, &P.tw, &P.th, &P.td);
-    P.ntw = (k.jw + P.tw - 1) / P.tw; P.nth = (k.jh + P.th - 1) / P.th; P.ntd = (k.jd + P.td - 1) / P.td;
-    P.nct = k.n_rows / BN;
-    P.chunks = k.a_c / KC;
-    const int64_t tiles = (int64_t)g.n * k.nclass * P.ntd * P.nth * P.ntw * P.nct;
+    P.tw = T.tw; P.th = T.th; P.td = T.td;
+    P.ntw = T.ntw; P.nth = T.nth; P.ntd = T.ntd;
+    P.nct = T.nct;
+    P.chunks = T.chunks;
+    P.ksplit = split ? T.ksplit : 1;
+    P.part_stride = split ? out_vox : 0;
+    const int64_t tiles = T.tiles * P.ksplit;
     if (tiles > 0x7FFFFFFF) return LAMP_ERR_UNSUPPORTED;
     P.total_tiles = (int32_t)tiles;
-    P.co = k.n_rows; P.y_f32 = y.f32; P.y_pitch = y.pitch; P.y = y.p;
-    P.bias = bias; P.stats = stats; P.status = status_word_ptr();
+    P.co = k.n_rows; P.status = status_word_ptr();
+    if (split) {
+        P.y_f32 = 1; P.y_pitch = k.n_rows; P.y = part; P.bias = nullptr; P.stats = nullptr;
+    } else {
+        P.y_f32 = y.f32; P.y_pitch = y.pitch; P.y = y.p; P.bias = bias; P.stats = stats;
+    }
     fill_taps(kind, &P.taps);
 
     CUtensorMap mx, mw;
@@ -526,7 +659,13 @@ lamp_status_t umma_conv(int kind, const ConvGeom &g, const TView &a, const bf16 
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return LAMP_ERR_CUDA;
     }
-    return KC == 64 ? launch_bn<64>(BN, mx, mw, P, st) : launch_bn<32>(BN, mx, mw, P, st);
+    const lamp_status_t s = KC == 64 ? launch_bn<64>(BN, mx, mw, P, st) : launch_bn<32>(BN, mx, mw, P, st);
+    if (s != LAMP_OK || !split) return s;
+    const int64_t vox_per_n = (int64_t)k.od * k.oh * k.ow;
+    const dim3 grid((unsigned)((vox_per_n + FIN_VOX - 1) / FIN_VOX), (unsigned)((k.n_rows / 4 + FIN_CG - 1) / FIN_CG), (unsigned)g.n);
+    splitk_finish_kernel<<<grid, FIN_THREADS, 0, st>>>((const float *)part, out_vox * k.n_rows, P.ksplit, vox_per_n, k.n_rows,
+                                                      bias, y.p, y.f32, y.pitch, stats);
+    return launch_status();
 }
 
 }  // namespace lamp

@@ -9,23 +9,13 @@ namespace lamp {
 namespace {
 
 // ------------------------------------------------------------------ InstanceNorm forward
-__global__ void finalize_stats_kernel(const double *__restrict__ stats, float *__restrict__ mr, int64_t nc,
-                                      double inv_v, float eps)
-{
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= nc) return;
-    const double mu = stats[2 * i] * inv_v;
-    double var = stats[2 * i + 1] * inv_v - mu * mu;
-    if (var < 0.0) var = 0.0;
-    mr[2 * i] = (float)mu;
-    mr[2 * i + 1] = (float)(1.0 / sqrt(var + (double)eps));
-}
-
 // thread = (voxel row r of the block, group g of 8 channels); the per-channel constants stay in registers
-// while the thread walks its voxels
+// while the thread walks its voxels.  Every thread derives (mu, rstd) of its 8 channels from the fp64 sums - the
+// mean and variance in fp64, the reciprocal square root as one correctly rounded fp32 operation - and the
+// first block of each sample also stores them for the backward pass.
 __global__ void __launch_bounds__(256)
-instnorm_relu_fwd_kernel(const bf16 *__restrict__ y, int64_t yp, const float *__restrict__ mr,
-                         bf16 *__restrict__ z, int64_t zp, int64_t Vn, int C, int64_t v_per_block)
+instnorm_relu_fwd_kernel(const bf16 *__restrict__ y, int64_t yp, const double *__restrict__ stats, double inv_v, float eps,
+                         float *__restrict__ mr, bf16 *__restrict__ z, int64_t zp, int64_t Vn, int C, int64_t v_per_block)
 {
     const int G = C >> 3, RB = 256 / G;
     const int g = threadIdx.x % G, r = threadIdx.x / G;
@@ -34,8 +24,13 @@ instnorm_relu_fwd_kernel(const bf16 *__restrict__ y, int64_t yp, const float *__
     float mu[8], rs[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        mu[j] = mr[((int64_t)n * C + g * 8 + j) * 2];
-        rs[j] = mr[((int64_t)n * C + g * 8 + j) * 2 + 1];
+        const int64_t i = (int64_t)n * C + g * 8 + j;
+        const double m = stats[2 * i] * inv_v;
+        double var = stats[2 * i + 1] * inv_v - m * m;
+        if (var < 0.0) var = 0.0;
+        mu[j] = (float)m;
+        rs[j] = __frsqrt_rn((float)var + eps);
+        if (blockIdx.x == 0 && r == 0) { mr[2 * i] = mu[j]; mr[2 * i + 1] = rs[j]; }
     }
     const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = min(Vn, v0 + v_per_block);
 #pragma unroll 4
@@ -494,14 +489,8 @@ overlap_add_kernel(const float *__restrict__ pp, int Krt, int D, int H, int W, i
 
 }  // namespace
 
-lamp_status_t k_finalize_stats(const double *stats, float *mu_rstd, int64_t nc, double inv_v, float eps, cudaStream_t st)
-{
-    if (nc == 0) return LAMP_OK;
-    finalize_stats_kernel<<<(unsigned)((nc + 127) / 128), 128, 0, st>>>(stats, mu_rstd, nc, inv_v, eps);
-    return launch_status();
-}
-
-lamp_status_t k_instnorm_relu_fwd(const TView &y, const float *mu_rstd, const TView &z, cudaStream_t st)
+lamp_status_t k_instnorm_relu_fwd(const TView &y, const double *stats, float eps, float *mu_rstd, const TView &z,
+                                  cudaStream_t st)
 {
     const int64_t Vn = (int64_t)y.d * y.h * y.w;
     if (Vn == 0 || y.n == 0) return LAMP_OK;
@@ -510,7 +499,8 @@ lamp_status_t k_instnorm_relu_fwd(const TView &y, const float *mu_rstd, const TV
     int64_t vpb = (Vn / (148 * 16) + rb - 1) / rb * rb;
     if (vpb < rb * 8) vpb = rb * 8;
     dim3 grid((unsigned)((Vn + vpb - 1) / vpb), y.n);
-    instnorm_relu_fwd_kernel<<<grid, 256, 0, st>>>((const bf16 *)y.p, y.pitch, mu_rstd, (bf16 *)z.p, z.pitch, Vn, y.c, vpb);
+    instnorm_relu_fwd_kernel<<<grid, 256, 0, st>>>((const bf16 *)y.p, y.pitch, stats, 1.0 / (double)Vn, eps, mu_rstd,
+                                                   (bf16 *)z.p, z.pitch, Vn, y.c, vpb);
     return launch_status();
 }
 

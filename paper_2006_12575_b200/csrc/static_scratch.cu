@@ -36,11 +36,13 @@ extern "C" lamp_status_t lamp_conv3d_dgrad_static_scratch(const lamp_conv_desc_t
                                                           const void *w, lamp_tensor_t *dx, void *cuda_stream)
 {
     if (!desc || !dy || !w || !dx) return LAMP_ERR_INVALID_ARG;
-    const size_t need = lamp_conv3d_workspace_bytes(desc, dx, LAMP_PASS_DGRAD);
+    const size_t need = lamp_conv3d_workspace_min_bytes(desc, dx, LAMP_PASS_DGRAD);
     if (need > (size_t)LAMP_STATIC_SCRATCH_BYTES) return LAMP_ERR_SCRATCH_LIMIT;
     void *scratch = nullptr;
     const lamp_status_t s = scratch_for_current_device(&scratch);
     if (s != LAMP_OK) return s;
     // Nothing in the scratch has to start at zero: the pass overwrites the part it reads.
-    return lamp_conv3d_dgrad(desc, dy, w, dx, scratch, (size_t)LAMP_STATIC_SCRATCH_BYTES, cuda_stream);
+    // Exactly the smallest workspace is handed on, so the pass runs as lamp_conv3d_dgrad does with that workspace
+    // (reduction not split) whatever the layer's size: same kernels, same bits.
+    return lamp_conv3d_dgrad(desc, dy, w, dx, scratch, need, cuda_stream);
 }

@@ -60,6 +60,8 @@ struct Plan {
     float *probs;                       // [V][K] when the caller gave none
     double *dice;                       // [n][K][3]
     double *bwd_sums;                   // [n][cmax][2]
+    void *stats_pool;                   // fp64 [n][c_out][2] of every normalised layer, back to back
+    size_t stats_pool_bytes;
     void *scratch;                      // conv workspace (wgrad partials / transposed weights)
     size_t scratch_bytes;
     size_t total;
@@ -110,6 +112,12 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
     }
     bf16 *yshared = (mode == LAMP_MODE_INFER) ? (bf16 *)A.take(ymax * sizeof(bf16)) : nullptr;
     P->lb.resize(net->layers.size());
+    size_t stats_total = 0;
+    for (const Layer &Ly : net->layers)
+        if (Ly.kind == K_CONV || Ly.kind == K_DOWN) stats_total += align_up((size_t)n * Ly.c_out * 2 * sizeof(double), 256);
+    P->stats_pool = stats_total ? A.take(stats_total) : nullptr;
+    P->stats_pool_bytes = stats_total;
+    size_t stats_off = 0;
     TView cur = view((void *)x_ptr, n, d, h, w, S.in_channels, x_pitch, 0);
     size_t scratch = 0;
     for (size_t i = 0; i < net->layers.size(); ++i) {
@@ -128,7 +136,11 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
             g.transposed = B.desc.transposed;
             B.g = g;
         }
-        if (mode == LAMP_MODE_TRAIN) {
+        if (Ly.kind != K_HEAD) {
+            const size_t s0 = conv_ws_bytes(B.g, LAMP_PASS_FWD);
+            scratch = scratch > s0 ? scratch : s0;
+        }
+        if (mode == LAMP_MODE_TRAIN && Ly.kind != K_HEAD) {
             size_t s1 = conv_ws_bytes(B.g, LAMP_PASS_WGRAD), s2 = conv_ws_bytes(B.g, LAMP_PASS_DGRAD);
             scratch = scratch > s1 ? scratch : s1;
             scratch = scratch > s2 ? scratch : s2;
@@ -136,7 +148,8 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
         if (Ly.kind == K_CONV || Ly.kind == K_DOWN) {
             void *yp = yshared ? (void *)yshared : A.take(vox(l) * Ly.c_out * sizeof(bf16));
             B.y = view(yp, n, dd(l), hh(l), ww(l), Ly.c_out, Ly.c_out, 0);
-            B.stats = (double *)A.take((size_t)n * Ly.c_out * 2 * sizeof(double));
+            B.stats = P->stats_pool ? (double *)((char *)P->stats_pool + stats_off) : nullptr;
+            stats_off += align_up((size_t)n * Ly.c_out * 2 * sizeof(double), 256);
             B.mr = (float *)A.take((size_t)n * Ly.c_out * 2 * sizeof(float));
             if (Ly.to_cat) {
                 B.out = P->cat[l];
@@ -196,6 +209,8 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
                 g = B.din;
             }
         }
+    }
+    if (scratch) {
         P->scratch = A.take(scratch);
         P->scratch_bytes = scratch;
     }
@@ -225,19 +240,18 @@ lamp_status_t run_forward(const lamp_unet *net, const Plan &P, const bf16 *W, co
                           uint8_t *argmax, const uint8_t *labels, double *dice, cudaStream_t st)
 {
     const lamp_unet_spec_t &S = net->spec;
+    // the InstanceNorm sums of all layers sit in one pool: one memset clears them
+    if (P.stats_pool_bytes) LAMP_CUDA_OK(cudaMemsetAsync(P.stats_pool, 0, P.stats_pool_bytes, st));
     for (size_t i = 0; i < net->layers.size(); ++i) {
         const Layer &Ly = net->layers[i];
         const LayerBuf &B = P.lb[i];
         const bf16 *w = W + Ly.w_off;
         const float *b = Bv + Ly.b_off;
         if (Ly.kind == K_CONV || Ly.kind == K_DOWN) {
-            const int64_t Vn = (int64_t)B.y.d * B.y.h * B.y.w;
-            LAMP_CUDA_OK(cudaMemsetAsync(B.stats, 0, (size_t)B.y.n * Ly.c_out * 2 * sizeof(double), st));
-            TRY(conv_fwd(B.g, B.in, w, b, B.y, B.stats, st));
-            TRY(k_finalize_stats(B.stats, B.mr, (int64_t)B.y.n * Ly.c_out, 1.0 / (double)Vn, S.in_eps, st));
-            TRY(k_instnorm_relu_fwd(B.y, B.mr, B.out, st));
+            TRY(conv_fwd(B.g, B.in, w, b, B.y, B.stats, P.scratch, P.scratch_bytes, st));
+            TRY(k_instnorm_relu_fwd(B.y, B.stats, S.in_eps, B.mr, B.out, st));
         } else if (Ly.kind == K_UP) {
-            TRY(conv_fwd(B.g, B.in, w, b, B.out, nullptr, st));
+            TRY(conv_fwd(B.g, B.in, w, b, B.out, nullptr, P.scratch, P.scratch_bytes, st));
         } else {
             TRY(k_head_softmax(B.in, w, b, S.num_classes, probs, argmax, labels, dice, st));
         }

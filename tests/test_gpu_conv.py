@@ -47,6 +47,10 @@ CASES = [
     ("t_c256_h32", 1, 3, 32, 8, 256, 256, 3, 1, 1, 0),
     ("t_c512_to_256", 1, 2, 32, 8, 512, 256, 3, 1, 1, 0),
     ("t_c128_to_384", 1, 2, 30, 16, 128, 384, 3, 1, 1, 0),
+    ("deep_512_cube8", 1, 8, 8, 8, 512, 512, 3, 1, 1, 0),
+    ("deep_512_to_256_ragged", 2, 3, 5, 7, 512, 256, 3, 1, 1, 0),
+    ("deep_down_256_512", 1, 8, 8, 8, 256, 512, 3, 2, 1, 0),
+    ("deep_up_512_256", 1, 4, 4, 4, 512, 256, 2, 2, 0, 1),
     ("tiny_volume", 1, 2, 2, 2, 64, 64, 3, 1, 1, 0),
     ("single_voxel", 1, 1, 1, 1, 32, 32, 3, 1, 1, 0),
 ]
@@ -83,7 +87,9 @@ def test_conv_fwd_matches_oracle(case):
     assert B.lamp_get_async_status() == 0
     assert_close(host_f64(y32), ref, f"{name} fwd f32", rel=2e-5, mx=2e-5)
     s_ref = np.stack([ref.sum(axis=(1, 2, 3)), (ref ** 2).sum(axis=(1, 2, 3))], axis=-1)
-    assert_close(host_f64(stats), s_ref, f"{name} stats", rel=1e-5, mx=1e-4)
+    # the sum of zero-mean values cancels, so its error relative to its own size exceeds that of a single y (fp32
+    # accumulation over up to 27 * 512 products)
+    assert_close(host_f64(stats), s_ref, f"{name} stats", rel=5e-5, mx=1e-4)
     # bf16 output into a channel slice of a wider buffer, no bias
     pitch, off = Co + 16, 8
     ybuf = torch.full(oshape[:4] + (pitch,), 7.0, dtype=torch.bfloat16, device="cuda")
@@ -95,6 +101,24 @@ def test_conv_fwd_matches_oracle(case):
     y2 = torch.empty_like(y32)
     B.lamp_conv3d_fwd(desc, xd, wd, bd, y2)
     assert torch.equal(y2, y32)
+    # with the full workspace a small volume splits its reduction over several CTAs: same checks again
+    nbytes = B.lamp_conv3d_workspace_bytes(desc, xd, B.PASS_FWD)
+    assert B.lamp_conv3d_workspace_min_bytes(desc, xd, B.PASS_FWD) == 0
+    if nbytes:
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        y3 = torch.full(oshape, float("nan"), dtype=torch.float32, device="cuda")
+        stats.zero_()
+        B.lamp_conv3d_fwd(desc, xd, wd, bd, y3, stats, ws)
+        assert B.lamp_get_async_status() == 0
+        assert_close(host_f64(y3), ref, f"{name} fwd f32 split", rel=2e-5, mx=2e-5)
+        assert_close(host_f64(stats), s_ref, f"{name} stats split", rel=5e-5, mx=1e-4)
+        ybuf.fill_(7.0)
+        B.lamp_conv3d_fwd(desc, xd, wd, None, B.tensor(ybuf, Co, off), None, ws)
+        assert_close(host_f64(ybuf[..., off:off + Co]), ops.bf16_round(refnb), f"{name} fwd bf16 slice split")
+        assert (ybuf[..., :off] == 7.0).all() and (ybuf[..., off + Co:] == 7.0).all()
+        y4 = torch.empty_like(y32)
+        B.lamp_conv3d_fwd(desc, xd, wd, bd, y4, None, ws)
+        assert torch.equal(y4, y3)
 
 
 @pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
@@ -119,6 +143,18 @@ def test_conv_dgrad_matches_oracle(case):
         B.lamp_conv3d_dgrad(desc, B.tensor(dyp, Co, 8), wd, B.tensor(dxb, Ci, off), ws)
         assert_close(host_f64(dxb[..., off:]), ops.bf16_round(ref), f"{name} dgrad bf16 slice")
         assert (dxb[..., :off] == 3.0).all()
+    # the smallest accepted workspace (reduction not split) gives the same result within rounding
+    nmin = B.lamp_conv3d_workspace_min_bytes(desc, dx, B.PASS_DGRAD)
+    assert nmin <= nbytes
+    if nmin < nbytes:
+        dx2 = torch.full((N, D, H, W, Ci), float("nan"), dtype=torch.float32, device="cuda")
+        B.lamp_conv3d_dgrad(desc, dyd, wd, dx2, ws[:max(nmin, 16)])
+        assert B.lamp_get_async_status() == 0
+        assert_close(host_f64(dx2), ref, f"{name} dgrad f32 unsplit", rel=2e-5, mx=2e-5)
+    if nmin > 256:
+        with pytest.raises(B.LampError) as e:
+            B.lamp_conv3d_dgrad(desc, dyd, wd, dx, ws[:256])
+        assert e.value.status == 3
 
 
 @pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
