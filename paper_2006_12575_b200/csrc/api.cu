@@ -309,8 +309,8 @@ lamp_status_t lamp_instnorm_relu_bwd(const lamp_tensor_t *dz_a, const lamp_tenso
     }
     TView vb{};
     if (dz_b) vb = make_view(dz_b);
-    return k_instnorm_relu_bwd(make_view(dz_a), dz_b ? &vb : nullptr, make_view(y), mu_rstd, sums, make_view(dy),
-                               (cudaStream_t)cuda_stream);
+    return k_instnorm_relu_bwd(make_view(dz_a), dz_b ? &vb : nullptr, make_view(y), mu_rstd, sums, false, make_view(dy),
+                               nullptr, nullptr, nullptr, (cudaStream_t)cuda_stream);
 }
 
 lamp_status_t lamp_get_async_status(void *cuda_stream)

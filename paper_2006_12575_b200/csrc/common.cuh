@@ -132,14 +132,18 @@ lamp_status_t ct_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, cons
 // z = relu((y - mu) * rstd) with (mu, rstd) derived from the fp64 sums; also stores (mu, rstd) to mu_rstd
 lamp_status_t k_instnorm_relu_fwd(const TView &y, const double *stats, float eps, float *mu_rstd, const TView &z,
                                   cudaStream_t st);
+// sums: fp64 [n][c][2] scratch (cleared here unless sums_are_zero).  db != NULL: also db[c] = sum of the stored dy over
+// voxels and samples, through db_acc (fp64 [c]) and the ticket counter db_count, both zero on entry.
 lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TView &y, const float *mu_rstd,
-                                  double *sums, const TView &dy, cudaStream_t st);
+                                  double *sums, bool sums_are_zero, const TView &dy, double *db_acc, unsigned *db_count,
+                                  float *db, cudaStream_t st);
 lamp_status_t k_head_softmax(const TView &z, const bf16 *w, const float *b, int K, float *probs, uint8_t *argmax,
                              const uint8_t *labels, double *dice_sums, cudaStream_t st);
 lamp_status_t k_dice_loss(const double *dice_sums, int N, int K, float *loss, cudaStream_t st);
+size_t        head_bwd_ws(int64_t Vn, int n, int K, int C);
 lamp_status_t k_head_bwd(const TView &z, const bf16 *w, int K, const float *probs, const uint8_t *labels,
                          const double *dice_sums, const TView &dz, float *dw, float *db, float *dlogits,
-                         cudaStream_t st);
+                         void *ws, size_t ws_bytes, cudaStream_t st);
 lamp_status_t k_gather_patches(const TView &vol, const TView &patches, int first_patch, const int32_t nst[3],
                                const int32_t stride[3], cudaStream_t st);
 lamp_status_t k_overlap_add(const float *pp, int K, int D, int H, int W, const int32_t patch[3],

@@ -102,28 +102,36 @@ instnorm_bwd_sums_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *_
     }
 }
 
-// pass 2: dy = rstd * (g - m1 - xhat * m2); same thread layout as the forward kernel
+// pass 2: dy = rstd * (g - m1 - xhat * m2); same thread layout as the forward kernel.
+// With DB the kernel also forms the bias gradient of the conv in front, db[c] = sum over all voxels and samples of
+// the dy values as stored (bf16): block sums go to db_acc (fp64 atomics, zero on entry) and the block that
+// finishes last (ticket counter db_count, zero on entry) converts the totals to fp32.
+template <bool DB>
 __global__ void __launch_bounds__(256)
 instnorm_bwd_apply_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *__restrict__ dzb, int64_t bp,
                           const bf16 *__restrict__ y, int64_t yp, const float *__restrict__ mr,
                           const double *__restrict__ sums, bf16 *__restrict__ dy, int64_t dp, int64_t Vn, int C,
-                          int64_t v_per_block)
+                          int64_t v_per_block, double *__restrict__ db_acc, unsigned *__restrict__ db_count,
+                          float *__restrict__ db_out)
 {
+    extern __shared__ float cred[];          // DB: [RB][C] column sums of the block
+    __shared__ int is_last;
     const int G = C >> 3, RB = 256 / G;
     const int g = threadIdx.x % G, r = threadIdx.x / G;
-    if (r >= RB) return;
+    const bool active = r < RB;
     const int n = blockIdx.y;
     const float inv_v = 1.0f / (float)Vn;
-    float mu[8], rs[8], m1[8], m2[8];
+    float mu[8], rs[8], m1[8], m2[8], cs[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int64_t i = (int64_t)n * C + g * 8 + j;
-        mu[j] = mr[2 * i];
-        rs[j] = mr[2 * i + 1];
-        m1[j] = (float)sums[2 * i] * inv_v;
-        m2[j] = (float)sums[2 * i + 1] * inv_v;
+        mu[j] = active ? mr[2 * i] : 0.f;
+        rs[j] = active ? mr[2 * i + 1] : 0.f;
+        m1[j] = active ? (float)sums[2 * i] * inv_v : 0.f;
+        m2[j] = active ? (float)sums[2 * i + 1] * inv_v : 0.f;
+        cs[j] = 0.f;
     }
-    const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = min(Vn, v0 + v_per_block);
+    const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = active ? min(Vn, v0 + v_per_block) : v0;
 #pragma unroll 2
     for (int64_t vv = v0 + r; vv < v1; vv += RB) {
         const int64_t v = (int64_t)n * Vn + vv;
@@ -142,68 +150,120 @@ instnorm_bwd_apply_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *
             const float gg = xh > 0.f ? fa[j] : 0.f;
             fa[j] = rs[j] * (gg - m1[j] - xh * m2[j]);
         }
-        *reinterpret_cast<uint4 *>(dy + v * dp + g * 8) = pack8(fa);
+        const uint4 q = pack8(fa);
+        *reinterpret_cast<uint4 *>(dy + v * dp + g * 8) = q;
+        if (DB) {
+            unpack8(q, fa);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) cs[j] += fa[j];
+        }
+    }
+    if (!DB) return;
+    if (active) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) cred[r * C + g * 8 + j] = cs[j];
+    }
+    __syncthreads();
+    for (int c = threadIdx.x; c < C; c += 256) {
+        float a = 0.f;
+        for (int rr = 0; rr < RB; ++rr) a += cred[rr * C + c];
+        atomicAdd(db_acc + c, (double)a);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned total = gridDim.x * gridDim.y;
+        is_last = atomicAdd(db_count, 1u) == total - 1;
+    }
+    __syncthreads();
+    if (is_last) {
+        __threadfence();
+        for (int c = threadIdx.x; c < C; c += 256) db_out[c] = (float)__ldcg(db_acc + c);
     }
 }
 
 // ------------------------------------------------------------------ head: 1x1x1 conv + softmax (+ Dice sums)
 constexpr int KMAX = 16;
 
+// KP = K rounded up to a multiple of 4 (rows k >= K of the weights are zero, their logits are masked).  A block walks
+// tiles of 256 consecutive voxels, one voxel per thread; the probabilities of a tile leave through shared memory so
+// that the [voxel][K] rows are written as one contiguous run.
+template <int KP>
 __global__ void __launch_bounds__(256)
 head_softmax_kernel(const bf16 *__restrict__ z, int64_t zp, int C, const bf16 *__restrict__ w,
                     const float *__restrict__ b, int K, float *__restrict__ probs, uint8_t *__restrict__ amax,
                     const uint8_t *__restrict__ labels, double *__restrict__ dice, int64_t Vn, int64_t v_per_block)
 {
-    extern __shared__ float sm[];           // w as float [K][C], then bias [K], then reduce [3*KMAX]
-    float *sw = sm, *sb = sm + K * C, *sred = sb + KMAX;
-    for (int i = threadIdx.x; i < K * C; i += 256) sw[i] = bf2f(w[i]);
-    if (threadIdx.x < KMAX) sb[threadIdx.x] = (threadIdx.x < K && b) ? b[threadIdx.x] : 0.f;
+    extern __shared__ __align__(16) float sm[];   // w as float [KP][C], bias [KP], reduce [3*KMAX], probability tile [256][K]
+    float *sw = sm, *sb = sm + KP * C, *sred = sb + KP, *sp = sred + 3 * KMAX;
+    for (int i = threadIdx.x; i < KP * C; i += 256) sw[i] = i < K * C ? bf2f(w[i]) : 0.f;
+    if (threadIdx.x < KP) sb[threadIdx.x] = (threadIdx.x < K && b) ? b[threadIdx.x] : 0.f;
     if (threadIdx.x < 3 * KMAX) sred[threadIdx.x] = 0.f;
     __syncthreads();
     const int n = blockIdx.y;
-    float sP[KMAX], sI[KMAX], sG[KMAX];
+    float sP[KP], sI[KP], sG[KP];
 #pragma unroll
-    for (int k = 0; k < KMAX; ++k) { sP[k] = 0.f; sI[k] = 0.f; sG[k] = 0.f; }
+    for (int k = 0; k < KP; ++k) { sP[k] = 0.f; sI[k] = 0.f; sG[k] = 0.f; }
     const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = min(Vn, v0 + v_per_block);
-    for (int64_t vv = v0 + threadIdx.x; vv < v1; vv += 256) {
+    for (int64_t base = v0; base < v1; base += 256) {
+        const int64_t vv = base + threadIdx.x;
+        const bool live = vv < v1;
         const int64_t v = (int64_t)n * Vn + vv;
-        float l[KMAX];
+        if (live) {
+            float l[KP];
 #pragma unroll
-        for (int k = 0; k < KMAX; ++k) l[k] = sb[k];
-        for (int c0 = 0; c0 < C; c0 += 8) {
-            float f[8];
-            unpack8(__ldg(reinterpret_cast<const uint4 *>(z + v * zp + c0)), f);
+            for (int k = 0; k < KP; ++k) l[k] = sb[k];
+            const uint4 *zr = reinterpret_cast<const uint4 *>(z + v * zp);
+            for (int c0 = 0; c0 < C; c0 += 32) {
+                uint4 q[4];
 #pragma unroll
-            for (int k = 0; k < KMAX; ++k) {
-                if (k < K) {
+                for (int u = 0; u < 4; ++u) q[u] = (c0 + 8 * u < C) ? __ldg(zr + (c0 >> 3) + u) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) l[k] = fmaf(f[j], sw[k * C + c0 + j], l[k]);
+                for (int u = 0; u < 4; ++u) {
+                    if (c0 + 8 * u < C) {
+                        float f[8];
+                        unpack8(q[u], f);
+#pragma unroll
+                        for (int k = 0; k < KP; ++k) {
+                            const float4 wa = *reinterpret_cast<const float4 *>(sw + k * C + c0 + 8 * u);
+                            const float4 wb = *reinterpret_cast<const float4 *>(sw + k * C + c0 + 8 * u + 4);
+                            l[k] = fmaf(f[0], wa.x, l[k]); l[k] = fmaf(f[1], wa.y, l[k]);
+                            l[k] = fmaf(f[2], wa.z, l[k]); l[k] = fmaf(f[3], wa.w, l[k]);
+                            l[k] = fmaf(f[4], wb.x, l[k]); l[k] = fmaf(f[5], wb.y, l[k]);
+                            l[k] = fmaf(f[6], wb.z, l[k]); l[k] = fmaf(f[7], wb.w, l[k]);
+                        }
+                    }
                 }
             }
-        }
-        float mx = l[0];
-        int am = 0;
+            float mx = l[0];
+            int am = 0;
 #pragma unroll
-        for (int k = 1; k < KMAX; ++k) if (k < K && l[k] > mx) { mx = l[k]; am = k; }
-        float sum = 0.f;
+            for (int k = 1; k < KP; ++k) if (k < K && l[k] > mx) { mx = l[k]; am = k; }
+            float sum = 0.f;
 #pragma unroll
-        for (int k = 0; k < KMAX; ++k) if (k < K) { l[k] = expf(l[k] - mx); sum += l[k]; }
-        const float inv = 1.0f / sum;
-        const int lab = labels ? labels[v] : -1;
+            for (int k = 0; k < KP; ++k) { l[k] = k < K ? expf(l[k] - mx) : 0.f; sum += l[k]; }
+            const float inv = 1.0f / sum;
+            const int lab = labels ? labels[v] : -1;
 #pragma unroll
-        for (int k = 0; k < KMAX; ++k) {
-            if (k < K) {
+            for (int k = 0; k < KP; ++k) {
                 const float p = l[k] * inv;
-                if (probs) probs[v * K + k] = p;
+                if (k < K) sp[threadIdx.x * K + k] = p;
                 sP[k] += p;
                 if (k == lab) { sI[k] += p; sG[k] += 1.f; }
             }
+            if (amax) amax[v] = (uint8_t)am;
         }
-        if (amax) amax[v] = (uint8_t)am;
+        if (probs) {
+            __syncthreads();
+            const int nv = (int)((v1 - base) < 256 ? (v1 - base) : 256);
+            float *dst = probs + ((int64_t)n * Vn + base) * K;
+            for (int i = threadIdx.x; i < nv * K; i += 256) dst[i] = sp[i];
+            __syncthreads();
+        }
     }
     if (dice) {
 #pragma unroll
-        for (int k = 0; k < KMAX; ++k) {
+        for (int k = 0; k < KP; ++k) {
             if (k < K) {
                 float a = sP[k], bb = sI[k], c = sG[k];
 #pragma unroll
@@ -242,98 +302,135 @@ __global__ void dice_loss_kernel(const double *__restrict__ dice, int N, int K, 
 }
 
 // Head backward: dl = dL/dlogits from (probs, labels, Dice sums); dz = dl * W (bf16);
-// dW[k][c] += sum_v dl[v,k] z[v,c]; db[k] += sum_v dl[v,k].   dW/db must be zero on entry.
+// dW[k][c] = sum_v dl[v,k] z[v,c]; db[k] = sum_v dl[v,k].
+// A block walks tiles of 256 voxels.  Step 1, one voxel per thread: dl (kept in shared memory) and the dz row.
+// Step 2, thread = (pair of channels, voxel lane): the outer products dl x z of the tile's voxels, accumulated in
+// registers over all tiles.  At the end the voxel lanes are added in lane order and the block writes ITS sums to
+// partW[block][K*C], partB[block][K]; a fixed-order reduction over the blocks follows (deterministic).
+template <int KP>
 __global__ void __launch_bounds__(256)
 head_bwd_kernel(const bf16 *__restrict__ z, int64_t zp, int C, const bf16 *__restrict__ w, int K,
                 const float *__restrict__ probs, const uint8_t *__restrict__ labels, const double *__restrict__ dice,
-                int N, bf16 *__restrict__ dz, int64_t dzp, float *__restrict__ dw, float *__restrict__ db,
+                int N, bf16 *__restrict__ dz, int64_t dzp, float *__restrict__ partW, float *__restrict__ partB,
                 float *__restrict__ dlog, int64_t Vn, int64_t v_per_block)
 {
-    extern __shared__ float sm[];
-    // [K*C] weights, [2*KMAX] dice coefficients, [256*KMAX] dl tile, then bf16 z tile [256][C]
-    float *sw = sm, *sa = sm + K * C, *sbq = sa + KMAX, *sdl = sbq + KMAX;
-    bf16 *sz = reinterpret_cast<bf16 *>(sdl + 256 * KMAX);
+    extern __shared__ __align__(16) float sm[];
+    // [KP*C] weights, [KP] + [KP] dice coefficients, then the tile: dl [256][KP], probabilities [256][K], z [256][C] bf16
+    float *sw = sm, *sa = sm + KP * C, *sbq = sa + KP, *sdl = sbq + KP, *sp = sdl + 256 * KP;
+    bf16 *sz = reinterpret_cast<bf16 *>(sp + 256 * K);          // every offset so far is a multiple of 4 floats
     const int n = blockIdx.y;
-    for (int i = threadIdx.x; i < K * C; i += 256) sw[i] = bf2f(w[i]);
-    if (threadIdx.x < K) {
-        const double eps = 1e-5;
-        const double *q = dice + ((int64_t)n * K + threadIdx.x) * 3;
-        const double den = q[1] + q[2] + eps;
-        sa[threadIdx.x] = (float)(2.0 / (den * N * K));
-        sbq[threadIdx.x] = (float)((2.0 * q[0] + eps) / (den * den * N * K));
+    for (int i = threadIdx.x; i < KP * C; i += 256) sw[i] = i < K * C ? bf2f(w[i]) : 0.f;
+    if (threadIdx.x < KP) {
+        float a = 0.f, bq = 0.f;
+        if (threadIdx.x < K) {
+            const double eps = 1e-5;
+            const double *q = dice + ((int64_t)n * K + threadIdx.x) * 3;
+            const double den = q[1] + q[2] + eps;
+            a = (float)(2.0 / (den * N * K));
+            bq = (float)((2.0 * q[0] + eps) / (den * den * N * K));
+        }
+        sa[threadIdx.x] = a;
+        sbq[threadIdx.x] = bq;
     }
-    __syncthreads();
-    const int entries = K * (C + 1);                 // (k, c) for c < C, plus (k, C) = bias
-    constexpr int EPT = 5;                           // entries per thread: K*(C+1) <= 16*65 = 1040 <= 256*5
-    float acc[EPT];
+    const int C8 = C >> 3, CP = C >> 1, VL = 256 / CP;
+    const int cp = threadIdx.x % CP, vl = threadIdx.x / CP;
+    float acc[KP][2], accb[KP];
 #pragma unroll
-    for (int j = 0; j < EPT; ++j) acc[j] = 0.f;
+    for (int k = 0; k < KP; ++k) { acc[k][0] = 0.f; acc[k][1] = 0.f; accb[k] = 0.f; }
     const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = min(Vn, v0 + v_per_block);
     for (int64_t base = v0; base < v1; base += 256) {
-        const int64_t vv = base + threadIdx.x;
-        const bool live = vv < v1;
-        const int64_t v = (int64_t)n * Vn + vv;
-        float dl[KMAX];
-        if (live) {
-            const int lab = labels[v];
-            float p[KMAX], dp[KMAX], dotp = 0.f;
+        const int nv = (int)((v1 - base) < 256 ? (v1 - base) : 256);
+        const int64_t vb = (int64_t)n * Vn + base;
+        __syncthreads();                                         // the previous tile has been consumed
+        for (int i = threadIdx.x; i < nv * K; i += 256) sp[i] = __ldg(probs + vb * K + i);
+        for (int i = threadIdx.x; i < 256 * C8; i += 256) {
+            const int row = i / C8, col = i - row * C8;
+            reinterpret_cast<uint4 *>(sz)[i] =
+                row < nv ? __ldg(reinterpret_cast<const uint4 *>(z + (vb + row) * zp) + col) : make_uint4(0, 0, 0, 0);
+        }
+        __syncthreads();
+        {
+            float dl[KP];
+            if (threadIdx.x < nv) {
+                const int64_t v = vb + threadIdx.x;
+                const int lab = labels[v];
+                float p[KP], dp[KP], dotp = 0.f;
 #pragma unroll
-            for (int k = 0; k < KMAX; ++k) {
-                if (k < K) {
-                    p[k] = probs[v * K + k];
+                for (int k = 0; k < KP; ++k) {
+                    p[k] = k < K ? sp[threadIdx.x * K + k] : 0.f;
                     dp[k] = -((k == lab ? sa[k] : 0.f) - sbq[k]);
                     dotp = fmaf(p[k], dp[k], dotp);
                 }
+#pragma unroll
+                for (int k = 0; k < KP; ++k) {
+                    dl[k] = p[k] * (dp[k] - dotp);
+                    if (k < K && dlog) dlog[v * K + k] = dl[k];
+                }
+                for (int c0 = 0; c0 < C; c0 += 8) {
+                    float f[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) f[j] = 0.f;
+#pragma unroll
+                    for (int k = 0; k < KP; ++k) {
+                        const float4 wa = *reinterpret_cast<const float4 *>(sw + k * C + c0);
+                        const float4 wb = *reinterpret_cast<const float4 *>(sw + k * C + c0 + 4);
+                        f[0] = fmaf(dl[k], wa.x, f[0]); f[1] = fmaf(dl[k], wa.y, f[1]);
+                        f[2] = fmaf(dl[k], wa.z, f[2]); f[3] = fmaf(dl[k], wa.w, f[3]);
+                        f[4] = fmaf(dl[k], wb.x, f[4]); f[5] = fmaf(dl[k], wb.y, f[5]);
+                        f[6] = fmaf(dl[k], wb.z, f[6]); f[7] = fmaf(dl[k], wb.w, f[7]);
+                    }
+                    *reinterpret_cast<uint4 *>(dz + v * dzp + c0) = pack8(f);
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < KP; ++k) dl[k] = 0.f;
             }
 #pragma unroll
-            for (int k = 0; k < KMAX; ++k) {
-                dl[k] = (k < K) ? p[k] * (dp[k] - dotp) : 0.f;
-                if (k < K && dlog) dlog[v * K + k] = dl[k];
-            }
-            for (int c0 = 0; c0 < C; c0 += 8) {
-                float f[8];
+            for (int k4 = 0; k4 < KP / 4; ++k4)
+                *reinterpret_cast<float4 *>(sdl + threadIdx.x * KP + 4 * k4) =
+                    make_float4(dl[4 * k4], dl[4 * k4 + 1], dl[4 * k4 + 2], dl[4 * k4 + 3]);
+        }
+        __syncthreads();
+        if (vl < VL) {
+            for (int t = vl; t < 256; t += VL) {
+                const __nv_bfloat162 zz = *reinterpret_cast<const __nv_bfloat162 *>(sz + t * C + 2 * cp);
+                const float z0 = __low2float(zz), z1 = __high2float(zz);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) f[j] = 0.f;
+                for (int k4 = 0; k4 < KP / 4; ++k4) {
+                    const float4 d = *reinterpret_cast<const float4 *>(sdl + t * KP + 4 * k4);
+                    const float dd[4] = {d.x, d.y, d.z, d.w};
 #pragma unroll
-                for (int k = 0; k < KMAX; ++k) {
-                    if (k < K) {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) f[j] = fmaf(dl[k], sw[k * C + c0 + j], f[j]);
+                    for (int u = 0; u < 4; ++u) {
+                        acc[4 * k4 + u][0] = fmaf(dd[u], z0, acc[4 * k4 + u][0]);
+                        acc[4 * k4 + u][1] = fmaf(dd[u], z1, acc[4 * k4 + u][1]);
+                        if (cp == 0) accb[4 * k4 + u] += dd[u];
                     }
                 }
-                *reinterpret_cast<uint4 *>(dz + v * dzp + c0) = pack8(f);
-                *reinterpret_cast<uint4 *>(sz + (size_t)threadIdx.x * C + c0) =
-                    __ldg(reinterpret_cast<const uint4 *>(z + v * zp + c0));
-            }
-        } else {
-#pragma unroll
-            for (int k = 0; k < KMAX; ++k) dl[k] = 0.f;
-        }
-#pragma unroll
-        for (int k = 0; k < KMAX; ++k) sdl[threadIdx.x * KMAX + k] = dl[k];
-        __syncthreads();
-        const int nv = (int)((v1 - base) < 256 ? (v1 - base) : 256);
-#pragma unroll
-        for (int j = 0; j < EPT; ++j) {
-            const int e = threadIdx.x + j * 256;
-            if (e < entries) {
-                const int k = e / (C + 1), c = e % (C + 1);
-                float a = acc[j];
-                if (c < C) for (int t = 0; t < nv; ++t) a = fmaf(sdl[t * KMAX + k], bf2f(sz[(size_t)t * C + c]), a);
-                else       for (int t = 0; t < nv; ++t) a += sdl[t * KMAX + k];
-                acc[j] = a;
             }
         }
-        __syncthreads();
     }
+    // block totals: red[vl][k][c] over the tile region of shared memory, then entry threads add the lanes in order
+    __syncthreads();
+    float *red = sdl, *redb = sdl + VL * KP * C;
+    if (vl < VL) {
 #pragma unroll
-    for (int j = 0; j < EPT; ++j) {
-        const int e = threadIdx.x + j * 256;
-        if (e < entries) {
-            const int k = e / (C + 1), c = e % (C + 1);
-            if (c < C) atomicAdd(&dw[k * C + c], acc[j]);
-            else if (db) atomicAdd(&db[k], acc[j]);
+        for (int k = 0; k < KP; ++k) {
+            red[(vl * KP + k) * C + 2 * cp] = acc[k][0];
+            red[(vl * KP + k) * C + 2 * cp + 1] = acc[k][1];
+            if (cp == 0) redb[vl * KP + k] = accb[k];
         }
+    }
+    __syncthreads();
+    const int64_t blk = (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
+    for (int e = threadIdx.x; e < K * C; e += 256) {
+        float a = 0.f;
+        for (int r = 0; r < VL; ++r) a += red[r * KP * C + e];      // e = k * C + c
+        partW[blk * K * C + e] = a;
+    }
+    if (threadIdx.x < K) {
+        float a = 0.f;
+        for (int r = 0; r < VL; ++r) a += redb[r * KP + threadIdx.x];
+        partB[blk * K + threadIdx.x] = a;
     }
 }
 
@@ -505,13 +602,17 @@ lamp_status_t k_instnorm_relu_fwd(const TView &y, const double *stats, float eps
 }
 
 lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TView &y, const float *mu_rstd,
-                                  double *sums, const TView &dy, cudaStream_t st)
+                                  double *sums, bool sums_are_zero, const TView &dy, double *db_acc, unsigned *db_count,
+                                  float *db, cudaStream_t st)
 {
     const int64_t Vn = (int64_t)y.d * y.h * y.w;
     const int C = y.c, G = C / 8;
     if (G > 256) return LAMP_ERR_UNSUPPORTED;
-    LAMP_CUDA_OK(cudaMemsetAsync(sums, 0, (size_t)y.n * C * 2 * sizeof(double), st));
-    if (Vn == 0 || y.n == 0) return LAMP_OK;
+    if (!sums_are_zero) LAMP_CUDA_OK(cudaMemsetAsync(sums, 0, (size_t)y.n * C * 2 * sizeof(double), st));
+    if (Vn == 0 || y.n == 0) {
+        if (db) LAMP_CUDA_OK(cudaMemsetAsync(db, 0, (size_t)C * sizeof(float), st));
+        return LAMP_OK;
+    }
     const int RB = 256 / G;
     int64_t blocks = (148 * 8 + y.n - 1) / y.n;
     const int64_t max_blocks = (Vn + RB - 1) / RB;
@@ -525,9 +626,14 @@ lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TVie
     int64_t vpa = (Vn / (148 * 16) + RB - 1) / RB * RB;
     if (vpa < (int64_t)RB * 8) vpa = (int64_t)RB * 8;
     dim3 grid((unsigned)((Vn + vpa - 1) / vpa), y.n);
-    instnorm_bwd_apply_kernel<<<grid, 256, 0, st>>>(
-        (const bf16 *)dza.p, dza.pitch, dzb ? (const bf16 *)dzb->p : nullptr, dzb ? dzb->pitch : 0,
-        (const bf16 *)y.p, y.pitch, mu_rstd, sums, (bf16 *)dy.p, dy.pitch, Vn, C, vpa);
+    if (db)
+        instnorm_bwd_apply_kernel<true><<<grid, 256, (size_t)RB * C * sizeof(float), st>>>(
+            (const bf16 *)dza.p, dza.pitch, dzb ? (const bf16 *)dzb->p : nullptr, dzb ? dzb->pitch : 0,
+            (const bf16 *)y.p, y.pitch, mu_rstd, sums, (bf16 *)dy.p, dy.pitch, Vn, C, vpa, db_acc, db_count, db);
+    else
+        instnorm_bwd_apply_kernel<false><<<grid, 256, 0, st>>>(
+            (const bf16 *)dza.p, dza.pitch, dzb ? (const bf16 *)dzb->p : nullptr, dzb ? dzb->pitch : 0,
+            (const bf16 *)y.p, y.pitch, mu_rstd, sums, (bf16 *)dy.p, dy.pitch, Vn, C, vpa, nullptr, nullptr, nullptr);
     return launch_status();
 }
 
@@ -542,18 +648,30 @@ static void head_grid(int64_t Vn, int n, int64_t &blocks, int64_t &vpb)
     blocks = (Vn + vpb - 1) / vpb;
 }
 
+static int head_kp(int K) { return (K + 3) / 4 * 4; }
+
 lamp_status_t k_head_softmax(const TView &z, const bf16 *w, const float *b, int K, float *probs, uint8_t *argmax,
                              const uint8_t *labels, double *dice_sums, cudaStream_t st)
 {
     const int64_t Vn = (int64_t)z.d * z.h * z.w;
-    if (K > KMAX || K < 1) return LAMP_ERR_UNSUPPORTED;
+    if (K > KMAX || K < 1 || z.c > 64 || z.c % 8) return LAMP_ERR_UNSUPPORTED;
     if (dice_sums) LAMP_CUDA_OK(cudaMemsetAsync(dice_sums, 0, (size_t)z.n * K * 3 * sizeof(double), st));
     if (Vn == 0 || z.n == 0) return LAMP_OK;
     int64_t blocks, vpb;
     head_grid(Vn, z.n, blocks, vpb);
-    const size_t smem = ((size_t)K * z.c + KMAX + 3 * KMAX) * sizeof(float);
-    head_softmax_kernel<<<dim3((unsigned)blocks, z.n), 256, smem, st>>>(
-        (const bf16 *)z.p, z.pitch, z.c, w, b, K, probs, argmax, labels, dice_sums, Vn, vpb);
+    const int KP = head_kp(K);
+    const size_t smem = ((size_t)KP * z.c + KP + 3 * KMAX + 256 * K) * sizeof(float);
+    const dim3 grid((unsigned)blocks, z.n);
+#define LAMP_HEAD_FWD(kp)                                                                                         \
+    head_softmax_kernel<kp><<<grid, 256, smem, st>>>((const bf16 *)z.p, z.pitch, z.c, w, b, K, probs, argmax, labels, \
+                                                     dice_sums, Vn, vpb)
+    switch (KP) {
+    case 4:  LAMP_HEAD_FWD(4); break;
+    case 8:  LAMP_HEAD_FWD(8); break;
+    case 12: LAMP_HEAD_FWD(12); break;
+    default: LAMP_HEAD_FWD(16); break;
+    }
+#undef LAMP_HEAD_FWD
     return launch_status();
 }
 
@@ -563,28 +681,63 @@ lamp_status_t k_dice_loss(const double *dice_sums, int N, int K, float *loss, cu
     return launch_status();
 }
 
+size_t head_bwd_ws(int64_t Vn, int n, int K, int C)
+{
+    if (Vn <= 0 || n <= 0) return 0;
+    int64_t blocks, vpb;
+    head_grid(Vn, n, blocks, vpb);
+    return align_up((size_t)blocks * n * K * C * sizeof(float), 256) + align_up((size_t)blocks * n * K * sizeof(float), 256);
+}
+
+template <int KP>
+static lamp_status_t launch_head_bwd(const TView &z, const bf16 *w, int K, const float *probs, const uint8_t *labels,
+                                     const double *dice_sums, const TView &dz, float *partW, float *partB, float *dlogits,
+                                     int64_t Vn, int64_t blocks, int64_t vpb, cudaStream_t st)
+{
+    const int C = z.c;
+    // the tile region (dl, probabilities, z) is reused for the end-of-block reduction [lanes][KP][C] + [lanes][KP]
+    const size_t lanes = 256 / (C / 2);
+    const size_t tile = (size_t)256 * KP + 256 * K + 128 * C, red = lanes * KP * C + lanes * KP;
+    const size_t smem = ((size_t)KP * C + 2 * KP + (tile > red ? tile : red)) * sizeof(float);
+    static bool attr_set = false;
+    if (!attr_set) {
+        LAMP_CUDA_OK(cudaFuncSetAttribute(head_bwd_kernel<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
+        attr_set = true;
+    }
+    head_bwd_kernel<KP><<<dim3((unsigned)blocks, z.n), 256, smem, st>>>(
+        (const bf16 *)z.p, z.pitch, C, w, K, probs, labels, dice_sums, z.n, (bf16 *)dz.p, dz.pitch, partW, partB, dlogits,
+        Vn, vpb);
+    return launch_status();
+}
+
+// ws: head_bwd_ws bytes (per-block partial sums of dW and db)
 lamp_status_t k_head_bwd(const TView &z, const bf16 *w, int K, const float *probs, const uint8_t *labels,
                          const double *dice_sums, const TView &dz, float *dw, float *db, float *dlogits,
-                         cudaStream_t st)
+                         void *ws, size_t ws_bytes, cudaStream_t st)
 {
     const int64_t Vn = (int64_t)z.d * z.h * z.w;
     const int C = z.c;
-    if (K > KMAX || C > 64) return LAMP_ERR_UNSUPPORTED;
-    LAMP_CUDA_OK(cudaMemsetAsync(dw, 0, (size_t)K * C * sizeof(float), st));
-    if (db) LAMP_CUDA_OK(cudaMemsetAsync(db, 0, (size_t)K * sizeof(float), st));
-    if (Vn == 0 || z.n == 0) return LAMP_OK;
+    if (K > KMAX || C > 64 || C % 8) return LAMP_ERR_UNSUPPORTED;
+    if (Vn == 0 || z.n == 0) {
+        LAMP_CUDA_OK(cudaMemsetAsync(dw, 0, (size_t)K * C * sizeof(float), st));
+        if (db) LAMP_CUDA_OK(cudaMemsetAsync(db, 0, (size_t)K * sizeof(float), st));
+        return LAMP_OK;
+    }
+    if (!ws || ws_bytes < head_bwd_ws(Vn, z.n, K, C)) return LAMP_ERR_WORKSPACE;
     int64_t blocks, vpb;
     head_grid(Vn, z.n, blocks, vpb);
-    const size_t smem = ((size_t)K * C + 2 * KMAX + 256 * KMAX) * sizeof(float) + (size_t)256 * C * sizeof(bf16);
-    static bool attr_set = false;
-    if (!attr_set) {
-        LAMP_CUDA_OK(cudaFuncSetAttribute(head_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
-        attr_set = true;
+    float *partW = (float *)ws;
+    float *partB = (float *)((char *)ws + align_up((size_t)blocks * z.n * K * C * sizeof(float), 256));
+    lamp_status_t s;
+    switch (head_kp(K)) {
+    case 4:  s = launch_head_bwd<4>(z, w, K, probs, labels, dice_sums, dz, partW, partB, dlogits, Vn, blocks, vpb, st); break;
+    case 8:  s = launch_head_bwd<8>(z, w, K, probs, labels, dice_sums, dz, partW, partB, dlogits, Vn, blocks, vpb, st); break;
+    case 12: s = launch_head_bwd<12>(z, w, K, probs, labels, dice_sums, dz, partW, partB, dlogits, Vn, blocks, vpb, st); break;
+    default: s = launch_head_bwd<16>(z, w, K, probs, labels, dice_sums, dz, partW, partB, dlogits, Vn, blocks, vpb, st); break;
     }
-    head_bwd_kernel<<<dim3((unsigned)blocks, z.n), 256, smem, st>>>(
-        (const bf16 *)z.p, z.pitch, C, w, K, probs, labels, dice_sums, z.n, (bf16 *)dz.p, dz.pitch, dw, db,
-        dlogits, Vn, vpb);
-    return launch_status();
+    if (s != LAMP_OK) return s;
+    if ((s = reduce_partials(partW, (int64_t)K * C, (int)(blocks * z.n), dw, st)) != LAMP_OK) return s;
+    return db ? reduce_partials(partB, K, (int)(blocks * z.n), db, st) : LAMP_OK;
 }
 
 lamp_status_t k_gather_patches(const TView &vol, const TView &patches, int first_patch, const int32_t nst[3],

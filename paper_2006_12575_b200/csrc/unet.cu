@@ -47,6 +47,9 @@ struct LayerBuf {
     TView y;                    // raw conv output (norm layers)
     double *stats;              // [n][c_out][2]
     float *mr;                  // [n][c_out][2]
+    double *bsums;              // InstanceNorm backward sums [n][c_out][2] (train mode)
+    double *db_acc;             // bias-gradient totals [c_out] in fp64 and the ticket counter of their reduction
+    unsigned *db_count;
     TView dy;                   // gradient w.r.t. the raw conv output (norm layers; train mode)
     TView din;                  // gradient w.r.t. the layer's input (train mode; empty for layer 0)
     TView dout, dout2;          // gradient w.r.t. the layer's output: main source and skip source (may be empty)
@@ -59,7 +62,8 @@ struct Plan {
     std::vector<TView> cat, dcat;       // per level (levels - 1 entries)
     float *probs;                       // [V][K] when the caller gave none
     double *dice;                       // [n][K][3]
-    double *bwd_sums;                   // [n][cmax][2]
+    void *bwd_pool;                     // per normalised layer: fp64 sums [n][c][2], fp64 db totals [c], ticket counter
+    size_t bwd_pool_bytes;
     void *stats_pool;                   // fp64 [n][c_out][2] of every normalised layer, back to back
     size_t stats_pool_bytes;
     void *scratch;                      // conv workspace (wgrad partials / transposed weights)
@@ -105,10 +109,9 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
         void *p = A.take(vox(l) * 2 * S.channels[l] * sizeof(bf16));
         P->cat[l] = view(p, n, dd(l), hh(l), ww(l), 2 * S.channels[l], 2 * S.channels[l], 0);
     }
-    size_t ymax = 0, cmax = 0;
+    size_t ymax = 0;
     for (const Layer &Ly : net->layers) {
         if (Ly.kind == K_CONV || Ly.kind == K_DOWN) ymax = ymax > vox(Ly.level) * Ly.c_out ? ymax : vox(Ly.level) * Ly.c_out;
-        cmax = cmax > (size_t)Ly.c_out ? cmax : (size_t)Ly.c_out;
     }
     bf16 *yshared = (mode == LAMP_MODE_INFER) ? (bf16 *)A.take(ymax * sizeof(bf16)) : nullptr;
     P->lb.resize(net->layers.size());
@@ -140,6 +143,10 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
             const size_t s0 = conv_ws_bytes(B.g, LAMP_PASS_FWD);
             scratch = scratch > s0 ? scratch : s0;
         }
+        if (mode == LAMP_MODE_TRAIN && Ly.kind == K_HEAD) {
+            const size_t s3 = head_bwd_ws((int64_t)cur.d * cur.h * cur.w, n, S.num_classes, Ly.c_in);
+            scratch = scratch > s3 ? scratch : s3;
+        }
         if (mode == LAMP_MODE_TRAIN && Ly.kind != K_HEAD) {
             size_t s1 = conv_ws_bytes(B.g, LAMP_PASS_WGRAD), s2 = conv_ws_bytes(B.g, LAMP_PASS_DGRAD);
             scratch = scratch > s1 ? scratch : s1;
@@ -170,14 +177,36 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
     }
     const size_t V0 = vox(0);
     P->probs = need_probs ? (float *)A.take(V0 * S.num_classes * sizeof(float)) : nullptr;
-    P->dice = nullptr; P->bwd_sums = nullptr;
+    P->dice = nullptr; P->bwd_pool = nullptr; P->bwd_pool_bytes = 0;
     P->scratch = nullptr; P->scratch_bytes = 0;
-    for (LayerBuf &B : P->lb) { B.dy = TView{}; B.din = TView{}; B.dout = TView{}; B.dout2 = TView{}; }
+    for (LayerBuf &B : P->lb) {
+        B.dy = TView{}; B.din = TView{}; B.dout = TView{}; B.dout2 = TView{};
+        B.bsums = nullptr; B.db_acc = nullptr; B.db_count = nullptr;
+    }
     if (mode == LAMP_MODE_TRAIN) {
         // Every gradient tensor gets its own buffer (nothing is recycled), so that each step of the
         // backward pass can be inspected after the call.
         P->dice = (double *)A.take((size_t)n * S.num_classes * 3 * sizeof(double));
-        P->bwd_sums = (double *)A.take((size_t)n * cmax * 2 * sizeof(double));
+        size_t pool = 0;
+        for (const Layer &Ly : net->layers)
+            if (Ly.kind == K_CONV || Ly.kind == K_DOWN)
+                pool += align_up((size_t)n * Ly.c_out * 2 * sizeof(double), 256) + align_up((size_t)Ly.c_out * sizeof(double), 256) + 256;
+        P->bwd_pool = A.take(pool);
+        P->bwd_pool_bytes = pool;
+        size_t poff = 0;
+        for (size_t i = 0; i < net->layers.size(); ++i) {
+            const Layer &Ly = net->layers[i];
+            LayerBuf &B = P->lb[i];
+            B.bsums = nullptr; B.db_acc = nullptr; B.db_count = nullptr;
+            if (Ly.kind != K_CONV && Ly.kind != K_DOWN) continue;
+            char *base = (char *)P->bwd_pool;
+            B.bsums = base ? (double *)(base + poff) : nullptr;
+            poff += align_up((size_t)n * Ly.c_out * 2 * sizeof(double), 256);
+            B.db_acc = base ? (double *)(base + poff) : nullptr;
+            poff += align_up((size_t)Ly.c_out * sizeof(double), 256);
+            B.db_count = base ? (unsigned *)(base + poff) : nullptr;
+            poff += 256;
+        }
         for (int l = 0; l + 1 < L; ++l) {
             void *p = A.take(vox(l) * 2 * S.channels[l] * sizeof(bf16));
             P->dcat[l] = view(p, n, dd(l), hh(l), ww(l), 2 * S.channels[l], 2 * S.channels[l], 0);
@@ -405,19 +434,22 @@ lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_b
     TRY(run_forward(net, P, W, biases_f32, probs, nullptr, labels, P.dice, st));
     TRY(k_dice_loss(P.dice, x->n, S.num_classes, loss, st));
 
-    // backward, last layer first
+    // backward, last layer first; one memset clears every layer's reduction scratch
+    LAMP_CUDA_OK(cudaMemsetAsync(P.bwd_pool, 0, P.bwd_pool_bytes, st));
     for (int i = (int)net->layers.size() - 1; i >= 0; --i) {
         const Layer &Ly = net->layers[i];
         const LayerBuf &B = P.lb[i];
         const bf16 *w = W + Ly.w_off;
         float *dw = grad_w + Ly.w_off, *db = grad_b + Ly.b_off;
         if (Ly.kind == K_HEAD) {
-            TRY(k_head_bwd(B.in, w, S.num_classes, probs, labels, P.dice, B.din, dw, db, nullptr, st));
+            TRY(k_head_bwd(B.in, w, S.num_classes, probs, labels, P.dice, B.din, dw, db, nullptr, P.scratch, P.scratch_bytes, st));
             continue;
         }
         if (Ly.kind != K_UP)
-            TRY(k_instnorm_relu_bwd(B.dout, Ly.to_cat ? &B.dout2 : nullptr, B.y, B.mr, P.bwd_sums, B.dy, st));
-        TRY(conv_wgrad(B.g, B.in, B.dy, dw, db, P.scratch, P.scratch_bytes, st));
+            TRY(k_instnorm_relu_bwd(B.dout, Ly.to_cat ? &B.dout2 : nullptr, B.y, B.mr, B.bsums, true, B.dy, B.db_acc,
+                                    B.db_count, db, st));
+        // the bias gradient of a normalised layer came out of the InstanceNorm backward kernel above
+        TRY(conv_wgrad(B.g, B.in, B.dy, dw, Ly.kind == K_UP ? db : nullptr, P.scratch, P.scratch_bytes, st));
         if (i == 0) break;
         TRY(conv_dgrad(B.g, B.dy, w, B.din, P.scratch, P.scratch_bytes, st));
     }
