@@ -93,6 +93,10 @@ lamp_status_t simt_conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy
 
 // out[e] = sum_s part[s][e] in a fixed order; dbias[co] = sum_v dy[v][co] (ws: bias_grad_ws bytes)
 lamp_status_t reduce_partials(const float *part, int64_t entries, int splits, float *out, cudaStream_t st);
+// out[t][b][a] = sum_s in[s][t][a][b] (A, B multiples of 32, see transpose_sum_supported); bf16 form: one split
+bool          transpose_sum_supported(int64_t taps, int A, int B);
+lamp_status_t transpose_sum_f32(const float *in, int64_t taps, int A, int B, int splits, float *out, cudaStream_t st);
+lamp_status_t transpose_bf16(const bf16 *in, int64_t taps, int A, int B, bf16 *out, cudaStream_t st);
 size_t        bias_grad_ws(int64_t voxels, int co);
 lamp_status_t bias_grad(const TView &dy, float *db, void *ws, cudaStream_t st);
 

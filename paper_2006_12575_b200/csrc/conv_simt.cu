@@ -407,6 +407,47 @@ reduce_parts_kernel(const float *__restrict__ part, int64_t entries, int splits,
     }
 }
 
+// The same sum for few splits over many entries: a thread owns 4 consecutive entries and adds the splits in order.
+__global__ void __launch_bounds__(256)
+reduce_parts_vec4_kernel(const float4 *__restrict__ part, int64_t entries4, int splits, float4 *__restrict__ out)
+{
+    const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (e >= entries4) return;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+    for (int s = 0; s < splits; ++s) {
+        const float4 t = __ldcg(part + (int64_t)s * entries4 + e);
+        a.x += t.x; a.y += t.y; a.z += t.z; a.w += t.w;
+    }
+    out[e] = a;
+}
+
+// out[t][b][a] = sum_s in[s][t][a][b] through 32 x 32 shared-memory tiles (A, B multiples of 32): reads run along b,
+// writes along a.  With one split and bf16 data this is the per-tap transpose of a weight tensor.
+template <typename T>
+__global__ void __launch_bounds__(256)
+transpose_sum_kernel(const T *__restrict__ in, int64_t split_stride, int splits, int A, int B, T *__restrict__ out)
+{
+    __shared__ float tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;           // 32 x 8
+    const int b0 = blockIdx.x * 32, a0 = blockIdx.y * 32;
+    const int64_t t = blockIdx.z;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int a = a0 + ty + 8 * i;
+        const int64_t src = (t * A + a) * B + b0 + tx;
+        float acc = 0.f;
+        for (int s = 0; s < splits; ++s) acc += (float)in[(int64_t)s * split_stride + src];
+        tile[ty + 8 * i][tx] = acc;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int b = b0 + ty + 8 * i;
+        out[(t * B + b) * A + a0 + tx] = (T)tile[tx][ty + 8 * i];
+    }
+}
+
 // xpad[v][0] = x[v], xpad[v][1..31] = 0 (the 1-channel input widened to one 32-channel chunk)
 __global__ void __launch_bounds__(256)
 pad_c1_kernel(const bf16 *__restrict__ x, int64_t xp, bf16 *__restrict__ xpad, int64_t V)
@@ -500,7 +541,25 @@ lamp_status_t simt_conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w,
 lamp_status_t reduce_partials(const float *part, int64_t entries, int splits, float *out, cudaStream_t st)
 {
     if (entries == 0) return LAMP_OK;
-    reduce_parts_kernel<<<(unsigned)((entries + 31) / 32), 256, 0, st>>>(part, entries, splits, out);
+    if (splits <= 16 && entries >= 32768 && entries % 4 == 0 && (((uintptr_t)part | (uintptr_t)out) & 15) == 0)
+        reduce_parts_vec4_kernel<<<(unsigned)((entries / 4 + 255) / 256), 256, 0, st>>>(
+            (const float4 *)part, entries / 4, splits, (float4 *)out);
+    else
+        reduce_parts_kernel<<<(unsigned)((entries + 31) / 32), 256, 0, st>>>(part, entries, splits, out);
+    return launch_status();
+}
+
+bool transpose_sum_supported(int64_t taps, int A, int B) { return A % 32 == 0 && B % 32 == 0 && taps > 0 && taps <= 65535; }
+
+lamp_status_t transpose_sum_f32(const float *in, int64_t taps, int A, int B, int splits, float *out, cudaStream_t st)
+{
+    transpose_sum_kernel<float><<<dim3(B / 32, A / 32, (unsigned)taps), 256, 0, st>>>(in, taps * A * B, splits, A, B, out);
+    return launch_status();
+}
+
+lamp_status_t transpose_bf16(const bf16 *in, int64_t taps, int A, int B, bf16 *out, cudaStream_t st)
+{
+    transpose_sum_kernel<bf16><<<dim3(B / 32, A / 32, (unsigned)taps), 256, 0, st>>>(in, 0, 1, A, B, out);
     return launch_status();
 }
 

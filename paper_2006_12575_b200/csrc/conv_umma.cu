@@ -594,6 +594,7 @@ size_t umma_dgrad_ws(const ConvGeom &g)
 lamp_status_t umma_transpose_weights(const bf16 *w, bf16 *wt, int taps, int co, int ci, cudaStream_t st)
 {
     const int64_t total = (int64_t)taps * co * ci;
+    if (transpose_sum_supported(taps, co, ci)) return transpose_bf16(w, taps, co, ci, wt, st);
     transpose_weights_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w, wt, co, ci, total);
     return launch_status();
 }

@@ -418,6 +418,9 @@ lamp_status_t umma_wgrad(const ConvGeom &g, const TView &x, const TView &dy, flo
     }
     if (s != LAMP_OK || direct) return s;
     if (!pl.g_is_x) return reduce_partials(pl.P.part, pl.P.entries, pl.P.nsplit, dw, st);
+    // partials are [tap][c_in][c_out]; dw is [tap][c_out][c_in]
+    const int taps = g.k * g.k * g.k;
+    if (transpose_sum_supported(taps, g.ci, g.co)) return transpose_sum_f32(pl.P.part, taps, g.ci, g.co, pl.P.nsplit, dw, st);
     reduce_transposed_kernel<<<(unsigned)((pl.P.entries + 255) / 256), 256, 0, st>>>(pl.P.part, pl.P.entries, pl.P.nsplit, g.ci, g.co, dw);
     return launch_status();
 }
