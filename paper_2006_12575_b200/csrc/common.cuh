@@ -117,7 +117,8 @@ lamp_status_t win_wgrad(const ConvGeom &g, const TView &x, const TView &dy, floa
                         cudaStream_t st);
 
 // conv_umma.cu (tcgen05 implicit GEMM, voxels x channels form; see the file header for the kinds)
-enum { UK_S1_FWD = 0, UK_S1_DGRAD = 1, UK_S2_FWD = 2, UK_S2_DGRAD = 3, UK_T_FWD = 4, UK_T_DGRAD = 5 };
+enum { UK_S1_FWD = 0, UK_S1_DGRAD = 1, UK_S2_FWD = 2, UK_S2_DGRAD = 3, UK_T_FWD = 4, UK_T_DGRAD = 5,
+       UK_T_FWD_MERGED = 6 /* internal: chosen by umma_conv for UK_T_FWD when c_out % 32 == 0 and no statistics */ };
 bool          umma_conv_supported(int kind, const ConvGeom &g, const TView &a, const TView &y);
 // part / part_bytes: optional scratch of umma_splitk_ws bytes; with it a pass that has too few tiles to fill the
 // GPU splits its K range over several CTAs (fp32 partial results, added in a fixed order by a second kernel)

@@ -54,7 +54,9 @@ struct UmmaParams {
     int32_t chunks;                // c_in / KC
     int32_t total_tiles;
     int32_t co;                    // c_out
+    int32_t merge_co;              // > 0: the N axis carries (parity class, channel) pairs, class = column / merge_co
     int32_t y_f32;
+    int32_t st32;                  // output rows may be written with 32-byte stores (base, pitch and slice offset allow it)
     int64_t y_pitch;
     void   *y;
     const float *bias;
@@ -78,28 +80,57 @@ __device__ __forceinline__ Tile decode_tile(const UmmaParams &P, int t)
     return r;
 }
 
-constexpr int NUM_THREADS = 192;
 constexpr int MAX_STAGES = 8;
+constexpr int MAX_ACC = 4;
+constexpr int MAX_SBIAS = 2048;         // bias vectors up to this length are staged in shared memory
+
+// Column sums of a 32 x 32 tile held one row per lane: after the exchange with lane ^ 16 a lane keeps 16 columns
+// (two rows added), after lane ^ 8 eight columns, ... and finally lane j holds column j summed over all rows.
+__device__ __forceinline__ float warp_colsum32(const float (&v)[32], int lane)
+{
+    float a[16], b[8], c[4], d[2];
+    const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4, h2 = lane & 2, h1 = lane & 1;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) a[i] = (h16 ? v[i + 16] : v[i]) + __shfl_xor_sync(0xffffffffu, h16 ? v[i] : v[i + 16], 16);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) b[i] = (h8 ? a[i + 8] : a[i]) + __shfl_xor_sync(0xffffffffu, h8 ? a[i] : a[i + 8], 8);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) c[i] = (h4 ? b[i + 4] : b[i]) + __shfl_xor_sync(0xffffffffu, h4 ? b[i] : b[i + 4], 4);
+#pragma unroll
+    for (int i = 0; i < 2; ++i) d[i] = (h2 ? c[i + 2] : c[i]) + __shfl_xor_sync(0xffffffffu, h2 ? c[i] : c[i + 2], 2);
+    return (h1 ? d[1] : d[0]) + __shfl_xor_sync(0xffffffffu, h1 ? d[0] : d[1], 1);
+}
+
+__device__ __forceinline__ void st_global_32B(void *p, const uint32_t (&u)[8])
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 :: "l"(p), "r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7])
+                 : "memory");
+}
 
 template <int KC, int BN>
 struct SmemLayout {
     static constexpr int A_BYTES = 128 * KC * 2;
     static constexpr int B_BYTES = BN * KC * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;      // multiple of 1024 for every (KC, BN)
-    static constexpr int EPI_BYTES = 4 * 32 * 33 * 4;
+    static constexpr int EPI_BYTES = MAX_SBIAS * 4;                    // the staged bias
+    // accumulators in TMEM, each drained by its own set of four epilogue warps (one warp per TMEM lane quarter)
+    static constexpr int NACC = BN >= 256 ? 2 : (BN >= 64 ? 3 : 4);
+    static constexpr int THREADS = 64 + 128 * NACC;
     static constexpr int CTRL_BYTES = 1024;
     static constexpr int BUDGET = 227 * 1024 - 1024 /* alignment slack */ - EPI_BYTES - CTRL_BYTES;
     static constexpr int STAGES = (BUDGET / STAGE_BYTES) < MAX_STAGES ? (BUDGET / STAGE_BYTES) : MAX_STAGES;
     static constexpr int TOTAL = 1024 + STAGES * STAGE_BYTES + EPI_BYTES + CTRL_BYTES;
-    static constexpr int TMEM_COLS = (2 * BN <= 32) ? 32 : (2 * BN <= 64) ? 64 : (2 * BN <= 128) ? 128 : (2 * BN <= 256) ? 256 : 512;
+    static constexpr int TMEM_COLS = (NACC * BN <= 32) ? 32 : (NACC * BN <= 64) ? 64 : (NACC * BN <= 128) ? 128 : (NACC * BN <= 256) ? 256 : 512;
 };
 
 template <int KC, int BN>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(SmemLayout<KC, BN>::THREADS, 1)
 conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const UmmaParams P)
 {
     using L = SmemLayout<KC, BN>;
     constexpr int STAGES = L::STAGES;
+    constexpr int NACC = L::NACC;
     constexpr uint32_t SWZ = (KC == 64) ? 2u : 4u;
     constexpr uint32_t SBO = 8 * KC * 2;                       // bytes per 8-row group
     constexpr uint32_t IDESC = make_idesc(BN);
@@ -109,21 +140,25 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     uint8_t *stage_base = smem;
     float *epi = (float *)(smem + STAGES * L::STAGE_BYTES);
     uint64_t *bars = (uint64_t *)(smem + STAGES * L::STAGE_BYTES + L::EPI_BYTES);
-    // bars: full[STAGES], empty[STAGES], tfull[2], tempty[2]; then tmem base (u32) and abort flag (int)
-    uint32_t *tmem_slot = (uint32_t *)(bars + 2 * MAX_STAGES + 4);
+    // bars: full[STAGES], empty[STAGES], tfull[NACC], tempty[NACC]; then tmem base (u32) and abort flag (int)
+    uint32_t *tmem_slot = (uint32_t *)(bars + 2 * MAX_STAGES + 2 * MAX_ACC);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + MAX_STAGES);
-    const uint32_t tfull0 = smem_u32(bars + 2 * MAX_STAGES), tempty0 = smem_u32(bars + 2 * MAX_STAGES + 2);
+    const uint32_t tfull0 = smem_u32(bars + 2 * MAX_STAGES), tempty0 = smem_u32(bars + 2 * MAX_STAGES + MAX_ACC);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 4); }
+        for (int a = 0; a < NACC; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 4); }
         *abort_flag = 0;
         mbar_init_fence();
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), L::TMEM_COLS);
+    float *sbias = epi;
+    const bool bias_staged = P.bias && P.co <= MAX_SBIAS;
+    if (bias_staged)
+        for (int i = threadIdx.x; i < P.co; i += L::THREADS) sbias[i] = P.bias[i];
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -181,15 +216,16 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 }
                 if (!ok) break;
                 umma_commit(tfull0 + 8 * acc);              // accumulator complete
-                acc ^= 1;
-                if (acc == 0) acc_phase ^= 1;
+                if (++acc == NACC) { acc = 0; acc_phase ^= 1; }
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        // ------------------------------------------------------------------ epilogue (warps 2 .. 2 + 4 NACC)
+        // set e = (warp - 2) / 4 drains accumulator e, i.e. every NACC-th tile of this CTA
         const int q = warp & 3;                             // TMEM lane quarter this warp may read
-        float *tr = epi + (warp - 2) * 32 * 33;
-        uint32_t acc = 0, acc_phase = 0;
+        const uint32_t acc = (uint32_t)(warp - 2) >> 2;
+        uint32_t acc_phase = 0;
+        int it = 0;
         float s1[BN / 32 + 1], s2[BN / 32 + 1];             // per-lane column sums: column (c0 + lane) of each chunk
 #pragma unroll
         for (int i = 0; i < BN / 32 + 1; ++i) { s1[i] = 0.f; s2[i] = 0.f; }
@@ -209,74 +245,112 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 }
             }
         };
-        for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
+        for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, ++it) {
+            if ((uint32_t)(it % NACC) != acc) continue;
             const Tile T = decode_tile(P, tile);
             const int ct = T.ct, n = T.n;
             if (n != stat_n || ct != stat_ct) { flush(); stat_n = n; stat_ct = ct; }
             const int m = q * 32 + lane;
             const int wx = m % P.tw, hy = (m / P.tw) % P.th, dz = m / (P.tw * P.th);
             const int jw = T.w0 + wx, jh = T.h0 + hy, jd = T.d0 + dz;
-            const int w = P.out_scale * jw + (T.cls & 1), h = P.out_scale * jh + ((T.cls >> 1) & 1),
-                      d = P.out_scale * jd + ((T.cls >> 2) & 1);
-            const bool valid = (jw < P.W) && (jh < P.H) && (jd < P.D) && (w < P.OW) && (h < P.OH) && (d < P.OD);
-            const int64_t vox = (((int64_t)n * P.OD + d) * P.OH + h) * P.OW + w + T.ks * P.part_stride;
+            const bool inside = (jw < P.W) && (jh < P.H) && (jd < P.D);
             // the whole warp takes the same decision, so no lane is left behind at a __syncwarp
             ok = __all_sync(0xffffffffu, mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag));
             if (!ok) break;
             tc_fence_after();
             const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
+            uint32_t r[32];
+            if (BN >= 32) tmem_ld32(trow, r); else tmem_ld16(trow, r);
 #pragma unroll
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 const int ncol = (BN - c0) < 32 ? (BN - c0) : 32;       // 32, or 16 for the last chunk
-                uint32_t r[32];
-                if (ncol == 32) tmem_ld32(trow + c0, r); else tmem_ld16(trow + c0, r);
+                // output voxel and first channel of this chunk of columns
+                int cls = T.cls, ch0 = ct * BN + c0;
+                if (P.merge_co) { cls = ch0 / P.merge_co; ch0 -= cls * P.merge_co; }
+                const int w = P.out_scale * jw + (cls & 1), h = P.out_scale * jh + ((cls >> 1) & 1),
+                          d = P.out_scale * jd + ((cls >> 2) & 1);
+                const bool valid = inside && (w < P.OW) && (h < P.OH) && (d < P.OD);
+                const int64_t vox = (((int64_t)n * P.OD + d) * P.OH + h) * P.OW + w + T.ks * P.part_stride;
                 tmem_ld_wait();
                 float v[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    if (j < ncol) {
-                        float f = __uint_as_float(r[j]);
-                        if (P.bias) f += __ldg(P.bias + ct * BN + c0 + j);
-                        v[j] = valid ? f : 0.f;
-                    } else v[j] = 0.f;
+                for (int j = 0; j < 32; ++j) v[j] = (j < ncol && valid) ? __uint_as_float(r[j]) : 0.f;
+                // the next chunk's accumulator columns travel while this one is converted and stored
+                if (c0 + 32 < BN) {
+                    if (BN - (c0 + 32) >= 32) tmem_ld32(trow + c0 + 32, r); else tmem_ld16(trow + c0 + 32, r);
+                }
+                if (valid && P.bias) {
+                    if (bias_staged) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            if (j < ncol) {
+                                const float4 b4 = *reinterpret_cast<const float4 *>(sbias + ch0 + j);
+                                v[j] += b4.x; v[j + 1] += b4.y; v[j + 2] += b4.z; v[j + 3] += b4.w;
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) if (j < ncol) v[j] += __ldg(P.bias + ch0 + j);
+                    }
                 }
                 if (valid) {
                     if (P.y_f32) {
-                        float4 *dst = reinterpret_cast<float4 *>((float *)P.y + vox * P.y_pitch + ct * BN + c0);
+                        float *dst = (float *)P.y + vox * P.y_pitch + ch0;
+                        if (P.st32) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            if (4 * j < ncol) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                            for (int j = 0; j < 4; ++j) {
+                                if (8 * j < ncol) {
+                                    uint32_t u[8];
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) u[e] = __float_as_uint(v[8 * j + e]);
+                                    st_global_32B(dst + 8 * j, u);
+                                }
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                if (4 * j < ncol)
+                                    reinterpret_cast<float4 *>(dst)[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                        }
                     } else {
-                        uint4 *dst = reinterpret_cast<uint4 *>((bf16 *)P.y + vox * P.y_pitch + ct * BN + c0);
+                        bf16 *dst = (bf16 *)P.y + vox * P.y_pitch + ch0;
+                        uint4 q4[4];
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            if (8 * j < ncol) {
-                                float f8[8];
+                            float f8[8];
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) f8[e] = v[8 * j + e];
-                                dst[j] = pack8(f8);
+                            for (int e = 0; e < 8; ++e) f8[e] = v[8 * j + e];
+                            q4[j] = pack8(f8);
+                        }
+                        if (P.st32) {
+#pragma unroll
+                            for (int j = 0; j < 2; ++j) {
+                                if (16 * j < ncol) {
+                                    const uint32_t u[8] = {q4[2 * j].x, q4[2 * j].y, q4[2 * j].z, q4[2 * j].w,
+                                                           q4[2 * j + 1].x, q4[2 * j + 1].y, q4[2 * j + 1].z, q4[2 * j + 1].w};
+                                    st_global_32B(dst + 16 * j, u);
+                                }
                             }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                if (8 * j < ncol) reinterpret_cast<uint4 *>(dst)[j] = q4[j];
                         }
                     }
                 }
                 if (P.stats) {
-                    // transpose through shared memory: lane j then sums column j over the warp's 32 rows
-                    __syncwarp();
+                    // lane j ends up with the sum (and sum of squares) of column j over the warp's 32 rows
+                    float sq[32];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) tr[lane * 33 + j] = v[j];
-                    __syncwarp();
-                    float a = 0.f, b = 0.f;
-#pragma unroll
-                    for (int rr = 0; rr < 32; ++rr) { const float f = tr[rr * 33 + lane]; a += f; b = fmaf(f, f, b); }
-                    s1[c0 / 32] += a;
-                    s2[c0 / 32] += b;
+                    for (int j = 0; j < 32; ++j) sq[j] = v[j] * v[j];
+                    s1[c0 / 32] += warp_colsum32(v, lane);
+                    s2[c0 / 32] += warp_colsum32(sq, lane);
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
-            acc ^= 1;
-            if (acc == 0) acc_phase ^= 1;
+            acc_phase ^= 1;
         }
         flush();
     }
@@ -440,7 +514,7 @@ lamp_status_t launch(const CUtensorMap &mx, const CUtensorMap &mw, const UmmaPar
     }
     const int sms = sm_count();
     const int grid = P.total_tiles < sms ? P.total_tiles : sms;
-    conv3_umma_kernel<KC, BN><<<grid, NUM_THREADS, L::TOTAL, st>>>(mx, mw, P);
+    conv3_umma_kernel<KC, BN><<<grid, L::THREADS, L::TOTAL, st>>>(mx, mw, P);
     return launch_status();
 }
 
@@ -496,6 +570,11 @@ bool kind_info(int kind, const ConvGeom &g, KindInfo *k)
         if (!tr) return false;
         *k = KindInfo{g.co, g.ci, 8, g.od, g.oh, g.ow, g.d, g.h, g.w, g.d, g.h, g.w, 2, 1, 1};
         return true;
+    case UK_T_FWD_MERGED:
+        // the eight taps side by side on N: one GEMM [voxels x c_in] x [c_in x 8 c_out], each input tile read once
+        if (!tr || g.co % 32) return false;
+        *k = KindInfo{g.ci, 8 * g.co, 1, g.d, g.h, g.w, g.d, g.h, g.w, g.od, g.oh, g.ow, 1, 2, 1};
+        return true;
     }
     return false;
 }
@@ -511,6 +590,8 @@ void fill_taps(int kind, TapTable *T)
         // tap (kd,kh,kw) reads the input at shift k - 1; the data gradient uses the mirrored weight tap
         for (int t = 0; t < 27; ++t)
             set(0, kind == UK_S1_DGRAD ? 26 - t : t, t / 9 - 1, (t / 3) % 3 - 1, t % 3 - 1);
+    } else if (kind == UK_T_FWD_MERGED) {
+        set(0, 0, 0, 0, 0);
     } else if (kind == UK_T_DGRAD) {
         for (int t = 0; t < 8; ++t) set(0, t, t >> 2, (t >> 1) & 1, t & 1);
     } else if (kind == UK_T_FWD) {
@@ -553,7 +634,7 @@ TilePlan plan_tiles(int kind, const ConvGeom &g, const KindInfo &k)
     for (int c = 0; c < k.nclass; ++c) min_taps = tt.ntaps[c] < min_taps ? tt.ntaps[c] : min_taps;
     const int sms = sm_count();
     T.ksplit = 1;
-    if (T.tiles > 0 && T.tiles * 2 <= sms) {
+    if (kind != UK_T_FWD_MERGED && T.tiles > 0 && T.tiles * 2 <= sms) {
         int s = (int)(sms / T.tiles);
         const int cap = min_taps * T.chunks / 4;          // at least four (tap, chunk) steps per CTA
         if (s > cap) s = cap;
@@ -567,6 +648,7 @@ TilePlan plan_tiles(int kind, const ConvGeom &g, const KindInfo &k)
 size_t umma_splitk_ws(int kind, const ConvGeom &g)
 {
     KindInfo k;
+    if (kind == UK_T_FWD && kind_info(UK_T_FWD_MERGED, g, &k)) return 0;     // runs merged (when no statistics are asked for)
     if (!kind_info(kind, g, &k)) return 0;
     if (k.a_c % 32 || k.n_rows % 16 || !bn_instantiated(pick_bn(k.n_rows))) return 0;
     const TilePlan T = plan_tiles(kind, g, k);
@@ -605,6 +687,8 @@ lamp_status_t umma_conv(int kind, const ConvGeom &g, const TView &a, const bf16 
                         double *stats, void *part, size_t part_bytes, cudaStream_t st)
 {
     KindInfo k;
+    if (kind == UK_T_FWD && !stats && kind_info(UK_T_FWD_MERGED, g, &k) && bn_instantiated(pick_bn(k.n_rows)))
+        kind = UK_T_FWD_MERGED;
     if (!kind_info(kind, g, &k)) return LAMP_ERR_UNSUPPORTED;
     if ((int64_t)g.n * k.jd * k.jh * k.jw == 0) return LAMP_OK;
     PFN_cuTensorMapEncodeTiled_v12000 encode = get_encode();
@@ -629,11 +713,14 @@ lamp_status_t umma_conv(int kind, const ConvGeom &g, const TView &a, const bf16 
     if (tiles > 0x7FFFFFFF) return LAMP_ERR_UNSUPPORTED;
     P.total_tiles = (int32_t)tiles;
     P.co = k.n_rows; P.status = status_word_ptr();
+    P.merge_co = kind == UK_T_FWD_MERGED ? g.co : 0;
     if (split) {
         P.y_f32 = 1; P.y_pitch = k.n_rows; P.y = part; P.bias = nullptr; P.stats = nullptr;
     } else {
         P.y_f32 = y.f32; P.y_pitch = y.pitch; P.y = y.p; P.bias = bias; P.stats = stats;
     }
+    // a chunk of columns starts at a multiple of 16 channels, so rows are 32-byte aligned when base and pitch are
+    P.st32 = ((uintptr_t)P.y & 31) == 0 && (P.y_pitch * (P.y_f32 ? 4 : 2)) % 32 == 0;
     fill_taps(kind, &P.taps);
 
     CUtensorMap mx, mw;
