@@ -140,6 +140,7 @@ lamp_status_t conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const f
                        double *stats, void *ws, size_t ws_bytes, cudaStream_t st)
 {
     if (ct_conv_fwd_supported(g, x, y)) return ct_conv_fwd(g, x, w, bias, y, stats, 0, st);
+    if (c1_umma_supported(g, x, y)) return c1_umma_fwd(g, x, w, bias, y, stats, st);
     const int kind = fwd_kind(g);
     if (kind >= 0 && umma_conv_supported(kind, g, x, y)) return umma_conv(kind, g, x, w, bias, y, stats, ws, ws_bytes, st);
     return simt_conv_fwd(g, x, w, bias, y, stats, st);

@@ -128,6 +128,11 @@ size_t        umma_splitk_ws(int kind, const ConvGeom &g);
 size_t        umma_dgrad_ws(const ConvGeom &g);
 lamp_status_t umma_transpose_weights(const bf16 *w, bf16 *wt, int taps, int co, int ci, cudaStream_t st);
 
+// conv_c1_umma.cu (tcgen05 first layer: c_in = 1, banded weight matrices along w)
+bool          c1_umma_supported(const ConvGeom &g, const TView &x, const TView &y);
+lamp_status_t c1_umma_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
+                          double *stats, cudaStream_t st);
+
 // conv_t.cu (tcgen05 "weights x voxels" implicit GEMM over shared-memory-resident planes, c_out <= 128)
 bool          ct_conv_fwd_supported(const ConvGeom &g, const TView &x, const TView &y);
 lamp_status_t ct_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,

@@ -86,7 +86,8 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     constexpr uint32_t IDESC = make_idesc(256);
 
     extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    // aligned by offsetting the shared array itself, so that the compiler still sees shared-memory pointers
+    uint8_t *smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t *p_base = smem;
     uint8_t *w_base = p_base + (size_t)P.np * P.plane_bytes;
     float *epi = (float *)(w_base + (size_t)P.nw * WST_BYTES);

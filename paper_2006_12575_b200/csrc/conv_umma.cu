@@ -84,29 +84,6 @@ constexpr int MAX_STAGES = 8;
 constexpr int MAX_ACC = 4;
 constexpr int MAX_SBIAS = 2048;         // bias vectors up to this length are staged in shared memory
 
-// Column sums of a 32 x 32 tile held one row per lane: after the exchange with lane ^ 16 a lane keeps 16 columns
-// (two rows added), after lane ^ 8 eight columns, ... and finally lane j holds column j summed over all rows.
-__device__ __forceinline__ float warp_colsum32(const float (&v)[32], int lane)
-{
-    float a[16], b[8], c[4], d[2];
-    const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4, h2 = lane & 2, h1 = lane & 1;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) a[i] = (h16 ? v[i + 16] : v[i]) + __shfl_xor_sync(0xffffffffu, h16 ? v[i] : v[i + 16], 16);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) b[i] = (h8 ? a[i + 8] : a[i]) + __shfl_xor_sync(0xffffffffu, h8 ? a[i] : a[i + 8], 8);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) c[i] = (h4 ? b[i + 4] : b[i]) + __shfl_xor_sync(0xffffffffu, h4 ? b[i] : b[i + 4], 4);
-#pragma unroll
-    for (int i = 0; i < 2; ++i) d[i] = (h2 ? c[i + 2] : c[i]) + __shfl_xor_sync(0xffffffffu, h2 ? c[i] : c[i + 2], 2);
-    return (h1 ? d[1] : d[0]) + __shfl_xor_sync(0xffffffffu, h1 ? d[0] : d[1], 1);
-}
-
-__device__ __forceinline__ void st_global_32B(void *p, const uint32_t (&u)[8])
-{
-    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                 :: "l"(p), "r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7])
-                 : "memory");
-}
 
 template <int KC, int BN>
 struct SmemLayout {
@@ -136,7 +113,8 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     constexpr uint32_t IDESC = make_idesc(BN);
 
     extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    // aligned by offsetting the shared array itself, so that the compiler still sees shared-memory pointers
+    uint8_t *smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t *stage_base = smem;
     float *epi = (float *)(smem + STAGES * L::STAGE_BYTES);
     uint64_t *bars = (uint64_t *)(smem + STAGES * L::STAGE_BYTES + L::EPI_BYTES);

@@ -77,7 +77,8 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     constexpr int ABOXES = 128 / BOXA, XBOXES = NC / BOXB;
 
     extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    // aligned by offsetting the shared array itself, so that the compiler still sees shared-memory pointers
+    uint8_t *smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t *xs_base = smem;
     uint8_t *as_base = smem + NX * L::X_BYTES;
     uint64_t *bars = (uint64_t *)(as_base + NA * A_STAGE_BYTES);

@@ -84,7 +84,8 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     constexpr int ACC_COLS = 256;                               // TMEM column stride between the two accumulators
 
     extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    // aligned by offsetting the shared array itself, so that the compiler still sees shared-memory pointers
+    uint8_t *smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
     uint64_t *bars = (uint64_t *)(smem + (size_t)P.nst * P.stage_bytes);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + MAX_ST);
     const uint32_t done_bar = smem_u32(bars + 2 * MAX_ST), drained_bar = smem_u32(bars + 2 * MAX_ST + 1);

@@ -18,6 +18,9 @@ CASES = [
     ("first_layer_c1_64", 1, 6, 5, 21, 1, 64, 3, 1, 1, 0),
     ("first_layer_c1_32_wide", 2, 4, 32, 16, 1, 32, 3, 1, 1, 0),
     ("first_layer_c1_64_wide", 1, 3, 16, 24, 1, 64, 3, 1, 1, 0),
+    ("first_layer_c1_32_ragged_lines", 1, 20, 36, 40, 1, 32, 3, 1, 1, 0),
+    ("first_layer_c1_96_batch", 3, 5, 9, 16, 1, 96, 3, 1, 1, 0),
+    ("first_layer_c1_64_cube", 1, 32, 32, 32, 1, 64, 3, 1, 1, 0),
     ("narrow_16_24", 2, 6, 5, 9, 16, 24, 3, 1, 1, 0),
     ("down_8_16", 1, 8, 6, 10, 8, 16, 3, 2, 1, 0),
     ("down_32_64", 1, 16, 8, 12, 32, 64, 3, 2, 1, 0),
