@@ -532,6 +532,35 @@ def run_hbm(args):
         ms = timed(lambda: B.lamp_instnorm_relu_bwd(dz, None, y, mr, sums, dy), flush)
         res[f"instnorm_relu_bwd C={C}"] = dict(ms=round(ms, 4), bytes=10 * n, gbs=round(10 * n / ms / 1e6, 1))
         del y, dz, z, dy, yf
+    # convolutions of the network whose FLOPs per byte sit below the machine balance: the one-channel first layer,
+    # the 2x2x2 transposed (up) conv into a concat slice and the stride-2 (down) conv at the top level
+    x1 = torch.randn((1, D, H, W, 1), device="cuda").to(torch.bfloat16)
+    for C in (32, 64):
+        w1 = (torch.randn((27, C, 1), device="cuda") * 0.2).to(torch.bfloat16)
+        b1 = torch.zeros(C, device="cuda")
+        y1 = torch.empty((1, D, H, W, C), dtype=torch.bfloat16, device="cuda")
+        st1 = torch.zeros((1, C, 2), dtype=torch.float64, device="cuda")
+        desc = B.conv_desc(1, C, 3, 1, 1, False)
+        nb = x1.numel() * 2 + y1.numel() * 2
+        ms = timed(lambda: B.lamp_conv3d_fwd(desc, x1, w1, b1, y1, st1), flush)
+        res[f"first-layer conv 1->{C}"] = dict(ms=round(ms, 4), bytes=nb, gbs=round(nb / ms / 1e6, 1))
+        del y1
+    xu = torch.randn((1, D // 2, H // 2, W // 2, 64), device="cuda").to(torch.bfloat16)
+    wu = (torch.randn((8, 32, 64), device="cuda") * 0.1).to(torch.bfloat16)
+    cat = torch.zeros((1, D, H, W, 64), dtype=torch.bfloat16, device="cuda")
+    desc = B.conv_desc(64, 32, 2, 2, 0, True)
+    nb = xu.numel() * 2 + cat.numel()                    # the written slice is half of the concat buffer
+    ms = timed(lambda: B.lamp_conv3d_fwd(desc, xu, wu, torch.zeros(32, device="cuda"), B.tensor(cat, 32, 32)), flush)
+    res["up conv 64->32 into concat slice"] = dict(ms=round(ms, 4), bytes=nb, gbs=round(nb / ms / 1e6, 1))
+    xd = torch.randn((1, D, H, W, 32), device="cuda").to(torch.bfloat16)
+    wd = (torch.randn((27, 64, 32), device="cuda") * 0.05).to(torch.bfloat16)
+    yd = torch.empty((1, D // 2, H // 2, W // 2, 64), dtype=torch.bfloat16, device="cuda")
+    std = torch.zeros((1, 64, 2), dtype=torch.float64, device="cuda")
+    desc = B.conv_desc(32, 64, 3, 2, 1, False)
+    nb = xd.numel() * 2 + yd.numel() * 2
+    ms = timed(lambda: B.lamp_conv3d_fwd(desc, xd, wd, torch.zeros(64, device="cuda"), yd, std), flush)
+    res["down conv 32->64 stride 2"] = dict(ms=round(ms, 4), bytes=nb, gbs=round(nb / ms / 1e6, 1))
+    del xu, cat, xd, yd
     # overlap-add on the 512 x 512 x 128 volume: 363 patches of 64^3, K = 10
     K, P = 10, (64, 64, 64)
     Dv, Hv, Wv = 512, 512, 128
