@@ -126,6 +126,10 @@ lamp_status_t umma_conv(int kind, const ConvGeom &g, const TView &a, const bf16 
                         double *stats, void *part, size_t part_bytes, cudaStream_t st);
 size_t        umma_splitk_ws(int kind, const ConvGeom &g);
 size_t        umma_dgrad_ws(const ConvGeom &g);
+// head (1x1x1 conv + softmax + arg max + Dice sums) on the tensor cores; dice_sums must be zero on entry
+bool          umma_head_supported(const TView &z, int K);
+lamp_status_t umma_head(const TView &z, const bf16 *w, const float *b, int K, float *probs, uint8_t *argmax,
+                        const uint8_t *labels, double *dice_sums, cudaStream_t st);
 lamp_status_t umma_transpose_weights(const bf16 *w, bf16 *wt, int taps, int co, int ci, cudaStream_t st);
 
 // conv_c1_umma.cu (tcgen05 first layer: c_in = 1, banded weight matrices along w)

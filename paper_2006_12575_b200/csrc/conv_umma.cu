@@ -53,6 +53,7 @@ struct UmmaParams {
     int64_t part_stride;           // voxels between the partial results of consecutive splits
     int32_t chunks;                // c_in / KC
     int32_t total_tiles;
+    int32_t step[7];               // the grid size in the tiles' mixed radix (ksplit, nct, ntw, nth, ntd, nclass, N)
     int32_t co;                    // c_out
     int32_t merge_co;              // > 0: the N axis carries (parity class, channel) pairs, class = column / merge_co
     int32_t y_f32;
@@ -62,23 +63,52 @@ struct UmmaParams {
     const float *bias;
     double *stats;                 // [N][co][2] or NULL
     int    *status;
+    // head mode (1x1x1 conv + softmax over the hK <= 16 columns of a row): outputs instead of y
+    int32_t hK;
+    float *probs;                  // [voxel][hK] or NULL
+    uint8_t *amax;                 // [voxel] or NULL
+    const uint8_t *labels;         // [voxel], with dice
+    double *dice;                  // [n][hK][3] = (sum p at the label, sum p, label count) or NULL
     TapTable taps;
 };
 
 struct Tile { int ks, ct, w0, h0, d0, cls, n; };
 
-__device__ __forceinline__ Tile decode_tile(const UmmaParams &P, int t)
-{
-    Tile r;
-    r.ks = t % P.ksplit; t /= P.ksplit;
-    r.ct = t % P.nct; t /= P.nct;
-    r.w0 = (t % P.ntw) * P.tw; t /= P.ntw;
-    r.h0 = (t % P.nth) * P.th; t /= P.nth;
-    r.d0 = (t % P.ntd) * P.td; t /= P.ntd;
-    r.cls = t % P.nclass;
-    r.n = t / P.nclass;
-    return r;
-}
+// A CTA visits tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The tile index is a number in the mixed radix
+// (ksplit, nct, ntw, nth, ntd, nclass, N); instead of dividing for every tile the walker divides once and then adds
+// the grid size digit by digit (tiles with one short reduction step are otherwise bound by this index arithmetic).
+struct TileWalker {
+    int dg[7];
+    __device__ __forceinline__ void init(const UmmaParams &P, int t)
+    {
+        dg[0] = t % P.ksplit; t /= P.ksplit;
+        dg[1] = t % P.nct; t /= P.nct;
+        dg[2] = t % P.ntw; t /= P.ntw;
+        dg[3] = t % P.nth; t /= P.nth;
+        dg[4] = t % P.ntd; t /= P.ntd;
+        dg[5] = t % P.nclass;
+        dg[6] = t / P.nclass;
+    }
+    __device__ __forceinline__ void next(const UmmaParams &P)
+    {
+        const int radix[6] = {P.ksplit, P.nct, P.ntw, P.nth, P.ntd, P.nclass};
+        int carry = 0;
+#pragma unroll
+        for (int i = 0; i < 6; ++i) {
+            int v = dg[i] + P.step[i] + carry;
+            carry = v >= radix[i];
+            if (carry) v -= radix[i];
+            dg[i] = v;
+        }
+        dg[6] += P.step[6] + carry;
+    }
+    __device__ __forceinline__ Tile tile(const UmmaParams &P) const
+    {
+        Tile r;
+        r.ks = dg[0]; r.ct = dg[1]; r.w0 = dg[2] * P.tw; r.h0 = dg[3] * P.th; r.d0 = dg[4] * P.td; r.cls = dg[5]; r.n = dg[6];
+        return r;
+    }
+};
 
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_ACC = 4;
@@ -101,7 +131,8 @@ struct SmemLayout {
     static constexpr int TMEM_COLS = (NACC * BN <= 32) ? 32 : (NACC * BN <= 64) ? 64 : (NACC * BN <= 128) ? 128 : (NACC * BN <= 256) ? 256 : 512;
 };
 
-template <int KC, int BN>
+// HEAD: 0, or the number of classes rounded up to a multiple of 4 (head mode, BN = 16)
+template <int KC, int BN, int HEAD = 0>
 __global__ void __launch_bounds__(SmemLayout<KC, BN>::THREADS, 1)
 conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const UmmaParams P)
 {
@@ -148,8 +179,10 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
-                const Tile T = decode_tile(P, tile);
+            TileWalker tw_;
+            tw_.init(P, blockIdx.x);
+            for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, tw_.next(P)) {
+                const Tile T = tw_.tile(P);
                 const int kit = P.taps.ntaps[T.cls] * P.chunks;
                 const int k1 = kit * (T.ks + 1) / P.ksplit;
                 for (int ki = kit * T.ks / P.ksplit; ki < k1; ++ki) {
@@ -174,8 +207,10 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             int stage = 0;
             uint32_t phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
-                const Tile T = decode_tile(P, tile);
+            TileWalker tw_;
+            tw_.init(P, blockIdx.x);
+            for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, tw_.next(P)) {
+                const Tile T = tw_.tile(P);
                 const int kit = P.taps.ntaps[T.cls] * P.chunks;
                 const int kiters = kit * (T.ks + 1) / P.ksplit - kit * T.ks / P.ksplit;   // >= 1: ksplit <= taps * chunks
                 if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag)) { ok = false; break; }
@@ -209,7 +244,30 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         for (int i = 0; i < BN / 32 + 1; ++i) { s1[i] = 0.f; s2[i] = 0.f; }
         int stat_n = -1, stat_ct = 0;
         bool ok = true;
+        constexpr int HK = HEAD ? HEAD : 1;
+        float hP[HK], hI[HK], hG[HK];                       // head mode: Dice sums of this thread's voxels
+#pragma unroll
+        for (int k = 0; k < HK; ++k) { hP[k] = 0.f; hI[k] = 0.f; hG[k] = 0.f; }
         auto flush = [&]() {
+            if (HEAD && P.dice && stat_n >= 0) {
+#pragma unroll
+                for (int k = 0; k < HK; ++k) {
+                    if (k < P.hK) {
+                        float a = hI[k], b = hP[k], c = hG[k];
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            a += __shfl_xor_sync(0xffffffffu, a, o);
+                            b += __shfl_xor_sync(0xffffffffu, b, o);
+                            c += __shfl_xor_sync(0xffffffffu, c, o);
+                        }
+                        if (lane == 0) {
+                            double *dst = P.dice + ((int64_t)stat_n * P.hK + k) * 3;
+                            atomicAdd(dst, (double)a); atomicAdd(dst + 1, (double)b); atomicAdd(dst + 2, (double)c);
+                        }
+                    }
+                    hP[k] = 0.f; hI[k] = 0.f; hG[k] = 0.f;
+                }
+            }
             if (P.stats && stat_n >= 0) {
 #pragma unroll
                 for (int i = 0; i < (BN + 31) / 32; ++i) {
@@ -223,9 +281,11 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 }
             }
         };
-        for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, ++it) {
+        TileWalker tw_;
+        tw_.init(P, blockIdx.x);
+        for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, ++it, tw_.next(P)) {
             if ((uint32_t)(it % NACC) != acc) continue;
-            const Tile T = decode_tile(P, tile);
+            const Tile T = tw_.tile(P);
             const int ct = T.ct, n = T.n;
             if (n != stat_n || ct != stat_ct) { flush(); stat_n = n; stat_ct = ct; }
             const int m = q * 32 + lane;
@@ -239,6 +299,35 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
             uint32_t r[32];
             if (BN >= 32) tmem_ld32(trow, r); else tmem_ld16(trow, r);
+            if constexpr (HEAD > 0) {
+                // the row holds the logits of the thread's voxel: softmax, arg max and the Dice sums
+                tmem_ld_wait();
+                const int64_t vox = (((int64_t)n * P.OD + jd) * P.OH + jh) * P.OW + jw;
+                float l[HK];
+#pragma unroll
+                for (int k = 0; k < HK; ++k) l[k] = k < P.hK ? __uint_as_float(r[k]) + (bias_staged ? sbias[k] : 0.f) : -INFINITY;
+                float mx = l[0];
+                int am = 0;
+#pragma unroll
+                for (int k = 1; k < HK; ++k) if (l[k] > mx) { mx = l[k]; am = k; }
+                float sum = 0.f;
+                // exp(x) for x <= 0 as one exp2 of x * log2(e): relative error of a few 1e-7, far inside the
+                // tolerance of the probabilities; classes beyond K contribute exp2(-inf) = 0
+#pragma unroll
+                for (int k = 0; k < HK; ++k) { l[k] = exp2f((l[k] - mx) * 1.4426950408889634f); sum += l[k]; }
+                const float inv = 1.0f / sum;
+                if (inside) {
+                    const int lab = P.dice ? (int)P.labels[vox] : -1;
+#pragma unroll
+                    for (int k = 0; k < HK; ++k) {
+                        const float p = l[k] * inv;
+                        if (k < P.hK && P.probs) P.probs[vox * P.hK + k] = p;
+                        hP[k] += p;
+                        if (k == lab) { hI[k] += p; hG[k] += 1.f; }
+                    }
+                    if (P.amax) P.amax[vox] = (uint8_t)am;
+                }
+            } else {
 #pragma unroll
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 const int ncol = (BN - c0) < 32 ? (BN - c0) : 32;       // 32, or 16 for the last chunk
@@ -324,6 +413,7 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     s1[c0 / 32] += warp_colsum32(v, lane);
                     s2[c0 / 32] += warp_colsum32(sq, lane);
                 }
+            }
             }
             tc_fence_before();
             __syncwarp();
@@ -481,18 +571,25 @@ void pick_tile(int D, int H, int W, int *tw, int *th, int *td)
         }
 }
 
-template <int KC, int BN>
+template <int KC, int BN, int HEAD = 0>
 lamp_status_t launch(const CUtensorMap &mx, const CUtensorMap &mw, const UmmaParams &P, cudaStream_t st)
 {
     using L = SmemLayout<KC, BN>;
     static bool attr = false;
     if (!attr) {
-        LAMP_CUDA_OK(cudaFuncSetAttribute(conv3_umma_kernel<KC, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
+        LAMP_CUDA_OK(cudaFuncSetAttribute(conv3_umma_kernel<KC, BN, HEAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
         attr = true;
     }
     const int sms = sm_count();
     const int grid = P.total_tiles < sms ? P.total_tiles : sms;
-    conv3_umma_kernel<KC, BN><<<grid, L::THREADS, L::TOTAL, st>>>(mx, mw, P);
+    UmmaParams Q = P;
+    {
+        const int radix[6] = {Q.ksplit, Q.nct, Q.ntw, Q.nth, Q.ntd, Q.nclass};
+        int t = grid;
+        for (int i = 0; i < 6; ++i) { Q.step[i] = t % radix[i]; t /= radix[i]; }
+        Q.step[6] = t;
+    }
+    conv3_umma_kernel<KC, BN, HEAD><<<grid, L::THREADS, L::TOTAL, st>>>(mx, mw, Q);
     return launch_status();
 }
 
@@ -646,6 +743,66 @@ bool umma_conv_supported(int kind, const ConvGeom &g, const TView &a, const TVie
     return true;
 }
 
+bool umma_head_supported(const TView &z, int K)
+{
+    return K >= 1 && K <= 16 && z.c % 32 == 0 && z.c <= 256 && z.pitch % 8 == 0 && ((uintptr_t)z.p & 15) == 0;
+}
+
+// Head of the network on the tensor cores: logits = z * w^T + b as one [voxels x c] x [c x 16] GEMM (rows of w beyond
+// K are out-of-range rows of the TMA box and arrive as zeros), softmax / arg max / Dice sums in the epilogue.
+lamp_status_t umma_head(const TView &z, const bf16 *w, const float *b, int K, float *probs, uint8_t *argmax,
+                        const uint8_t *labels, double *dice_sums, cudaStream_t st)
+{
+    if ((int64_t)z.n * z.d * z.h * z.w == 0) return LAMP_OK;
+    PFN_cuTensorMapEncodeTiled_v12000 encode = get_encode();
+    if (!encode) return LAMP_ERR_CUDA;
+    const int KC = (z.c % 64 == 0) ? 64 : 32;
+    UmmaParams P;
+    memset(&P, 0, sizeof(P));
+    P.N = z.n; P.D = z.d; P.H = z.h; P.W = z.w;
+    P.OD = z.d; P.OH = z.h; P.OW = z.w;
+    P.in_scale = 1; P.out_scale = 1; P.nclass = 1;
+    pick_tile(z.d, z.h, z.w, &P.tw, &P.th, &P.td);
+    P.ntw = (z.w + P.tw - 1) / P.tw; P.nth = (z.h + P.th - 1) / P.th; P.ntd = (z.d + P.td - 1) / P.td;
+    P.nct = 1; P.ksplit = 1; P.part_stride = 0;
+    P.chunks = z.c / KC;
+    const int64_t tiles = (int64_t)z.n * P.ntd * P.nth * P.ntw;
+    if (tiles > 0x7FFFFFFF) return LAMP_ERR_UNSUPPORTED;
+    P.total_tiles = (int32_t)tiles;
+    P.co = K; P.merge_co = 0;
+    P.bias = b; P.status = status_word_ptr();
+    P.hK = K; P.probs = probs; P.amax = argmax; P.labels = labels; P.dice = dice_sums;
+    P.taps.ntaps[0] = 1;                                   // one tap, no shift, weight tile 0
+    CUtensorMap mx, mw;
+    {
+        const cuuint64_t dims[5] = {(cuuint64_t)z.c, (cuuint64_t)z.w, (cuuint64_t)z.h, (cuuint64_t)z.d, (cuuint64_t)z.n};
+        const cuuint64_t strides[4] = {(cuuint64_t)z.pitch * 2, (cuuint64_t)z.pitch * 2 * z.w,
+                                       (cuuint64_t)z.pitch * 2 * z.w * z.h, (cuuint64_t)z.pitch * 2 * z.w * z.h * z.d};
+        const cuuint32_t box[5] = {(cuuint32_t)KC, (cuuint32_t)P.tw, (cuuint32_t)P.th, (cuuint32_t)P.td, 1};
+        const cuuint32_t es[5] = {1, 1, 1, 1, 1};
+        if (encode(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, z.p, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   KC == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return LAMP_ERR_CUDA;
+    }
+    {
+        const cuuint64_t dims[3] = {(cuuint64_t)z.c, (cuuint64_t)K, 1};
+        const cuuint64_t strides[2] = {(cuuint64_t)z.c * 2, (cuuint64_t)z.c * 2 * K};
+        const cuuint32_t box[3] = {(cuuint32_t)KC, 16, 1};
+        const cuuint32_t es[3] = {1, 1, 1};
+        if (encode(&mw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void *)w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   KC == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return LAMP_ERR_CUDA;
+    }
+    switch ((K + 3) / 4) {
+    case 1:  return KC == 64 ? launch<64, 16, 4>(mx, mw, P, st) : launch<32, 16, 4>(mx, mw, P, st);
+    case 2:  return KC == 64 ? launch<64, 16, 8>(mx, mw, P, st) : launch<32, 16, 8>(mx, mw, P, st);
+    case 3:  return KC == 64 ? launch<64, 16, 12>(mx, mw, P, st) : launch<32, 16, 12>(mx, mw, P, st);
+    default: return KC == 64 ? launch<64, 16, 16>(mx, mw, P, st) : launch<32, 16, 16>(mx, mw, P, st);
+    }
+}
+
 size_t umma_dgrad_ws(const ConvGeom &g)
 {
     return align_up((size_t)g.k * g.k * g.k * g.co * g.ci * sizeof(bf16), 256);
@@ -692,6 +849,7 @@ lamp_status_t umma_conv(int kind, const ConvGeom &g, const TView &a, const bf16 
     P.total_tiles = (int32_t)tiles;
     P.co = k.n_rows; P.status = status_word_ptr();
     P.merge_co = kind == UK_T_FWD_MERGED ? g.co : 0;
+    P.hK = 0; P.probs = nullptr; P.amax = nullptr; P.labels = nullptr; P.dice = nullptr;
     if (split) {
         P.y_f32 = 1; P.y_pitch = k.n_rows; P.y = part; P.bias = nullptr; P.stats = nullptr;
     } else {

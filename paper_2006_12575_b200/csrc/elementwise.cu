@@ -657,6 +657,7 @@ lamp_status_t k_head_softmax(const TView &z, const bf16 *w, const float *b, int 
     if (K > KMAX || K < 1 || z.c > 64 || z.c % 8) return LAMP_ERR_UNSUPPORTED;
     if (dice_sums) LAMP_CUDA_OK(cudaMemsetAsync(dice_sums, 0, (size_t)z.n * K * 3 * sizeof(double), st));
     if (Vn == 0 || z.n == 0) return LAMP_OK;
+    if (umma_head_supported(z, K) && ((uintptr_t)w & 15) == 0) return umma_head(z, w, b, K, probs, argmax, labels, dice_sums, st);
     int64_t blocks, vpb;
     head_grid(Vn, z.n, blocks, vpb);
     const int KP = head_kp(K);
