@@ -37,8 +37,7 @@ using namespace ptx;
 
 struct TapTable {                  // per parity class: the taps that contribute, their weight tile and input shift
     int8_t ntaps[8];
-    int8_t wtap[8][27];
-    int8_t sd[8][27], sh[8][27], sw[8][27];
+    uint32_t tap[8][27];           // one word per tap: bytes (weight tile, shift d, shift h, shift w), shifts signed
 };
 
 struct UmmaParams {
@@ -184,13 +183,18 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, tw_.next(P)) {
                 const Tile T = tw_.tile(P);
                 const int kit = P.taps.ntaps[T.cls] * P.chunks;
-                const int k1 = kit * (T.ks + 1) / P.ksplit;
-                for (int ki = kit * T.ks / P.ksplit; ki < k1; ++ki) {
-                    const int tp = ki / P.chunks, ch = ki - tp * P.chunks;
-                    const int cw = P.in_scale * T.w0 + P.taps.sw[T.cls][tp];
-                    const int chh = P.in_scale * T.h0 + P.taps.sh[T.cls][tp];
-                    const int cd = P.in_scale * T.d0 + P.taps.sd[T.cls][tp];
-                    const int wt = P.taps.wtap[T.cls][tp];
+                int k0 = 0, k1 = kit, tp = 0, ch = 0;
+                if (P.ksplit > 1) {
+                    k0 = kit * T.ks / P.ksplit; k1 = kit * (T.ks + 1) / P.ksplit;
+                    tp = k0 / P.chunks; ch = k0 - tp * P.chunks;
+                }
+                const int3 bw0 = make_int3(P.in_scale * T.w0, P.in_scale * T.h0, P.in_scale * T.d0);
+                for (int ki = k0; ki < k1; ++ki) {
+                    const uint32_t tw4 = P.taps.tap[T.cls][tp];
+                    const int wt = (int)(tw4 & 0xFF);
+                    const int cd = bw0.z + ((int)(tw4 << 16) >> 24);
+                    const int chh = bw0.y + ((int)(tw4 << 8) >> 24);
+                    const int cw = bw0.x + ((int)tw4 >> 24);
                     if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
                     const uint32_t fb = full0 + 8 * stage;
                     mbar_expect_tx(fb, L::STAGE_BYTES);
@@ -198,6 +202,7 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     tma_load_5d(sa, &map_x, fb, ch * KC, cw, chh, cd, T.n);
                     tma_load_3d(sa + L::A_BYTES, &map_w, fb, ch * KC, T.ct * BN, wt);
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    if (++ch == P.chunks) { ch = 0; ++tp; }
                 }
             }
         }
@@ -212,7 +217,8 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, tw_.next(P)) {
                 const Tile T = tw_.tile(P);
                 const int kit = P.taps.ntaps[T.cls] * P.chunks;
-                const int kiters = kit * (T.ks + 1) / P.ksplit - kit * T.ks / P.ksplit;   // >= 1: ksplit <= taps * chunks
+                // >= 1: ksplit <= taps * chunks
+                const int kiters = P.ksplit > 1 ? kit * (T.ks + 1) / P.ksplit - kit * T.ks / P.ksplit : kit;
                 if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
@@ -659,7 +665,7 @@ void fill_taps(int kind, TapTable *T)
     memset(T, 0, sizeof(*T));
     auto set = [&](int cls, int wtap, int sd, int sh, int sw) {
         const int i = T->ntaps[cls]++;
-        T->wtap[cls][i] = (int8_t)wtap; T->sd[cls][i] = (int8_t)sd; T->sh[cls][i] = (int8_t)sh; T->sw[cls][i] = (int8_t)sw;
+        T->tap[cls][i] = (uint32_t)(wtap & 0xFF) | ((uint32_t)(sd & 0xFF) << 8) | ((uint32_t)(sh & 0xFF) << 16) | ((uint32_t)(sw & 0xFF) << 24);
     };
     if (kind == UK_S1_FWD || kind == UK_S2_FWD || kind == UK_S1_DGRAD) {
         // tap (kd,kh,kw) reads the input at shift k - 1; the data gradient uses the mirrored weight tap
