@@ -84,13 +84,20 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                                                                // too little work per tap to pay a barrier round trip each
     constexpr uint32_t WST_BYTES = TPS * W_BYTES;
     constexpr uint32_t IDESC = make_idesc(256);
+    // 32 -> 32 channels: all weights stay in shared memory.  Per in-plane tap the region [0 0 0 k0 k1 k2] of 32-row
+    // blocks (kd = 0, 1, 2 after three zero blocks; three more zero blocks close the last region): the 128 stacked rows
+    // of input plane pi are the four consecutive blocks that start at block pi (forward) or 5 - pi (mirrored taps).
+    constexpr bool WRES = (KC == 32 && COB == 32);
+    constexpr uint32_t BLK_BYTES = 32 * ROWB;                  // one block of 32 output channels
+    constexpr uint32_t WRES_TAP_BYTES = 6 * BLK_BYTES;
+    constexpr uint32_t WRES_BYTES = 9 * WRES_TAP_BYTES + 3 * BLK_BYTES;
 
     extern __shared__ uint8_t smem_raw[];
     // aligned by offsetting the shared array itself, so that the compiler still sees shared-memory pointers
     uint8_t *smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t *p_base = smem;
     uint8_t *w_base = p_base + (size_t)P.np * P.plane_bytes;
-    float *epi = (float *)(w_base + (size_t)P.nw * WST_BYTES);
+    float *epi = (float *)(w_base + (WRES ? (size_t)WRES_BYTES : (size_t)P.nw * WST_BYTES));
     uint64_t *bars = (uint64_t *)((uint8_t *)epi + 4 * 32 * 33 * 4);
     const uint32_t pfull0 = smem_u32(bars), pempty0 = smem_u32(bars + MAX_NP);
     const uint32_t wfull0 = smem_u32(bars + 2 * MAX_NP), wempty0 = smem_u32(bars + 2 * MAX_NP + MAX_NW);
@@ -107,6 +114,14 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         mbar_init_fence();
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+    if (WRES) {
+        // zero blocks of the resident weights (the kd blocks arrive by TMA below)
+        for (uint32_t i = threadIdx.x; i < WRES_BYTES / 16; i += CT_THREADS) {
+            const uint32_t off = i * 16, in_tap = off % WRES_TAP_BYTES;
+            if (off >= 9 * WRES_TAP_BYTES || in_tap < 3 * BLK_BYTES) *reinterpret_cast<uint4 *>(w_base + off) = make_uint4(0, 0, 0, 0);
+        }
+        fence_proxy_async();
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -139,7 +154,13 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             int ws = 0;
             uint32_t wph = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
+            if (WRES) {
+                // once: the three kd blocks of every in-plane tap (mirrored taps read tap 8 - t9)
+                mbar_expect_tx(wfull0, 27 * BLK_BYTES);
+                for (int t9 = 0; t9 < 9; ++t9)
+                    tma_load_4d(smem_u32(w_base + t9 * WRES_TAP_BYTES + 3 * BLK_BYTES), &map_w, wfull0, 0, 0, 0, P.mirror ? 8 - t9 : t9);
+            }
+            for (int item = blockIdx.x; item < P.total_items && ok && !WRES; item += gridDim.x) {
                 const Item it = decode_item<S>(P, item);
                 for (int pi = 0; pi < S + 2 && ok; ++pi) {
                     const int p = it.o0 - 1 + pi;
@@ -166,6 +187,7 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             int ps = 0, ws = 0;
             uint32_t pph = 0, wph = 0, acc = 0, acc_phase = 0;
             bool ok = true;
+            if (WRES) { ok = mbar_wait(wfull0, 0, abort_flag); tc_fence_after(); }
             for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
                 const Item it = decode_item<S>(P, item);
                 if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag)) { ok = false; break; }
@@ -179,7 +201,20 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         if (!mbar_wait(pfull0 + 8 * ps, pph, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t plane = smem_u32(p_base + (size_t)ps * P.plane_bytes);
-                        for (int t9 = 0; t9 < 9; t9 += TPS) {
+                        if (WRES) {
+                            const uint32_t wwin = smem_u32(w_base) + (uint32_t)(P.mirror ? 5 - pi : pi) * BLK_BYTES;
+#pragma unroll
+                            for (int t9 = 0; t9 < 9; ++t9) {
+                                const uint64_t da = make_desc(wwin + t9 * WRES_TAP_BYTES, 0, 8 * ROWB, SWZ);
+                                const uint64_t db = make_desc(plane + ((t9 / 3) * HALO_W + t9 % 3) * ROWB, 0, HALO_W * ROWB, SWZ);
+#pragma unroll
+                                for (int k = 0; k < KC / 16; ++k) {
+                                    umma_bf16(d_tmem, da + 2 * k, db + 2 * k, IDESC, accumulate);
+                                    accumulate = 1;
+                                }
+                            }
+                        }
+                        for (int t9 = 0; t9 < 9 && !WRES; t9 += TPS) {
                             if (!mbar_wait(wfull0 + 8 * ws, wph, abort_flag)) { ok = false; break; }
                             tc_fence_after();
 #pragma unroll
@@ -346,6 +381,9 @@ bool make_ct_plan(const ConvGeom &g, CtPlan *out)
     int nw = (budget - np * P.plane_bytes) / w_bytes;
     if (nw > MAX_NW) nw = MAX_NW;
     if (nw < 3) return false;
+    // 32 -> 32 channels: the weights are resident (nine regions of six 2 KB blocks plus three closing zero blocks)
+    const bool wres = KC == 32 && COB == 32;
+    const size_t wres_bytes = (size_t)(9 * 6 + 3) * 32 * rowb;
     P.np = np; P.nw = nw;
     P.nwt = (g.w + TW - 1) / TW;
     P.nht = (g.h + TH - 1) / TH;
@@ -359,7 +397,8 @@ bool make_ct_plan(const ConvGeom &g, CtPlan *out)
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     out->KC = KC; out->COB = COB;
-    out->smem = 1024 + (size_t)np * P.plane_bytes + (size_t)nw * w_bytes + EPI_BYTES + CTRL_BYTES;
+    out->smem = 1024 + (size_t)np * P.plane_bytes + (wres ? wres_bytes : (size_t)nw * w_bytes) + EPI_BYTES + CTRL_BYTES;
+    if (out->smem > (size_t)SMEM_LIMIT) return false;
     out->grid = (int)(items < sms ? items : sms);
     return true;
 }
@@ -418,7 +457,9 @@ lamp_status_t ct_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, cons
         // weights viewed as (c_in, c_out, kd, kh*3+kw): a box spans the stacked kd blocks, then the taps of a stage
         const cuuint64_t dims[4] = {(cuuint64_t)g.ci, (cuuint64_t)g.co, 3, 9};
         const cuuint64_t strides[3] = {(cuuint64_t)g.ci * 2, (cuuint64_t)g.ci * 2 * g.co * 9, (cuuint64_t)g.ci * 2 * g.co};
-        const cuuint32_t box[4] = {(cuuint32_t)pl.KC, (cuuint32_t)pl.COB, (cuuint32_t)(128 / pl.COB), (cuuint32_t)(pl.KC == 32 ? 3 : 1)};
+        const bool wres = pl.KC == 32 && pl.COB == 32;      // resident weights: one box = the three kd blocks of a tap
+        const cuuint32_t box[4] = {(cuuint32_t)pl.KC, (cuuint32_t)pl.COB, (cuuint32_t)(wres ? 3 : 128 / pl.COB),
+                                   (cuuint32_t)(wres ? 1 : (pl.KC == 32 ? 3 : 1))};
         const cuuint32_t es[4] = {1, 1, 1, 1};
         if (encode(&mw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void *)w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
