@@ -561,6 +561,15 @@ def run_hbm(args):
     ms = timed(lambda: B.lamp_conv3d_fwd(desc, xd, wd, torch.zeros(64, device="cuda"), yd, std), flush)
     res["down conv 32->64 stride 2"] = dict(ms=round(ms, 4), bytes=nb, gbs=round(nb / ms / 1e6, 1))
     del xu, cat, xd, yd
+    # parameter update over a flat buffer the size of the 175 M-parameter network's weights
+    npar = 175 * 1000 * 1000
+    gq = torch.randn(npar, device="cuda")
+    wq = torch.randn(npar, device="cuda")
+    vq = torch.rand(npar, device="cuda")
+    wq16 = torch.empty(npar, dtype=torch.bfloat16, device="cuda")
+    ms = timed(lambda: B.lamp_rmsprop_step(gq, wq, vq, wq16, 1e-3, 0.99, 1e-8), flush)
+    res["rmsprop step 175 M parameters"] = dict(ms=round(ms, 4), bytes=22 * npar, gbs=round(22 * npar / ms / 1e6, 1))
+    del gq, wq, vq, wq16
     # overlap-add on the 512 x 512 x 128 volume: 363 patches of 64^3, K = 10
     K, P = 10, (64, 64, 64)
     Dv, Hv, Wv = 512, 512, 128

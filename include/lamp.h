@@ -257,6 +257,21 @@ lamp_status_t lamp_overlap_add(const float *patch_probs, int32_t k, int32_t d, i
                                const int32_t patch[3], float overlap, int32_t window,
                                float *probs_planar, uint8_t *argmax, void *cuda_stream);
 
+/* ------------------------------------------------------------------------
+ * Parameter update (Sec. 3, training setup: RMSProp, learning rate 1e-3; the update is the
+ * one of the lecture the paper cites, without momentum or centring).
+ * ---------------------------------------------------------------------- */
+
+/* For each of the n elements:  v = alpha * v + (1 - alpha) * g^2;  master -= lr * g / (sqrt(v) + eps);
+ * param_bf16 = bf16(master) (round to nearest even).
+ * grad, master, v: device fp32 [n] (v is the running mean of squared gradients, zero before the
+ * first step); param_bf16: device bf16 [n], or NULL for parameters that are used in fp32 (biases).
+ * master and v are updated in place.  n == 0 is a no-op.  Arithmetic in fp32.
+ * The flat layouts of lamp_unet_param_layout fit: one call for the weights (with the bf16 copy
+ * that the network calls read), one for the biases (param_bf16 = NULL, master = the bias vector). */
+lamp_status_t lamp_rmsprop_step(int64_t n, const float *grad, float *master, float *v, void *param_bf16,
+                                float lr, float alpha, float eps, void *cuda_stream);
+
 /* Synchronises `cuda_stream`, then returns and clears the device-side status word
  * (LAMP_OK, or LAMP_ERR_TIMEOUT if a bounded wait inside a kernel ran out). */
 lamp_status_t lamp_get_async_status(void *cuda_stream);

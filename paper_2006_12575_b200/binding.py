@@ -76,6 +76,7 @@ def lib():
             "lamp_sliding_window_workspace_bytes": (sz, [vp, i32, i32, i32, I3, f32, i32]),
             "lamp_sliding_window_infer": (C.c_int, [vp, vp, vp, TP, I3, f32, i32, i32, vp, vp, vp, sz, vp]),
             "lamp_overlap_add": (C.c_int, [vp, i32, i32, i32, i32, I3, f32, i32, vp, vp, vp]),
+            "lamp_rmsprop_step": (C.c_int, [C.c_int64, vp, vp, vp, vp, f32, f32, f32, vp]),
             "lamp_get_async_status": (C.c_int, [vp]),
             "lamp_selftest_wait_timeout": (C.c_int, [vp]),
             "lamp_status_string": (C.c_char_p, [C.c_int]),
@@ -95,7 +96,7 @@ EXPORTS = ["lamp_conv3d_workspace_bytes", "lamp_conv3d_workspace_min_bytes", "la
            "lamp_unet_num_layers", "lamp_unet_weight_count", "lamp_unet_bias_count", "lamp_unet_param_layout",
            "lamp_unet_workspace_bytes", "lamp_unet_tensor_layout", "lamp_unet_forward", "lamp_unet_train_step",
            "lamp_sliding_window_workspace_bytes", "lamp_sliding_window_infer", "lamp_overlap_add",
-           "lamp_get_async_status", "lamp_selftest_wait_timeout", "lamp_status_string", "lamp_version"]
+           "lamp_rmsprop_step", "lamp_get_async_status", "lamp_selftest_wait_timeout", "lamp_status_string", "lamp_version"]
 
 
 def _check(st, what):
@@ -260,6 +261,11 @@ def lamp_sliding_window_infer(net, weights, biases, volume, patch, overlap, sw_b
 def lamp_overlap_add(patch_probs, k, d, h, w, patch, overlap, window, probs_planar, argmax):
     _check(lib().lamp_overlap_add(_ptr(patch_probs), k, d, h, w, _i3(patch), overlap, window, _ptr(probs_planar),
                                   _ptr(argmax), _stream()), "lamp_overlap_add")
+
+
+def lamp_rmsprop_step(grad, master, v, param_bf16=None, lr=1e-3, alpha=0.99, eps=1e-8):
+    _check(lib().lamp_rmsprop_step(grad.numel(), _ptr(grad), _ptr(master), _ptr(v), _ptr(param_bf16), lr, alpha, eps,
+                                   _stream()), "lamp_rmsprop_step")
 
 
 def lamp_get_async_status():

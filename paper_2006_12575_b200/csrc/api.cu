@@ -314,6 +314,17 @@ lamp_status_t lamp_instnorm_relu_bwd(const lamp_tensor_t *dz_a, const lamp_tenso
                                nullptr, nullptr, nullptr, (cudaStream_t)cuda_stream);
 }
 
+lamp_status_t lamp_rmsprop_step(int64_t n, const float *grad, float *master, float *v, void *param_bf16,
+                                float lr, float alpha, float eps, void *cuda_stream)
+{
+    if (n < 0) return LAMP_ERR_INVALID_ARG;
+    if (n == 0) return LAMP_OK;
+    if (!grad || !master || !v) return LAMP_ERR_INVALID_ARG;
+    if (!(lr >= 0.f) || !(alpha >= 0.f && alpha <= 1.f) || !(eps >= 0.f)) return LAMP_ERR_INVALID_ARG;
+    if ((((uintptr_t)grad | (uintptr_t)master | (uintptr_t)v) & 3) || ((uintptr_t)param_bf16 & 1)) return LAMP_ERR_INVALID_ARG;
+    return k_rmsprop(n, grad, master, v, (bf16 *)param_bf16, lr, alpha, eps, (cudaStream_t)cuda_stream);
+}
+
 lamp_status_t lamp_get_async_status(void *cuda_stream)
 {
     if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return LAMP_ERR_CUDA;

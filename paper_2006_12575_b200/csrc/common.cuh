@@ -158,6 +158,8 @@ size_t        head_bwd_ws(int64_t Vn, int n, int K, int C);
 lamp_status_t k_head_bwd(const TView &z, const bf16 *w, int K, const float *probs, const uint8_t *labels,
                          const double *dice_sums, const TView &dz, float *dw, float *db, float *dlogits,
                          void *ws, size_t ws_bytes, cudaStream_t st);
+lamp_status_t k_rmsprop(int64_t n, const float *g, float *w, float *v, bf16 *wb, float lr, float alpha, float eps,
+                        cudaStream_t st);
 lamp_status_t k_gather_patches(const TView &vol, const TView &patches, int first_patch, const int32_t nst[3],
                                const int32_t stride[3], cudaStream_t st);
 lamp_status_t k_overlap_add(const float *pp, int K, int D, int H, int W, const int32_t patch[3],

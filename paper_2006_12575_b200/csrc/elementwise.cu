@@ -434,6 +434,41 @@ head_bwd_kernel(const bf16 *__restrict__ z, int64_t zp, int C, const bf16 *__res
     }
 }
 
+// ------------------------------------------------------------------ parameter update
+// v = alpha v + (1 - alpha) g^2; w -= lr g / (sqrt(v) + eps); bf16 copy.  Four elements per thread when the
+// pointers allow 16-byte accesses (22 bytes of traffic per element: HBM-bound).
+__global__ void __launch_bounds__(256)
+rmsprop_kernel(int64_t n, const float *__restrict__ g, float *__restrict__ w, float *__restrict__ v,
+               bf16 *__restrict__ wb, float lr, float alpha, float eps, int vec)
+{
+    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    auto upd = [&](float gi, float &wi, float &vi) {
+        vi = fmaf(alpha, vi, (1.0f - alpha) * gi * gi);
+        wi -= lr * gi / (sqrtf(vi) + eps);
+    };
+    if (vec) {
+        if (4 * i >= n) return;
+        const float4 g4 = __ldg(reinterpret_cast<const float4 *>(g) + i);
+        float4 w4 = reinterpret_cast<float4 *>(w)[i], v4 = reinterpret_cast<float4 *>(v)[i];
+        upd(g4.x, w4.x, v4.x); upd(g4.y, w4.y, v4.y); upd(g4.z, w4.z, v4.z); upd(g4.w, w4.w, v4.w);
+        reinterpret_cast<float4 *>(w)[i] = w4;
+        reinterpret_cast<float4 *>(v)[i] = v4;
+        if (wb) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(w4.x, w4.y), hi = __floats2bfloat162_rn(w4.z, w4.w);
+            uint2 u;
+            u.x = *reinterpret_cast<uint32_t *>(&lo);
+            u.y = *reinterpret_cast<uint32_t *>(&hi);
+            reinterpret_cast<uint2 *>(wb)[i] = u;
+        }
+    } else {
+        if (i >= n) return;
+        float wi = w[i], vi = v[i];
+        upd(g[i], wi, vi);
+        w[i] = wi; v[i] = vi;
+        if (wb) wb[i] = f2bf(wi);
+    }
+}
+
 // ------------------------------------------------------------------ sliding window
 __device__ __forceinline__ int patch_origin(int i, int nst, int stride, int len, int patch)
 {
@@ -739,6 +774,16 @@ lamp_status_t k_head_bwd(const TView &z, const bf16 *w, int K, const float *prob
     if (s != LAMP_OK) return s;
     if ((s = reduce_partials(partW, (int64_t)K * C, (int)(blocks * z.n), dw, st)) != LAMP_OK) return s;
     return db ? reduce_partials(partB, K, (int)(blocks * z.n), db, st) : LAMP_OK;
+}
+
+lamp_status_t k_rmsprop(int64_t n, const float *g, float *w, float *v, bf16 *wb, float lr, float alpha, float eps,
+                        cudaStream_t st)
+{
+    if (n == 0) return LAMP_OK;
+    const bool vec = n % 4 == 0 && (((uintptr_t)g | (uintptr_t)w | (uintptr_t)v) & 15) == 0 && ((uintptr_t)wb & 7) == 0;
+    const int64_t threads = vec ? n / 4 : n;
+    rmsprop_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(n, g, w, v, wb, lr, alpha, eps, vec ? 1 : 0);
+    return launch_status();
 }
 
 lamp_status_t k_gather_patches(const TView &vol, const TView &patches, int first_patch, const int32_t nst[3],
