@@ -21,6 +21,15 @@ instnorm_relu_fwd_kernel(const bf16 *__restrict__ y, int64_t yp, const double *_
     const int g = threadIdx.x % G, r = threadIdx.x / G;
     if (r >= RB) return;
     const int n = blockIdx.y;
+    const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = min(Vn, v0 + v_per_block);
+    // the first voxels are requested before the per-channel constants: their latency overlaps the fp64 arithmetic
+    constexpr int PF = 4;
+    uint4 pre[PF];
+#pragma unroll
+    for (int k = 0; k < PF; ++k) {
+        const int64_t vv = v0 + r + (int64_t)k * RB;
+        pre[k] = vv < v1 ? __ldg(reinterpret_cast<const uint4 *>(y + ((int64_t)n * Vn + vv) * yp + g * 8)) : make_uint4(0, 0, 0, 0);
+    }
     float mu[8], rs[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
@@ -32,15 +41,27 @@ instnorm_relu_fwd_kernel(const bf16 *__restrict__ y, int64_t yp, const double *_
         rs[j] = __frsqrt_rn((float)var + eps);
         if (blockIdx.x == 0 && r == 0) { mr[2 * i] = mu[j]; mr[2 * i + 1] = rs[j]; }
     }
-    const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = min(Vn, v0 + v_per_block);
-#pragma unroll 4
-    for (int64_t vv = v0 + r; vv < v1; vv += RB) {
-        const int64_t v = (int64_t)n * Vn + vv;
-        float f[8];
-        unpack8(__ldg(reinterpret_cast<const uint4 *>(y + v * yp + g * 8)), f);
+    // groups of PF voxels: the next group's loads are issued before the current group is normalised and stored
+    for (int64_t vb = v0 + r; vb < v1; vb += (int64_t)PF * RB) {
+        uint4 cur[PF];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) f[j] = fmaxf((f[j] - mu[j]) * rs[j], 0.f);
-        *reinterpret_cast<uint4 *>(z + v * zp + g * 8) = pack8(f);
+        for (int k = 0; k < PF; ++k) cur[k] = pre[k];
+#pragma unroll
+        for (int k = 0; k < PF; ++k) {
+            const int64_t vv = vb + (int64_t)(PF + k) * RB;
+            pre[k] = vv < v1 ? __ldg(reinterpret_cast<const uint4 *>(y + ((int64_t)n * Vn + vv) * yp + g * 8)) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int k = 0; k < PF; ++k) {
+            const int64_t vv = vb + (int64_t)k * RB;
+            if (vv < v1) {
+                float f[8];
+                unpack8(cur[k], f);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) f[j] = fmaxf((f[j] - mu[j]) * rs[j], 0.f);
+                *reinterpret_cast<uint4 *>(z + ((int64_t)n * Vn + vv) * zp + g * 8) = pack8(f);
+            }
+        }
     }
 }
 
@@ -68,24 +89,39 @@ instnorm_bwd_sums_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *_
         }
         const int64_t v0 = (int64_t)blockIdx.x * v_per_block;
         const int64_t v1 = min(Vn, v0 + v_per_block);
-#pragma unroll 4
-        for (int64_t vv = v0 + r; vv < v1; vv += RB) {
+        // groups of PF voxels, the next group's loads in flight while the current one is summed; voxels past the end
+        // arrive as zero gradients and add nothing
+        constexpr int PF = 2;
+        const uint4 zero4 = make_uint4(0, 0, 0, 0);
+        uint4 py[PF], pa[PF], pb[PF];
+        auto fetch = [&](int64_t vv, uint4 &qy, uint4 &qa, uint4 &qb) {
+            const bool in = vv < v1;
             const int64_t v = (int64_t)n * Vn + vv;
-            float fy[8], fa[8];
-            unpack8(__ldg(reinterpret_cast<const uint4 *>(y + v * yp + g * 8)), fy);
-            unpack8(__ldg(reinterpret_cast<const uint4 *>(dza + v * ap + g * 8)), fa);
-            if (dzb) {
-                float fb[8];
-                unpack8(__ldg(reinterpret_cast<const uint4 *>(dzb + v * bp + g * 8)), fb);
+            qy = in ? __ldg(reinterpret_cast<const uint4 *>(y + v * yp + g * 8)) : zero4;
+            qa = in ? __ldg(reinterpret_cast<const uint4 *>(dza + v * ap + g * 8)) : zero4;
+            qb = (in && dzb) ? __ldg(reinterpret_cast<const uint4 *>(dzb + v * bp + g * 8)) : zero4;
+        };
 #pragma unroll
-                for (int j = 0; j < 8; ++j) fa[j] += fb[j];
-            }
+        for (int k = 0; k < PF; ++k) fetch(v0 + r + (int64_t)k * RB, py[k], pa[k], pb[k]);
+        for (int64_t vb = v0 + r; vb < v1; vb += (int64_t)PF * RB) {
+            uint4 cy[PF], ca[PF], cb[PF];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float xh = (fy[j] - mu[j]) * rs[j];
-                const float gg = xh > 0.f ? fa[j] : 0.f;
-                s[j] += gg;
-                s[8 + j] = fmaf(gg, xh, s[8 + j]);
+            for (int k = 0; k < PF; ++k) { cy[k] = py[k]; ca[k] = pa[k]; cb[k] = pb[k]; }
+#pragma unroll
+            for (int k = 0; k < PF; ++k) fetch(vb + (int64_t)(PF + k) * RB, py[k], pa[k], pb[k]);
+#pragma unroll
+            for (int k = 0; k < PF; ++k) {
+                float fy[8], fa[8], fb[8];
+                unpack8(cy[k], fy);
+                unpack8(ca[k], fa);
+                unpack8(cb[k], fb);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float xh = (fy[j] - mu[j]) * rs[j];
+                    const float gg = xh > 0.f ? fa[j] + fb[j] : 0.f;
+                    s[j] += gg;
+                    s[8 + j] = fmaf(gg, xh, s[8 + j]);
+                }
             }
         }
 #pragma unroll
@@ -132,30 +168,47 @@ instnorm_bwd_apply_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *
         cs[j] = 0.f;
     }
     const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = active ? min(Vn, v0 + v_per_block) : v0;
-#pragma unroll 2
-    for (int64_t vv = v0 + r; vv < v1; vv += RB) {
+    // groups of PF voxels, the next group's loads in flight while the current one is processed
+    constexpr int PF = 2;
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    uint4 py[PF], pa[PF], pb[PF];
+    auto fetch = [&](int64_t vv, uint4 &qy, uint4 &qa, uint4 &qb) {
+        const bool in = vv < v1;
         const int64_t v = (int64_t)n * Vn + vv;
-        float fy[8], fa[8];
-        unpack8(__ldg(reinterpret_cast<const uint4 *>(y + v * yp + g * 8)), fy);
-        unpack8(__ldg(reinterpret_cast<const uint4 *>(dza + v * ap + g * 8)), fa);
-        if (dzb) {
-            float fb[8];
-            unpack8(__ldg(reinterpret_cast<const uint4 *>(dzb + v * bp + g * 8)), fb);
+        qy = in ? __ldg(reinterpret_cast<const uint4 *>(y + v * yp + g * 8)) : zero4;
+        qa = in ? __ldg(reinterpret_cast<const uint4 *>(dza + v * ap + g * 8)) : zero4;
+        qb = (in && dzb) ? __ldg(reinterpret_cast<const uint4 *>(dzb + v * bp + g * 8)) : zero4;
+    };
 #pragma unroll
-            for (int j = 0; j < 8; ++j) fa[j] += fb[j];
-        }
+    for (int k = 0; k < PF; ++k) fetch(v0 + r + (int64_t)k * RB, py[k], pa[k], pb[k]);
+    for (int64_t vb = v0 + r; vb < v1; vb += (int64_t)PF * RB) {
+        uint4 cy[PF], ca[PF], cb[PF];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const float xh = (fy[j] - mu[j]) * rs[j];
-            const float gg = xh > 0.f ? fa[j] : 0.f;
-            fa[j] = rs[j] * (gg - m1[j] - xh * m2[j]);
-        }
-        const uint4 q = pack8(fa);
-        *reinterpret_cast<uint4 *>(dy + v * dp + g * 8) = q;
-        if (DB) {
-            unpack8(q, fa);
+        for (int k = 0; k < PF; ++k) { cy[k] = py[k]; ca[k] = pa[k]; cb[k] = pb[k]; }
 #pragma unroll
-            for (int j = 0; j < 8; ++j) cs[j] += fa[j];
+        for (int k = 0; k < PF; ++k) fetch(vb + (int64_t)(PF + k) * RB, py[k], pa[k], pb[k]);
+#pragma unroll
+        for (int k = 0; k < PF; ++k) {
+            const int64_t vv = vb + (int64_t)k * RB;
+            if (vv >= v1) break;
+            const int64_t v = (int64_t)n * Vn + vv;
+            float fy[8], fa[8], fb[8];
+            unpack8(cy[k], fy);
+            unpack8(ca[k], fa);
+            unpack8(cb[k], fb);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float xh = (fy[j] - mu[j]) * rs[j];
+                const float gg = xh > 0.f ? fa[j] + fb[j] : 0.f;
+                fa[j] = rs[j] * (gg - m1[j] - xh * m2[j]);
+            }
+            const uint4 q = pack8(fa);
+            *reinterpret_cast<uint4 *>(dy + v * dp + g * 8) = q;
+            if (DB) {
+                unpack8(q, fa);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) cs[j] += fa[j];
+            }
         }
     }
     if (!DB) return;
