@@ -74,6 +74,36 @@ static inline lamp_status_t launch_status()
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Programmatic dependent launch.  A kernel launched through launch_pdl may be scheduled while the kernel in front
+// of it on the stream is still running: its blocks set up shared memory, barriers and tensor memory, then stop at
+// pdl_wait() until that kernel has completed and its writes are visible.  Rules every such kernel follows:
+//   * every thread executes pdl_wait() before its first access to global memory and before any return, so that
+//     the completion of this kernel implies the completion of all kernels in front of it;
+//   * pdl_launch_dependents() (no memory semantics) is executed at the top, which lets the next kernel's blocks
+//     take over SMs as this kernel's blocks retire.
+// Kernels launched with <<<>>> keep the plain stream order on both sides.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline lamp_status_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                       Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...) == cudaSuccess ? LAMP_OK : LAMP_ERR_CUDA;
+}
+#endif
+
 // ---------------------------------------------------------------------------
 // Internal launchers (one per kernel family); all enqueue on `st`.
 // ---------------------------------------------------------------------------

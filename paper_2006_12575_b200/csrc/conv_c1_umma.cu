@@ -94,6 +94,7 @@ conv_c1_umma_kernel(const __grid_constant__ CUtensorMap map_x, const C1Params P)
     const int part = blockIdx.x % P.nparts;                     // the CTA's block of 32 output channels
     const int first = blockIdx.x / P.nparts, step = gridDim.x / P.nparts;
 
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 4); }
@@ -101,6 +102,7 @@ conv_c1_umma_kernel(const __grid_constant__ CUtensorMap map_x, const C1Params P)
         mbar_init_fence();
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+    pdl_wait();                 // everything above touched shared and tensor memory only
     // the nine banded matrices: row (j, c), position i -> w[kd][kh][i - 7 - j][part * 32 + c] inside the band
     for (int idx = threadIdx.x; idx < 9 * 256 * 4; idx += C1_THREADS) {
         const int tap = idx / 1024, r = (idx >> 2) & 255, ch = idx & 3;
@@ -357,7 +359,8 @@ lamp_status_t c1_umma_fwd(const ConvGeom &g, const TView &x, const bf16 *w, cons
     if (per_part < 1) per_part = 1;
     if (per_part > tiles) per_part = tiles;
     const int grid = (int)(per_part * P.nparts);
-    conv_c1_umma_kernel<<<grid, C1_THREADS, C1_SMEM, st>>>(mx, P);
+    const lamp_status_t ls = launch_pdl(conv_c1_umma_kernel, dim3(grid), dim3(C1_THREADS), (size_t)C1_SMEM, st, mx, P);
+    if (ls != LAMP_OK) return ls;
     return launch_status();
 }
 

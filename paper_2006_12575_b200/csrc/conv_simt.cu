@@ -207,6 +207,8 @@ __global__ void __launch_bounds__(256)
 colsum_vec_kernel(const bf16 *__restrict__ dy, int64_t dyp, int co, int64_t V, int64_t v_per_block, float *__restrict__ part)
 {
     extern __shared__ float red[];          // [RB][G][8]
+    pdl_launch_dependents();
+    pdl_wait();
     const int G = co >> 3, RB = 256 / G;
     const int g = threadIdx.x % G, r = threadIdx.x / G;
     const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = min(V, v0 + v_per_block);
@@ -392,6 +394,8 @@ __global__ void __launch_bounds__(256)
 reduce_parts_kernel(const float *__restrict__ part, int64_t entries, int splits, float *__restrict__ out)
 {
     __shared__ float red[8][32];
+    pdl_launch_dependents();
+    pdl_wait();
     const int el = threadIdx.x & 31, sl = threadIdx.x >> 5;
     const int64_t e = (int64_t)blockIdx.x * 32 + el;
     float acc = 0.f;
@@ -411,6 +415,8 @@ reduce_parts_kernel(const float *__restrict__ part, int64_t entries, int splits,
 __global__ void __launch_bounds__(256)
 reduce_parts_vec4_kernel(const float4 *__restrict__ part, int64_t entries4, int splits, float4 *__restrict__ out)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;
     if (e >= entries4) return;
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -429,6 +435,8 @@ __global__ void __launch_bounds__(256)
 transpose_sum_kernel(const T *__restrict__ in, int64_t split_stride, int splits, int A, int B, T *__restrict__ out)
 {
     __shared__ float tile[32][33];
+    pdl_launch_dependents();
+    pdl_wait();
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;           // 32 x 8
     const int b0 = blockIdx.x * 32, a0 = blockIdx.y * 32;
     const int64_t t = blockIdx.z;
@@ -452,6 +460,8 @@ transpose_sum_kernel(const T *__restrict__ in, int64_t split_stride, int splits,
 __global__ void __launch_bounds__(256)
 pad_c1_kernel(const bf16 *__restrict__ x, int64_t xp, bf16 *__restrict__ xpad, int64_t V)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;      // one 16-byte group of 8 channels
     if (e >= V * 4) return;
     const int64_t v = e >> 2;
@@ -464,6 +474,8 @@ pad_c1_kernel(const bf16 *__restrict__ x, int64_t xp, bf16 *__restrict__ xpad, i
 __global__ void __launch_bounds__(256)
 take_c0_kernel(const float *__restrict__ dw32, float *__restrict__ dw, int n)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int i = blockIdx.x * 256 + threadIdx.x;
     if (i < n) dw[i] = dw32[(int64_t)i * 32];
 }
@@ -542,25 +554,22 @@ lamp_status_t reduce_partials(const float *part, int64_t entries, int splits, fl
 {
     if (entries == 0) return LAMP_OK;
     if (splits <= 16 && entries >= 32768 && entries % 4 == 0 && (((uintptr_t)part | (uintptr_t)out) & 15) == 0)
-        reduce_parts_vec4_kernel<<<(unsigned)((entries / 4 + 255) / 256), 256, 0, st>>>(
-            (const float4 *)part, entries / 4, splits, (float4 *)out);
+        return launch_pdl(reduce_parts_vec4_kernel, dim3((unsigned)((entries / 4 + 255) / 256)), dim3(256), 0, st,
+                          (const float4 *)part, entries / 4, splits, (float4 *)out);
     else
-        reduce_parts_kernel<<<(unsigned)((entries + 31) / 32), 256, 0, st>>>(part, entries, splits, out);
-    return launch_status();
+        return launch_pdl(reduce_parts_kernel, dim3((unsigned)((entries + 31) / 32)), dim3(256), 0, st, part, entries, splits, out);
 }
 
 bool transpose_sum_supported(int64_t taps, int A, int B) { return A % 32 == 0 && B % 32 == 0 && taps > 0 && taps <= 65535; }
 
 lamp_status_t transpose_sum_f32(const float *in, int64_t taps, int A, int B, int splits, float *out, cudaStream_t st)
 {
-    transpose_sum_kernel<float><<<dim3(B / 32, A / 32, (unsigned)taps), 256, 0, st>>>(in, taps * A * B, splits, A, B, out);
-    return launch_status();
+    return launch_pdl(transpose_sum_kernel<float>, dim3(B / 32, A / 32, (unsigned)taps), dim3(256), 0, st, in, taps * A * B, splits, A, B, out);
 }
 
 lamp_status_t transpose_bf16(const bf16 *in, int64_t taps, int A, int B, bf16 *out, cudaStream_t st)
 {
-    transpose_sum_kernel<bf16><<<dim3(B / 32, A / 32, (unsigned)taps), 256, 0, st>>>(in, 0, 1, A, B, out);
-    return launch_status();
+    return launch_pdl(transpose_sum_kernel<bf16>, dim3(B / 32, A / 32, (unsigned)taps), dim3(256), 0, st, in, (int64_t)0, 1, A, B, out);
 }
 
 static void bias_plan(int64_t V, int *blocks, int64_t *vpb)
@@ -586,7 +595,9 @@ lamp_status_t bias_grad(const TView &dy, float *db, void *ws, cudaStream_t st)
     bias_plan(V, &b, &vpb);
     if (dy.c % 8 == 0 && dy.c <= 2048 && dy.pitch % 8 == 0 && ((uintptr_t)dy.p & 15) == 0) {
         const int G = dy.c / 8, RB = 256 / G;
-        colsum_vec_kernel<<<b, 256, (size_t)RB * dy.c * sizeof(float), st>>>((const bf16 *)dy.p, dy.pitch, dy.c, V, vpb, (float *)ws);
+        if (launch_pdl(colsum_vec_kernel, dim3(b), dim3(256), (size_t)RB * dy.c * sizeof(float), st, (const bf16 *)dy.p, dy.pitch, dy.c, V, vpb,
+                       (float *)ws) != LAMP_OK)
+            return LAMP_ERR_CUDA;
     } else {
         colsum_kernel<<<b, 256, 0, st>>>((const bf16 *)dy.p, dy.pitch, dy.c, V, vpb, (float *)ws);
     }
@@ -613,14 +624,12 @@ lamp_status_t pad_c1(const TView &x, bf16 *xpad, cudaStream_t st)
 {
     const int64_t V = (int64_t)x.n * x.d * x.h * x.w;
     if (V == 0) return LAMP_OK;
-    pad_c1_kernel<<<(unsigned)((V * 4 + 255) / 256), 256, 0, st>>>((const bf16 *)x.p, x.pitch, xpad, V);
-    return launch_status();
+    return launch_pdl(pad_c1_kernel, dim3((unsigned)((V * 4 + 255) / 256)), dim3(256), 0, st, (const bf16 *)x.p, x.pitch, xpad, V);
 }
 
 lamp_status_t take_c0(const float *dw32, float *dw, int n, cudaStream_t st)
 {
-    take_c0_kernel<<<(n + 255) / 256, 256, 0, st>>>(dw32, dw, n);
-    return launch_status();
+    return launch_pdl(take_c0_kernel, dim3((n + 255) / 256), dim3(256), 0, st, dw32, dw, n);
 }
 
 size_t simt_conv_wgrad_ws(const ConvGeom &g)

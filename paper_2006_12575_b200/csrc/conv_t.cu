@@ -106,6 +106,7 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_NP; ++s) { mbar_init(pfull0 + 8 * s, 1); mbar_init(pempty0 + 8 * s, 1); }
         for (int s = 0; s < MAX_NW; ++s) { mbar_init(wfull0 + 8 * s, 1); mbar_init(wempty0 + 8 * s, 1); }
@@ -122,6 +123,7 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
         fence_proxy_async();
     }
+    pdl_wait();                 // everything above touched shared and tensor memory only
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -411,8 +413,7 @@ lamp_status_t launch_ct(const CUtensorMap &mx, const CUtensorMap &mw, const CtPl
         LAMP_CUDA_OK(cudaFuncSetAttribute(conv3_t_kernel<KC, COB>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT));
         attr = true;
     }
-    conv3_t_kernel<KC, COB><<<pl.grid, CT_THREADS, pl.smem, st>>>(mx, mw, pl.P);
-    return launch_status();
+    return launch_pdl(conv3_t_kernel<KC, COB>, dim3(pl.grid), dim3(CT_THREADS), pl.smem, st, mx, mw, pl.P);
 }
 
 }  // namespace

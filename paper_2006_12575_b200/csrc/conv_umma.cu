@@ -156,6 +156,7 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + MAX_STAGES);
     const uint32_t tfull0 = smem_u32(bars + 2 * MAX_STAGES), tempty0 = smem_u32(bars + 2 * MAX_STAGES + MAX_ACC);
 
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         for (int a = 0; a < NACC; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 4); }
@@ -163,6 +164,7 @@ conv3_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         mbar_init_fence();
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), L::TMEM_COLS);
+    pdl_wait();                 // everything above touched shared and tensor memory only
     float *sbias = epi;
     const bool bias_staged = P.bias && P.co <= MAX_SBIAS;
     if (bias_staged)
@@ -456,6 +458,8 @@ splitk_finish_kernel(const float *__restrict__ part, int64_t split_elems, int ks
                      double *__restrict__ stats)
 {
     __shared__ float4 red[2][FIN_THREADS];
+    pdl_launch_dependents();
+    pdl_wait();
     const int n = blockIdx.z;
     const int cl = threadIdx.x % FIN_CG, vl = threadIdx.x / FIN_CG;
     const int cg = blockIdx.y * FIN_CG + cl;                       // group of 4 channels
@@ -595,8 +599,7 @@ lamp_status_t launch(const CUtensorMap &mx, const CUtensorMap &mw, const UmmaPar
         for (int i = 0; i < 6; ++i) { Q.step[i] = t % radix[i]; t /= radix[i]; }
         Q.step[6] = t;
     }
-    conv3_umma_kernel<KC, BN, HEAD><<<grid, L::THREADS, L::TOTAL, st>>>(mx, mw, Q);
-    return launch_status();
+    return launch_pdl(conv3_umma_kernel<KC, BN, HEAD>, dim3(grid), dim3(L::THREADS), L::TOTAL, st, mx, mw, Q);
 }
 
 template <int KC>
@@ -893,9 +896,8 @@ lamp_status_t umma_conv(int kind, const ConvGeom &g, const TView &a, const bf16 
     if (s != LAMP_OK || !split) return s;
     const int64_t vox_per_n = (int64_t)k.od * k.oh * k.ow;
     const dim3 grid((unsigned)((vox_per_n + FIN_VOX - 1) / FIN_VOX), (unsigned)((k.n_rows / 4 + FIN_CG - 1) / FIN_CG), (unsigned)g.n);
-    splitk_finish_kernel<<<grid, FIN_THREADS, 0, st>>>((const float *)part, out_vox * k.n_rows, P.ksplit, vox_per_n, k.n_rows,
-                                                      bias, y.p, y.f32, y.pitch, stats);
-    return launch_status();
+    return launch_pdl(splitk_finish_kernel, grid, dim3(FIN_THREADS), 0, st, (const float *)part, out_vox * k.n_rows, P.ksplit,
+                      vox_per_n, k.n_rows, bias, y.p, y.f32, y.pitch, stats);
 }
 
 }  // namespace lamp

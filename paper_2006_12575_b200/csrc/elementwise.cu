@@ -17,11 +17,15 @@ __global__ void __launch_bounds__(256)
 instnorm_relu_fwd_kernel(const bf16 *__restrict__ y, int64_t yp, const double *__restrict__ stats, double inv_v, float eps,
                          float *__restrict__ mr, bf16 *__restrict__ z, int64_t zp, int64_t Vn, int C, int64_t v_per_block)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int G = C >> 3, RB = 256 / G;
     const int g = threadIdx.x % G, r = threadIdx.x / G;
     if (r >= RB) return;
     const int n = blockIdx.y;
-    const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = min(Vn, v0 + v_per_block);
+    // blocks are numbered back to front: the convolution in front wrote y front to back, so the tensor's tail is what
+    // the L2 cache still holds, and the head of z is what the next convolution finds there
+    const int64_t v0 = (int64_t)(gridDim.x - 1 - blockIdx.x) * v_per_block, v1 = min(Vn, v0 + v_per_block);
     // the first voxels are requested before the per-channel constants: their latency overlaps the fp64 arithmetic
     constexpr int PF = 4;
     uint4 pre[PF];
@@ -72,6 +76,8 @@ instnorm_bwd_sums_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *_
                          const bf16 *__restrict__ y, int64_t yp, const float *__restrict__ mr,
                          double *__restrict__ sums, int64_t Vn, int C, int64_t v_per_block)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     extern __shared__ float red[];          // [RB][G][16]
     const int G = C >> 3;
     const int RB = 256 / G;
@@ -87,7 +93,9 @@ instnorm_bwd_sums_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *_
             mu[j] = mr[((int64_t)n * C + g * 8 + j) * 2];
             rs[j] = mr[((int64_t)n * C + g * 8 + j) * 2 + 1];
         }
-        const int64_t v0 = (int64_t)blockIdx.x * v_per_block;
+        // back to front (the tail of the gradient just written is still in L2); pass 2 then walks front to back
+        // and finds the head of dz and y that this pass read last
+        const int64_t v0 = (int64_t)(gridDim.x - 1 - blockIdx.x) * v_per_block;
         const int64_t v1 = min(Vn, v0 + v_per_block);
         // groups of PF voxels, the next group's loads in flight while the current one is summed; voxels past the end
         // arrive as zero gradients and add nothing
@@ -150,6 +158,8 @@ instnorm_bwd_apply_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *
                           int64_t v_per_block, double *__restrict__ db_acc, unsigned *__restrict__ db_count,
                           float *__restrict__ db_out)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     extern __shared__ float cred[];          // DB: [RB][C] column sums of the block
     __shared__ int is_last;
     const int G = C >> 3, RB = 256 / G;
@@ -247,6 +257,8 @@ head_softmax_kernel(const bf16 *__restrict__ z, int64_t zp, int C, const bf16 *_
                     const float *__restrict__ b, int K, float *__restrict__ probs, uint8_t *__restrict__ amax,
                     const uint8_t *__restrict__ labels, double *__restrict__ dice, int64_t Vn, int64_t v_per_block)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     extern __shared__ __align__(16) float sm[];   // w as float [KP][C], bias [KP], reduce [3*KMAX], probability tile [256][K]
     float *sw = sm, *sb = sm + KP * C, *sred = sb + KP, *sp = sred + 3 * KMAX;
     for (int i = threadIdx.x; i < KP * C; i += 256) sw[i] = i < K * C ? bf2f(w[i]) : 0.f;
@@ -340,6 +352,8 @@ head_softmax_kernel(const bf16 *__restrict__ z, int64_t zp, int C, const bf16 *_
 // dice[n][k][3] = (I, P, G)  ->  loss = mean_n (1 - mean_k (2I + e)/(P + G + e))
 __global__ void dice_loss_kernel(const double *__restrict__ dice, int N, int K, float *__restrict__ loss)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     const double eps = 1e-5;
     double L = 0.0;
@@ -367,6 +381,8 @@ head_bwd_kernel(const bf16 *__restrict__ z, int64_t zp, int C, const bf16 *__res
                 int N, bf16 *__restrict__ dz, int64_t dzp, float *__restrict__ partW, float *__restrict__ partB,
                 float *__restrict__ dlog, int64_t Vn, int64_t v_per_block)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     extern __shared__ __align__(16) float sm[];
     // [KP*C] weights, [KP] + [KP] dice coefficients, then the tile: dl [256][KP], probabilities [256][K], z [256][C] bf16
     float *sw = sm, *sa = sm + KP * C, *sbq = sa + KP, *sdl = sbq + KP, *sp = sdl + 256 * KP;
@@ -494,6 +510,8 @@ __global__ void __launch_bounds__(256)
 rmsprop_kernel(int64_t n, const float *__restrict__ g, float *__restrict__ w, float *__restrict__ v,
                bf16 *__restrict__ wb, float lr, float alpha, float eps, int vec)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
     auto upd = [&](float gi, float &wi, float &vi) {
         vi = fmaf(alpha, vi, (1.0f - alpha) * gi * gi);
@@ -535,6 +553,8 @@ gather_patches_kernel(const bf16 *__restrict__ vol, int64_t vp, int D, int H, in
                       bf16 *__restrict__ out, int64_t op, int B, int PD, int PH, int PW, int first,
                       int nd, int nh, int nw, int sd, int sh, int sw)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int64_t per = (int64_t)PD * PH * PW * C;
     const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;
     if (e >= per * B) return;
@@ -562,6 +582,8 @@ overlap_add_kernel(const float *__restrict__ pp, int Krt, int D, int H, int W, i
                    int nd, int nh, int nw, int sd, int sh, int sw, int window, int aligned4,
                    float *__restrict__ planar, uint8_t *__restrict__ amax)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int K = KT > 0 ? KT : Krt;
     extern __shared__ float tab[];          // 1-D window factors: [PD] [PH] [PW], each normalised to max 1
     float *td = tab, *th = tab + PD, *tw = th + PH;
@@ -684,7 +706,7 @@ lamp_status_t k_instnorm_relu_fwd(const TView &y, const double *stats, float eps
     int64_t vpb = (Vn / (148 * 16) + rb - 1) / rb * rb;
     if (vpb < rb * 8) vpb = rb * 8;
     dim3 grid((unsigned)((Vn + vpb - 1) / vpb), y.n);
-    instnorm_relu_fwd_kernel<<<grid, 256, 0, st>>>((const bf16 *)y.p, y.pitch, stats, 1.0 / (double)Vn, eps, mu_rstd,
+    (void)launch_pdl(instnorm_relu_fwd_kernel, grid, dim3(256), (size_t)(0), st, (const bf16 *)y.p, y.pitch, stats, 1.0 / (double)Vn, eps, mu_rstd,
                                                    (bf16 *)z.p, z.pitch, Vn, y.c, vpb);
     return launch_status();
 }
@@ -708,18 +730,18 @@ lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TVie
     const int64_t vpb = (Vn + blocks - 1) / blocks;
     blocks = (Vn + vpb - 1) / vpb;
     const size_t smem = (size_t)RB * G * 16 * sizeof(float);
-    instnorm_bwd_sums_kernel<<<dim3((unsigned)blocks, y.n), 256, smem, st>>>(
+    (void)launch_pdl(instnorm_bwd_sums_kernel, dim3((unsigned)blocks, y.n), dim3(256), (size_t)(smem), st, 
         (const bf16 *)dza.p, dza.pitch, dzb ? (const bf16 *)dzb->p : nullptr, dzb ? dzb->pitch : 0,
         (const bf16 *)y.p, y.pitch, mu_rstd, sums, Vn, C, vpb);
     int64_t vpa = (Vn / (148 * 16) + RB - 1) / RB * RB;
     if (vpa < (int64_t)RB * 8) vpa = (int64_t)RB * 8;
     dim3 grid((unsigned)((Vn + vpa - 1) / vpa), y.n);
     if (db)
-        instnorm_bwd_apply_kernel<true><<<grid, 256, (size_t)RB * C * sizeof(float), st>>>(
+        (void)launch_pdl(instnorm_bwd_apply_kernel<true>, grid, dim3(256), (size_t)((size_t)RB * C * sizeof(float)), st, 
             (const bf16 *)dza.p, dza.pitch, dzb ? (const bf16 *)dzb->p : nullptr, dzb ? dzb->pitch : 0,
             (const bf16 *)y.p, y.pitch, mu_rstd, sums, (bf16 *)dy.p, dy.pitch, Vn, C, vpa, db_acc, db_count, db);
     else
-        instnorm_bwd_apply_kernel<false><<<grid, 256, 0, st>>>(
+        (void)launch_pdl(instnorm_bwd_apply_kernel<false>, grid, dim3(256), (size_t)(0), st, 
             (const bf16 *)dza.p, dza.pitch, dzb ? (const bf16 *)dzb->p : nullptr, dzb ? dzb->pitch : 0,
             (const bf16 *)y.p, y.pitch, mu_rstd, sums, (bf16 *)dy.p, dy.pitch, Vn, C, vpa, nullptr, nullptr, nullptr);
     return launch_status();
@@ -752,7 +774,7 @@ lamp_status_t k_head_softmax(const TView &z, const bf16 *w, const float *b, int 
     const size_t smem = ((size_t)KP * z.c + KP + 3 * KMAX + 256 * K) * sizeof(float);
     const dim3 grid((unsigned)blocks, z.n);
 #define LAMP_HEAD_FWD(kp)                                                                                         \
-    head_softmax_kernel<kp><<<grid, 256, smem, st>>>((const bf16 *)z.p, z.pitch, z.c, w, b, K, probs, argmax, labels, \
+    (void)launch_pdl(head_softmax_kernel<kp>, grid, dim3(256), (size_t)(smem), st, (const bf16 *)z.p, z.pitch, z.c, w, b, K, probs, argmax, labels, \
                                                      dice_sums, Vn, vpb)
     switch (KP) {
     case 4:  LAMP_HEAD_FWD(4); break;
@@ -766,7 +788,7 @@ lamp_status_t k_head_softmax(const TView &z, const bf16 *w, const float *b, int 
 
 lamp_status_t k_dice_loss(const double *dice_sums, int N, int K, float *loss, cudaStream_t st)
 {
-    dice_loss_kernel<<<1, 32, 0, st>>>(dice_sums, N, K, loss);
+    (void)launch_pdl(dice_loss_kernel, dim3(1), dim3(32), (size_t)(0), st, dice_sums, N, K, loss);
     return launch_status();
 }
 
@@ -793,7 +815,7 @@ static lamp_status_t launch_head_bwd(const TView &z, const bf16 *w, int K, const
         LAMP_CUDA_OK(cudaFuncSetAttribute(head_bwd_kernel<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
         attr_set = true;
     }
-    head_bwd_kernel<KP><<<dim3((unsigned)blocks, z.n), 256, smem, st>>>(
+    (void)launch_pdl(head_bwd_kernel<KP>, dim3((unsigned)blocks, z.n), dim3(256), (size_t)(smem), st, 
         (const bf16 *)z.p, z.pitch, C, w, K, probs, labels, dice_sums, z.n, (bf16 *)dz.p, dz.pitch, partW, partB, dlogits,
         Vn, vpb);
     return launch_status();
@@ -835,7 +857,7 @@ lamp_status_t k_rmsprop(int64_t n, const float *g, float *w, float *v, bf16 *wb,
     if (n == 0) return LAMP_OK;
     const bool vec = n % 4 == 0 && (((uintptr_t)g | (uintptr_t)w | (uintptr_t)v) & 15) == 0 && ((uintptr_t)wb & 7) == 0;
     const int64_t threads = vec ? n / 4 : n;
-    rmsprop_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(n, g, w, v, wb, lr, alpha, eps, vec ? 1 : 0);
+    (void)launch_pdl(rmsprop_kernel, dim3((unsigned)((threads + 255) / 256)), dim3(256), (size_t)(0), st, n, g, w, v, wb, lr, alpha, eps, vec ? 1 : 0);
     return launch_status();
 }
 
@@ -844,7 +866,7 @@ lamp_status_t k_gather_patches(const TView &vol, const TView &patches, int first
 {
     const int64_t total = (int64_t)patches.n * patches.d * patches.h * patches.w * patches.c;
     if (total == 0) return LAMP_OK;
-    gather_patches_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
+    (void)launch_pdl(gather_patches_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), (size_t)(0), st, 
         (const bf16 *)vol.p, vol.pitch, vol.d, vol.h, vol.w, vol.c, (bf16 *)patches.p, patches.pitch, patches.n,
         patches.d, patches.h, patches.w, first_patch, nst[0], nst[1], nst[2], stride[0], stride[1], stride[2]);
     return launch_status();
@@ -861,7 +883,7 @@ lamp_status_t k_overlap_add(const float *pp, int K, int D, int H, int W, const i
     const int aligned4 = vec && patch[2] % 4 == 0 && (nst[2] == 1 || stride[2] % 4 == 0) && (W - patch[2]) % 4 == 0 &&
                          ((uintptr_t)pp % 16 == 0);
 #define LAMP_OA(VECN, KTN)                                                                                              \
-    overlap_add_kernel<VECN, KTN><<<(unsigned)((total + 255) / 256), 256, smem, st>>>(                                \
+    (void)launch_pdl(overlap_add_kernel<VECN, KTN>, dim3((unsigned)((total + 255) / 256)), dim3(256), (size_t)(smem), st,                                 \
         pp, K, D, H, W, patch[0], patch[1], patch[2], nst[0], nst[1], nst[2], stride[0], stride[1], stride[2], window, \
         aligned4, planar, argmax)
     if (vec) {

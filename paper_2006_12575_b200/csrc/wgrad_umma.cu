@@ -90,6 +90,7 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < NX; ++s) { mbar_init(xfull0 + 8 * s, 1); mbar_init(xempty0 + 8 * s, 1); }
         for (int s = 0; s < NA; ++s) { mbar_init(afull0 + 8 * s, 1); mbar_init(aempty0 + 8 * s, 1); }
@@ -99,6 +100,7 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         mbar_init_fence();
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), L::TMEM_COLS);
+    pdl_wait();                 // everything above touched shared and tensor memory only
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -366,7 +368,8 @@ lamp_status_t launch_wg(const CUtensorMap &mx, const CUtensorMap &mdy, const WgP
         LAMP_CUDA_OK(cudaFuncSetAttribute(wgrad_umma_kernel<NC, BOXA, BOXB>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
         attr = true;
     }
-    wgrad_umma_kernel<NC, BOXA, BOXB><<<pl.grid, WG_THREADS, L::TOTAL, st>>>(mx, mdy, pl.P);
+    const lamp_status_t ls = launch_pdl(wgrad_umma_kernel<NC, BOXA, BOXB>, dim3(pl.grid), dim3(WG_THREADS), L::TOTAL, st, mx, mdy, pl.P);
+    if (ls != LAMP_OK) return ls;
     return launch_status();
 }
 

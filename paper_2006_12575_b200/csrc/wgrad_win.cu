@@ -93,6 +93,7 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_ST; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         mbar_init(done_bar, 1);
@@ -101,6 +102,7 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         mbar_init_fence();
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+    pdl_wait();                 // everything above touched shared and tensor memory only
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -330,7 +332,8 @@ lamp_status_t launch_ww(const CUtensorMap &mx, const CUtensorMap &mdy, const WwP
         LAMP_CUDA_OK(cudaFuncSetAttribute(wgrad_win_kernel<CBA, CBB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr = true;
     }
-    wgrad_win_kernel<CBA, CBB><<<pl.grid, WW_THREADS, pl.smem, st>>>(mx, mdy, pl.P);
+    const lamp_status_t ls = launch_pdl(wgrad_win_kernel<CBA, CBB>, dim3(pl.grid), dim3(WW_THREADS), pl.smem, st, mx, mdy, pl.P);
+    if (ls != LAMP_OK) return ls;
     return launch_status();
 }
 
