@@ -227,7 +227,13 @@ lamp_status_t lamp_unet_forward(const lamp_unet_t *net, const void *weights_bf16
  *   L = mean_n [ 1 - (1/K) sum_k (2 I_k + e)/(P_k + G_k + e) ],  I = sum p g, P = sum p, G = sum g, e = 1e-5.
  * labels: uint8 [n*d*h*w], values < num_classes.  loss: fp32 device scalar.
  * grad_w: fp32, laid out like the weight buffer; grad_b: fp32, like the bias buffer.
- * probs: fp32 [n*d*h*w][num_classes] or NULL (then taken from the workspace). */
+ * probs: fp32 [n*d*h*w][num_classes] or NULL (then taken from the workspace).
+ * Streams: the weight gradients (and the per-step transposes of the weights the data gradients read) run on a
+ * second stream owned by the handle, ordered against cuda_stream with events; that stream starts after all
+ * work enqueued on cuda_stream before the call and is joined into cuda_stream before the call returns, so the
+ * caller sees ordinary stream semantics.  The stream and its events are created by the first training step of a
+ * handle on a device (no device memory is involved); that first call must therefore come before any stream
+ * capture.  One handle must not run training steps from several host threads at once. */
 lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
                                    const lamp_tensor_t *x, const uint8_t *labels, float *loss,
                                    float *grad_w, float *grad_b, float *probs,

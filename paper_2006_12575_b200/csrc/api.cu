@@ -146,24 +146,46 @@ lamp_status_t conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const f
     return simt_conv_fwd(g, x, w, bias, y, stats, st);
 }
 
+// Every tensor-core data gradient reads the weights as [tap][c_in][c_out]: conv_dgrad_prepare writes that form into
+// wt (conv_ws_min_bytes(g, LAMP_PASS_DGRAD) bytes; nothing to do for passes that run on the CUDA cores),
+// conv_dgrad_run takes it from there.  Callers that run many passes with the same weights prepare once.
+static bool dgrad_reads_transposed(const ConvGeom &g, const TView &dy, const TView &dx)
+{
+    const int kind = dgrad_kind(g);
+    return kind >= 0 && umma_conv_supported(kind, g, dy, dx);
+}
+
+lamp_status_t conv_dgrad_prepare(const ConvGeom &g, const TView &dy, const TView &dx, const bf16 *w, void *wt,
+                                 size_t wt_bytes, cudaStream_t st)
+{
+    if (!dgrad_reads_transposed(g, dy, dx)) return LAMP_OK;
+    if (!wt || wt_bytes < umma_dgrad_ws(g) || !aligned16(wt)) return LAMP_ERR_WORKSPACE;
+    return umma_transpose_weights(w, (bf16 *)wt, g.k * g.k * g.k, g.co, g.ci, st);
+}
+
+lamp_status_t conv_dgrad_run(const ConvGeom &g, const TView &dy, const bf16 *w, const void *wt, const TView &dx,
+                             void *part, size_t part_bytes, cudaStream_t st)
+{
+    if (!dgrad_reads_transposed(g, dy, dx)) return simt_conv_dgrad(g, dy, w, dx, st);
+    if (!wt) return LAMP_ERR_WORKSPACE;
+    const int kind = dgrad_kind(g);
+    if (kind == UK_S1_DGRAD) {
+        ConvGeom t = g;
+        t.ci = g.co; t.co = g.ci;
+        if (ct_conv_fwd_supported(t, dy, dx)) return ct_conv_fwd(t, dy, (const bf16 *)wt, nullptr, dx, nullptr, 1, st);
+    }
+    return umma_conv(kind, g, dy, (const bf16 *)wt, nullptr, dx, nullptr, part, part_bytes, st);
+}
+
 lamp_status_t conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w, const TView &dx, void *ws, size_t ws_bytes,
                          cudaStream_t st)
 {
-    const int kind = dgrad_kind(g);
-    if (kind >= 0 && umma_conv_supported(kind, g, dy, dx)) {
-        // every tensor-core data gradient reads the weights as [tap][c_in][c_out]
-        const size_t need = umma_dgrad_ws(g);
-        if (!ws || ws_bytes < need || !aligned16(ws)) return LAMP_ERR_WORKSPACE;
-        lamp_status_t s = umma_transpose_weights(w, (bf16 *)ws, g.k * g.k * g.k, g.co, g.ci, st);
-        if (s != LAMP_OK) return s;
-        if (kind == UK_S1_DGRAD) {
-            ConvGeom t = g;
-            t.ci = g.co; t.co = g.ci;
-            if (ct_conv_fwd_supported(t, dy, dx)) return ct_conv_fwd(t, dy, (const bf16 *)ws, nullptr, dx, nullptr, 1, st);
-        }
-        return umma_conv(kind, g, dy, (const bf16 *)ws, nullptr, dx, nullptr, (char *)ws + need, ws_bytes - need, st);
-    }
-    return simt_conv_dgrad(g, dy, w, dx, st);
+    if (!dgrad_reads_transposed(g, dy, dx)) return simt_conv_dgrad(g, dy, w, dx, st);
+    const size_t need = umma_dgrad_ws(g);
+    if (!ws || ws_bytes < need || !aligned16(ws)) return LAMP_ERR_WORKSPACE;
+    const lamp_status_t s = conv_dgrad_prepare(g, dy, dx, w, ws, ws_bytes, st);
+    if (s != LAMP_OK) return s;
+    return conv_dgrad_run(g, dy, w, ws, dx, (char *)ws + need, ws_bytes - need, st);
 }
 
 // The one-channel first layer borrows the windowed tensor-core kernel: x is widened to 32 channels (zeros)

@@ -204,6 +204,12 @@ lamp_status_t conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const f
                        double *stats, void *ws, size_t ws_bytes, cudaStream_t st);
 lamp_status_t conv_dgrad(const ConvGeom &g, const TView &dy, const bf16 *w, const TView &dx, void *ws, size_t ws_bytes,
                          cudaStream_t st);
+// the data gradient in two steps: the transposed weights written once (wt: conv_ws_min_bytes(g, LAMP_PASS_DGRAD)
+// bytes), then any number of passes that read them (part: optional split-K scratch, see umma_conv)
+lamp_status_t conv_dgrad_prepare(const ConvGeom &g, const TView &dy, const TView &dx, const bf16 *w, void *wt,
+                                 size_t wt_bytes, cudaStream_t st);
+lamp_status_t conv_dgrad_run(const ConvGeom &g, const TView &dy, const bf16 *w, const void *wt, const TView &dx,
+                             void *part, size_t part_bytes, cudaStream_t st);
 lamp_status_t conv_wgrad(const ConvGeom &g, const TView &x, const TView &dy, float *dw, float *db, void *ws,
                          size_t ws_bytes, cudaStream_t st);
 

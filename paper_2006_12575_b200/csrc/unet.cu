@@ -26,6 +26,12 @@ struct lamp_unet {
     lamp_unet_spec_t spec;
     std::vector<Layer> layers;
     size_t n_w, n_b;
+    // Host-side resources of the training step: a second stream on which the weight gradients (and the per-step
+    // weight transposes) run beside the data-gradient chain, and the events that order the two.  Created on the
+    // first training step on a device, destroyed with the handle.
+    mutable int side_dev = -1;
+    mutable cudaStream_t side = nullptr;
+    mutable cudaEvent_t ev_fork = nullptr, ev_wt = nullptr, ev_dy = nullptr, ev_join = nullptr;
 };
 
 namespace {
@@ -66,8 +72,12 @@ struct Plan {
     size_t bwd_pool_bytes;
     void *stats_pool;                   // fp64 [n][c_out][2] of every normalised layer, back to back
     size_t stats_pool_bytes;
-    void *scratch;                      // conv workspace (wgrad partials / transposed weights)
+    void *scratch;                      // conv workspace of the main chain (split-K partials, head backward)
     size_t scratch_bytes;
+    void *scratch_side;                 // conv workspace of the weight-gradient passes (train mode)
+    size_t scratch_side_bytes;
+    std::vector<void *> wt;             // per layer: the weights as the data gradient reads them (train mode), or NULL
+    std::vector<size_t> wt_bytes;
     size_t total;
 };
 
@@ -122,7 +132,7 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
     P->stats_pool_bytes = stats_total;
     size_t stats_off = 0;
     TView cur = view((void *)x_ptr, n, d, h, w, S.in_channels, x_pitch, 0);
-    size_t scratch = 0;
+    size_t scratch = 0, scratch_side = 0;
     for (size_t i = 0; i < net->layers.size(); ++i) {
         const Layer &Ly = net->layers[i];
         LayerBuf &B = P->lb[i];
@@ -148,8 +158,10 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
             scratch = scratch > s3 ? scratch : s3;
         }
         if (mode == LAMP_MODE_TRAIN && Ly.kind != K_HEAD) {
-            size_t s1 = conv_ws_bytes(B.g, LAMP_PASS_WGRAD), s2 = conv_ws_bytes(B.g, LAMP_PASS_DGRAD);
-            scratch = scratch > s1 ? scratch : s1;
+            // the data gradient's transposed weights have their own per-layer buffers (below)
+            const size_t s1 = conv_ws_bytes(B.g, LAMP_PASS_WGRAD);
+            const size_t s2 = conv_ws_bytes(B.g, LAMP_PASS_DGRAD) - conv_ws_min_bytes(B.g, LAMP_PASS_DGRAD);
+            scratch_side = scratch_side > s1 ? scratch_side : s1;
             scratch = scratch > s2 ? scratch : s2;
         }
         if (Ly.kind == K_CONV || Ly.kind == K_DOWN) {
@@ -179,6 +191,9 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
     P->probs = need_probs ? (float *)A.take(V0 * S.num_classes * sizeof(float)) : nullptr;
     P->dice = nullptr; P->bwd_pool = nullptr; P->bwd_pool_bytes = 0;
     P->scratch = nullptr; P->scratch_bytes = 0;
+    P->scratch_side = nullptr; P->scratch_side_bytes = 0;
+    P->wt.assign(net->layers.size(), nullptr);
+    P->wt_bytes.assign(net->layers.size(), 0);
     for (LayerBuf &B : P->lb) {
         B.dy = TView{}; B.din = TView{}; B.dout = TView{}; B.dout2 = TView{};
         B.bsums = nullptr; B.db_acc = nullptr; B.db_count = nullptr;
@@ -243,6 +258,19 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
         P->scratch = A.take(scratch);
         P->scratch_bytes = scratch;
     }
+    if (mode == LAMP_MODE_TRAIN) {
+        if (scratch_side) {
+            P->scratch_side = A.take(scratch_side);
+            P->scratch_side_bytes = scratch_side;
+        }
+        for (size_t i = 1; i < net->layers.size(); ++i) {
+            if (net->layers[i].kind == K_HEAD) continue;
+            const size_t b = conv_ws_min_bytes(P->lb[i].g, LAMP_PASS_DGRAD);
+            if (!b) continue;
+            P->wt[i] = A.take(b);
+            P->wt_bytes[i] = b;
+        }
+    }
     P->total = align_up(A.off, 256);
 }
 
@@ -286,6 +314,40 @@ lamp_status_t run_forward(const lamp_unet *net, const Plan &P, const bf16 *W, co
         }
     }
     return LAMP_OK;
+}
+
+void release_side(const lamp_unet *net)
+{
+    if (net->ev_fork) cudaEventDestroy(net->ev_fork);
+    if (net->ev_wt) cudaEventDestroy(net->ev_wt);
+    if (net->ev_dy) cudaEventDestroy(net->ev_dy);
+    if (net->ev_join) cudaEventDestroy(net->ev_join);
+    if (net->side) cudaStreamDestroy(net->side);
+    net->ev_fork = net->ev_wt = net->ev_dy = net->ev_join = nullptr;
+    net->side = nullptr;
+    net->side_dev = -1;
+}
+
+// The side stream and its events on the current device; false if they cannot be had (the step then runs on one
+// stream).  Creation is not allowed while the caller's stream is being captured, hence "first call before capture".
+bool ensure_side(const lamp_unet *net)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (net->side && net->side_dev == dev) return true;
+    release_side(net);
+    bool ok = cudaStreamCreateWithFlags(&net->side, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&net->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&net->ev_wt, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&net->ev_dy, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&net->ev_join, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+        (void)cudaGetLastError();
+        release_side(net);
+        return false;
+    }
+    net->side_dev = dev;
+    return true;
 }
 
 }  // namespace
@@ -335,7 +397,12 @@ lamp_status_t lamp_unet_create(const lamp_unet_spec_t *spec, lamp_unet_t **out)
     return LAMP_OK;
 }
 
-void lamp_unet_destroy(lamp_unet_t *net) { delete net; }
+void lamp_unet_destroy(lamp_unet_t *net)
+{
+    if (!net) return;
+    release_side(net);
+    delete net;
+}
 int32_t lamp_unet_num_layers(const lamp_unet_t *net) { return net ? (int32_t)net->layers.size() : 0; }
 size_t lamp_unet_weight_count(const lamp_unet_t *net) { return net ? net->n_w : 0; }
 size_t lamp_unet_bias_count(const lamp_unet_t *net) { return net ? net->n_b : 0; }
@@ -431,29 +498,63 @@ lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_b
     if (P.total > ws_bytes) return LAMP_ERR_WORKSPACE;
     const bf16 *W = (const bf16 *)weights_bf16;
     if (!probs) probs = P.probs;
-    TRY(run_forward(net, P, W, biases_f32, probs, nullptr, labels, P.dice, st));
-    TRY(k_dice_loss(P.dice, x->n, S.num_classes, loss, st));
-
-    // backward, last layer first; one memset clears every layer's reduction scratch
-    LAMP_CUDA_OK(cudaMemsetAsync(P.bwd_pool, 0, P.bwd_pool_bytes, st));
-    for (int i = (int)net->layers.size() - 1; i >= 0; --i) {
-        const Layer &Ly = net->layers[i];
-        const LayerBuf &B = P.lb[i];
-        const bf16 *w = W + Ly.w_off;
-        float *dw = grad_w + Ly.w_off, *db = grad_b + Ly.b_off;
-        if (Ly.kind == K_HEAD) {
-            TRY(k_head_bwd(B.in, w, S.num_classes, probs, labels, P.dice, B.din, dw, db, nullptr, P.scratch, P.scratch_bytes, st));
-            continue;
-        }
-        if (Ly.kind != K_UP)
-            TRY(k_instnorm_relu_bwd(B.dout, Ly.to_cat ? &B.dout2 : nullptr, B.y, B.mr, B.bsums, true, B.dy, B.db_acc,
-                                    B.db_count, db, st));
-        // the bias gradient of a normalised layer came out of the InstanceNorm backward kernel above
-        TRY(conv_wgrad(B.g, B.in, B.dy, dw, Ly.kind == K_UP ? db : nullptr, P.scratch, P.scratch_bytes, st));
-        if (i == 0) break;
-        TRY(conv_dgrad(B.g, B.dy, w, B.din, P.scratch, P.scratch_bytes, st));
+    // Two streams.  The caller's stream carries the chain forward pass -> loss -> InstanceNorm backward / data
+    // gradient, layer by layer.  The side stream carries what nothing in that chain waits for: first the per-step
+    // transposes of the weights the data gradients read (beside the forward pass), then every weight gradient as soon
+    // as its dy exists - tensor-core work that runs beside the HBM-bound InstanceNorm backward of the next layer and
+    // fills the SMs the small deep-level kernels leave idle.  The side stream starts after everything the caller
+    // enqueued before this call and is joined before the call returns.
+    const bool two = ensure_side(net);
+    const cudaStream_t sd = two ? net->side : st;
+    if (two) {
+        LAMP_CUDA_OK(cudaEventRecord(net->ev_fork, st));
+        LAMP_CUDA_OK(cudaStreamWaitEvent(sd, net->ev_fork, 0));
     }
-    return LAMP_OK;
+    lamp_status_t rs = LAMP_OK;
+    auto body = [&]() -> lamp_status_t {
+        for (size_t i = 1; i < net->layers.size(); ++i) {
+            if (net->layers[i].kind == K_HEAD) continue;
+            const LayerBuf &B = P.lb[i];
+            TRY(conv_dgrad_prepare(B.g, B.dy, B.din, W + net->layers[i].w_off, P.wt[i], P.wt_bytes[i], sd));
+        }
+        if (two) LAMP_CUDA_OK(cudaEventRecord(net->ev_wt, sd));
+        TRY(run_forward(net, P, W, biases_f32, probs, nullptr, labels, P.dice, st));
+        TRY(k_dice_loss(P.dice, x->n, S.num_classes, loss, st));
+
+        // backward, last layer first; one memset clears every layer's reduction scratch
+        LAMP_CUDA_OK(cudaMemsetAsync(P.bwd_pool, 0, P.bwd_pool_bytes, st));
+        if (two) LAMP_CUDA_OK(cudaStreamWaitEvent(st, net->ev_wt, 0));
+        for (int i = (int)net->layers.size() - 1; i >= 0; --i) {
+            const Layer &Ly = net->layers[i];
+            const LayerBuf &B = P.lb[i];
+            const bf16 *w = W + Ly.w_off;
+            float *dw = grad_w + Ly.w_off, *db = grad_b + Ly.b_off;
+            if (Ly.kind == K_HEAD) {
+                TRY(k_head_bwd(B.in, w, S.num_classes, probs, labels, P.dice, B.din, dw, db, nullptr, P.scratch, P.scratch_bytes, st));
+                continue;
+            }
+            if (Ly.kind != K_UP)
+                TRY(k_instnorm_relu_bwd(B.dout, Ly.to_cat ? &B.dout2 : nullptr, B.y, B.mr, B.bsums, true, B.dy, B.db_acc,
+                                        B.db_count, db, st));
+            // dy is complete on the caller's stream: the weight gradient starts from here on the side stream (the
+            // bias gradient of a normalised layer came out of the InstanceNorm backward kernel above)
+            if (two) {
+                LAMP_CUDA_OK(cudaEventRecord(net->ev_dy, st));
+                LAMP_CUDA_OK(cudaStreamWaitEvent(sd, net->ev_dy, 0));
+            }
+            TRY(conv_wgrad(B.g, B.in, B.dy, dw, Ly.kind == K_UP ? db : nullptr, P.scratch_side, P.scratch_side_bytes, sd));
+            if (i == 0) break;
+            TRY(conv_dgrad_run(B.g, B.dy, w, P.wt[i], B.din, P.scratch, P.scratch_bytes, st));
+        }
+        return LAMP_OK;
+    };
+    rs = body();
+    if (two) {
+        // joined on every path, so that a stream capture of the caller never ends with the side stream still forked
+        const bool j = cudaEventRecord(net->ev_join, sd) == cudaSuccess && cudaStreamWaitEvent(st, net->ev_join, 0) == cudaSuccess;
+        if (!j && rs == LAMP_OK) rs = LAMP_ERR_CUDA;
+    }
+    return rs;
 }
 
 static void window_grid(int len, int patch, float overlap, int32_t *nst, int32_t *stride)
