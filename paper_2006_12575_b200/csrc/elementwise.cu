@@ -71,7 +71,10 @@ instnorm_relu_fwd_kernel(const bf16 *__restrict__ y, int64_t yp, const double *_
 
 // ------------------------------------------------------------------ InstanceNorm backward
 // pass 1: per (n, c)  sum g  and  sum g * xhat,  g = (dza + dzb) * [xhat > 0]
-__global__ void __launch_bounds__(256)
+// HAS_B: a second gradient source exists.  PF voxels per thread are in flight while PF others are summed; without the
+// second source twice as many fit in the same registers (the kernel is bound by the bytes it keeps in flight).
+template <bool HAS_B, int PF>
+__global__ void __launch_bounds__(256, 2)
 instnorm_bwd_sums_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *__restrict__ dzb, int64_t bp,
                          const bf16 *__restrict__ y, int64_t yp, const float *__restrict__ mr,
                          double *__restrict__ sums, int64_t Vn, int C, int64_t v_per_block)
@@ -99,7 +102,6 @@ instnorm_bwd_sums_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *_
         const int64_t v1 = min(Vn, v0 + v_per_block);
         // groups of PF voxels, the next group's loads in flight while the current one is summed; voxels past the end
         // arrive as zero gradients and add nothing
-        constexpr int PF = 2;
         const uint4 zero4 = make_uint4(0, 0, 0, 0);
         uint4 py[PF], pa[PF], pb[PF];
         auto fetch = [&](int64_t vv, uint4 &qy, uint4 &qa, uint4 &qb) {
@@ -107,7 +109,7 @@ instnorm_bwd_sums_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *_
             const int64_t v = (int64_t)n * Vn + vv;
             qy = in ? __ldg(reinterpret_cast<const uint4 *>(y + v * yp + g * 8)) : zero4;
             qa = in ? __ldg(reinterpret_cast<const uint4 *>(dza + v * ap + g * 8)) : zero4;
-            qb = (in && dzb) ? __ldg(reinterpret_cast<const uint4 *>(dzb + v * bp + g * 8)) : zero4;
+            qb = (HAS_B && in) ? __ldg(reinterpret_cast<const uint4 *>(dzb + v * bp + g * 8)) : zero4;
         };
 #pragma unroll
         for (int k = 0; k < PF; ++k) fetch(v0 + r + (int64_t)k * RB, py[k], pa[k], pb[k]);
@@ -126,7 +128,7 @@ instnorm_bwd_sums_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *_
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const float xh = (fy[j] - mu[j]) * rs[j];
-                    const float gg = xh > 0.f ? fa[j] + fb[j] : 0.f;
+                    const float gg = xh > 0.f ? (HAS_B ? fa[j] + fb[j] : fa[j]) : 0.f;
                     s[j] += gg;
                     s[8 + j] = fmaf(gg, xh, s[8 + j]);
                 }
@@ -150,8 +152,8 @@ instnorm_bwd_sums_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *_
 // With DB the kernel also forms the bias gradient of the conv in front, db[c] = sum over all voxels and samples of
 // the dy values as stored (bf16): block sums go to db_acc (fp64 atomics, zero on entry) and the block that
 // finishes last (ticket counter db_count, zero on entry) converts the totals to fp32.
-template <bool DB>
-__global__ void __launch_bounds__(256)
+template <bool DB, bool HAS_B, int PF>
+__global__ void __launch_bounds__(256, 2)
 instnorm_bwd_apply_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *__restrict__ dzb, int64_t bp,
                           const bf16 *__restrict__ y, int64_t yp, const float *__restrict__ mr,
                           const double *__restrict__ sums, bf16 *__restrict__ dy, int64_t dp, int64_t Vn, int C,
@@ -179,7 +181,6 @@ instnorm_bwd_apply_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *
     }
     const int64_t v0 = (int64_t)blockIdx.x * v_per_block, v1 = active ? min(Vn, v0 + v_per_block) : v0;
     // groups of PF voxels, the next group's loads in flight while the current one is processed
-    constexpr int PF = 2;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
     uint4 py[PF], pa[PF], pb[PF];
     auto fetch = [&](int64_t vv, uint4 &qy, uint4 &qa, uint4 &qb) {
@@ -187,7 +188,7 @@ instnorm_bwd_apply_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *
         const int64_t v = (int64_t)n * Vn + vv;
         qy = in ? __ldg(reinterpret_cast<const uint4 *>(y + v * yp + g * 8)) : zero4;
         qa = in ? __ldg(reinterpret_cast<const uint4 *>(dza + v * ap + g * 8)) : zero4;
-        qb = (in && dzb) ? __ldg(reinterpret_cast<const uint4 *>(dzb + v * bp + g * 8)) : zero4;
+        qb = (HAS_B && in) ? __ldg(reinterpret_cast<const uint4 *>(dzb + v * bp + g * 8)) : zero4;
     };
 #pragma unroll
     for (int k = 0; k < PF; ++k) fetch(v0 + r + (int64_t)k * RB, py[k], pa[k], pb[k]);
@@ -209,7 +210,7 @@ instnorm_bwd_apply_kernel(const bf16 *__restrict__ dza, int64_t ap, const bf16 *
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const float xh = (fy[j] - mu[j]) * rs[j];
-                const float gg = xh > 0.f ? fa[j] + fb[j] : 0.f;
+                const float gg = xh > 0.f ? (HAS_B ? fa[j] + fb[j] : fa[j]) : 0.f;
                 fa[j] = rs[j] * (gg - m1[j] - xh * m2[j]);
             }
             const uint4 q = pack8(fa);
@@ -724,26 +725,34 @@ lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TVie
         return LAMP_OK;
     }
     const int RB = 256 / G;
+    // pass 1: at most 8 blocks per SM, and at least 16 voxels per thread: every block ends with 2 C fp64 atomics, which
+    // dominate when a small tensor is cut into many blocks
     int64_t blocks = (148 * 8 + y.n - 1) / y.n;
-    const int64_t max_blocks = (Vn + RB - 1) / RB;
+    const int64_t max_blocks = (Vn + RB * 16 - 1) / (RB * 16);
     if (blocks > max_blocks) blocks = max_blocks;
     const int64_t vpb = (Vn + blocks - 1) / blocks;
     blocks = (Vn + vpb - 1) / vpb;
     const size_t smem = (size_t)RB * G * 16 * sizeof(float);
-    (void)launch_pdl(instnorm_bwd_sums_kernel, dim3((unsigned)blocks, y.n), dim3(256), (size_t)(smem), st, 
-        (const bf16 *)dza.p, dza.pitch, dzb ? (const bf16 *)dzb->p : nullptr, dzb ? dzb->pitch : 0,
-        (const bf16 *)y.p, y.pitch, mu_rstd, sums, Vn, C, vpb);
+    const bf16 *pa = (const bf16 *)dza.p, *pb = dzb ? (const bf16 *)dzb->p : nullptr, *py = (const bf16 *)y.p;
+    const int64_t bpitch = dzb ? dzb->pitch : 0;
+    const dim3 sgrid((unsigned)blocks, y.n);
+    if (pb)
+        (void)launch_pdl(instnorm_bwd_sums_kernel<true, 2>, sgrid, dim3(256), smem, st, pa, dza.pitch, pb, bpitch, py, y.pitch,
+                         mu_rstd, sums, Vn, C, vpb);
+    else
+        (void)launch_pdl(instnorm_bwd_sums_kernel<false, 4>, sgrid, dim3(256), smem, st, pa, dza.pitch, pb, bpitch, py, y.pitch,
+                         mu_rstd, sums, Vn, C, vpb);
     int64_t vpa = (Vn / (148 * 16) + RB - 1) / RB * RB;
     if (vpa < (int64_t)RB * 8) vpa = (int64_t)RB * 8;
     dim3 grid((unsigned)((Vn + vpa - 1) / vpa), y.n);
-    if (db)
-        (void)launch_pdl(instnorm_bwd_apply_kernel<true>, grid, dim3(256), (size_t)((size_t)RB * C * sizeof(float)), st, 
-            (const bf16 *)dza.p, dza.pitch, dzb ? (const bf16 *)dzb->p : nullptr, dzb ? dzb->pitch : 0,
-            (const bf16 *)y.p, y.pitch, mu_rstd, sums, (bf16 *)dy.p, dy.pitch, Vn, C, vpa, db_acc, db_count, db);
-    else
-        (void)launch_pdl(instnorm_bwd_apply_kernel<false>, grid, dim3(256), (size_t)(0), st, 
-            (const bf16 *)dza.p, dza.pitch, dzb ? (const bf16 *)dzb->p : nullptr, dzb ? dzb->pitch : 0,
-            (const bf16 *)y.p, y.pitch, mu_rstd, sums, (bf16 *)dy.p, dy.pitch, Vn, C, vpa, nullptr, nullptr, nullptr);
+    const size_t dsmem = db ? (size_t)RB * C * sizeof(float) : 0;
+    bf16 *pd = (bf16 *)dy.p;
+#define LAMP_IN_APPLY(DBV, HB, PFV)                                                                                       \
+    (void)launch_pdl(instnorm_bwd_apply_kernel<DBV, HB, PFV>, grid, dim3(256), dsmem, st, pa, dza.pitch, pb, bpitch, py,  \
+                     y.pitch, mu_rstd, (const double *)sums, pd, dy.pitch, Vn, C, vpa, db_acc, db_count, db)
+    if (db) { if (pb) LAMP_IN_APPLY(true, true, 2); else LAMP_IN_APPLY(true, false, 4); }
+    else    { if (pb) LAMP_IN_APPLY(false, true, 2); else LAMP_IN_APPLY(false, false, 4); }
+#undef LAMP_IN_APPLY
     return launch_status();
 }
 
