@@ -485,6 +485,29 @@ def run_unet(args):
         raise SystemExit("device status not ok")
     out.update(value=round(V / (ms * 1e-3), 1), ms_per_step=round(ms, 3), tflops=round(flops / (ms * 1e-3) / 1e12, 2),
                seconds_per_volume=round(ms * 1e-3, 5))
+    # the same call captured once in a CUDA graph and replayed: what the launch-bound deep levels cost in host launches
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                fn()
+            for _ in range(max(1, args.warmup)):
+                g.replay()
+            side.synchronize()
+            t0, t1 = ev(), ev()
+            t0.record()
+            for _ in range(args.steps):
+                g.replay()
+            t1.record()
+            side.synchronize()
+        gms = t0.elapsed_time(t1) / args.steps
+        if B.lamp_get_async_status() != 0:
+            raise SystemExit("device status not ok")
+        out["graph_replay"] = dict(ms_per_step=round(gms, 3), value=round(V / (gms * 1e-3), 1))
+    except RuntimeError as e:
+        out["graph_replay"] = dict(error=str(e)[:120])
     print(json.dumps(out), flush=True)
 
 

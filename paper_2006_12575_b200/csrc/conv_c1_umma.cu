@@ -359,7 +359,7 @@ lamp_status_t c1_umma_fwd(const ConvGeom &g, const TView &x, const bf16 *w, cons
     if (per_part < 1) per_part = 1;
     if (per_part > tiles) per_part = tiles;
     const int grid = (int)(per_part * P.nparts);
-    const lamp_status_t ls = launch_pdl(conv_c1_umma_kernel, dim3(grid), dim3(C1_THREADS), (size_t)C1_SMEM, st, mx, P);
+    const lamp_status_t ls = launch_pdl(tiles * P.nparts <= 16 * (int64_t)grid, conv_c1_umma_kernel, dim3(grid), dim3(C1_THREADS), (size_t)C1_SMEM, st, mx, P);
     if (ls != LAMP_OK) return ls;
     return launch_status();
 }

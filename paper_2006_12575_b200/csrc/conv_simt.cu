@@ -389,9 +389,10 @@ conv_c1_wgrad_kernel(ConvGeom g, const bf16 *__restrict__ x, int64_t xp, const b
 }
 
 // out[e] = sum_s part[s][e], fixed order: 32 entries x 8 split slices per block; slice j adds splits j, j + 8, ...
-// and the eight slice sums are then added in slice order.
+// into four interleaved running sums (independent loads in flight), and the eight slice sums are then added in
+// slice order.  out may be the first split of part (a block reads all splits of its entries before it writes them).
 __global__ void __launch_bounds__(256)
-reduce_parts_kernel(const float *__restrict__ part, int64_t entries, int splits, float *__restrict__ out)
+reduce_parts_kernel(const float *part, int64_t entries, int splits, float *out)
 {
     __shared__ float red[8][32];
     pdl_launch_dependents();
@@ -399,8 +400,19 @@ reduce_parts_kernel(const float *__restrict__ part, int64_t entries, int splits,
     const int el = threadIdx.x & 31, sl = threadIdx.x >> 5;
     const int64_t e = (int64_t)blockIdx.x * 32 + el;
     float acc = 0.f;
-    if (e < entries)
-        for (int s = sl; s < splits; s += 8) acc += part[(int64_t)s * entries + e];
+    if (e < entries) {
+        float a4[4] = {0.f, 0.f, 0.f, 0.f};
+        int s = sl;
+        for (; s + 24 < splits; s += 32) {
+            float t[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) t[u] = __ldcg(part + (int64_t)(s + 8 * u) * entries + e);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) a4[u] += t[u];
+        }
+        for (int u = 0; s < splits; s += 8, ++u) a4[u] += __ldcg(part + (int64_t)s * entries + e);
+        acc = (a4[0] + a4[1]) + (a4[2] + a4[3]);
+    }
     red[sl][el] = acc;
     __syncthreads();
     if (sl == 0 && e < entries) {
@@ -411,9 +423,10 @@ reduce_parts_kernel(const float *__restrict__ part, int64_t entries, int splits,
     }
 }
 
-// The same sum for few splits over many entries: a thread owns 4 consecutive entries and adds the splits in order.
+// The same sum for few splits over many entries: a thread owns 4 consecutive entries and adds the splits in order
+// (out may be the first split of part).
 __global__ void __launch_bounds__(256)
-reduce_parts_vec4_kernel(const float4 *__restrict__ part, int64_t entries4, int splits, float4 *__restrict__ out)
+reduce_parts_vec4_kernel(const float4 *part, int64_t entries4, int splits, float4 *out)
 {
     pdl_launch_dependents();
     pdl_wait();
@@ -554,22 +567,30 @@ lamp_status_t reduce_partials(const float *part, int64_t entries, int splits, fl
 {
     if (entries == 0) return LAMP_OK;
     if (splits <= 16 && entries >= 32768 && entries % 4 == 0 && (((uintptr_t)part | (uintptr_t)out) & 15) == 0)
-        return launch_pdl(reduce_parts_vec4_kernel, dim3((unsigned)((entries / 4 + 255) / 256)), dim3(256), 0, st,
+        return launch_pdl(true, reduce_parts_vec4_kernel, dim3((unsigned)((entries / 4 + 255) / 256)), dim3(256), 0, st,
                           (const float4 *)part, entries / 4, splits, (float4 *)out);
     else
-        return launch_pdl(reduce_parts_kernel, dim3((unsigned)((entries + 31) / 32)), dim3(256), 0, st, part, entries, splits, out);
+        return launch_pdl(true, reduce_parts_kernel, dim3((unsigned)((entries + 31) / 32)), dim3(256), 0, st, part, entries, splits, out);
 }
 
 bool transpose_sum_supported(int64_t taps, int A, int B) { return A % 32 == 0 && B % 32 == 0 && taps > 0 && taps <= 65535; }
 
 lamp_status_t transpose_sum_f32(const float *in, int64_t taps, int A, int B, int splits, float *out, cudaStream_t st)
 {
-    return launch_pdl(transpose_sum_kernel<float>, dim3(B / 32, A / 32, (unsigned)taps), dim3(256), 0, st, in, taps * A * B, splits, A, B, out);
+    if (!transpose_sum_supported(taps, A, B)) return LAMP_ERR_UNSUPPORTED;
+    if (splits > 4) {
+        // many splits: the transpose kernel would add them one after the other in few threads; the partials are added
+        // first, by the well-spread reduction, into the first split, which is then transposed on its own
+        const lamp_status_t s = reduce_partials(in, taps * A * B, splits, const_cast<float *>(in), st);
+        if (s != LAMP_OK) return s;
+        splits = 1;
+    }
+    return launch_pdl(true, transpose_sum_kernel<float>, dim3(B / 32, A / 32, (unsigned)taps), dim3(256), 0, st, in, taps * A * B, splits, A, B, out);
 }
 
 lamp_status_t transpose_bf16(const bf16 *in, int64_t taps, int A, int B, bf16 *out, cudaStream_t st)
 {
-    return launch_pdl(transpose_sum_kernel<bf16>, dim3(B / 32, A / 32, (unsigned)taps), dim3(256), 0, st, in, (int64_t)0, 1, A, B, out);
+    return launch_pdl(true, transpose_sum_kernel<bf16>, dim3(B / 32, A / 32, (unsigned)taps), dim3(256), 0, st, in, (int64_t)0, 1, A, B, out);
 }
 
 static void bias_plan(int64_t V, int *blocks, int64_t *vpb)
@@ -595,7 +616,7 @@ lamp_status_t bias_grad(const TView &dy, float *db, void *ws, cudaStream_t st)
     bias_plan(V, &b, &vpb);
     if (dy.c % 8 == 0 && dy.c <= 2048 && dy.pitch % 8 == 0 && ((uintptr_t)dy.p & 15) == 0) {
         const int G = dy.c / 8, RB = 256 / G;
-        if (launch_pdl(colsum_vec_kernel, dim3(b), dim3(256), (size_t)RB * dy.c * sizeof(float), st, (const bf16 *)dy.p, dy.pitch, dy.c, V, vpb,
+        if (launch_pdl(true, colsum_vec_kernel, dim3(b), dim3(256), (size_t)RB * dy.c * sizeof(float), st, (const bf16 *)dy.p, dy.pitch, dy.c, V, vpb,
                        (float *)ws) != LAMP_OK)
             return LAMP_ERR_CUDA;
     } else {
@@ -624,12 +645,12 @@ lamp_status_t pad_c1(const TView &x, bf16 *xpad, cudaStream_t st)
 {
     const int64_t V = (int64_t)x.n * x.d * x.h * x.w;
     if (V == 0) return LAMP_OK;
-    return launch_pdl(pad_c1_kernel, dim3((unsigned)((V * 4 + 255) / 256)), dim3(256), 0, st, (const bf16 *)x.p, x.pitch, xpad, V);
+    return launch_pdl(true, pad_c1_kernel, dim3((unsigned)((V * 4 + 255) / 256)), dim3(256), 0, st, (const bf16 *)x.p, x.pitch, xpad, V);
 }
 
 lamp_status_t take_c0(const float *dw32, float *dw, int n, cudaStream_t st)
 {
-    return launch_pdl(take_c0_kernel, dim3((n + 255) / 256), dim3(256), 0, st, dw32, dw, n);
+    return launch_pdl(true, take_c0_kernel, dim3((n + 255) / 256), dim3(256), 0, st, dw32, dw, n);
 }
 
 size_t simt_conv_wgrad_ws(const ConvGeom &g)

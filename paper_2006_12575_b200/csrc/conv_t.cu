@@ -413,7 +413,7 @@ lamp_status_t launch_ct(const CUtensorMap &mx, const CUtensorMap &mw, const CtPl
         LAMP_CUDA_OK(cudaFuncSetAttribute(conv3_t_kernel<KC, COB>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT));
         attr = true;
     }
-    return launch_pdl(conv3_t_kernel<KC, COB>, dim3(pl.grid), dim3(CT_THREADS), pl.smem, st, mx, mw, pl.P);
+    return launch_pdl(pl.P.total_items <= 4 * pl.grid, conv3_t_kernel<KC, COB>, dim3(pl.grid), dim3(CT_THREADS), pl.smem, st, mx, mw, pl.P);
 }
 
 }  // namespace

@@ -599,7 +599,7 @@ lamp_status_t launch(const CUtensorMap &mx, const CUtensorMap &mw, const UmmaPar
         for (int i = 0; i < 6; ++i) { Q.step[i] = t % radix[i]; t /= radix[i]; }
         Q.step[6] = t;
     }
-    return launch_pdl(conv3_umma_kernel<KC, BN, HEAD>, dim3(grid), dim3(L::THREADS), L::TOTAL, st, mx, mw, Q);
+    return launch_pdl(P.total_tiles <= 4 * grid, conv3_umma_kernel<KC, BN, HEAD>, dim3(grid), dim3(L::THREADS), L::TOTAL, st, mx, mw, Q);
 }
 
 template <int KC>
@@ -896,7 +896,7 @@ lamp_status_t umma_conv(int kind, const ConvGeom &g, const TView &a, const bf16 
     if (s != LAMP_OK || !split) return s;
     const int64_t vox_per_n = (int64_t)k.od * k.oh * k.ow;
     const dim3 grid((unsigned)((vox_per_n + FIN_VOX - 1) / FIN_VOX), (unsigned)((k.n_rows / 4 + FIN_CG - 1) / FIN_CG), (unsigned)g.n);
-    return launch_pdl(splitk_finish_kernel, grid, dim3(FIN_THREADS), 0, st, (const float *)part, out_vox * k.n_rows, P.ksplit,
+    return launch_pdl(true, splitk_finish_kernel, grid, dim3(FIN_THREADS), 0, st, (const float *)part, out_vox * k.n_rows, P.ksplit,
                       vox_per_n, k.n_rows, bias, y.p, y.f32, y.pitch, stats);
 }
 

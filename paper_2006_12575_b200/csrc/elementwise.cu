@@ -697,6 +697,9 @@ overlap_add_kernel(const float *__restrict__ pp, int Krt, int D, int H, int W, i
 
 }  // namespace
 
+// launches over at most this many elements count as short (see launch_pdl)
+constexpr int64_t SHORT_ELEMS = (int64_t)32 << 20;
+
 lamp_status_t k_instnorm_relu_fwd(const TView &y, const double *stats, float eps, float *mu_rstd, const TView &z,
                                   cudaStream_t st)
 {
@@ -707,7 +710,7 @@ lamp_status_t k_instnorm_relu_fwd(const TView &y, const double *stats, float eps
     int64_t vpb = (Vn / (148 * 16) + rb - 1) / rb * rb;
     if (vpb < rb * 8) vpb = rb * 8;
     dim3 grid((unsigned)((Vn + vpb - 1) / vpb), y.n);
-    (void)launch_pdl(instnorm_relu_fwd_kernel, grid, dim3(256), (size_t)(0), st, (const bf16 *)y.p, y.pitch, stats, 1.0 / (double)Vn, eps, mu_rstd,
+    (void)launch_pdl((int64_t)y.n * Vn * y.c <= SHORT_ELEMS, instnorm_relu_fwd_kernel, grid, dim3(256), (size_t)(0), st, (const bf16 *)y.p, y.pitch, stats, 1.0 / (double)Vn, eps, mu_rstd,
                                                    (bf16 *)z.p, z.pitch, Vn, y.c, vpb);
     return launch_status();
 }
@@ -736,11 +739,12 @@ lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TVie
     const bf16 *pa = (const bf16 *)dza.p, *pb = dzb ? (const bf16 *)dzb->p : nullptr, *py = (const bf16 *)y.p;
     const int64_t bpitch = dzb ? dzb->pitch : 0;
     const dim3 sgrid((unsigned)blocks, y.n);
+    const bool early = (int64_t)y.n * Vn * C <= SHORT_ELEMS;
     if (pb)
-        (void)launch_pdl(instnorm_bwd_sums_kernel<true, 2>, sgrid, dim3(256), smem, st, pa, dza.pitch, pb, bpitch, py, y.pitch,
+        (void)launch_pdl(early, instnorm_bwd_sums_kernel<true, 2>, sgrid, dim3(256), smem, st, pa, dza.pitch, pb, bpitch, py, y.pitch,
                          mu_rstd, sums, Vn, C, vpb);
     else
-        (void)launch_pdl(instnorm_bwd_sums_kernel<false, 4>, sgrid, dim3(256), smem, st, pa, dza.pitch, pb, bpitch, py, y.pitch,
+        (void)launch_pdl(early, instnorm_bwd_sums_kernel<false, 4>, sgrid, dim3(256), smem, st, pa, dza.pitch, pb, bpitch, py, y.pitch,
                          mu_rstd, sums, Vn, C, vpb);
     int64_t vpa = (Vn / (148 * 16) + RB - 1) / RB * RB;
     if (vpa < (int64_t)RB * 8) vpa = (int64_t)RB * 8;
@@ -748,7 +752,7 @@ lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TVie
     const size_t dsmem = db ? (size_t)RB * C * sizeof(float) : 0;
     bf16 *pd = (bf16 *)dy.p;
 #define LAMP_IN_APPLY(DBV, HB, PFV)                                                                                       \
-    (void)launch_pdl(instnorm_bwd_apply_kernel<DBV, HB, PFV>, grid, dim3(256), dsmem, st, pa, dza.pitch, pb, bpitch, py,  \
+    (void)launch_pdl(early, instnorm_bwd_apply_kernel<DBV, HB, PFV>, grid, dim3(256), dsmem, st, pa, dza.pitch, pb, bpitch, py,  \
                      y.pitch, mu_rstd, (const double *)sums, pd, dy.pitch, Vn, C, vpa, db_acc, db_count, db)
     if (db) { if (pb) LAMP_IN_APPLY(true, true, 2); else LAMP_IN_APPLY(true, false, 4); }
     else    { if (pb) LAMP_IN_APPLY(false, true, 2); else LAMP_IN_APPLY(false, false, 4); }
@@ -783,7 +787,7 @@ lamp_status_t k_head_softmax(const TView &z, const bf16 *w, const float *b, int 
     const size_t smem = ((size_t)KP * z.c + KP + 3 * KMAX + 256 * K) * sizeof(float);
     const dim3 grid((unsigned)blocks, z.n);
 #define LAMP_HEAD_FWD(kp)                                                                                         \
-    (void)launch_pdl(head_softmax_kernel<kp>, grid, dim3(256), (size_t)(smem), st, (const bf16 *)z.p, z.pitch, z.c, w, b, K, probs, argmax, labels, \
+    (void)launch_pdl((int64_t)z.n * Vn <= SHORT_ELEMS / 32, head_softmax_kernel<kp>, grid, dim3(256), (size_t)(smem), st, (const bf16 *)z.p, z.pitch, z.c, w, b, K, probs, argmax, labels, \
                                                      dice_sums, Vn, vpb)
     switch (KP) {
     case 4:  LAMP_HEAD_FWD(4); break;
@@ -797,7 +801,7 @@ lamp_status_t k_head_softmax(const TView &z, const bf16 *w, const float *b, int 
 
 lamp_status_t k_dice_loss(const double *dice_sums, int N, int K, float *loss, cudaStream_t st)
 {
-    (void)launch_pdl(dice_loss_kernel, dim3(1), dim3(32), (size_t)(0), st, dice_sums, N, K, loss);
+    (void)launch_pdl(true, dice_loss_kernel, dim3(1), dim3(32), (size_t)(0), st, dice_sums, N, K, loss);
     return launch_status();
 }
 
@@ -824,7 +828,7 @@ static lamp_status_t launch_head_bwd(const TView &z, const bf16 *w, int K, const
         LAMP_CUDA_OK(cudaFuncSetAttribute(head_bwd_kernel<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
         attr_set = true;
     }
-    (void)launch_pdl(head_bwd_kernel<KP>, dim3((unsigned)blocks, z.n), dim3(256), (size_t)(smem), st, 
+    (void)launch_pdl((int64_t)z.n * Vn <= SHORT_ELEMS / 32, head_bwd_kernel<KP>, dim3((unsigned)blocks, z.n), dim3(256), (size_t)(smem), st, 
         (const bf16 *)z.p, z.pitch, C, w, K, probs, labels, dice_sums, z.n, (bf16 *)dz.p, dz.pitch, partW, partB, dlogits,
         Vn, vpb);
     return launch_status();
@@ -866,7 +870,7 @@ lamp_status_t k_rmsprop(int64_t n, const float *g, float *w, float *v, bf16 *wb,
     if (n == 0) return LAMP_OK;
     const bool vec = n % 4 == 0 && (((uintptr_t)g | (uintptr_t)w | (uintptr_t)v) & 15) == 0 && ((uintptr_t)wb & 7) == 0;
     const int64_t threads = vec ? n / 4 : n;
-    (void)launch_pdl(rmsprop_kernel, dim3((unsigned)((threads + 255) / 256)), dim3(256), (size_t)(0), st, n, g, w, v, wb, lr, alpha, eps, vec ? 1 : 0);
+    (void)launch_pdl(n <= SHORT_ELEMS, rmsprop_kernel, dim3((unsigned)((threads + 255) / 256)), dim3(256), (size_t)(0), st, n, g, w, v, wb, lr, alpha, eps, vec ? 1 : 0);
     return launch_status();
 }
 
@@ -875,7 +879,7 @@ lamp_status_t k_gather_patches(const TView &vol, const TView &patches, int first
 {
     const int64_t total = (int64_t)patches.n * patches.d * patches.h * patches.w * patches.c;
     if (total == 0) return LAMP_OK;
-    (void)launch_pdl(gather_patches_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), (size_t)(0), st, 
+    (void)launch_pdl(total <= SHORT_ELEMS, gather_patches_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), (size_t)(0), st, 
         (const bf16 *)vol.p, vol.pitch, vol.d, vol.h, vol.w, vol.c, (bf16 *)patches.p, patches.pitch, patches.n,
         patches.d, patches.h, patches.w, first_patch, nst[0], nst[1], nst[2], stride[0], stride[1], stride[2]);
     return launch_status();
@@ -892,7 +896,7 @@ lamp_status_t k_overlap_add(const float *pp, int K, int D, int H, int W, const i
     const int aligned4 = vec && patch[2] % 4 == 0 && (nst[2] == 1 || stride[2] % 4 == 0) && (W - patch[2]) % 4 == 0 &&
                          ((uintptr_t)pp % 16 == 0);
 #define LAMP_OA(VECN, KTN)                                                                                              \
-    (void)launch_pdl(overlap_add_kernel<VECN, KTN>, dim3((unsigned)((total + 255) / 256)), dim3(256), (size_t)(smem), st,                                 \
+    (void)launch_pdl(total <= SHORT_ELEMS / 32, overlap_add_kernel<VECN, KTN>, dim3((unsigned)((total + 255) / 256)), dim3(256), (size_t)(smem), st,                                 \
         pp, K, D, H, W, patch[0], patch[1], patch[2], nst[0], nst[1], nst[2], stride[0], stride[1], stride[2], window, \
         aligned4, planar, argmax)
     if (vec) {

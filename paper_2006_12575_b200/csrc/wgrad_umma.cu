@@ -368,7 +368,7 @@ lamp_status_t launch_wg(const CUtensorMap &mx, const CUtensorMap &mdy, const WgP
         LAMP_CUDA_OK(cudaFuncSetAttribute(wgrad_umma_kernel<NC, BOXA, BOXB>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
         attr = true;
     }
-    const lamp_status_t ls = launch_pdl(wgrad_umma_kernel<NC, BOXA, BOXB>, dim3(pl.grid), dim3(WG_THREADS), L::TOTAL, st, mx, mdy, pl.P);
+    const lamp_status_t ls = launch_pdl((int64_t)pl.P.ntiles * pl.P.nunits <= 64 * (int64_t)pl.grid * pl.P.nsplit, wgrad_umma_kernel<NC, BOXA, BOXB>, dim3(pl.grid), dim3(WG_THREADS), L::TOTAL, st, mx, mdy, pl.P);
     if (ls != LAMP_OK) return ls;
     return launch_status();
 }

@@ -332,7 +332,7 @@ lamp_status_t launch_ww(const CUtensorMap &mx, const CUtensorMap &mdy, const WwP
         LAMP_CUDA_OK(cudaFuncSetAttribute(wgrad_win_kernel<CBA, CBB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr = true;
     }
-    const lamp_status_t ls = launch_pdl(wgrad_win_kernel<CBA, CBB>, dim3(pl.grid), dim3(WW_THREADS), pl.smem, st, mx, mdy, pl.P);
+    const lamp_status_t ls = launch_pdl((int64_t)pl.P.ntiles * pl.P.nsets <= 64 * (int64_t)pl.grid, wgrad_win_kernel<CBA, CBB>, dim3(pl.grid), dim3(WW_THREADS), pl.smem, st, mx, mdy, pl.P);
     if (ls != LAMP_OK) return ls;
     return launch_status();
 }

@@ -363,3 +363,47 @@ def test_overlap_add_vector_path_matches_oracle(K):
         assert_close(host_f64(planar), A.transpose(3, 0, 1, 2), "overlap-add vector path", rel=1e-5, mx=1e-5)
         agree, strict, near = tie_aware_agreement(am.cpu().numpy().reshape(D, H, W), A)
         assert agree == 1.0
+
+
+def test_train_step_replayed_from_a_cuda_graph_matches_the_eager_call():
+    """The training step forks onto the handle's side stream and joins again before it returns, so a stream
+    capture of the call must close and its replay must give what the eager call gives (loss, weight and bias
+    gradients; the InstanceNorm sums are fp64 atomics, so the comparison is to rounding, not bitwise)."""
+    net, spec, lay, ws, bs, wd, bd, offs = make_net(3, [32, 64, 128], 2, 4, 21)
+    D = H = W = 16
+    V = D * H * W
+    x = dev_bf16(synth.bf16_round(synth.blurred_noise((D, H, W), 1.5, 22))[None, ..., None])
+    lab = torch.from_numpy(synth.labels_quartiles((D, H, W), 23, 4)[None]).cuda().reshape(-1)
+    nw, nb = B.lamp_unet_weight_count(net), B.lamp_unet_bias_count(net)
+    wsb = torch.empty(B.lamp_unet_workspace_bytes(net, 1, D, H, W, B.MODE_TRAIN), dtype=torch.uint8, device="cuda")
+    res = []
+    for mode in ("eager", "graph"):
+        loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+        gw = torch.full((nw,), 7.0, dtype=torch.float32, device="cuda")
+        gb = torch.full((nb,), 7.0, dtype=torch.float32, device="cuda")
+        call = lambda: B.lamp_unet_train_step(net, wd, bd, x, lab, loss, gw, gb, None, wsb)
+        if mode == "eager":
+            call()                      # also the first step of the handle: creates the side stream before any capture
+        else:
+            s = torch.cuda.Stream()
+            s.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(s):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=s):
+                    call()
+                gw.fill_(7.0)
+                gb.fill_(7.0)
+                g.replay()
+                g.replay()
+            s.synchronize()
+        torch.cuda.synchronize()
+        assert B.lamp_get_async_status() == 0
+        res.append((float(loss.item()), host_f64(gw), host_f64(gb)))
+    (l0, w0, b0), (l1, w1, b1) = res
+    assert abs(l0 - l1) <= 1e-6 * abs(l0)
+    for i, l in enumerate(lay):
+        wo, bo = offs[i]
+        n = ws[i].size
+        assert_close(w1[wo:wo + n], w0[wo:wo + n], f"layer {i} dW, graph vs eager", rel=1e-5, mx=1e-4)
+    assert np.abs(b1 - b0).max() <= 1e-4 * max(np.abs(b0).max(), 1e-6) + 1e-7
+    B.lamp_unet_destroy(net)
