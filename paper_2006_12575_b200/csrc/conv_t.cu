@@ -22,6 +22,14 @@
 //    InstanceNorm sums are per-thread scalars; a 32 x 32 shared-memory transpose per warp turns
 //    TMEM rows into 64-byte (bf16) or 128-byte (fp32) channel runs per voxel for the NDHWC store.
 //
+//  * Stride 2 (ST = 2, the down-sampling conv).  Output voxel (h', w') reads input rows 2h' + kh - 1 and columns
+//    2w' + kw - 1: per input plane FOUR parity boxes are loaded, each by one TMA box with element stride 2 along
+//    w and h (9 x 33 voxels starting at (2 w0 - pw, 2 h0 - ph), pw / ph = 1 for the odd lattice).  Tap kw = 1 is a
+//    window of the even-w box, kw = 0 and kw = 2 are the windows 0 and 1 voxels into the odd-w box (the same along
+//    h), so every input voxel is fetched once per plane instead of once per tap.  Output plane o reads input
+//    planes 2o - 1 .. 2o + 1: stacked block j carries tap kd = pi - 2j of input plane 2 o0 - 1 + pi (the weight box
+//    walks kd with element stride 2).  Channels go in chunks of 32 so that two planes of four boxes fit.
+//
 // Warps: 0 = activation-plane TMA producer, 1 = MMA issuer (+ TMEM owner), 2 = weight-tile TMA
 // producer, 3..6 = epilogue.  All waits are bounded (LAMP_ERR_TIMEOUT on expiry).
 #include <cuda.h>
@@ -40,8 +48,12 @@ constexpr int TW = 8, TH = 32;          // output window: 8 (w) x 32 (h) = 256 v
 constexpr int HALO_W = TW + 2, HALO_H = TH + 2;
 constexpr int MAX_NP = 4, MAX_NW = 8;
 
+constexpr int S2_BOX_W = TW + 1, S2_BOX_H = TH + 1;      // voxels a stride-2 parity box delivers
+constexpr int S2_SUB_BYTES = ((S2_BOX_W * S2_BOX_H * 64 + 1023) / 1024) * 1024;   // one parity box of 32 channels
+
 struct CtParams {
-    int32_t N, D, H, W;
+    int32_t N, D, H, W;                 // extents of the OUTPUT tensor
+    int32_t ID;                         // depth of the input tensor (= D for stride 1)
     int32_t nwt, nht, ngr, nct;         // tiles along w, h; plane groups; c_out blocks of 128
     int32_t chunks;                     // c_in / KC
     int32_t total_items;
@@ -71,23 +83,26 @@ __device__ __forceinline__ Item decode_item(const CtParams &P, int item)
 
 // KC: channels per chunk (64: 128-byte swizzle, 32: 64-byte swizzle).  COB: output channels per plane
 // inside the 128 rows (128, 64 or 32); S = 128 / COB output planes are stacked.
-template <int KC, int COB>
+template <int KC, int COB, int ST>
 __global__ void __launch_bounds__(CT_THREADS, 1)
 conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const CtParams P)
 {
     constexpr int S = 128 / COB;
     constexpr int ROWB = KC * 2;
     constexpr uint32_t SWZ = KC == 64 ? 2u : 4u;
-    constexpr uint32_t PLANE_BOX_BYTES = HALO_W * HALO_H * ROWB;
+    static_assert(ST == 1 || KC == 32, "the stride-2 form works on 32-channel chunks");
+    constexpr uint32_t S2_BOX_BYTES = S2_BOX_W * S2_BOX_H * ROWB;          // bytes one parity box delivers
+    constexpr uint32_t PLANE_BOX_BYTES = ST == 1 ? HALO_W * HALO_H * ROWB : 4 * S2_BOX_BYTES;
+    constexpr int NPL = ST == 1 ? S + 2 : 2 * S + 1;           // input planes an item of S output planes reads
     constexpr uint32_t W_BYTES = 128 * ROWB;                  // one tap's weight tile
-    constexpr int TPS = KC == 32 ? 3 : 1;                      // taps (one kh row) per weight stage: 32-channel chunks carry
+    constexpr int TPS = (KC == 32 && ST == 1) ? 3 : 1;         // taps (one kh row) per weight stage: 32-channel chunks carry
                                                                // too little work per tap to pay a barrier round trip each
     constexpr uint32_t WST_BYTES = TPS * W_BYTES;
     constexpr uint32_t IDESC = make_idesc(256);
     // 32 -> 32 channels: all weights stay in shared memory.  Per in-plane tap the region [0 0 0 k0 k1 k2] of 32-row
     // blocks (kd = 0, 1, 2 after three zero blocks; three more zero blocks close the last region): the 128 stacked rows
     // of input plane pi are the four consecutive blocks that start at block pi (forward) or 5 - pi (mirrored taps).
-    constexpr bool WRES = (KC == 32 && COB == 32);
+    constexpr bool WRES = (KC == 32 && COB == 32 && ST == 1);
     constexpr uint32_t BLK_BYTES = 32 * ROWB;                  // one block of 32 output channels
     constexpr uint32_t WRES_TAP_BYTES = 6 * BLK_BYTES;
     constexpr uint32_t WRES_BYTES = 9 * WRES_TAP_BYTES + 3 * BLK_BYTES;
@@ -137,14 +152,22 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             bool ok = true;
             for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
                 const Item it = decode_item<S>(P, item);
-                for (int pi = 0; pi < S + 2 && ok; ++pi) {
-                    const int p = it.o0 - 1 + pi;
-                    if (p < 0 || p >= P.D) continue;
+                for (int pi = 0; pi < NPL && ok; ++pi) {
+                    const int p = ST * it.o0 - 1 + pi;
+                    if (p < 0 || p >= P.ID) continue;
                     for (int c = 0; c < P.chunks; ++c) {
                         if (!mbar_wait(pempty0 + 8 * ps, pph ^ 1, abort_flag)) { ok = false; break; }
                         mbar_expect_tx(pfull0 + 8 * ps, PLANE_BOX_BYTES);
-                        tma_load_5d(smem_u32(p_base + (size_t)ps * P.plane_bytes), &map_x, pfull0 + 8 * ps, c * KC, it.w0 - 1,
-                                    it.h0 - 1, p, it.n);
+                        const uint32_t dst = smem_u32(p_base + (size_t)ps * P.plane_bytes);
+                        if (ST == 1) {
+                            tma_load_5d(dst, &map_x, pfull0 + 8 * ps, c * KC, it.w0 - 1, it.h0 - 1, p, it.n);
+                        } else {
+                            // parity box (ph, pw): every second voxel from (2 h0 - ph, 2 w0 - pw)
+#pragma unroll
+                            for (int sb = 0; sb < 4; ++sb)
+                                tma_load_5d(dst + sb * S2_SUB_BYTES, &map_x, pfull0 + 8 * ps, c * KC, 2 * it.w0 - (sb & 1),
+                                            2 * it.h0 - (sb >> 1), p, it.n);
+                        }
                         if (++ps == P.np) { ps = 0; pph ^= 1; }
                     }
                 }
@@ -164,9 +187,9 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             }
             for (int item = blockIdx.x; item < P.total_items && ok && !WRES; item += gridDim.x) {
                 const Item it = decode_item<S>(P, item);
-                for (int pi = 0; pi < S + 2 && ok; ++pi) {
-                    const int p = it.o0 - 1 + pi;
-                    if (p < 0 || p >= P.D) continue;
+                for (int pi = 0; pi < NPL && ok; ++pi) {
+                    const int p = ST * it.o0 - 1 + pi;
+                    if (p < 0 || p >= P.ID) continue;
                     for (int c = 0; c < P.chunks && ok; ++c) {
                         for (int t9 = 0; t9 < 9; t9 += TPS) {
                             if (!mbar_wait(wempty0 + 8 * ws, wph ^ 1, abort_flag)) { ok = false; break; }
@@ -175,8 +198,9 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                             // kd = pi - (S - 1) + b (forward) or, with mirrored taps, the weight tap (2 - pi + b, 8 - t9 - (TPS - 1) + s);
                             // kd outside 0..2 is outside the tensor and arrives as zeros
                             const uint32_t dst = smem_u32(w_base + (size_t)ws * WST_BYTES);
+                            // (stride 2: the box walks kd with element stride 2, block b holds kd = pi - 2 (S - 1) + 2 b)
                             if (P.mirror) tma_load_4d(dst, &map_w, wfull0 + 8 * ws, c * KC, it.ct * 128, 2 - pi, 8 - t9 - (TPS - 1));
-                            else          tma_load_4d(dst, &map_w, wfull0 + 8 * ws, c * KC, it.ct * 128, pi - (S - 1), t9);
+                            else          tma_load_4d(dst, &map_w, wfull0 + 8 * ws, c * KC, it.ct * 128, pi - ST * (S - 1), t9);
                             if (++ws == P.nw) { ws = 0; wph ^= 1; }
                         }
                     }
@@ -196,9 +220,9 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * 256;
                 uint32_t accumulate = 0;
-                for (int pi = 0; pi < S + 2 && ok; ++pi) {
-                    const int p = it.o0 - 1 + pi;
-                    if (p < 0 || p >= P.D) continue;
+                for (int pi = 0; pi < NPL && ok; ++pi) {
+                    const int p = ST * it.o0 - 1 + pi;
+                    if (p < 0 || p >= P.ID) continue;
                     for (int c = 0; c < P.chunks && ok; ++c) {
                         if (!mbar_wait(pfull0 + 8 * ps, pph, abort_flag)) { ok = false; break; }
                         tc_fence_after();
@@ -224,7 +248,11 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                                 const int t = P.mirror ? t9 + TPS - 1 - sl : t9 + sl;        // conv tap whose weights sit in slot sl
                                 const int kh = t / 3, kw = t - kh * 3;
                                 const uint64_t da = make_desc(smem_u32(w_base + (size_t)ws * WST_BYTES + sl * W_BYTES), 0, 8 * ROWB, SWZ);
-                                const uint64_t db = make_desc(plane + (kh * HALO_W + kw) * ROWB, 0, HALO_W * ROWB, SWZ);
+                                // stride 2: tap 1 reads the even box, taps 0 and 2 the odd box 0 and 1 voxels in
+                                const uint64_t db = ST == 1
+                                    ? make_desc(plane + (kh * HALO_W + kw) * ROWB, 0, HALO_W * ROWB, SWZ)
+                                    : make_desc(plane + ((kh != 1) * 2 + (kw != 1)) * S2_SUB_BYTES + ((kh == 2) * S2_BOX_W + (kw == 2)) * ROWB,
+                                                0, S2_BOX_W * ROWB, SWZ);
 #pragma unroll
                                 for (int k = 0; k < KC / 16; ++k) {
                                     umma_bf16(d_tmem, da + 2 * k, db + 2 * k, IDESC, accumulate);
@@ -356,7 +384,7 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode()
     return fn;
 }
 
-struct CtPlan { CtParams P; int KC, COB; size_t smem; int grid; };
+struct CtPlan { CtParams P; int KC, COB, ST; size_t smem; int grid; };
 
 constexpr int EPI_BYTES = 4 * 32 * 33 * 4;
 constexpr int CTRL_BYTES = 1024;
@@ -364,32 +392,34 @@ constexpr int SMEM_LIMIT = 227 * 1024;
 
 bool make_ct_plan(const ConvGeom &g, CtPlan *out)
 {
-    if (!(g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed)) return false;
+    if (!(g.k == 3 && (g.s == 1 || g.s == 2) && g.p == 1 && !g.transposed)) return false;
     if (g.ci % 32) return false;
+    const int ST = g.s;
     int COB;
     if (g.co == 32 || g.co == 64) COB = g.co;
     else if (g.co % 128 == 0) COB = 128;
     else return false;
-    const int KC = g.ci % 64 == 0 ? 64 : 32;
+    const int KC = (g.ci % 64 == 0 && ST == 1) ? 64 : 32;
     const int S = 128 / COB;
     CtParams &P = out->P;
-    P.N = g.n; P.D = g.d; P.H = g.h; P.W = g.w;
+    P.N = g.n; P.D = g.od; P.H = g.oh; P.W = g.ow;            // the tiles cover the output tensor
+    P.ID = g.d;
     P.chunks = g.ci / KC;
     const int rowb = KC * 2;
-    P.plane_bytes = (int)align_up((size_t)HALO_W * HALO_H * rowb, 1024);
-    const int w_bytes = 128 * rowb * (KC == 32 ? 3 : 1);      // bytes of one weight stage
+    P.plane_bytes = ST == 1 ? (int)align_up((size_t)HALO_W * HALO_H * rowb, 1024) : 4 * S2_SUB_BYTES;
+    const int w_bytes = 128 * rowb * ((KC == 32 && ST == 1) ? 3 : 1);      // bytes of one weight stage
     const int budget = SMEM_LIMIT - 1024 - EPI_BYTES - CTRL_BYTES;
-    int np = KC == 64 ? 2 : 4;
+    int np = (KC == 64 || ST == 2) ? 2 : 4;
     int nw = (budget - np * P.plane_bytes) / w_bytes;
     if (nw > MAX_NW) nw = MAX_NW;
     if (nw < 3) return false;
     // 32 -> 32 channels: the weights are resident (nine regions of six 2 KB blocks plus three closing zero blocks)
-    const bool wres = KC == 32 && COB == 32;
+    const bool wres = KC == 32 && COB == 32 && ST == 1;
     const size_t wres_bytes = (size_t)(9 * 6 + 3) * 32 * rowb;
     P.np = np; P.nw = nw;
-    P.nwt = (g.w + TW - 1) / TW;
-    P.nht = (g.h + TH - 1) / TH;
-    P.ngr = (g.d + S - 1) / S;
+    P.nwt = (g.ow + TW - 1) / TW;
+    P.nht = (g.oh + TH - 1) / TH;
+    P.ngr = (g.od + S - 1) / S;
     P.nct = g.co / (COB == 128 ? 128 : COB);
     const int64_t items = (int64_t)g.n * P.ngr * P.nht * P.nwt * P.nct;
     if (items > 0x7FFFFFFF || items <= 0) return false;
@@ -398,22 +428,22 @@ bool make_ct_plan(const ConvGeom &g, CtPlan *out)
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    out->KC = KC; out->COB = COB;
+    out->KC = KC; out->COB = COB; out->ST = ST;
     out->smem = 1024 + (size_t)np * P.plane_bytes + (wres ? wres_bytes : (size_t)nw * w_bytes) + EPI_BYTES + CTRL_BYTES;
     if (out->smem > (size_t)SMEM_LIMIT) return false;
     out->grid = (int)(items < sms ? items : sms);
     return true;
 }
 
-template <int KC, int COB>
+template <int KC, int COB, int ST = 1>
 lamp_status_t launch_ct(const CUtensorMap &mx, const CUtensorMap &mw, const CtPlan &pl, cudaStream_t st)
 {
     static bool attr = false;
     if (!attr) {
-        LAMP_CUDA_OK(cudaFuncSetAttribute(conv3_t_kernel<KC, COB>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT));
+        LAMP_CUDA_OK(cudaFuncSetAttribute(conv3_t_kernel<KC, COB, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT));
         attr = true;
     }
-    return launch_pdl(pl.P.total_items <= 4 * pl.grid, conv3_t_kernel<KC, COB>, dim3(pl.grid), dim3(CT_THREADS), pl.smem, st, mx, mw, pl.P);
+    return launch_pdl(pl.P.total_items <= 4 * pl.grid, conv3_t_kernel<KC, COB, ST>, dim3(pl.grid), dim3(CT_THREADS), pl.smem, st, mx, mw, pl.P);
 }
 
 }  // namespace
@@ -424,7 +454,7 @@ bool ct_conv_fwd_supported(const ConvGeom &g, const TView &x, const TView &y)
     if ((int64_t)g.n * g.d * g.h * g.w == 0) return false;
     if (!make_ct_plan(g, &pl)) return false;
     // the 8 x 32 window must not be mostly padding
-    const double used = (double)g.h * g.w / ((double)pl.P.nht * TH * pl.P.nwt * TW);
+    const double used = (double)g.oh * g.ow / ((double)pl.P.nht * TH * pl.P.nwt * TW);
     if (used < 0.55) return false;
     if (x.pitch % 8 || ((uintptr_t)x.p & 15)) return false;
     if (y.f32 ? (y.pitch % 4 != 0) : (y.pitch % 8 != 0)) return false;
@@ -448,8 +478,10 @@ lamp_status_t ct_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, cons
         const cuuint64_t dims[5] = {(cuuint64_t)g.ci, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.d, (cuuint64_t)g.n};
         const cuuint64_t strides[4] = {(cuuint64_t)x.pitch * 2, (cuuint64_t)x.pitch * 2 * g.w,
                                        (cuuint64_t)x.pitch * 2 * g.w * g.h, (cuuint64_t)x.pitch * 2 * g.w * g.h * g.d};
-        const cuuint32_t box[5] = {(cuuint32_t)pl.KC, (cuuint32_t)HALO_W, (cuuint32_t)HALO_H, 1, 1};
-        const cuuint32_t es[5] = {1, 1, 1, 1, 1};
+        // stride 2: a parity box takes every second voxel along w and h (the box spans twice what it delivers)
+        const cuuint32_t s2 = pl.ST == 2;
+        const cuuint32_t box[5] = {(cuuint32_t)pl.KC, s2 ? 2u * S2_BOX_W : (cuuint32_t)HALO_W, s2 ? 2u * S2_BOX_H : (cuuint32_t)HALO_H, 1, 1};
+        const cuuint32_t es[5] = {1, s2 ? 2u : 1u, s2 ? 2u : 1u, 1, 1};
         if (encode(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, x.p, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return LAMP_ERR_CUDA;
@@ -458,13 +490,24 @@ lamp_status_t ct_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, cons
         // weights viewed as (c_in, c_out, kd, kh*3+kw): a box spans the stacked kd blocks, then the taps of a stage
         const cuuint64_t dims[4] = {(cuuint64_t)g.ci, (cuuint64_t)g.co, 3, 9};
         const cuuint64_t strides[3] = {(cuuint64_t)g.ci * 2, (cuuint64_t)g.ci * 2 * g.co * 9, (cuuint64_t)g.ci * 2 * g.co};
-        const bool wres = pl.KC == 32 && pl.COB == 32;      // resident weights: one box = the three kd blocks of a tap
-        const cuuint32_t box[4] = {(cuuint32_t)pl.KC, (cuuint32_t)pl.COB, (cuuint32_t)(wres ? 3 : 128 / pl.COB),
-                                   (cuuint32_t)(wres ? 1 : (pl.KC == 32 ? 3 : 1))};
-        const cuuint32_t es[4] = {1, 1, 1, 1};
+        const bool wres = pl.KC == 32 && pl.COB == 32 && pl.ST == 1;      // resident weights: one box = the three kd blocks of a tap
+        // stride 2: the stacked blocks are two kd apart (block b of input plane pi carries kd = pi - 2 (S - 1) + 2 b)
+        const cuuint32_t nblk = 128 / pl.COB;
+        const cuuint32_t box[4] = {(cuuint32_t)pl.KC, (cuuint32_t)pl.COB, (cuuint32_t)(wres ? 3 : nblk * (pl.ST == 2 ? 2 : 1)),
+                                   (cuuint32_t)(wres ? 1 : ((pl.KC == 32 && pl.ST == 1) ? 3 : 1))};
+        const cuuint32_t es[4] = {1, 1, (cuuint32_t)(pl.ST == 2 ? 2 : 1), 1};
         if (encode(&mw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void *)w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return LAMP_ERR_CUDA;
+    }
+    if (pl.ST == 2) {
+        if (mirror_taps) return LAMP_ERR_UNSUPPORTED;
+        switch (pl.COB) {
+        case 32:  return launch_ct<32, 32, 2>(mx, mw, pl, st);
+        case 64:  return launch_ct<32, 64, 2>(mx, mw, pl, st);
+        case 128: return launch_ct<32, 128, 2>(mx, mw, pl, st);
+        }
+        return LAMP_ERR_UNSUPPORTED;
     }
     const int key = pl.KC * 1000 + pl.COB;
     switch (key) {

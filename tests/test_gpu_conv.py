@@ -50,6 +50,10 @@ CASES = [
     ("t_c256_h32", 1, 3, 32, 8, 256, 256, 3, 1, 1, 0),
     ("t_c512_to_256", 1, 2, 32, 8, 512, 256, 3, 1, 1, 0),
     ("t_c128_to_384", 1, 2, 30, 16, 128, 384, 3, 1, 1, 0),
+    ("t_down_32_64", 1, 12, 64, 16, 32, 64, 3, 2, 1, 0),
+    ("t_down_64_128_ragged_odd", 1, 7, 60, 31, 64, 128, 3, 2, 1, 0),
+    ("t_down_32_32_batch", 2, 8, 64, 16, 32, 32, 3, 2, 1, 0),
+    ("t_down_128_256", 1, 4, 64, 16, 128, 256, 3, 2, 1, 0),
     ("deep_512_cube8", 1, 8, 8, 8, 512, 512, 3, 1, 1, 0),
     ("deep_512_to_256_ragged", 2, 3, 5, 7, 512, 256, 3, 1, 1, 0),
     ("deep_down_256_512", 1, 8, 8, 8, 256, 512, 3, 2, 1, 0),
