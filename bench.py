@@ -485,6 +485,9 @@ def run_unet(args):
         raise SystemExit("device status not ok")
     out.update(value=round(V / (ms * 1e-3), 1), ms_per_step=round(ms, 3), tflops=round(flops / (ms * 1e-3) / 1e12, 2),
                seconds_per_volume=round(ms * 1e-3, 5))
+    if args.no_graph:
+        print(json.dumps(out), flush=True)
+        return
     # the same call captured once in a CUDA graph and replayed: what the launch-bound deep levels cost in host launches
     try:
         side = torch.cuda.Stream()
@@ -509,6 +512,90 @@ def run_unet(args):
     except RuntimeError as e:
         out["graph_replay"] = dict(error=str(e)[:120])
     print(json.dumps(out), flush=True)
+
+
+def run_unet_dp(args):
+    """Data-parallel training: every rank runs the U-Net training step on its own volume, the flat fp32 gradients
+    are averaged over the ranks (bucketed all-reduce of the process group), and RMSProp updates the fp32 master copy
+    and the bf16 copy the convolutions read.  One JSON line from rank 0: voxels of all ranks over the slowest rank."""
+    import torch
+    import torch.distributed as dist
+    from paper_2006_12575_b200 import binding as B
+    from paper_2006_12575_b200 import build as lamp_build
+    from paper_2006_12575_b200 import replicas, synth
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        lamp_build.build()
+    if world > 1:
+        dist.barrier()
+    cfg = UNET_CFGS[args.cfg]
+    D, H, W = cfg["vol"]
+    V = D * H * W
+    net = B.lamp_unet_create(B.unet_spec(cfg["levels"], cfg["ch"], cfg["cpl"], 1, cfg["K"]))
+    g = torch.Generator().manual_seed(10 * args.cfg + 1)              # the same initial weights on every rank
+    master = torch.zeros(B.lamp_unet_weight_count(net), dtype=torch.float32)
+    for i in range(B.lamp_unet_num_layers(net)):
+        wo, bo, d = B.lamp_unet_param_layout(net, i)
+        taps = d.ksize ** 3
+        n = taps * d.c_in * d.c_out
+        master[wo:wo + n] = torch.randn(n, generator=g) * (2.0 / ((1 if d.transposed else taps) * d.c_in)) ** 0.5
+    master = master.to(dev)
+    wd = master.to(torch.bfloat16)
+    bmaster = torch.zeros(B.lamp_unet_bias_count(net), dtype=torch.float32, device=dev)
+    vw, vb = torch.zeros_like(master), torch.zeros_like(bmaster)
+    x = torch.from_numpy(synth.blurred_noise((D, H, W), 2.0, 10 * args.cfg + 100 * rank)).to(torch.bfloat16).reshape(1, D, H, W, 1).to(dev)
+    lab = torch.from_numpy(synth.labels_quartiles((D, H, W), 10 * args.cfg + 2 + 100 * rank, cfg["K"], 4.0)).reshape(-1).to(dev)
+    loss = torch.zeros(1, dtype=torch.float32, device=dev)
+    gw, gb = torch.empty_like(master), torch.empty_like(bmaster)
+    ws = torch.empty(B.lamp_unet_workspace_bytes(net, 1, D, H, W, B.MODE_TRAIN), dtype=torch.uint8, device=dev)
+
+    def step():
+        B.lamp_unet_train_step(net, wd, bmaster, x, lab, loss, gw, gb, None, ws)
+        replicas.allreduce_mean_(gw)
+        replicas.allreduce_mean_(gb)
+        B.lamp_rmsprop_step(gw, master, vw, wd)
+        B.lamp_rmsprop_step(gb, bmaster, vb, None)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    losses = []
+    for _ in range(args.warmup):
+        step()
+        losses.append(float(loss.item()))
+    sync_all()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        step()
+    t1.record()
+    sync_all()
+    losses.append(float(loss.item()))
+    ms = replicas.job_time_ms(t0.elapsed_time(t1), dev) / args.steps
+    status = B.lamp_get_async_status()
+    if rank == 0:
+        if status != 0:
+            raise SystemExit("device status not ok")
+        out = dict(metric="unet_data_parallel_train_voxels_per_s", value=round(world * V / (ms * 1e-3), 1), unit="voxels/s",
+                   n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=round(ms, 3), higher_is_better=True,
+                   scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
+                   config=dict(workload=f"configs[{args.cfg}] U-Net training step + gradient average over {world} replica(s) "
+                                        "+ RMSProp update", gradient_bytes=int(gw.numel() + gb.numel()) * 4,
+                               exchange="bucketed all-reduce after the backward pass (not overlapped with it)"),
+                   loss_first_last=[round(losses[0], 5), round(losses[-1], 5)] if losses else None)
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
 
 
 def run_hbm(args):
@@ -616,12 +703,16 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="lamp", choices=["lamp", "reference"])
     ap.add_argument("--channels", default=",".join(str(c) for c in CHANNELS))
-    ap.add_argument("--workload", default="conv_sweep", choices=["conv_sweep", "unet_train", "unet_infer", "sliding", "hbm"])
+    ap.add_argument("--workload", default="conv_sweep", choices=["conv_sweep", "unet_train", "unet_infer", "sliding", "hbm", "unet_train_dp"])
     ap.add_argument("--cfg", type=int, default=2)
     ap.add_argument("--sw-batch", type=int, default=32)
+    ap.add_argument("--no-graph", action="store_true", help="U-Net workloads: skip the CUDA-graph replay timing")
     args = ap.parse_args()
     if args.workload == "hbm":
         run_hbm(args)
+        return
+    if args.workload == "unet_train_dp":
+        run_unet_dp(args)
         return
     if args.workload != "conv_sweep":
         run_unet(args)
