@@ -75,11 +75,10 @@ def _ws_view(wsb, layout):
                             (t.d * t.h * t.w * t.c_pitch, t.h * t.w * t.c_pitch, t.w * t.c_pitch, t.c_pitch, 1))
 
 
-def test_standard_unet_train_step_at_full_size_sampled():
-    """128^3 volume, widths 32..512, K = 10: one training step; every kind of layer is checked on sampled
-    outputs against the oracle evaluated on the tensors the GPU stored as that layer's input."""
-    levels, ch, cpl, K = 5, [32, 64, 128, 256, 512], 2, 10
-    D = H = W = 128
+def _train_step_sampled(levels, ch, cpl, K, dhw, checked, head_planes):
+    """One training step at a benchmark size; the layers named in `checked` (every kind of layer and kernel) are
+    checked on sampled outputs against the oracle evaluated on the tensors the GPU stored as that layer's input."""
+    D, H, W = dhw
     V = D * H * W
     net = B.lamp_unet_create(B.unet_spec(levels, ch, cpl, 1, K))
     spec = O.UNetSpec(levels, ch, cpl, 1, K)
@@ -111,8 +110,7 @@ def test_standard_unet_train_step_at_full_size_sampled():
     rs = np.random.default_rng(5)
     names = {l.name: i for i, l in enumerate(lay)}
     gw_h = gw.cpu().numpy().astype(np.float64)
-    for name in ["enc0.conv0", "enc0.conv1", "down0", "enc1.conv1", "down2", "enc4.conv1", "up3", "dec1.conv0", "up0",
-                 "dec0.conv0", "dec0.conv1"]:
+    for name in checked:
         i = names[name]
         l = lay[i]
         w64 = wl[i].astype(np.float64)
@@ -145,11 +143,26 @@ def test_standard_unet_train_step_at_full_size_sampled():
             assert_close(host_f64(u_gpu[idx]), ops.bf16_round(ref), f"{name} out (sampled)")
     # head: probabilities from the stored input, all voxels of a few planes
     hi = len(lay) - 1
-    z = host_f64(_ws_view(wsb, lay_of(hi, B.T_IN))[:, 60:64])
+    d0, d1 = head_planes
+    z = host_f64(_ws_view(wsb, lay_of(hi, B.T_IN))[:, d0:d1])
     bo = offs[hi][1]
     p_ref = ops.softmax(ops.conv3d_fwd(z, wl[hi].astype(np.float64), bflat[bo:bo + K].astype(np.float64), 1, 1, 0))
-    assert_close(p_gpu[:, 60:64], p_ref, "head probs", rel=1e-5, mx=1e-5)
+    assert_close(p_gpu[:, d0:d1], p_ref, "head probs", rel=1e-5, mx=1e-5)
     B.lamp_unet_destroy(net)
+
+
+def test_standard_unet_train_step_at_full_size_sampled():
+    """128^3 volume, widths 32..512, two convs per level, K = 10."""
+    _train_step_sampled(5, [32, 64, 128, 256, 512], 2, 10, (128, 128, 128),
+                        ["enc0.conv0", "enc0.conv1", "down0", "enc1.conv1", "down2", "enc4.conv1", "up3", "dec1.conv0", "up0",
+                         "dec0.conv0", "dec0.conv1"], (60, 64))
+
+
+def test_large_unet_train_step_at_full_size_sampled():
+    """192 x 192 x 64 volume, widths 64..1024, three convs per level, K = 10 (the large-context network)."""
+    _train_step_sampled(5, [64, 128, 256, 512, 1024], 3, 10, (192, 192, 64),
+                        ["enc0.conv0", "enc0.conv2", "down0", "enc1.conv1", "down3", "enc4.conv2", "up3", "dec1.conv0", "up0",
+                         "dec0.conv0", "dec0.conv2"], (30, 32))
 
 
 def test_sliding_window_full_size_blend_sampled():
