@@ -220,3 +220,78 @@ def test_sliding_window_full_size_blend_sampled():
     assert ok.mean() >= 0.9999
     assert np.allclose(got.sum(1), 1, atol=1e-5)
     B.lamp_unet_destroy(net)
+
+
+def test_whole_volume_512x512x128_top_level_layers_on_high_address_slabs():
+    """The whole-volume workload (512 x 512 x 128, widths 32..512): its top-level tensors hold more than 2^31 elements,
+    so every index on the way has to be 64-bit.  One training step keeps every tensor; the top-level layers are then
+    checked on slabs of planes at the far end of the tensors (and at the near end), where a 32-bit offset would have
+    wrapped: a 3x3x3 conv output plane depends on three input planes only, so the oracle runs on those three planes."""
+    levels, ch, cpl, K = 5, [32, 64, 128, 256, 512], 2, 10
+    D, H, W = 512, 512, 128
+    V = D * H * W
+    net = B.lamp_unet_create(B.unet_spec(levels, ch, cpl, 1, K))
+    spec = O.UNetSpec(levels, ch, cpl, 1, K)
+    lay = O.unet_layers(spec)
+    names = {l.name: i for i, l in enumerate(lay)}
+    nw, nb = B.lamp_unet_weight_count(net), B.lamp_unet_bias_count(net)
+    wflat = np.zeros(nw, dtype=np.float32)
+    wl, offs = [], []
+    for i, l in enumerate(lay):
+        wo, bo, d = B.lamp_unet_param_layout(net, i)
+        w = synth.bf16_round(synth.rng(500 + i).standard_normal((l.taps, l.c_out, l.c_in)) * (2.0 / l.fan_in) ** 0.5)
+        wflat[wo:wo + w.size] = w.ravel()
+        wl.append(w.astype(np.float64))
+        offs.append((wo, bo))
+    bflat = (0.05 * synth.rng(51).standard_normal(nb)).astype(np.float32)
+    wd = torch.from_numpy(wflat).cuda().to(torch.bfloat16)
+    bd = torch.from_numpy(bflat).cuda()
+    xh = _randn_bf16((1, D, H, W, 1), 52)
+    xd = xh.cuda()
+    lab = torch.randint(0, K, (V,), dtype=torch.uint8, generator=torch.Generator().manual_seed(53)).cuda()
+    loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+    gw = torch.empty(nw, dtype=torch.float32, device="cuda")
+    gb = torch.empty(nb, dtype=torch.float32, device="cuda")
+    probs = torch.empty((V, K), dtype=torch.float32, device="cuda")
+    nbytes = B.lamp_unet_workspace_bytes(net, 1, D, H, W, B.MODE_TRAIN)
+    assert nbytes < 120e9
+    wsb = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    B.lamp_unet_train_step(net, wd, bd, xd, lab, loss, gw, gb, probs, wsb)
+    torch.cuda.synchronize()
+    assert B.lamp_get_async_status() == 0 and np.isfinite(float(loss.item()))
+    lay_of = lambda i, which: B.lamp_unet_tensor_layout(net, 1, D, H, W, B.MODE_TRAIN, i, which)
+    view = lambda i, which: _ws_view(wsb, lay_of(i, which))
+    bias = lambda i: bflat[offs[i][1]:offs[i][1] + lay[i].c_out].astype(np.float64)
+    for d0 in (D - 3, 1):
+        sl = slice(d0 - 1, d0 + 2)
+        for name in ("enc0.conv0", "enc0.conv1", "dec0.conv0", "dec0.conv1"):
+            i = names[name]
+            x_in = host_f64(xd[:, sl]) if i == 0 else host_f64(view(i, B.T_IN)[:, sl])
+            y_ref = ops.conv3d_fwd(x_in, wl[i], bias(i), 3, 1, 1)[:, 1]
+            y_gpu = host_f64(view(i, B.T_Y)[:, d0])
+            assert_close(y_gpu, ops.bf16_round(y_ref), f"{name} y, plane {d0}")
+            t, off = lay_of(i, B.T_MU_RSTD)
+            mr = wsb[off:off + lay[i].c_out * 8].view(torch.float32).cpu().numpy().astype(np.float64).reshape(-1, 2)
+            z_ref = ops.bf16_round(np.maximum((y_gpu - mr[:, 0]) * mr[:, 1], 0.0))
+            assert_close(host_f64(view(i, B.T_OUT)[:, d0]), z_ref, f"{name} z, plane {d0}", rel=2e-4, mx=4e-3)
+            if i > 0:
+                dy = host_f64(view(i, B.T_DY)[:, sl])
+                dx_ref = ops.conv3d_dgrad(dy, wl[i], (3, H, W), 3, 1, 1)[:, 1]
+                assert_close(host_f64(view(i, B.T_DIN)[:, d0]), ops.bf16_round(dx_ref), f"{name} din, plane {d0}")
+        # transposed conv into the concat slice: output planes 2j, 2j + 1 come from input plane j
+        i = names["up0"]
+        j = d0 // 2
+        xin = host_f64(view(i, B.T_IN)[:, j])                                  # [1, H/2, W/2, ci]
+        u_gpu = host_f64(view(i, B.T_OUT)[:, 2 * j:2 * j + 2])
+        for a in range(2):
+            for b_ in range(2):
+                for c in range(2):
+                    ref = np.einsum("nhwi,oi->nhwo", xin, wl[i][(a * 2 + b_) * 2 + c]) + bias(i)
+                    assert_close(u_gpu[:, a, b_::2, c::2], ops.bf16_round(ref), f"up0 out, plane {2 * j + a}")
+        # head
+        hi = names["head"]
+        z = host_f64(view(hi, B.T_IN)[:, d0:d0 + 1])
+        p_ref = ops.softmax(ops.conv3d_fwd(z, wl[hi], bias(hi), 1, 1, 0))
+        p_gpu = host_f64(probs.view(1, D, H, W, K)[:, d0:d0 + 1])
+        assert_close(p_gpu, p_ref, f"head probs, plane {d0}", rel=1e-5, mx=1e-5)
+    B.lamp_unet_destroy(net)
