@@ -295,3 +295,33 @@ def test_whole_volume_512x512x128_top_level_layers_on_high_address_slabs():
         p_gpu = host_f64(probs.view(1, D, H, W, K)[:, d0:d0 + 1])
         assert_close(p_gpu, p_ref, f"head probs, plane {d0}", rel=1e-5, mx=1e-5)
     B.lamp_unet_destroy(net)
+
+
+@pytest.mark.parametrize("ci,at_end", [(32, True), (32, False), (1, True)])
+def test_weight_gradient_512x512x128_from_a_slab_at_the_far_end(ci, at_end):
+    """Weight gradient over the 33.5 M-voxel volume with the operands laid out as in the network (x a 32-channel slice
+    of a 64-channel buffer, so its byte offsets pass 4 GB).  dy is zero except in two planes at one end of the volume:
+    the sum over voxels then equals the oracle's weight gradient of a four-plane slab, while the kernel still walks
+    the whole volume - a wrapped 32-bit offset at the far end would change the result."""
+    D, H, W, co = 512, 512, 128, 32
+    g = torch.Generator(device="cuda").manual_seed(60 + ci)
+    pitch = 64 if ci == 32 else 1
+    xbuf = torch.randn((1, D, H, W, pitch), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    dy = torch.zeros((1, D, H, W, co), dtype=torch.bfloat16, device="cuda")
+    lo = D - 4 if at_end else 0                                 # slab of four planes; dy lives in its two outer planes
+    dsl = slice(D - 2, D) if at_end else slice(0, 2)
+    dy[:, dsl] = torch.randn((1, 2, H, W, co), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    desc = B.conv_desc(ci, co)
+    xt = B.tensor(xbuf, ci, 0)
+    dw = torch.empty((27, co, ci), dtype=torch.float32, device="cuda")
+    db = torch.empty(co, dtype=torch.float32, device="cuda")
+    ws = torch.empty(B.lamp_conv3d_workspace_bytes(desc, xt, B.PASS_WGRAD), dtype=torch.uint8, device="cuda")
+    B.lamp_conv3d_wgrad(desc, xt, dy, dw, db, ws)
+    torch.cuda.synchronize()
+    assert B.lamp_get_async_status() == 0
+    x_slab = host_f64(xbuf[:, lo:lo + 4, :, :, :ci])
+    dy_slab = host_f64(dy[:, lo:lo + 4])
+    # the slab's inner face is not a volume border: the planes next to it carry no dy, so its zero padding adds nothing
+    dw_ref, db_ref = ops.conv3d_wgrad(x_slab, dy_slab, 3, 1, 1)
+    assert_close(host_f64(dw), dw_ref, "dw", rel=2e-5, mx=2e-5)
+    assert_close(host_f64(db), db_ref, "db", rel=1e-4, mx=1e-4)
