@@ -309,7 +309,47 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 uint32_t r[32];
                 tmem_ld32(trow + c0, r);
                 tmem_ld_wait();
-                if (plane_ok) {
+                if (plane_ok && !P.y_f32) {
+                    // bf16 output: two voxels of a channel are rounded and packed into one word BEFORE the transpose, a
+                    // lane then takes 16 channels of a voxel pair: half the shared-memory traffic of the fp32 form (the
+                    // epilogue's shared-memory work slows the tensor pipe, which reads its operands from there too)
+                    uint32_t *trw = reinterpret_cast<uint32_t *>(tr);
+                    __syncwarp();
+#pragma unroll
+                    for (int jp = 0; jp < 16; ++jp) {
+                        float f2[2];
+#pragma unroll
+                        for (int v = 0; v < 2; ++v) {
+                            const int col = c0 + 2 * jp + v;
+                            const bool valid = (it.w0 + (col & 7) < P.W) && (it.h0 + (col >> 3) < P.H);
+                            const float f = valid ? __uint_as_float(r[2 * jp + v]) + bias : 0.f;
+                            s1 += f;
+                            s2 = fmaf(f, f, s2);
+                            f2[v] = f;
+                        }
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(f2[0], f2[1]);
+                        trw[jp * 33 + lane] = *reinterpret_cast<uint32_t *>(&h2);
+                    }
+                    __syncwarp();
+                    const int jp = lane >> 1, ch0 = (lane & 1) * 16;
+                    uint32_t wv[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) wv[e] = trw[jp * 33 + ch0 + e];
+#pragma unroll
+                    for (int v = 0; v < 2; ++v) {
+                        const int col = c0 + 2 * jp + v;
+                        const int w = it.w0 + (col & 7), h = it.h0 + (col >> 3);
+                        if (w < P.W && h < P.H) {
+                            const int64_t vox = (((int64_t)it.n * P.D + o) * P.H + h) * P.W + w;
+                            uint4 *dst = reinterpret_cast<uint4 *>((bf16 *)P.y + vox * P.y_pitch + cbase + ch0);
+                            uint32_t ow[8];
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) ow[k] = __byte_perm(wv[2 * k], wv[2 * k + 1], v ? 0x7632 : 0x5410);
+                            dst[0] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                            dst[1] = make_uint4(ow[4], ow[5], ow[6], ow[7]);
+                        }
+                    }
+                } else if (plane_ok) {
                     // r[j] = channel (cbase + lane) at voxel column c0 + j: column = hl * 8 + wx
                     __syncwarp();
 #pragma unroll
