@@ -124,7 +124,9 @@ lamp_status_t lamp_conv3d_dgrad(const lamp_conv_desc_t *desc, const lamp_tensor_
  *    c_in * c_out = 77672, e.g. 256 x 256); otherwise LAMP_ERR_SCRATCH_LIMIT is returned and
  *    nothing is launched.  Variants that need no scratch are accepted at any size.
  *  - The first call on each device looks up the array's device address (with that device
- *    current) and keeps it; make that first call before starting any stream capture.
+ *    current) and keeps it; make that first call before starting any stream capture.  The kept
+ *    address belongs to the device's primary context and is not looked up again: do not use this
+ *    call after a cudaDeviceReset of a device on which it already ran.
  *  - All calls on a device share the one array, which keeps whatever the last call left in it.
  *    Nothing in it has to be zero beforehand (each call overwrites the part it reads), but two
  *    calls that overlap in time on the same GPU - different streams or threads - race on it:

@@ -13,6 +13,29 @@ int *status_word_ptr()
     return p;
 }
 
+void *tensor_map_encoder()
+{
+    // resolved once per process; the entry point does not depend on the device
+    static void *fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return p;
+    }();
+    return fn;
+}
+
+int sm_count()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        sms <= 0)
+        sms = 148;
+    return sms;
+}
+
 static bool aligned16(const void *p) { return ((uintptr_t)p & 15) == 0; }
 
 static lamp_status_t check_tensor(const lamp_tensor_t *t, bool allow_f32, bool any_channels)
@@ -96,7 +119,7 @@ static size_t splitk_ws(const ConvGeom &g, int pass)
     a.pitch = 8; b.pitch = 8;
     if (pass == LAMP_PASS_FWD) {
         a.d = g.d; a.h = g.h; a.w = g.w; a.c = g.ci;
-        if (ct_conv_fwd_supported(g, a, b)) return 0;
+        if (cr_conv_fwd_supported(g, a, b) || ct_conv_fwd_supported(g, a, b)) return 0;
         const int kind = fwd_kind(g);
         return kind >= 0 && umma_conv_supported(kind, g, a, b) ? umma_splitk_ws(kind, g) : 0;
     }
@@ -106,7 +129,7 @@ static size_t splitk_ws(const ConvGeom &g, int pass)
         ConvGeom t = g;
         t.ci = g.co; t.co = g.ci;
         a.d = g.d; a.h = g.h; a.w = g.w; a.c = g.co;
-        if (ct_conv_fwd_supported(t, a, b)) return 0;
+        if (cr_conv_fwd_supported(t, a, b) || ct_conv_fwd_supported(t, a, b)) return 0;
     }
     return umma_splitk_ws(kind, g);
 }
@@ -139,6 +162,7 @@ size_t conv_ws_bytes(const ConvGeom &g, int pass)
 lamp_status_t conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
                        double *stats, void *ws, size_t ws_bytes, cudaStream_t st)
 {
+    if (cr_conv_fwd_supported(g, x, y)) return cr_conv_fwd(g, x, w, bias, y, stats, 0, st);
     if (ct_conv_fwd_supported(g, x, y)) return ct_conv_fwd(g, x, w, bias, y, stats, 0, st);
     if (c1_umma_supported(g, x, y)) return c1_umma_fwd(g, x, w, bias, y, stats, st);
     const int kind = fwd_kind(g);
@@ -172,6 +196,7 @@ lamp_status_t conv_dgrad_run(const ConvGeom &g, const TView &dy, const bf16 *w, 
     if (kind == UK_S1_DGRAD) {
         ConvGeom t = g;
         t.ci = g.co; t.co = g.ci;
+        if (cr_conv_fwd_supported(t, dy, dx)) return cr_conv_fwd(t, dy, (const bf16 *)wt, nullptr, dx, nullptr, 1, st);
         if (ct_conv_fwd_supported(t, dy, dx)) return ct_conv_fwd(t, dy, (const bf16 *)wt, nullptr, dx, nullptr, 1, st);
     }
     return umma_conv(kind, g, dy, (const bf16 *)wt, nullptr, dx, nullptr, part, part_bytes, st);

@@ -74,6 +74,29 @@ static inline lamp_status_t launch_status()
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// api.cu.  The driver's cuTensorMapEncodeTiled, resolved once through the runtime (NULL if unavailable); declared
+// as void* so that this header needs no driver types.
+void *tensor_map_encoder();
+// api.cu.  Number of SMs of the current device.
+int sm_count();
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize is a per-device attribute of a kernel: a launcher keeps one of these
+// per kernel instantiation and asks it before every launch; the attribute is set on the first launch on each device
+// (bit i of `done` = device i; devices beyond 63 set it on every launch).  Safe to call from several host threads.
+struct SmemAttrOnce {
+    unsigned long long done = 0;
+    template <typename K> lamp_status_t ensure(K kernel, int bytes)
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return LAMP_ERR_CUDA;
+        const unsigned long long bit = dev >= 0 && dev < 64 ? 1ull << dev : 0ull;
+        if (bit && (__atomic_load_n(&done, __ATOMIC_ACQUIRE) & bit)) return LAMP_OK;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return LAMP_ERR_CUDA;
+        if (bit) __atomic_fetch_or(&done, bit, __ATOMIC_RELEASE);
+        return LAMP_OK;
+    }
+};
+
 // Programmatic dependent launch.  A kernel launched through launch_pdl may be scheduled while the kernel in front
 // of it on the stream is still running: its blocks set up shared memory, barriers and tensor memory, then stop at
 // pdl_wait() until that kernel has completed and its writes are visible.  Rules every such kernel follows:
@@ -173,6 +196,11 @@ lamp_status_t c1_umma_fwd(const ConvGeom &g, const TView &x, const bf16 *w, cons
 // conv_t.cu (tcgen05 "weights x voxels" implicit GEMM over shared-memory-resident planes, c_out <= 128)
 bool          ct_conv_fwd_supported(const ConvGeom &g, const TView &x, const TView &y);
 lamp_status_t ct_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
+                          double *stats, int mirror_taps, cudaStream_t st);
+
+// conv_r.cu (tcgen05 "voxels x (kd, channels)" implicit GEMM with rotating accumulator slots, c_out = 64 or 32)
+bool          cr_conv_fwd_supported(const ConvGeom &g, const TView &x, const TView &y);
+lamp_status_t cr_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, const float *bias, const TView &y,
                           double *stats, int mirror_taps, cudaStream_t st);
 
 // elementwise.cu

@@ -289,20 +289,7 @@ conv_c1_umma_kernel(const __grid_constant__ CUtensorMap map_x, const C1Params P)
     }
 }
 
-PFN_cuTensorMapEncodeTiled_v12000 get_encode()
-{
-    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (PFN_cuTensorMapEncodeTiled_v12000)p;
-    }
-    return fn;
-}
+PFN_cuTensorMapEncodeTiled_v12000 get_encode() { return (PFN_cuTensorMapEncodeTiled_v12000)tensor_map_encoder(); }
 
 }  // namespace
 
@@ -346,14 +333,9 @@ lamp_status_t c1_umma_fwd(const ConvGeom &g, const TView &x, const bf16 *w, cons
                    CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return LAMP_ERR_CUDA;
     }
-    static bool attr = false;
-    if (!attr) {
-        LAMP_CUDA_OK(cudaFuncSetAttribute(conv_c1_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C1_SMEM));
-        attr = true;
-    }
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-        sms = 148;
+    static SmemAttrOnce attr;
+    { const lamp_status_t as = attr.ensure(conv_c1_umma_kernel, (int)((int)C1_SMEM)); if (as != LAMP_OK) return as; }
+    const int sms = sm_count();
     // every CTA serves one channel block: the grid is a multiple of the number of blocks
     int64_t per_part = sms / P.nparts;
     if (per_part < 1) per_part = 1;

@@ -409,20 +409,7 @@ conv3_t_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
 }
 
-PFN_cuTensorMapEncodeTiled_v12000 get_encode()
-{
-    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (PFN_cuTensorMapEncodeTiled_v12000)p;
-    }
-    return fn;
-}
+PFN_cuTensorMapEncodeTiled_v12000 get_encode() { return (PFN_cuTensorMapEncodeTiled_v12000)tensor_map_encoder(); }
 
 struct CtPlan { CtParams P; int KC, COB, ST; size_t smem; int grid; };
 
@@ -465,9 +452,7 @@ bool make_ct_plan(const ConvGeom &g, CtPlan *out)
     if (items > 0x7FFFFFFF || items <= 0) return false;
     P.total_items = (int32_t)items;
     P.co = g.co;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     out->KC = KC; out->COB = COB; out->ST = ST;
     out->smem = 1024 + (size_t)np * P.plane_bytes + (wres ? wres_bytes : (size_t)nw * w_bytes) + EPI_BYTES + CTRL_BYTES;
     if (out->smem > (size_t)SMEM_LIMIT) return false;
@@ -478,11 +463,8 @@ bool make_ct_plan(const ConvGeom &g, CtPlan *out)
 template <int KC, int COB, int ST = 1>
 lamp_status_t launch_ct(const CUtensorMap &mx, const CUtensorMap &mw, const CtPlan &pl, cudaStream_t st)
 {
-    static bool attr = false;
-    if (!attr) {
-        LAMP_CUDA_OK(cudaFuncSetAttribute(conv3_t_kernel<KC, COB, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT));
-        attr = true;
-    }
+    static SmemAttrOnce attr;
+    { const lamp_status_t as = attr.ensure(conv3_t_kernel<KC, COB, ST>, (int)(SMEM_LIMIT)); if (as != LAMP_OK) return as; }
     return launch_pdl(pl.P.total_items <= 4 * pl.grid, conv3_t_kernel<KC, COB, ST>, dim3(pl.grid), dim3(CT_THREADS), pl.smem, st, mx, mw, pl.P);
 }
 

@@ -535,29 +535,7 @@ __global__ void transpose_weights_kernel(const bf16 *__restrict__ w, bf16 *__res
 // ----------------------------------------------------------------------------------------------
 // host side
 // ----------------------------------------------------------------------------------------------
-int sm_count()
-{
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        sms <= 0)
-        sms = 148;
-    return sms;
-}
-
-PFN_cuTensorMapEncodeTiled_v12000 get_encode()
-{
-    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (PFN_cuTensorMapEncodeTiled_v12000)p;
-    }
-    return fn;
-}
+PFN_cuTensorMapEncodeTiled_v12000 get_encode() { return (PFN_cuTensorMapEncodeTiled_v12000)tensor_map_encoder(); }
 
 int pick_bn(int co)
 {
@@ -585,11 +563,8 @@ template <int KC, int BN, int HEAD = 0>
 lamp_status_t launch(const CUtensorMap &mx, const CUtensorMap &mw, const UmmaParams &P, cudaStream_t st)
 {
     using L = SmemLayout<KC, BN>;
-    static bool attr = false;
-    if (!attr) {
-        LAMP_CUDA_OK(cudaFuncSetAttribute(conv3_umma_kernel<KC, BN, HEAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
-        attr = true;
-    }
+    static SmemAttrOnce attr;
+    { const lamp_status_t as = attr.ensure(conv3_umma_kernel<KC, BN, HEAD>, (int)(L::TOTAL)); if (as != LAMP_OK) return as; }
     const int sms = sm_count();
     const int grid = P.total_tiles < sms ? P.total_tiles : sms;
     UmmaParams Q = P;

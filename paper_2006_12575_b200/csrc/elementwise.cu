@@ -823,11 +823,8 @@ static lamp_status_t launch_head_bwd(const TView &z, const bf16 *w, int K, const
     const size_t lanes = 256 / (C / 2);
     const size_t tile = (size_t)256 * KP + 256 * K + 128 * C, red = lanes * KP * C + lanes * KP;
     const size_t smem = ((size_t)KP * C + 2 * KP + (tile > red ? tile : red)) * sizeof(float);
-    static bool attr_set = false;
-    if (!attr_set) {
-        LAMP_CUDA_OK(cudaFuncSetAttribute(head_bwd_kernel<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
-        attr_set = true;
-    }
+    static SmemAttrOnce attr;
+    { const lamp_status_t as = attr.ensure(head_bwd_kernel<KP>, (int)(96 * 1024)); if (as != LAMP_OK) return as; }
     (void)launch_pdl((int64_t)z.n * Vn <= SHORT_ELEMS / 32, head_bwd_kernel<KP>, dim3((unsigned)blocks, z.n), dim3(256), (size_t)(smem), st, 
         (const bf16 *)z.p, z.pitch, C, w, K, probs, labels, dice_sums, z.n, (bf16 *)dz.p, dz.pitch, partW, partB, dlogits,
         Vn, vpb);

@@ -13,7 +13,10 @@ namespace {
 static __device__ __align__(256) unsigned char g_static_scratch[LAMP_STATIC_SCRATCH_BYTES];
 
 constexpr int MAX_DEVICES = 64;
-void *g_scratch_addr[MAX_DEVICES];      // device address of g_static_scratch, per device, resolved on first use
+// device address of g_static_scratch, per device, resolved on first use.  Host threads may race to fill an entry:
+// all of them store the same value, and the accesses are atomic.  The cached address belongs to the device's
+// primary context: it does not survive a cudaDeviceReset of that device.
+void *g_scratch_addr[MAX_DEVICES];
 
 // In host code `g_static_scratch` is only a handle of the symbol, not an address a kernel may use:
 // the device address has to be asked for, with the device in question current.
@@ -21,12 +24,12 @@ lamp_status_t scratch_for_current_device(void **out)
 {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return LAMP_ERR_CUDA;
-    if (!g_scratch_addr[dev]) {
-        void *p = nullptr;
+    void *p = __atomic_load_n(&g_scratch_addr[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
         if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return LAMP_ERR_CUDA;
-        g_scratch_addr[dev] = p;
+        __atomic_store_n(&g_scratch_addr[dev], p, __ATOMIC_RELEASE);
     }
-    *out = g_scratch_addr[dev];
+    *out = p;
     return LAMP_OK;
 }
 

@@ -246,20 +246,7 @@ wgrad_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     }
 }
 
-PFN_cuTensorMapEncodeTiled_v12000 get_encode()
-{
-    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (PFN_cuTensorMapEncodeTiled_v12000)p;
-    }
-    return fn;
-}
+PFN_cuTensorMapEncodeTiled_v12000 get_encode() { return (PFN_cuTensorMapEncodeTiled_v12000)tensor_map_encoder(); }
 
 void pick_tile128(int D, int H, int W, int *tw, int *th, int *td)
 {
@@ -343,9 +330,7 @@ bool make_wg_plan(const ConvGeom &g, WgPlan *out)
     P.sps = 512 / NC < P.MB ? 512 / NC : P.MB;
     P.sets_per_chunk = (P.MB + P.sps - 1) / P.sps;
     P.nsets = P.nchunks * P.sets_per_chunk;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     int nsplit = sms / P.nsets;
     if (nsplit < 1) nsplit = 1;
     if (nsplit > P.ntiles) nsplit = P.ntiles;
@@ -363,11 +348,8 @@ template <int NC, int BOXA, int BOXB>
 lamp_status_t launch_wg(const CUtensorMap &mx, const CUtensorMap &mdy, const WgPlan &pl, cudaStream_t st)
 {
     using L = WgSmem<NC>;
-    static bool attr = false;
-    if (!attr) {
-        LAMP_CUDA_OK(cudaFuncSetAttribute(wgrad_umma_kernel<NC, BOXA, BOXB>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
-        attr = true;
-    }
+    static SmemAttrOnce attr;
+    { const lamp_status_t as = attr.ensure(wgrad_umma_kernel<NC, BOXA, BOXB>, (int)(L::TOTAL)); if (as != LAMP_OK) return as; }
     const lamp_status_t ls = launch_pdl((int64_t)pl.P.ntiles * pl.P.nunits <= 64 * (int64_t)pl.grid * pl.P.nsplit, wgrad_umma_kernel<NC, BOXA, BOXB>, dim3(pl.grid), dim3(WG_THREADS), L::TOTAL, st, mx, mdy, pl.P);
     if (ls != LAMP_OK) return ls;
     return launch_status();

@@ -243,20 +243,7 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     }
 }
 
-PFN_cuTensorMapEncodeTiled_v12000 get_encode()
-{
-    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (PFN_cuTensorMapEncodeTiled_v12000)p;
-    }
-    return fn;
-}
+PFN_cuTensorMapEncodeTiled_v12000 get_encode() { return (PFN_cuTensorMapEncodeTiled_v12000)tensor_map_encoder(); }
 
 bool encode_box(PFN_cuTensorMapEncodeTiled_v12000 encode, CUtensorMap *m, const TView &t, int box_c, int bw, int bh)
 {
@@ -309,9 +296,7 @@ bool make_ww_plan(const ConvGeom &g, WwPlan *out)
     if (nst > MAX_ST) nst = MAX_ST;
     if (nst < 2) return false;
     P.nst = nst;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     int nsplit = sms / P.nsets;
     if (nsplit < 1) nsplit = 1;
     if (nsplit > P.ntiles) nsplit = P.ntiles;
@@ -327,11 +312,8 @@ bool make_ww_plan(const ConvGeom &g, WwPlan *out)
 template <int CBA, int CBB>
 lamp_status_t launch_ww(const CUtensorMap &mx, const CUtensorMap &mdy, const WwPlan &pl, cudaStream_t st)
 {
-    static bool attr = false;
-    if (!attr) {
-        LAMP_CUDA_OK(cudaFuncSetAttribute(wgrad_win_kernel<CBA, CBB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attr = true;
-    }
+    static SmemAttrOnce attr;
+    { const lamp_status_t as = attr.ensure(wgrad_win_kernel<CBA, CBB>, (int)(227 * 1024)); if (as != LAMP_OK) return as; }
     const lamp_status_t ls = launch_pdl((int64_t)pl.P.ntiles * pl.P.nsets <= 64 * (int64_t)pl.grid, wgrad_win_kernel<CBA, CBB>, dim3(pl.grid), dim3(WW_THREADS), pl.smem, st, mx, mdy, pl.P);
     if (ls != LAMP_OK) return ls;
     return launch_status();

@@ -54,6 +54,15 @@ CASES = [
     ("t_down_64_128_ragged_odd", 1, 7, 60, 31, 64, 128, 3, 2, 1, 0),
     ("t_down_32_32_batch", 2, 8, 64, 16, 32, 32, 3, 2, 1, 0),
     ("t_down_128_256", 1, 4, 64, 16, 128, 256, 3, 2, 1, 0),
+    # narrow layers on volumes large enough for the rotating-slot kernel (runs of >= 10 planes per CTA, cut inside
+    # window columns; ragged windows; two samples; two channel chunks; columns shorter than a run)
+    ("r_c64_runs", 1, 38, 64, 160, 64, 64, 3, 1, 1, 0),
+    ("r_c64_ragged_batch", 2, 33, 70, 60, 64, 64, 3, 1, 1, 0),
+    ("r_c128_to_64", 1, 25, 96, 160, 128, 64, 3, 1, 1, 0),
+    ("r_c64_thin_columns", 1, 3, 352, 288, 64, 64, 3, 1, 1, 0),
+    ("r_c32_runs", 1, 40, 96, 136, 32, 32, 3, 1, 1, 0),
+    ("r_c64_to_32_ragged", 1, 37, 90, 140, 64, 32, 3, 1, 1, 0),
+    ("r_c32_to_64", 1, 30, 128, 104, 32, 64, 3, 1, 1, 0),
     ("deep_512_cube8", 1, 8, 8, 8, 512, 512, 3, 1, 1, 0),
     ("deep_512_to_256_ragged", 2, 3, 5, 7, 512, 256, 3, 1, 1, 0),
     ("deep_down_256_512", 1, 8, 8, 8, 256, 512, 3, 2, 1, 0),

@@ -31,15 +31,43 @@ def make_net(levels, ch, cpl, K, seed, cin=1, bias_scale=0.1):
     return net, spec, lay, ws, bs, dev_bf16(wflat), torch.from_numpy(bflat).cuda(), offs
 
 
-def tie_aware_agreement(seg, ref_scores):
+def tie_aware_agreement(seg, ref_scores, tau=None):
     """Fraction of voxels whose class equals the oracle's, counting either of the oracle's two best
-    classes as correct where their margin is below 1e-3 of the largest score."""
+    classes as correct where their margin is below tau (default: 1e-3 of the largest score)."""
     order = np.argsort(-ref_scores, axis=-1, kind="stable")
     best, second = order[..., 0], order[..., 1]
     top = np.take_along_axis(ref_scores, order[..., :2], axis=-1)
-    near = (top[..., 0] - top[..., 1]) < 1e-3 * np.abs(ref_scores).max()
+    if tau is None:
+        tau = 1e-3 * np.abs(ref_scores).max()
+    near = (top[..., 0] - top[..., 1]) < tau
     ok = (seg == best) | (near & (seg == second))
     return float(ok.mean()), float((seg == best).mean()), int(near.sum())
+
+
+def end_to_end_figures(got, ref_q, ref_f, what):
+    """End-to-end comparison of class scores [..., K] with the storage-mirrored oracle (ref_q), held to the
+    arithmetic's own budget: the distance between the mirrored and the unrounded oracle (ref_f) is the bf16
+    storage error of the chain, and two correct bf16 evaluations can differ by about that much (their roundings
+    flip on fp32-level differences).  Asserted: rel-L2 <= max(1e-3, 2 budget); max-abs <= max(1e-2 max|ref|,
+    2 max-abs budget); arg max agreement >= 99.99 % where either of the oracle's two best classes counts once
+    their margin is inside twice the max-abs budget.  The strict figure and the one at the 1e-3 margin are
+    returned (and printed by the callers) beside the budgets."""
+    got, ref_q, ref_f = (np.asarray(a, dtype=np.float64) for a in (got, ref_q, ref_f))
+    budget = np.linalg.norm(ref_q - ref_f) / np.linalg.norm(ref_f)
+    budget_abs = np.abs(ref_q - ref_f).max()
+    rel = np.linalg.norm(got - ref_q) / np.linalg.norm(ref_q)
+    mabs = np.abs(got - ref_q).max()
+    mref = np.abs(ref_q).max()
+    assert rel <= max(1e-3, 2.0 * budget), f"{what}: end-to-end rel L2 {rel:.3e}, budget {budget:.3e}"
+    assert mabs <= max(1e-2 * mref, 2.0 * budget_abs), f"{what}: end-to-end max abs {mabs:.3e}, budget {budget_abs:.3e}"
+    seg = np.argmax(got, axis=-1)
+    a_budget, strict, near_b = tie_aware_agreement(seg, ref_q, tau=max(1e-3 * mref, 2.0 * budget_abs))
+    a_1e3, _, near = tie_aware_agreement(seg, ref_q)
+    assert a_budget >= 0.9999, f"{what}: end-to-end arg max agreement {a_budget:.6f} (strict {strict:.6f})"
+    r = dict(rel_l2=rel, budget_rel_l2=budget, max_abs=mabs, budget_max_abs=budget_abs, argmax_strict=strict,
+             argmax_tie_1e3=a_1e3, argmax_tie_budget=a_budget, near_ties_1e3=near, near_ties_budget=near_b)
+    print(f"end to end, {what}: " + ", ".join(f"{k}={v:.4g}" for k, v in r.items()))
+    return r
 
 
 @pytest.mark.parametrize("shape,pitch,off", [((2, 5, 6, 7, 16), 16, 0), ((1, 9, 4, 11, 24), 48, 24),
@@ -179,9 +207,7 @@ def check_network_layer_by_layer(levels, ch, cpl, K, dhw, seed, x, lab, tight=2e
     bs64 = [a.astype(np.float64) for a in bs]
     loss_q, dWq, dBq, p_q = O.train_step(spec, ws64, bs64, x.astype(np.float64), lab, quantise=True)
     loss_f, dWf, dBf, p_f = O.train_step(spec, ws64, bs64, x.astype(np.float64), lab, quantise=False)
-    budget = np.linalg.norm(p_q - p_f) / np.linalg.norm(p_f)
-    e2e = np.linalg.norm(p_gpu - p_q) / np.linalg.norm(p_q)
-    assert e2e <= max(1e-3, 2.0 * budget), (e2e, budget)
+    fig = end_to_end_figures(p_gpu, p_q, p_f, "train step probabilities")
     assert abs(float(loss.item()) - loss_q) <= max(1e-3, 2.0 * abs(loss_q - loss_f) / abs(loss_f)) * abs(loss_q)
     for i, l in enumerate(lay):
         wo, _ = offs[i]
@@ -189,9 +215,8 @@ def check_network_layer_by_layer(levels, ch, cpl, K, dhw, seed, x, lab, tight=2e
         bud = np.linalg.norm(dWq[i] - dWf[i]) / np.linalg.norm(dWf[i])
         err = np.linalg.norm(got - dWq[i]) / np.linalg.norm(dWq[i])
         assert err <= max(1e-3, 2.0 * bud), (l.name, err, bud)
-    agree, strict, near = tie_aware_agreement(np.argmax(p_gpu, -1), p_q)
     B.lamp_unet_destroy(net)
-    return dict(e2e=e2e, budget=budget, argmax_e2e=agree)
+    return fig
 
 
 CFG0 = dict(levels=3, ch=[8, 16, 32], cpl=2, K=4)
@@ -249,9 +274,7 @@ def test_unet_forward_head_argmax_matches_oracle_on_stored_input():
     bs64 = [a.astype(np.float64) for a in bs]
     p_q = O.forward(spec, ws64, bs64, x.astype(np.float64), quantise=True).reshape(V, 4)
     p_f = O.forward(spec, ws64, bs64, x.astype(np.float64), quantise=False).reshape(V, 4)
-    budget = np.linalg.norm(p_q - p_f) / np.linalg.norm(p_f)
-    e2e = np.linalg.norm(host_f64(probs) - p_q) / np.linalg.norm(p_q)
-    assert e2e <= max(1e-3, 2 * budget), (e2e, budget)
+    end_to_end_figures(host_f64(probs), p_q, p_f, "forward pass, tiny U-Net")
     B.lamp_unet_destroy(net)
 
 
@@ -264,8 +287,7 @@ def test_unet_forward_batch_and_noncubic():
     wsb = torch.empty(B.lamp_unet_workspace_bytes(net, 2, 6, 8, 12, B.MODE_INFER), dtype=torch.uint8, device="cuda")
     B.lamp_unet_forward(net, wd, bd, dev_bf16(x), probs, None, wsb)
     full = O.forward(spec, ws, bs, x.astype(np.float64), quantise=False)
-    budget = np.linalg.norm(ref - full) / np.linalg.norm(full)
-    assert_close(host_f64(probs), ref.reshape(V, 3), "batched forward", rel=max(1e-3, 2 * budget), mx=0.2)
+    end_to_end_figures(host_f64(probs), ref.reshape(V, 3), full.reshape(V, 3), "batched forward")
     B.lamp_unet_destroy(net)
 
 
@@ -304,7 +326,6 @@ def test_sliding_window_matches_oracle_and_whole_patch_equals_forward():
     vol = synth.bf16_round(synth.ct_volume((D, H, W), 21))[None, ..., None]
     A, seg_ref, n_p = O.sliding_window(spec, ws, bs, vol.astype(np.float64), P, 0.25, gaussian=True, quantise=True)
     A_full, _, _ = O.sliding_window(spec, ws, bs, vol.astype(np.float64), P, 0.25, gaussian=True, quantise=False)
-    budget = np.linalg.norm(A - A_full) / np.linalg.norm(A_full)
     assert n_p == 2 * 1 * 2
     sd, sh, sw = (O.window_starts(n, p, 0.25) for n, p in zip((D, H, W), P))
     origins = [(a, b, c) for a in sd for b in sh for c in sw]
@@ -332,7 +353,7 @@ def test_sliding_window_matches_oracle_and_whole_patch_equals_forward():
         agree, strict, near = tie_aware_agreement(am.cpu().numpy().reshape(D, H, W), A_loc)
         assert agree >= 0.9999
         # (3) end to end against the mirrored oracle, within the bf16 storage budget
-        assert_close(host_f64(planar), A.transpose(3, 0, 1, 2), "sliding window end to end", rel=max(1e-3, 2 * budget), mx=0.2)
+        end_to_end_figures(host_f64(planar).transpose(1, 2, 3, 0), A, A_full, "sliding window")
     # patch = whole volume: identical to one forward pass
     probs = torch.empty((D * H * W, 3), dtype=torch.float32, device="cuda")
     wsf = torch.empty(B.lamp_unet_workspace_bytes(net, 1, D, H, W, B.MODE_INFER), dtype=torch.uint8, device="cuda")

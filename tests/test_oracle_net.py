@@ -229,6 +229,40 @@ def test_sliding_window_aggregation_properties():
     np.testing.assert_allclose(A[3, 0, 0], want, rtol=1e-13)
 
 
+def test_gaussian_window_closed_form_values():
+    """The blending window (paper silent: Sec. 3 gives patch sizes only; reading: separable Gaussian centred on the
+    patch, sigma = extent / 8 per axis, scaled to maximum 1, floored at 1e-3) against values worked out by hand.
+    P = 8: sigma = 1, offsets t = i - 3.5, so relative to the two centre samples (t = +-0.5) the per-axis weight is
+    exp(-(t^2 - 0.25) / 2): 1, e^-1, e^-3, e^-6 at |t| = 0.5, 1.5, 2.5, 3.5."""
+    w = unet.gaussian_window((8, 8, 8))
+    e = np.exp
+    np.testing.assert_allclose(w[3, 3, 3], 1.0, rtol=1e-15)
+    np.testing.assert_allclose(w[4, 3, 4], 1.0, rtol=1e-15)
+    np.testing.assert_allclose(w[2, 3, 4], e(-1.0), rtol=1e-13)            # 0.36788: sigma = P/4 would give e^-0.25
+    np.testing.assert_allclose(w[1, 3, 3], e(-3.0), rtol=1e-13)            # 0.049787
+    np.testing.assert_allclose(w[3, 6, 4], e(-3.0), rtol=1e-13)            # symmetric in the offset, any axis
+    np.testing.assert_allclose(w[0, 3, 3], e(-6.0), rtol=1e-13)            # 2.4788e-3: still above the floor
+    np.testing.assert_allclose(w[2, 5, 4], e(-2.0), rtol=1e-13)            # separable: e^-1 * e^-1
+    assert w[0, 2, 3] == 1e-3                                              # e^-7 = 9.12e-4 -> floored
+    assert w[0, 0, 0] == 1e-3                                              # e^-18 -> floored
+    assert w[7, 7, 7] == 1e-3
+    assert (w >= 1e-3).all() and w.max() == 1.0
+    # the whole window: exponents are sums of one of (0, 1, 3, 6) per axis, each combination occurring 8 times
+    total = sum(8 * max(e(-(a + b + c)), 1e-3) for a in (0, 1, 3, 6) for b in (0, 1, 3, 6) for c in (0, 1, 3, 6))
+    np.testing.assert_allclose(w.sum(), total, rtol=1e-13)
+    assert (w == 1e-3).sum() == 8 * sum(1 for a in (0, 1, 3, 6) for b in (0, 1, 3, 6) for c in (0, 1, 3, 6) if a + b + c >= 7)
+    # per-axis sigma follows the axis extent: (64, 32, 16) has sigma (8, 4, 2)
+    v = unet.gaussian_window((64, 32, 16))
+    np.testing.assert_allclose(v[31, 15, 7], 1.0, rtol=1e-15)
+    np.testing.assert_allclose(v[23, 15, 7], e(-0.5 * (8.5 ** 2 - 0.5 ** 2) / 64.0), rtol=1e-13)    # e^-0.5625
+    np.testing.assert_allclose(v[31, 11, 7], e(-0.5 * (4.5 ** 2 - 0.5 ** 2) / 16.0), rtol=1e-13)    # e^-0.625
+    np.testing.assert_allclose(v[31, 15, 5], e(-0.5 * (2.5 ** 2 - 0.5 ** 2) / 4.0), rtol=1e-13)     # e^-0.75
+    # odd extent: a single centre sample
+    u = unet.gaussian_window((5, 5, 5))
+    np.testing.assert_allclose(u[2, 2, 2], 1.0, rtol=1e-15)
+    np.testing.assert_allclose(u[1, 2, 2], e(-0.5 / 0.625 ** 2), rtol=1e-13)
+
+
 def test_bf16_storage_chain_amplifies_fp32_level_differences_beyond_1e3():
     """Why network-level parity is checked step by step: perturb every conv output of the oracle by a
     relative 1e-7 (the size of an fp32-vs-fp64 accumulation difference) before its bf16 storage rounding.
