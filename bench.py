@@ -31,10 +31,32 @@ CHANNELS = (32, 64, 128, 256)
 VOL = (128, 128, 128)
 SEED = 2
 NOMINAL_BF16_TFLOPS = 2250.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture summarised
-# under profiles/ (None: not captured for the kernel as it stands)
-NCU_TRAFFIC_BYTES = {"conv3_t_kernel (fwd+dgrad, C=256)": 2.166e9,     # profiles/conv3_t_c256_128cube.txt
-                     "wgrad_win_kernel (wgrad, C=256)": 2.151e9}       # profiles/wgrad_win_c256_128cube.txt
+PROFILES = os.path.join(ROOT, "profiles")
+
+
+def ncu_traffic_bytes(summary, sources):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch, as recorded in a profiles/ summary: the line
+    `traffic_bytes_per_launch: <bytes>`.  The summary also records `source_sha256: <hex>` of the kernel's source
+    files at the time of the capture; when the files differ today the counters no longer describe the kernel and
+    the answer is None."""
+    import hashlib
+    try:
+        text = open(os.path.join(PROFILES, summary)).read()
+    except OSError:
+        return None
+    val = sha = None
+    for line in text.splitlines():
+        if line.startswith("traffic_bytes_per_launch:"):
+            val = float(line.split(":", 1)[1].split()[0])
+        elif line.startswith("source_sha256:"):
+            sha = line.split(":", 1)[1].split()[0]
+    h = hashlib.sha256()
+    try:
+        for f in sources:
+            h.update(open(os.path.join(ROOT, "paper_2006_12575_b200", "csrc", f), "rb").read())
+    except OSError:
+        return None
+    return val if (val is not None and sha == h.hexdigest()) else None
 
 
 def pass_flops(C, vol=VOL):
@@ -320,8 +342,13 @@ def run_gpu(args):
                                       pct_measured=round(100 * tf / peaks["bf16"], 1))
     # kernel families (one CUDA kernel template each); the dgrad pass also holds the tiny weight-transpose launch
     cmax = max(chans)
-    fam = {f"conv3_t_kernel (fwd+dgrad, C={cmax})": [k for k in per if k[1] in ("fwd", "dgrad") and k[0] == cmax],
-           f"conv3_t_kernel (fwd+dgrad, C<{cmax})": [k for k in per if k[1] in ("fwd", "dgrad") and k[0] != cmax],
+    # (C >= 128: conv3_t_kernel; C = 64: conv3_r_kernel)
+    fwd_name = "conv3_t_kernel" if cmax >= 128 else "conv3_r_kernel" if cmax == 64 else "conv3_t_kernel"
+    traffic_of = {f"{fwd_name} (fwd+dgrad, C={cmax})": ("conv3_t_c256_128cube.txt", ["conv_t.cu", "umma_ptx.cuh"]) if cmax == 256 else
+                  ("conv3_r_c64_128cube.txt", ["conv_r.cu", "umma_ptx.cuh"]) if cmax == 64 else None,
+                  f"wgrad_win_kernel (wgrad, C={cmax})": ("wgrad_win_c256_128cube.txt", ["wgrad_win.cu", "umma_ptx.cuh"]) if cmax == 256 else None}
+    fam = {f"{fwd_name} (fwd+dgrad, C={cmax})": [k for k in per if k[1] in ("fwd", "dgrad") and k[0] == cmax],
+           f"conv3_t_kernel / conv3_r_kernel (fwd+dgrad, C<{cmax})": [k for k in per if k[1] in ("fwd", "dgrad") and k[0] != cmax],
            f"wgrad_win_kernel (wgrad, C={cmax})": [k for k in per if k[1] == "wgrad" and k[0] == cmax],
            f"wgrad_win_kernel (wgrad, C<{cmax})": [k for k in per if k[1] == "wgrad" and k[0] != cmax]}
     fam = {f: ks for f, ks in fam.items() if ks}
@@ -331,7 +358,8 @@ def run_gpu(args):
     dom_launches = sum(len(per[k]) for k in fam[dom])
     achieved = dom_flops / (fam_time[dom] * 1e-3) / 1e12
     roofline = dict(bound="tensor", kernel=dom, achieved=round(achieved, 2), peak=peaks["bf16"], unit="TFLOP/s",
-                    frac=round(achieved / peaks["bf16"], 4), traffic=NCU_TRAFFIC_BYTES.get(dom),
+                    frac=round(achieved / peaks["bf16"], 4),
+                    traffic=ncu_traffic_bytes(*traffic_of[dom]) if traffic_of.get(dom) else None,
                     peak_source=peaks["source"] + " cuBLAS bf16 burst", frac_of_nominal_2250=round(achieved / NOMINAL_BF16_TFLOPS, 4),
                     algorithmic_flops_per_launch=dom_flops / dom_launches,
                     avg_launch_ms=round(fam_time[dom] / dom_launches, 4),
@@ -359,6 +387,31 @@ def run_gpu(args):
         cpu["value"] = None
         cpu["error"] = str(e)[:200]
 
+    # the U-Net half of the metric, in the same process right after the sweep (one replica only: these workloads
+    # hold up to 31 GB and are quoted per GPU): training step of the standard network, whole-volume against
+    # sliding-window inference on the 512 x 512 x 128 volume
+    unet = None
+    if world == 1 and not args.no_unet:
+        del devb, host, hout
+        torch.cuda.empty_cache()
+        unet = {}
+        for key, wl, cfg_id, st_, wu_ in (("train_step_configs2", "unet_train", 2, 10, 3),
+                                          ("whole_volume_configs4", "unet_infer", 4, 5, 3),
+                                          ("sliding_window_configs4", "sliding", 4, 3, 3)):
+            smp = ClockSampler(local)
+            try:
+                r = measure_unet(wl, cfg_id, st_, wu_, args.sw_batch, graph=False)
+                r = {k: r[k] for k in ("metric", "value", "unit", "ms_per_step", "seconds_per_volume", "tflops", "steps", "warmup",
+                                       "config", "roofline")}
+            except Exception as e:                       # must not take the headline down with it
+                r = dict(error=str(e)[:200])
+            r["clocks"] = smp.stop()
+            unet[key] = r
+            torch.cuda.empty_cache()
+        a, b_ = unet.get("whole_volume_configs4", {}), unet.get("sliding_window_configs4", {})
+        if "seconds_per_volume" in a and "seconds_per_volume" in b_:
+            unet["whole_volume_speedup_over_sliding_window"] = round(b_["seconds_per_volume"] / a["seconds_per_volume"], 2)
+
     launches_per_C = 1 + 2 + 2     # fwd; dgrad = weight transpose + conv; wgrad = split-K kernel + fixed-order reduce
     out = dict(metric="conv3d_tflops", value=round(value, 3), unit="TFLOP/s", n_gpus=world, steps=args.steps,
                warmup=args.warmup, ms_per_step=round(ms / args.steps, 4), higher_is_better=True, scaling="weak",
@@ -373,6 +426,8 @@ def run_gpu(args):
                gpu_launches=args.steps * len(chans) * launches_per_C,
                roofline=roofline, cpu_baseline=cpu, passes=passes,
                pct_of_nominal_bf16=round(100 * value / world / NOMINAL_BF16_TFLOPS, 2))
+    if unet is not None:
+        out["unet"] = unet
     print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -410,14 +465,71 @@ def unet_fwd_flops(cfg):
     return fl + 2.0 * ch[0] * cfg["K"] * vox[0]
 
 
-def run_unet(args):
+def unet_floor_ms(cfg, train, peaks, vol=None):
+    """Roofline floor of one U-Net pass: the sum over its steps of max(FLOPs / tensor peak, algorithmic bytes /
+    HBM peak), with the measured peaks.  Bytes per step: a conv reads its input and writes its output once
+    (bf16) and reads its weights; normalise + ReLU moves 4 B per element; its backward 10 B per element; a data
+    gradient reads dy and writes dx; a weight gradient reads x and dy and writes fp32 weights; the head reads
+    its input and writes K fp32 probabilities and one label per voxel (training: reads them again and writes
+    the gradient of its input)."""
+    D, H, W = vol or cfg["vol"]
+    ch, L, K = cfg["ch"], cfg["levels"], cfg["K"]
+    vox = [(D >> l) * (H >> l) * (W >> l) for l in range(L)]
+    tf, bw = peaks["bf16"] * 1e12, peaks["hbm_gbs"] * 1e9
+    total = 0.0
+
+    def step(flops, nbytes):
+        nonlocal total
+        total += max(flops / tf, nbytes / bw)
+
+    def conv(ci, co, vin, vout, taps, norm, dgrad=True):
+        fl = 2.0 * taps * ci * co * vout
+        io = 2.0 * vin * ci + 2.0 * vout * co
+        step(fl, io + 2.0 * taps * ci * co)
+        if norm:
+            step(0, 4.0 * vout * co)
+        if train:
+            if norm:
+                step(0, 10.0 * vout * co)
+            if dgrad:
+                step(fl, io + 2.0 * taps * ci * co)
+            step(fl, io + 4.0 * taps * ci * co)
+
+    c = 1
+    for l in range(L):
+        for i in range(cfg["cpl"]):
+            conv(c, ch[l], vox[l], vox[l], 27, True, dgrad=not (l == 0 and i == 0))
+            c = ch[l]
+        if l < L - 1:
+            conv(ch[l], ch[l + 1], vox[l], vox[l + 1], 27, True)
+            c = ch[l + 1]
+    for l in range(L - 2, -1, -1):
+        # transposed conv: one tap per output voxel
+        fl = 2.0 * ch[l + 1] * ch[l] * vox[l]
+        io = 2.0 * vox[l + 1] * ch[l + 1] + 2.0 * vox[l] * ch[l]
+        step(fl, io)
+        if train:
+            step(fl, io)
+            step(fl, io)
+        c = 2 * ch[l]
+        for _ in range(cfg["cpl"]):
+            conv(c, ch[l], vox[l], vox[l], 27, True)
+            c = ch[l]
+    step(2.0 * ch[0] * K * vox[0], vox[0] * (2.0 * ch[0] + 4.0 * K + 1))
+    if train:
+        step(4.0 * ch[0] * K * vox[0], vox[0] * (4.0 * ch[0] + 4.0 * K + 1))
+    return total * 1e3
+
+
+def measure_unet(workload, cfg_id, steps, warmup, sw_batch=32, graph=True):
+    """Times one U-Net workload on cuda:0 through the C ABI; returns the fields of its JSON line."""
     import torch
     from paper_2006_12575_b200 import binding as B
-    from paper_2006_12575_b200 import build as lamp_build
     from paper_2006_12575_b200 import synth
-    lamp_build.build()
-    torch.cuda.set_device(0)
-    cfg = UNET_CFGS[args.cfg]
+    cfg = UNET_CFGS[cfg_id]
+    args = argparse.Namespace(cfg=cfg_id, workload=workload, steps=steps, warmup=warmup, sw_batch=sw_batch,
+                              no_graph=not graph)
+    peaks = measured_peaks()
     D, H, W = cfg["vol"]
     V = D * H * W
     net = B.lamp_unet_create(B.unet_spec(cfg["levels"], cfg["ch"], cfg["cpl"], 1, cfg["K"]))
@@ -450,6 +562,7 @@ def run_unet(args):
         ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
         fn = lambda: B.lamp_unet_train_step(net, wd, bd, x, lab, loss, gw, gb, None, ws)
         flops = 3 * unet_fwd_flops(cfg)
+        floor_ms = unet_floor_ms(cfg, True, peaks)
         out.update(metric="unet_train_step_voxels_per_s", config=dict(workload=f"configs[{args.cfg}] U-Net forward+backward",
                                                                          workspace_bytes=nbytes))
     elif args.workload == "unet_infer":
@@ -459,6 +572,7 @@ def run_unet(args):
         ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
         fn = lambda: B.lamp_unet_forward(net, wd, bd, x, probs, seg, ws)
         flops = unet_fwd_flops(cfg)
+        floor_ms = unet_floor_ms(cfg, False, peaks)
         out.update(metric="unet_whole_volume_infer_voxels_per_s",
                    config=dict(workload=f"configs[{args.cfg}] whole-volume forward", workspace_bytes=nbytes))
     else:
@@ -474,6 +588,9 @@ def run_unet(args):
             k = (n_ - p_) // s_ + 1
             npatch *= k + (1 if (k - 1) * s_ != n_ - p_ else 0)
         flops = npatch * unet_fwd_flops(pc)
+        # every patch's forward pass, then the blend: patch probabilities written and read once (fp32), one label out
+        floor_ms = npatch * unet_floor_ms(cfg, False, peaks, vol=patch) + \
+            (npatch * 64 ** 3 * 8.0 * cfg["K"] + V) / (peaks["hbm_gbs"] * 1e9) * 1e3
         out.update(metric="unet_sliding_window_infer_voxels_per_s",
                    config=dict(workload=f"configs[{args.cfg}] sliding window 64^3, overlap 0.25, gaussian", patches=npatch,
                                sw_batch=args.sw_batch, workspace_bytes=nbytes))
@@ -491,9 +608,12 @@ def run_unet(args):
         raise SystemExit("device status not ok")
     out.update(value=round(V / (ms * 1e-3), 1), ms_per_step=round(ms, 3), tflops=round(flops / (ms * 1e-3) / 1e12, 2),
                seconds_per_volume=round(ms * 1e-3, 5))
+    out["roofline"] = dict(bound="sum over the steps of max(tensor, hbm)", floor_ms=round(floor_ms, 3),
+                           frac=round(floor_ms / ms, 3), peak_source=peaks["source"],
+                           peaks=dict(bf16_tflops=peaks["bf16"], hbm_gbs=peaks["hbm_gbs"]))
     if args.no_graph:
-        print(json.dumps(out), flush=True)
-        return
+        B.lamp_unet_destroy(net)
+        return out
     # the same call captured once in a CUDA graph and replayed: what the launch-bound deep levels cost in host launches
     try:
         side = torch.cuda.Stream()
@@ -517,7 +637,16 @@ def run_unet(args):
         out["graph_replay"] = dict(ms_per_step=round(gms, 3), value=round(V / (gms * 1e-3), 1))
     except RuntimeError as e:
         out["graph_replay"] = dict(error=str(e)[:120])
-    print(json.dumps(out), flush=True)
+    B.lamp_unet_destroy(net)
+    return out
+
+
+def run_unet(args):
+    import torch
+    from paper_2006_12575_b200 import build as lamp_build
+    lamp_build.build()
+    torch.cuda.set_device(0)
+    print(json.dumps(measure_unet(args.workload, args.cfg, args.steps, args.warmup, args.sw_batch, not args.no_graph)), flush=True)
 
 
 def run_unet_dp(args):
@@ -713,6 +842,7 @@ def main():
     ap.add_argument("--cfg", type=int, default=2)
     ap.add_argument("--sw-batch", type=int, default=32)
     ap.add_argument("--no-graph", action="store_true", help="U-Net workloads: skip the CUDA-graph replay timing")
+    ap.add_argument("--no-unet", action="store_true", help="conv sweep: leave out the U-Net workloads that follow it")
     args = ap.parse_args()
     if args.workload == "hbm":
         run_hbm(args)

@@ -15,14 +15,22 @@
 // of a tile accordingly.  After input plane p the slot of output plane p - 1 is complete: the epilogue moves it
 // to registers, stores zeros in its place (it becomes the fresh slot of plane p + 2) and hands it back.
 //
+//  * c_out = 32 (J = 2).  Three kd blocks of 32 channels would leave N = 96, which costs 76 cycles instead of 48.  So a
+//    slot holds TWO output rows side by side: the 128 M rows are the voxels of every second h row (8 (w) x 16 rows, the
+//    descriptor steps two halo rows between 8-voxel groups), and column block (kd, jj) belongs to output row h + jj.
+//    A window that starts hs rows into the halo box is tap kh = hs - jj of block jj: four window shifts hs = 0..3 x three
+//    kw serve the nine in-plane taps of both rows, the blocks with kh outside 0..2 are fetched with an out-of-range tap
+//    coordinate and arrive as zeros: 18 of 24 blocks carry work (75 % of the full rate; the stacked-plane form reaches
+//    50 %).  Channels go in chunks of 32, and the three kw tiles of a shift share one pipeline stage.
 //  * Two voxel windows per CTA (h rows 0..15 and 16..31 of one 8 x 32 window, one TMA halo box of 10 x 34 voxels
 //    per input plane and channel chunk, out-of-volume voxels zero-filled = the zero padding) share every weight
 //    tile, which halves the L2 -> SM weight traffic per MMA (the tiles are streamed: 27 * c_in * c_out * 2 bytes
 //    do not fit beside the planes).  The nine in-plane taps are shifted windows of the halo box (descriptor
 //    start (kh * 10 + kw) rows in, 10 rows between 8-voxel groups; the swizzle is a function of the address).
-//  * The last two weight tiles of an input plane are issued window by window (window 0: taps 7, 8; then window
-//    1: taps 7, 8) and the first two of the next plane likewise, so each window's slot hand-over (TMEM -> registers,
-//    zero store, barrier) has two tiles of the other window's MMAs to hide behind.
+//  * Every weight tile is used by window 0, then by window 1; window 0's slot hand-over (TMEM -> registers, zero
+//    store, barrier) after the last tile of an input plane runs behind window 1's MMAs of that tile.  (Issuing the
+//    last two and first two tiles of a plane window by window, to give the hand-over twice that time, measured 9 %
+//    slower.)
 //  * A CTA owns a contiguous run of (window column, output plane) units; a run that starts or ends inside a
 //    column costs one extra input plane each (the halo along d), columns that end at the volume border none.
 //  * Epilogue: one voxel per thread with all its channels: bias, InstanceNorm sums (a transposing shuffle
@@ -42,8 +50,8 @@ namespace {
 using namespace ptx;
 
 constexpr int CR_THREADS = 384;
-constexpr int TW = 8, TH = 32;          // window pair: 8 (w) x 32 (h) voxels = two M = 128 windows
-constexpr int HALO_W = TW + 2, HALO_H = TH + 2;
+constexpr int TW = 8;                   // window pair: 8 (w) x 32 J (h) voxels = two windows of 128 M rows x J output rows
+constexpr int HALO_W = TW + 2;
 constexpr int MAX_NP = 4, MAX_NW = 8;
 constexpr int CTRL_BYTES = 1024;
 constexpr int SMEM_LIMIT = 227 * 1024;
@@ -74,7 +82,7 @@ struct PieceWalker {
         u = P.units * (int64_t)blockIdx.x / gridDim.x;
         u1 = P.units * (int64_t)(blockIdx.x + 1) / gridDim.x;
     }
-    __device__ __forceinline__ bool next(const CrParams &P, Piece &pc)
+    __device__ __forceinline__ bool next(const CrParams &P, Piece &pc, int TH)
     {
         if (u >= u1) return false;
         int64_t col = u / P.D;
@@ -99,17 +107,22 @@ __device__ __forceinline__ void tmem_st32_zero(uint32_t taddr)
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// KC: channels per chunk (64: 128-byte swizzle, 32: 64-byte swizzle).  CO: output channels (64 or 32).
-template <int KC, int CO>
+// KC: channels per chunk (64: 128-byte swizzle, 32: 64-byte swizzle).  CO x J = 64: output channels x output rows per slot.
+template <int KC, int CO, int J>
 __global__ void __launch_bounds__(CR_THREADS, 1)
 conv3_r_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const CrParams P)
 {
+    static_assert(CO * J == 64, "a slot is 64 accumulator columns");
     constexpr int ROWB = KC * 2;
     constexpr uint32_t SWZ = KC == 64 ? 2u : 4u;
+    constexpr int TH = 32 * J, HALO_H = TH + 2;
     constexpr uint32_t PLANE_BOX_BYTES = HALO_W * HALO_H * ROWB;
-    constexpr uint32_t BLK_BYTES = CO * ROWB;                  // one kd block of a weight tile
-    constexpr uint32_t WST_BYTES = 3 * BLK_BYTES;
-    constexpr int NCOL = 3 * CO;
+    constexpr uint32_t BLK_BYTES = CO * ROWB;                  // one (kd, jj) block of a weight tile
+    constexpr uint32_t TILE_BYTES = 3 * J * BLK_BYTES;         // one (window shift, kw) tile: N = 192 rows
+    constexpr int NT = 3 * (J + 2);                            // tiles per input plane and chunk: window shifts hs x kw
+    constexpr int TPS = J == 2 ? 3 : 1;                        // tiles per pipeline stage
+    constexpr uint32_t WST_BYTES = TPS * TILE_BYTES;
+    constexpr int NCOL = 192;
     constexpr uint32_t IDESC = make_idesc(NCOL);
 
     extern __shared__ uint8_t smem_raw[];
@@ -151,7 +164,7 @@ conv3_r_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             PieceWalker pw;
             Piece pc;
             pw.init(P);
-            while (ok && pw.next(P, pc)) {
+            while (ok && pw.next(P, pc, TH)) {
                 const int p_lo = pc.o_lo > 0 ? pc.o_lo - 1 : 0, p_hi = pc.o_hi < P.D ? pc.o_hi : P.D - 1;
                 for (int p = p_lo; p <= p_hi && ok; ++p) {
                     for (int c = 0; c < P.chunks; ++c) {
@@ -173,22 +186,33 @@ conv3_r_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             PieceWalker pw;
             Piece pc;
             pw.init(P);
-            while (ok && pw.next(P, pc)) {
+            while (ok && pw.next(P, pc, TH)) {
                 const int p_lo = pc.o_lo > 0 ? pc.o_lo - 1 : 0, p_hi = pc.o_hi < P.D ? pc.o_hi : P.D - 1;
                 for (int p = p_lo; p <= p_hi && ok; ++p) {
                     // kd block of output plane o = p + 1 - kd goes to slot o mod 3 of the tile
                     const int slot_kd0 = (p + 1) % 3;
                     for (int c = 0; c < P.chunks && ok; ++c) {
-                        for (int t9 = 0; t9 < 9; ++t9) {
+                        for (int t0 = 0; t0 < NT; t0 += TPS) {
                             if (!mbar_wait(wempty0 + 8 * ws, wph ^ 1, abort_flag)) { ok = false; break; }
                             mbar_expect_tx(wfull0 + 8 * ws, WST_BYTES);
                             const uint32_t dst = smem_u32(w_base + (size_t)ws * WST_BYTES);
 #pragma unroll
-                            for (int kd = 0; kd < 3; ++kd) {
-                                int slot = slot_kd0 - kd;
-                                if (slot < 0) slot += 3;
-                                const int tap = kd * 9 + t9;        // with mirrored taps the window (kd, t9) reads weight tap 26 - tap
-                                tma_load_3d(dst + slot * BLK_BYTES, &map_w, wfull0 + 8 * ws, c * KC, 0, P.mirror ? 26 - tap : tap);
+                            for (int ti = 0; ti < TPS; ++ti) {
+                                const int hs = (t0 + ti) / 3, kw = (t0 + ti) % 3;
+#pragma unroll
+                                for (int kd = 0; kd < 3; ++kd) {
+                                    int slot = slot_kd0 - kd;
+                                    if (slot < 0) slot += 3;
+#pragma unroll
+                                    for (int jj = 0; jj < J; ++jj) {
+                                        // block jj reads tap kh = hs - jj; outside 0..2 the coordinate is out of range (zeros).
+                                        // With mirrored taps the window (kd, kh, kw) reads weight tap (2 - kd, 2 - kh, 2 - kw).
+                                        const int kh = hs - jj;
+                                        const bool in = kh >= 0 && kh <= 2;
+                                        tma_load_5d(dst + ti * TILE_BYTES + (slot * J + jj) * BLK_BYTES, &map_w, wfull0 + 8 * ws, c * KC, 0,
+                                                    P.mirror ? 2 - kw : kw, in ? (P.mirror ? 2 - kh : kh) : 3, P.mirror ? 2 - kd : kd);
+                                    }
+                                }
                             }
                             if (++ws == P.nw) { ws = 0; wph ^= 1; }
                         }
@@ -205,46 +229,39 @@ conv3_r_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             PieceWalker pw;
             Piece pc;
             pw.init(P);
-            while (ok && pw.next(P, pc)) {
+            while (ok && pw.next(P, pc, TH)) {
                 const int p_lo = pc.o_lo > 0 ? pc.o_lo - 1 : 0, p_hi = pc.o_hi < P.D ? pc.o_hi : P.D - 1;
                 for (int p = p_lo; p <= p_hi && ok; ++p, ++gs) {
                     for (int c = 0; c < P.chunks && ok; ++c) {
                         if (!mbar_wait(pfull0 + 8 * ps, pph, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t plane = smem_u32(p_base + (size_t)ps * P.plane_bytes);
-                        for (int t9 = 0; t9 < 9 && ok;) {
-                            // the first two and the last two tiles of an input plane go window by window
-                            const bool first = c == 0 && t9 == 0, last = c == P.chunks - 1 && t9 == 7;
-                            const int g = (first || last) ? 2 : 1;
-                            int st[2];
-                            uint32_t sph[2];
-                            st[0] = ws; sph[0] = wph;
-                            st[1] = ws + 1; sph[1] = wph;
-                            if (st[1] == P.nw) { st[1] = 0; sph[1] ^= 1; }
-                            for (int s = 0; s < g && ok; ++s) ok = mbar_wait(wfull0 + 8 * st[s], sph[s], abort_flag);
-                            if (!ok) break;
+                        for (int t0 = 0; t0 < NT && ok; t0 += TPS) {
+                            if (!mbar_wait(wfull0 + 8 * ws, wph, abort_flag)) { ok = false; break; }
                             tc_fence_after();
 #pragma unroll
-                            for (int j = 0; j < 2; ++j) {
-                                if (first) {
-                                    if (!mbar_wait(free0 + 8 * j, gs & 1, abort_flag)) { ok = false; break; }
-                                    tc_fence_after();
-                                }
-                                const uint32_t d_tmem = tmem_base + j * WIN_COLS;
-                                for (int s = 0; s < g; ++s) {
-                                    const int t = t9 + s, kh = t / 3, kw = t - kh * 3;
-                                    const uint64_t da = make_desc(plane + ((kh + 16 * j) * HALO_W + kw) * ROWB, 0, HALO_W * ROWB, SWZ);
-                                    const uint64_t db = make_desc(smem_u32(w_base + (size_t)st[s] * WST_BYTES), 0, 8 * ROWB, SWZ);
+                            for (int ti = 0; ti < TPS; ++ti) {
+                                const int tt = t0 + ti, hs = tt / 3, kw = tt - hs * 3;
+                                const bool first = c == 0 && tt == 0, last = c == P.chunks - 1 && tt == NT - 1;
+                                const uint64_t db = make_desc(smem_u32(w_base + (size_t)ws * WST_BYTES) + ti * TILE_BYTES, 0, 8 * ROWB, SWZ);
 #pragma unroll
-                                    for (int k = 0; k < KC / 16; ++k) umma_bf16(d_tmem, da + 2 * k, db + 2 * k, IDESC, 1u);
+                                for (int j = 0; j < 2; ++j) {
+                                    if (first) {
+                                        // the slot that input plane p starts afresh has been zeroed
+                                        if (!mbar_wait(free0 + 8 * j, gs & 1, abort_flag)) { ok = false; break; }
+                                        tc_fence_after();
+                                    }
+                                    // window j: 16 groups of 8 voxels along w, J halo rows apart, from halo row hs + 16 J j
+                                    const uint64_t da = make_desc(plane + ((hs + 16 * J * j) * HALO_W + kw) * ROWB, 0, J * HALO_W * ROWB, SWZ);
+#pragma unroll
+                                    for (int k = 0; k < KC / 16; ++k) umma_bf16(tmem_base + j * WIN_COLS, da + 2 * k, db + 2 * k, IDESC, 1u);
+                                    if (last) umma_commit(done0 + 8 * j);
                                 }
-                                if (last) umma_commit(done0 + 8 * j);
+                                if (!ok) break;
                             }
                             if (!ok) break;
-                            for (int s = 0; s < g; ++s) umma_commit(wempty0 + 8 * st[s]);
-                            ws += g;
-                            if (ws >= P.nw) { ws -= P.nw; wph ^= 1; }
-                            t9 += g;
+                            umma_commit(wempty0 + 8 * ws);
+                            if (++ws == P.nw) { ws = 0; wph ^= 1; }
                         }
                         if (!ok) break;
                         umma_commit(pempty0 + 8 * ps);
@@ -257,8 +274,8 @@ conv3_r_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         // -------------------------------------------------------------------- epilogue
         const int q = warp & 3;                                 // TMEM lane quarter of this warp
         const int j = (warp - 4) >> 2;                          // window
-        const int m = q * 32 + lane;                            // voxel of the window: row hl, column wx
-        const int hl = 16 * j + (m >> 3), wx = m & 7;
+        const int m = q * 32 + lane;                            // M row of the window: output row(s) from hl, column wx
+        const int hl = J * (16 * j + (m >> 3)), wx = m & 7;
         const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + j * WIN_COLS;
         uint32_t gs = 0;
         float s1[CO / 32], s2[CO / 32];                         // lane l: sums of channel (32 i + l)
@@ -278,9 +295,11 @@ conv3_r_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 #pragma unroll
             for (int i = 0; i < CO / 32; ++i) { s1[i] = 0.f; s2[i] = 0.f; }
         };
-        // bias, statistics and store of 32 channels (first channel c0) of this thread's voxel of output plane o
-        auto emit = [&](const Piece &pc, int o, int c0, const uint32_t (&r)[32]) {
-            const int h = pc.h0 + hl, w = pc.w0 + wx;
+        // bias, statistics and store of 32 accumulator columns (the i-th 32 of the slot) of output plane o:
+        // J = 1: channels 32 i .. 32 i + 31 of this thread's voxel; J = 2: all 32 channels of the voxel in row hl + i
+        auto emit = [&](const Piece &pc, int o, int i32, const uint32_t (&r)[32]) {
+            const int c0 = J == 1 ? 32 * i32 : 0;
+            const int h = pc.h0 + hl + (J == 2 ? i32 : 0), w = pc.w0 + wx;
             const bool valid = h < P.H && w < P.W;
             float v[32];
 #pragma unroll
@@ -352,43 +371,43 @@ conv3_r_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         PieceWalker pw;
         Piece pc;
         pw.init(P);
-        while (ok && pw.next(P, pc)) {
+        while (ok && pw.next(P, pc, TH)) {
             if (pc.n != stat_n) { flush(); stat_n = pc.n; }
             const int p_lo = pc.o_lo > 0 ? pc.o_lo - 1 : 0, p_hi = pc.o_hi < P.D ? pc.o_hi : P.D - 1;
             for (int p = p_lo; p <= p_hi && ok; ++p, ++gs) {
                 ok = __all_sync(0xffffffffu, mbar_wait(done0 + 8 * j, gs & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t tdone = trow + (uint32_t)((p + 2) % 3) * CO;      // slot of output plane p - 1
-                uint32_t r[CO / 32][32];
+                const uint32_t tdone = trow + (uint32_t)((p + 2) % 3) * 64;      // slot of output plane p - 1
+                uint32_t r[2][32];
                 if (p < p_hi) {
 #pragma unroll
-                    for (int i = 0; i < CO / 32; ++i) tmem_ld32(tdone + 32 * i, r[i]);
+                    for (int i = 0; i < 2; ++i) tmem_ld32(tdone + 32 * i, r[i]);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < CO / 32; ++i) tmem_st32_zero(tdone + 32 * i);
+                    for (int i = 0; i < 2; ++i) tmem_st32_zero(tdone + 32 * i);
                     hand_back();
                     if (p - 1 >= pc.o_lo) {
 #pragma unroll
-                        for (int i = 0; i < CO / 32; ++i) emit(pc, p - 1, 32 * i, r[i]);
+                        for (int i = 0; i < 2; ++i) emit(pc, p - 1, i, r[i]);
                     }
                 } else {
                     // last input plane of the run: plane p - 1 is complete, and so is plane p where the volume ends;
                     // whatever the slots hold afterwards belongs to planes outside the run
                     if (p - 1 >= pc.o_lo) {
 #pragma unroll
-                        for (int i = 0; i < CO / 32; ++i) tmem_ld32(tdone + 32 * i, r[i]);
+                        for (int i = 0; i < 2; ++i) tmem_ld32(tdone + 32 * i, r[i]);
                         tmem_ld_wait();
 #pragma unroll
-                        for (int i = 0; i < CO / 32; ++i) emit(pc, p - 1, 32 * i, r[i]);
+                        for (int i = 0; i < 2; ++i) emit(pc, p - 1, i, r[i]);
                     }
                     if (p < pc.o_hi) {
-                        const uint32_t tlast = trow + (uint32_t)(p % 3) * CO;
+                        const uint32_t tlast = trow + (uint32_t)(p % 3) * 64;
 #pragma unroll
-                        for (int i = 0; i < CO / 32; ++i) tmem_ld32(tlast + 32 * i, r[i]);
+                        for (int i = 0; i < 2; ++i) tmem_ld32(tlast + 32 * i, r[i]);
                         tmem_ld_wait();
 #pragma unroll
-                        for (int i = 0; i < CO / 32; ++i) emit(pc, p, 32 * i, r[i]);
+                        for (int i = 0; i < 2; ++i) emit(pc, p, i, r[i]);
                     }
 #pragma unroll
                     for (int c0 = 0; c0 < NCOL; c0 += 32) tmem_st32_zero(trow + c0);
@@ -414,24 +433,26 @@ conv3_r_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
 }
 
-struct CrPlan { CrParams P; int KC, CO; size_t smem; int grid; };
+struct CrPlan { CrParams P; int KC, CO, J, TH; size_t smem; int grid; };
 
 bool make_cr_plan(const ConvGeom &g, CrPlan *out)
 {
     if (!(g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed)) return false;
     if (g.co != 64 && g.co != 32) return false;
     if (g.ci % 32 || g.ci <= 0) return false;
-    const int KC = g.ci % 64 == 0 ? 64 : 32;
+    const int J = g.co == 64 ? 1 : 2;
+    const int KC = (J == 1 && g.ci % 64 == 0) ? 64 : 32;       // two output rows per slot: planes twice as tall, 32-channel chunks
+    const int TH = 32 * J;
     const int rowb = KC * 2;
     CrParams &P = out->P;
     P.N = g.n; P.D = g.od; P.H = g.oh; P.W = g.ow;
     P.chunks = g.ci / KC;
-    P.plane_bytes = (int)align_up((size_t)HALO_W * HALO_H * rowb, 1024);
-    const int wst = 3 * g.co * rowb;
-    const int np = KC == 64 ? 2 : 3;
+    P.plane_bytes = (int)align_up((size_t)HALO_W * (TH + 2) * rowb, 1024);
+    const int wst = (J == 2 ? 3 : 1) * 192 * rowb;              // one stage: 1 or 3 tiles of 192 rows
+    const int np = (KC == 64 || J == 2) ? 2 : 3;
     int nw = (SMEM_LIMIT - 1024 - CTRL_BYTES - np * P.plane_bytes) / wst;
     if (nw > MAX_NW) nw = MAX_NW;
-    if (nw < 4) return false;                                  // the issuer holds two tiles at a time
+    if (nw < 3) return false;
     P.np = np; P.nw = nw;
     P.nwt = (g.ow + TW - 1) / TW;
     P.nht = (g.oh + TH - 1) / TH;
@@ -439,19 +460,19 @@ bool make_cr_plan(const ConvGeom &g, CrPlan *out)
     if (units <= 0 || units > 0x3FFFFFFF) return false;
     P.units = units;
     const int sms = sm_count();
-    out->KC = KC; out->CO = g.co;
+    out->KC = KC; out->CO = g.co; out->J = J; out->TH = TH;
     out->smem = 1024 + (size_t)np * P.plane_bytes + (size_t)nw * wst + CTRL_BYTES;
     if (out->smem > (size_t)SMEM_LIMIT) return false;
     out->grid = (int)(units < sms ? units : sms);
     return true;
 }
 
-template <int KC, int CO>
+template <int KC, int CO, int J>
 lamp_status_t launch_cr(const CUtensorMap &mx, const CUtensorMap &mw, const CrPlan &pl, cudaStream_t st)
 {
     static SmemAttrOnce attr;
-    { const lamp_status_t as = attr.ensure(conv3_r_kernel<KC, CO>, SMEM_LIMIT); if (as != LAMP_OK) return as; }
-    return launch_pdl(pl.P.units <= 4 * (int64_t)pl.grid, conv3_r_kernel<KC, CO>, dim3(pl.grid), dim3(CR_THREADS), pl.smem, st, mx, mw, pl.P);
+    { const lamp_status_t as = attr.ensure(conv3_r_kernel<KC, CO, J>, SMEM_LIMIT); if (as != LAMP_OK) return as; }
+    return launch_pdl(pl.P.units <= 4 * (int64_t)pl.grid, conv3_r_kernel<KC, CO, J>, dim3(pl.grid), dim3(CR_THREADS), pl.smem, st, mx, mw, pl.P);
 }
 
 }  // namespace
@@ -461,8 +482,8 @@ bool cr_conv_fwd_supported(const ConvGeom &g, const TView &x, const TView &y)
     CrPlan pl;
     if ((int64_t)g.n * g.d * g.h * g.w == 0) return false;
     if (!make_cr_plan(g, &pl)) return false;
-    // the 8 x 32 window pair must not be mostly padding
-    const double used = (double)g.oh * g.ow / ((double)pl.P.nht * TH * pl.P.nwt * TW);
+    // the window pair (8 x 32 or 8 x 64 voxels) must not be mostly padding
+    const double used = (double)g.oh * g.ow / ((double)pl.P.nht * pl.TH * pl.P.nwt * TW);
     if (used < 0.55) return false;
     // a run cut inside a column pays two extra input planes: worth it only for runs of some length (shorter ones
     // go to the stacked-plane kernel, which pays a fixed quarter)
@@ -492,27 +513,28 @@ lamp_status_t cr_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, cons
         const cuuint64_t dims[5] = {(cuuint64_t)g.ci, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.d, (cuuint64_t)g.n};
         const cuuint64_t strides[4] = {(cuuint64_t)x.pitch * 2, (cuuint64_t)x.pitch * 2 * g.w,
                                        (cuuint64_t)x.pitch * 2 * g.w * g.h, (cuuint64_t)x.pitch * 2 * g.w * g.h * g.d};
-        const cuuint32_t box[5] = {(cuuint32_t)pl.KC, (cuuint32_t)HALO_W, (cuuint32_t)HALO_H, 1, 1};
+        const cuuint32_t box[5] = {(cuuint32_t)pl.KC, (cuuint32_t)HALO_W, (cuuint32_t)(pl.TH + 2), 1, 1};
         const cuuint32_t es[5] = {1, 1, 1, 1, 1};
         if (encode(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, x.p, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return LAMP_ERR_CUDA;
     }
     {
-        // weights [tap][row = output channel of this pass][k = reduced channel]: one box = one kd block of a tile
-        const cuuint64_t dims[3] = {(cuuint64_t)g.ci, (cuuint64_t)g.co, 27};
-        const cuuint64_t strides[2] = {(cuuint64_t)g.ci * 2, (cuuint64_t)g.ci * 2 * g.co};
-        const cuuint32_t box[3] = {(cuuint32_t)pl.KC, (cuuint32_t)pl.CO, 1};
-        const cuuint32_t es[3] = {1, 1, 1};
-        if (encode(&mw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void *)w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+        // weights [kd][kh][kw][row = output channel of this pass][k = reduced channel] as a 5-D tensor, so that a tap
+        // coordinate outside 0..2 delivers a block of zeros; one box = one (kd, kh, kw) block of a tile
+        const cuuint64_t dims[5] = {(cuuint64_t)g.ci, (cuuint64_t)g.co, 3, 3, 3};
+        const cuuint64_t tapb = (cuuint64_t)g.ci * 2 * g.co;
+        const cuuint64_t strides[4] = {(cuuint64_t)g.ci * 2, tapb, 3 * tapb, 9 * tapb};
+        const cuuint32_t box[5] = {(cuuint32_t)pl.KC, (cuuint32_t)pl.CO, 1, 1, 1};
+        const cuuint32_t es[5] = {1, 1, 1, 1, 1};
+        if (encode(&mw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, (void *)w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return LAMP_ERR_CUDA;
     }
     lamp_status_t s;
-    if (pl.KC == 64 && pl.CO == 64) s = launch_cr<64, 64>(mx, mw, pl, st);
-    else if (pl.KC == 32 && pl.CO == 64) s = launch_cr<32, 64>(mx, mw, pl, st);
-    else if (pl.KC == 64 && pl.CO == 32) s = launch_cr<64, 32>(mx, mw, pl, st);
-    else s = launch_cr<32, 32>(mx, mw, pl, st);
+    if (pl.J == 2) s = launch_cr<32, 32, 2>(mx, mw, pl, st);
+    else if (pl.KC == 64) s = launch_cr<64, 64, 1>(mx, mw, pl, st);
+    else s = launch_cr<32, 64, 1>(mx, mw, pl, st);
     if (s != LAMP_OK) return s;
     return launch_status();
 }

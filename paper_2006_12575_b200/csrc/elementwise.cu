@@ -777,7 +777,7 @@ lamp_status_t k_head_softmax(const TView &z, const bf16 *w, const float *b, int 
                              const uint8_t *labels, double *dice_sums, cudaStream_t st)
 {
     const int64_t Vn = (int64_t)z.d * z.h * z.w;
-    if (K > KMAX || K < 1 || z.c > 64 || z.c % 8) return LAMP_ERR_UNSUPPORTED;
+    if (K > KMAX || K < 1 || z.c > 128 || z.c % 8) return LAMP_ERR_UNSUPPORTED;
     if (dice_sums) LAMP_CUDA_OK(cudaMemsetAsync(dice_sums, 0, (size_t)z.n * K * 3 * sizeof(double), st));
     if (Vn == 0 || z.n == 0) return LAMP_OK;
     if (umma_head_supported(z, K) && ((uintptr_t)w & 15) == 0) return umma_head(z, w, b, K, probs, argmax, labels, dice_sums, st);
@@ -824,7 +824,7 @@ static lamp_status_t launch_head_bwd(const TView &z, const bf16 *w, int K, const
     const size_t tile = (size_t)256 * KP + 256 * K + 128 * C, red = lanes * KP * C + lanes * KP;
     const size_t smem = ((size_t)KP * C + 2 * KP + (tile > red ? tile : red)) * sizeof(float);
     static SmemAttrOnce attr;
-    { const lamp_status_t as = attr.ensure(head_bwd_kernel<KP>, (int)(96 * 1024)); if (as != LAMP_OK) return as; }
+    { const lamp_status_t as = attr.ensure(head_bwd_kernel<KP>, (int)(128 * 1024)); if (as != LAMP_OK) return as; }
     (void)launch_pdl((int64_t)z.n * Vn <= SHORT_ELEMS / 32, head_bwd_kernel<KP>, dim3((unsigned)blocks, z.n), dim3(256), (size_t)(smem), st, 
         (const bf16 *)z.p, z.pitch, C, w, K, probs, labels, dice_sums, z.n, (bf16 *)dz.p, dz.pitch, partW, partB, dlogits,
         Vn, vpb);
@@ -838,7 +838,8 @@ lamp_status_t k_head_bwd(const TView &z, const bf16 *w, int K, const float *prob
 {
     const int64_t Vn = (int64_t)z.d * z.h * z.w;
     const int C = z.c;
-    if (K > KMAX || C > 64 || C % 8) return LAMP_ERR_UNSUPPORTED;
+    // the block's shared memory holds the weights, 256 voxels of z and the lane partials: 107 KB at C = 128, K = 16
+    if (K > KMAX || C > 128 || C % 8) return LAMP_ERR_UNSUPPORTED;
     if (Vn == 0 || z.n == 0) {
         LAMP_CUDA_OK(cudaMemsetAsync(dw, 0, (size_t)K * C * sizeof(float), st));
         if (db) LAMP_CUDA_OK(cudaMemsetAsync(db, 0, (size_t)K * sizeof(float), st));

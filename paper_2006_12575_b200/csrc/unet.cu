@@ -362,7 +362,7 @@ lamp_status_t lamp_unet_create(const lamp_unet_spec_t *spec, lamp_unet_t **out)
     if (spec->in_channels != 1 && (spec->in_channels <= 0 || spec->in_channels % 8)) return LAMP_ERR_UNSUPPORTED;
     for (int l = 0; l < spec->levels; ++l)
         if (spec->channels[l] <= 0 || spec->channels[l] % 8 || spec->channels[l] > 2048) return LAMP_ERR_UNSUPPORTED;
-    if (spec->channels[0] > 64) return LAMP_ERR_UNSUPPORTED;           // head kernel limit
+    if (spec->channels[0] > 128) return LAMP_ERR_UNSUPPORTED;          // the head's backward kernel keeps 256 voxels x channels[0] in shared memory
     if (!(spec->in_eps > 0.f)) return LAMP_ERR_INVALID_ARG;
     lamp_unet *net = new (std::nothrow) lamp_unet;
     if (!net) return LAMP_ERR_INVALID_ARG;

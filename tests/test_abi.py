@@ -62,10 +62,14 @@ def test_workspace_queries_scale_with_the_volume():
 def test_invalid_arguments_are_rejected_on_the_host():
     L = B.lib()
     bad = [B.unet_spec(0, [8]), B.unet_spec(2, [8, 12]), B.unet_spec(2, [8, 16], num_classes=40),
-           B.unet_spec(2, [8, 16], in_channels=3), B.unet_spec(1, [128])]
+           B.unet_spec(2, [8, 16], in_channels=3), B.unet_spec(1, [256])]
     for spec in bad:
         h = C.c_void_p()
         assert L.lamp_unet_create(C.byref(spec), C.byref(h)) in (1, 2)
+    # the widest network of the paper (Sec. 3: 128 filters in the first encoder block) is accepted
+    wide = B.lamp_unet_create(B.unet_spec(5, [128, 256, 512, 1024, 2048], 2, 1, 10))
+    assert B.lamp_unet_weight_count(wide) > 500e6
+    B.lamp_unet_destroy(wide)
     d = B.conv_desc(8, 8, 5, 1, 2)
     t = B.Tensor(16, B.LAMP_BF16, 1, 4, 4, 4, 8, 8, 0)
     assert L.lamp_conv3d_fwd(C.byref(d), C.byref(t), 16, None, C.byref(t), None, None, 0, None) == 2

@@ -60,8 +60,9 @@ CASES = [
     ("r_c64_ragged_batch", 2, 33, 70, 60, 64, 64, 3, 1, 1, 0),
     ("r_c128_to_64", 1, 25, 96, 160, 128, 64, 3, 1, 1, 0),
     ("r_c64_thin_columns", 1, 3, 352, 288, 64, 64, 3, 1, 1, 0),
-    ("r_c32_runs", 1, 40, 96, 136, 32, 32, 3, 1, 1, 0),
-    ("r_c64_to_32_ragged", 1, 37, 90, 140, 64, 32, 3, 1, 1, 0),
+    ("r_c32_runs", 1, 60, 128, 104, 32, 32, 3, 1, 1, 0),
+    ("r_c64_to_32_ragged", 1, 44, 90, 140, 64, 32, 3, 1, 1, 0),
+    ("r_c32_batch_odd_rows", 2, 29, 75, 100, 32, 32, 3, 1, 1, 0),
     ("r_c32_to_64", 1, 30, 128, 104, 32, 64, 3, 1, 1, 0),
     ("deep_512_cube8", 1, 8, 8, 8, 512, 512, 3, 1, 1, 0),
     ("deep_512_to_256_ragged", 2, 3, 5, 7, 512, 256, 3, 1, 1, 0),

@@ -19,7 +19,12 @@ def _sample_points(rs, N, D, H, W, n_rand, n_edge):
     pts = np.stack([rs.integers(0, N, n_rand), rs.integers(0, D, n_rand), rs.integers(0, H, n_rand),
                     rs.integers(0, W, n_rand)], axis=1)
     edge = np.stack([rs.integers(0, N, n_edge)] + [rs.choice([0, 1, n // 2, n - 2, n - 1], n_edge) for n in (D, H, W)], axis=1)
-    return np.concatenate([pts, edge]).astype(np.int32)
+    # voxels anywhere on the six faces: one coordinate pinned to its first or last value
+    face = np.stack([rs.integers(0, N, n_edge), rs.integers(0, D, n_edge), rs.integers(0, H, n_edge), rs.integers(0, W, n_edge)], axis=1)
+    ax = rs.integers(1, 4, n_edge)
+    last = np.array([N, D, H, W])[ax] - 1
+    face[np.arange(n_edge), ax] = np.where(rs.integers(0, 2, n_edge) == 1, last, 0)
+    return np.concatenate([pts, edge, face]).astype(np.int32)
 
 
 def _randn_bf16(shape, seed):
@@ -47,8 +52,9 @@ def test_conv_sweep_layer_at_benchmark_size(C):
     x64 = hx.to(torch.float64).numpy()
     dy64 = hdy.to(torch.float64).numpy()
     w64 = w.astype(np.float64)
-    n_pts = 1200 if C <= 128 else 500
-    pts = _sample_points(rs, 1, D, H, W, n_pts, n_pts // 3)
+    # 1e5 random voxels (every 8 x 32-voxel window of every CTA's run is hit about a dozen times) plus 6000 voxels on
+    # and next to the six faces, edges and corners; 1e4 weight entries (every tap about 370 times)
+    pts = _sample_points(rs, 1, D, H, W, 100000, 6000)
     idx = (pts[:, 0], pts[:, 1], pts[:, 2], pts[:, 3])
     ref = ops.conv3d_fwd_points(x64, w64, None, pts, 3, 1, 1)
     assert_close(host_f64(y[idx]), ops.bf16_round(ref), f"C={C} fwd (sampled)")
@@ -56,7 +62,7 @@ def test_conv_sweep_layer_at_benchmark_size(C):
     wm = np.ascontiguousarray(w64[::-1].transpose(0, 2, 1))
     ref = ops.conv3d_fwd_points(dy64, wm, None, pts, 3, 1, 1)
     assert_close(host_f64(dx[idx]), ops.bf16_round(ref), f"C={C} dgrad (sampled)")
-    ent = np.stack([rs.integers(0, 27, 160), rs.integers(0, C, 160), rs.integers(0, C, 160)], axis=1).astype(np.int32)
+    ent = np.stack([rs.integers(0, 27, 10000), rs.integers(0, C, 10000), rs.integers(0, C, 10000)], axis=1).astype(np.int32)
     ent[:27, 0] = np.arange(27)                      # every tap at least once
     ref = ops.conv3d_wgrad_points(x64, dy64, ent, 3, 1, 1)
     got = host_f64(dw[ent[:, 0], ent[:, 1], ent[:, 2]])
@@ -121,13 +127,15 @@ def _train_step_sampled(levels, ch, cpl, K, dhw, checked, head_planes):
             s = 2 if l.kind == "down" else 1
             y_gpu = _ws_view(wsb, lay_of(i, B.T_Y))
             _, Do, Ho, Wo, _ = y_gpu.shape
-            pts = _sample_points(rs, 1, Do, Ho, Wo, 300, 100)
+            pts = _sample_points(rs, 1, Do, Ho, Wo, 4000, 1000)
             ref = ops.conv3d_fwd_points(x_in, w64, b64, pts, 3, s, 1)
             idx = (pts[:, 0], pts[:, 1], pts[:, 2], pts[:, 3])
             assert_close(host_f64(y_gpu[idx]), ops.bf16_round(ref), f"{name} y (sampled)")
             # weight gradient on sampled entries, from the GPU's own stored dy
             dy_gpu = host_f64(_ws_view(wsb, lay_of(i, B.T_DY)))
-            ent = np.stack([rs.integers(0, 27, 40), rs.integers(0, l.c_out, 40), rs.integers(0, l.c_in, 40)], 1).astype(np.int32)
+            # 2000 entries (the whole tensor for the one-channel first layer): the relative L2 error over a handful
+            # of entries of a gradient whose terms nearly cancel is too noisy an estimate of the tensor's
+            ent = np.stack([rs.integers(0, 27, 2000), rs.integers(0, l.c_out, 2000), rs.integers(0, l.c_in, 2000)], 1).astype(np.int32)
             ref = ops.conv3d_wgrad_points(x_in, dy_gpu, ent, 3, s, 1)
             wo = offs[i][0]
             got = gw_h[wo:wo + wl[i].size].reshape(wl[i].shape)[ent[:, 0], ent[:, 1], ent[:, 2]]
@@ -135,7 +143,7 @@ def _train_step_sampled(levels, ch, cpl, K, dhw, checked, head_planes):
         else:
             u_gpu = _ws_view(wsb, lay_of(i, B.T_OUT))
             _, Do, Ho, Wo, _ = u_gpu.shape
-            pts = _sample_points(rs, 1, Do, Ho, Wo, 300, 100)
+            pts = _sample_points(rs, 1, Do, Ho, Wo, 4000, 1000)
             tap = ((pts[:, 1] & 1) * 2 + (pts[:, 2] & 1)) * 2 + (pts[:, 3] & 1)
             xi = x_in[pts[:, 0], pts[:, 1] // 2, pts[:, 2] // 2, pts[:, 3] // 2]          # [P, ci]
             ref = np.einsum("pi,poi->po", xi, w64[tap]) + b64

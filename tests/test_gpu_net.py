@@ -243,6 +243,15 @@ def test_train_step_wide_unet_every_step_matches_oracle():
     print("wide U-Net:", r)
 
 
+def test_train_step_unet_128_first_level_every_step_matches_oracle():
+    # the paper's widest first level (Sec. 3: 128 filters): head forward and backward on 128 channels
+    D, H, W = 8, 8, 16
+    x = synth.bf16_round(synth.blurred_noise((D, H, W), 1.5, 31))[None, ..., None]
+    lab = synth.labels_blobs((D, H, W), 32, 10, 1.5)[None]
+    r = check_network_layer_by_layer(2, [128, 256], 1, 10, (D, H, W), 3, x, lab)
+    print("U-Net-128:", r)
+
+
 def test_unet_forward_head_argmax_matches_oracle_on_stored_input():
     net, spec, lay, ws, bs, wd, bd, _ = make_net(CFG0["levels"], CFG0["ch"], CFG0["cpl"], CFG0["K"], seed=1)
     x, _ = _cfg0_inputs()
