@@ -178,44 +178,45 @@ conv3_r_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             }
         }
     } else if (warp == 2) {
-        if (lane == 0) {
-            // ---------------------------------------------------------------- weight tiles
-            int ws = 0;
-            uint32_t wph = 0;
-            bool ok = true;
-            PieceWalker pw;
-            Piece pc;
-            pw.init(P);
-            while (ok && pw.next(P, pc, TH)) {
-                const int p_lo = pc.o_lo > 0 ? pc.o_lo - 1 : 0, p_hi = pc.o_hi < P.D ? pc.o_hi : P.D - 1;
-                for (int p = p_lo; p <= p_hi && ok; ++p) {
-                    // kd block of output plane o = p + 1 - kd goes to slot o mod 3 of the tile
-                    const int slot_kd0 = (p + 1) % 3;
-                    for (int c = 0; c < P.chunks && ok; ++c) {
-                        for (int t0 = 0; t0 < NT; t0 += TPS) {
-                            if (!mbar_wait(wempty0 + 8 * ws, wph ^ 1, abort_flag)) { ok = false; break; }
-                            mbar_expect_tx(wfull0 + 8 * ws, WST_BYTES);
-                            const uint32_t dst = smem_u32(w_base + (size_t)ws * WST_BYTES);
-#pragma unroll
-                            for (int ti = 0; ti < TPS; ++ti) {
-                                const int hs = (t0 + ti) / 3, kw = (t0 + ti) % 3;
-#pragma unroll
-                                for (int kd = 0; kd < 3; ++kd) {
-                                    int slot = slot_kd0 - kd;
-                                    if (slot < 0) slot += 3;
-#pragma unroll
-                                    for (int jj = 0; jj < J; ++jj) {
-                                        // block jj reads tap kh = hs - jj; outside 0..2 the coordinate is out of range (zeros).
-                                        // With mirrored taps the window (kd, kh, kw) reads weight tap (2 - kd, 2 - kh, 2 - kw).
-                                        const int kh = hs - jj;
-                                        const bool in = kh >= 0 && kh <= 2;
-                                        tma_load_5d(dst + ti * TILE_BYTES + (slot * J + jj) * BLK_BYTES, &map_w, wfull0 + 8 * ws, c * KC, 0,
-                                                    P.mirror ? 2 - kw : kw, in ? (P.mirror ? 2 - kh : kh) : 3, P.mirror ? 2 - kd : kd);
-                                    }
-                                }
-                            }
-                            if (++ws == P.nw) { ws = 0; wph ^= 1; }
+        // -------------------------------------------------------------------- weight tiles
+        // The whole warp walks the stages; lane 0 waits for the stage and announces its bytes, then lane b issues box b
+        // (one box = the J blocks of one (tile, kd): issuing the boxes of a stage from one thread, one after the
+        // other, made the MMA issuer wait for weights a sixth of the time at 32 channels).
+        constexpr int NBOX = 3 * TPS;
+        const int ti = lane / 3, kd = lane - 3 * ti;            // this lane's box
+        int ws = 0;
+        uint32_t wph = 0;
+        bool ok = true;
+        PieceWalker pw;
+        Piece pc;
+        pw.init(P);
+        while (ok && pw.next(P, pc, TH)) {
+            const int p_lo = pc.o_lo > 0 ? pc.o_lo - 1 : 0, p_hi = pc.o_hi < P.D ? pc.o_hi : P.D - 1;
+            for (int p = p_lo; p <= p_hi && ok; ++p) {
+                // kd block of output plane o = p + 1 - kd goes to slot o mod 3 of the tile
+                int slot = (p + 1) % 3 - kd;
+                if (slot < 0) slot += 3;
+                for (int c = 0; c < P.chunks && ok; ++c) {
+                    for (int t0 = 0; t0 < NT; t0 += TPS) {
+                        bool got = true;
+                        if (lane == 0) {
+                            got = mbar_wait(wempty0 + 8 * ws, wph ^ 1, abort_flag);
+                            if (got) mbar_expect_tx(wfull0 + 8 * ws, WST_BYTES);
                         }
+                        ok = __shfl_sync(0xffffffffu, (int)got, 0) != 0;
+                        if (!ok) break;
+                        if (lane < NBOX) {
+                            // window shift hs serves tap kh = hs - jj of output row jj: the box spans kh = hs - J + 1 .. hs
+                            // (block order jj = J - 1 .. 0); with mirrored taps the window (kd, kh, kw) reads weight tap
+                            // (2 - kd, 2 - kh, 2 - kw), so the box spans 2 - hs .. 2 - hs + J - 1 (block order jj = 0 .. J - 1).
+                            // Taps outside 0..2 are outside the tensor and arrive as zeros.
+                            const int hs = (t0 + ti) / 3, kw = (t0 + ti) % 3;
+                            tma_load_5d(smem_u32(w_base + (size_t)ws * WST_BYTES) + ti * TILE_BYTES + slot * (J * BLK_BYTES), &map_w,
+                                        wfull0 + 8 * ws, c * KC, 0, P.mirror ? 2 - kw : kw, P.mirror ? 2 - hs : hs - J + 1,
+                                        P.mirror ? 2 - kd : kd);
+                        }
+                        __syncwarp();
+                        if (++ws == P.nw) { ws = 0; wph ^= 1; }
                     }
                 }
             }
@@ -299,7 +300,8 @@ conv3_r_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         // J = 1: channels 32 i .. 32 i + 31 of this thread's voxel; J = 2: all 32 channels of the voxel in row hl + i
         auto emit = [&](const Piece &pc, int o, int i32, const uint32_t (&r)[32]) {
             const int c0 = J == 1 ? 32 * i32 : 0;
-            const int h = pc.h0 + hl + (J == 2 ? i32 : 0), w = pc.w0 + wx;
+            // J = 2: the slot's halves are the two output rows in the order the weight box delivered their taps
+            const int h = pc.h0 + hl + (J == 2 ? (P.mirror ? i32 : 1 - i32) : 0), w = pc.w0 + wx;
             const bool valid = h < P.H && w < P.W;
             float v[32];
 #pragma unroll
@@ -521,11 +523,11 @@ lamp_status_t cr_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, cons
     }
     {
         // weights [kd][kh][kw][row = output channel of this pass][k = reduced channel] as a 5-D tensor, so that a tap
-        // coordinate outside 0..2 delivers a block of zeros; one box = one (kd, kh, kw) block of a tile
+        // coordinate outside 0..2 delivers a block of zeros; one box = the J consecutive kh blocks of one (kd, kw)
         const cuuint64_t dims[5] = {(cuuint64_t)g.ci, (cuuint64_t)g.co, 3, 3, 3};
         const cuuint64_t tapb = (cuuint64_t)g.ci * 2 * g.co;
         const cuuint64_t strides[4] = {(cuuint64_t)g.ci * 2, tapb, 3 * tapb, 9 * tapb};
-        const cuuint32_t box[5] = {(cuuint32_t)pl.KC, (cuuint32_t)pl.CO, 1, 1, 1};
+        const cuuint32_t box[5] = {(cuuint32_t)pl.KC, (cuuint32_t)pl.CO, 1, (cuuint32_t)pl.J, 1};
         const cuuint32_t es[5] = {1, 1, 1, 1, 1};
         if (encode(&mw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, (void *)w, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
