@@ -691,10 +691,15 @@ def run_unet_dp(args):
     gw, gb = torch.empty_like(master), torch.empty_like(bmaster)
     ws = torch.empty(B.lamp_unet_workspace_bytes(net, 1, D, H, W, B.MODE_TRAIN), dtype=torch.uint8, device=dev)
 
+    # gradient buckets of about 32 MB that end on layer boundaries; each one's all-reduce starts on its own stream as
+    # soon as the backward pass has finished it
+    offs = [B.lamp_unet_param_layout(net, i)[0] for i in range(B.lamp_unet_num_layers(net))]
+    starts = replicas.plan_buckets(offs, gw.numel(), 8 << 20)
+    events = [torch.cuda.Event() for _ in starts]
+    comm = torch.cuda.Stream()
+
     def step():
-        B.lamp_unet_train_step(net, wd, bmaster, x, lab, loss, gw, gb, None, ws)
-        replicas.allreduce_mean_(gw)
-        replicas.allreduce_mean_(gb)
+        replicas.train_step_overlapped(B, net, wd, bmaster, x, lab, loss, gw, gb, None, ws, starts, events, comm)
         B.lamp_rmsprop_step(gw, master, vw, wd)
         B.lamp_rmsprop_step(gb, bmaster, vb, None)
 
@@ -726,9 +731,84 @@ def run_unet_dp(args):
                    scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
                    config=dict(workload=f"configs[{args.cfg}] U-Net training step + gradient average over {world} replica(s) "
                                         "+ RMSProp update", gradient_bytes=int(gw.numel() + gb.numel()) * 4,
-                               exchange="bucketed all-reduce after the backward pass (not overlapped with it)"),
+                               exchange=f"{len(starts)} buckets, each all-reduced on a second stream as soon as the backward pass "
+                                        "has finished it"),
                    loss_first_last=[round(losses[0], 5), round(losses[-1], 5)] if losses else None)
         print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_sliding_dp(args):
+    """Sliding-window inference of one volume with the patches split over the replicas (one reduction of the class
+    sums and weight totals).  One JSON line from rank 0: voxels of the volume over the slowest rank's time."""
+    import torch
+    import torch.distributed as dist
+    from paper_2006_12575_b200 import binding as B
+    from paper_2006_12575_b200 import build as lamp_build
+    from paper_2006_12575_b200 import replicas, synth
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        lamp_build.build()
+    if world > 1:
+        dist.barrier()
+    cfg = UNET_CFGS[args.cfg]
+    D, H, W = cfg["vol"]
+    K = cfg["K"]
+    patch = (64, 64, 64)
+    net = B.lamp_unet_create(B.unet_spec(cfg["levels"], cfg["ch"], cfg["cpl"], 1, K))
+    g = torch.Generator().manual_seed(10 * args.cfg + 1)
+    wflat = torch.zeros(B.lamp_unet_weight_count(net), dtype=torch.float32)
+    for i in range(B.lamp_unet_num_layers(net)):
+        wo, bo, d = B.lamp_unet_param_layout(net, i)
+        taps = d.ksize ** 3
+        n = taps * d.c_in * d.c_out
+        wflat[wo:wo + n] = torch.randn(n, generator=g) * (2.0 / ((1 if d.transposed else taps) * d.c_in)) ** 0.5
+    wd = wflat.to(dev).to(torch.bfloat16)
+    bd = torch.zeros(B.lamp_unet_bias_count(net), dtype=torch.float32, device=dev)
+    vol = synth.ct_volume((D, H, W), 40) if args.cfg == 4 else synth.blurred_noise((D, H, W), 2.0, 10 * args.cfg)
+    x = torch.from_numpy(vol).to(torch.bfloat16).reshape(1, D, H, W, 1).to(dev)
+    sums = torch.empty((K, D, H, W), dtype=torch.float32, device=dev)
+    wsum = torch.empty((D, H, W), dtype=torch.float32, device=dev)
+    seg = torch.empty(D * H * W, dtype=torch.uint8, device=dev)
+    ws = torch.empty(B.lamp_sliding_window_workspace_bytes(net, D, H, W, patch, 0.25, args.sw_batch), dtype=torch.uint8, device=dev)
+    fn = lambda: replicas.sliding_window_sharded(B, net, wd, bd, x, patch, 0.25, args.sw_batch, 1, sums, wsum, seg, ws)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        fn()
+    sync_all()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        fn()
+    t1.record()
+    sync_all()
+    ms = replicas.job_time_ms(t0.elapsed_time(t1), dev) / args.steps
+    status = B.lamp_get_async_status()
+    if rank == 0:
+        if status != 0:
+            raise SystemExit("device status not ok")
+        print(json.dumps(dict(metric="unet_sliding_window_sharded_voxels_per_s", value=round(D * H * W / (ms * 1e-3), 1),
+                              unit="voxels/s", n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=round(ms, 3),
+                              seconds_per_volume=round(ms * 1e-3, 5), higher_is_better=True, scaling="strong", vs_baseline=None,
+                              dtype="bf16", data="synthetic",
+                              config=dict(workload=f"configs[{args.cfg}] sliding window 64^3, overlap 0.25, gaussian; patches split "
+                                                   f"over {world} replica(s), class sums and weight totals all-reduced",
+                                          patches=B.lamp_sliding_window_num_patches(D, H, W, patch, 0.25),
+                                          sw_batch=args.sw_batch, reduced_bytes=int(sums.numel() + wsum.numel()) * 4))), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
@@ -838,7 +918,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="lamp", choices=["lamp", "reference"])
     ap.add_argument("--channels", default=",".join(str(c) for c in CHANNELS))
-    ap.add_argument("--workload", default="conv_sweep", choices=["conv_sweep", "unet_train", "unet_infer", "sliding", "hbm", "unet_train_dp"])
+    ap.add_argument("--workload", default="conv_sweep", choices=["conv_sweep", "unet_train", "unet_infer", "sliding", "hbm", "unet_train_dp", "sliding_dp"])
     ap.add_argument("--cfg", type=int, default=2)
     ap.add_argument("--sw-batch", type=int, default=32)
     ap.add_argument("--no-graph", action="store_true", help="U-Net workloads: skip the CUDA-graph replay timing")
@@ -849,6 +929,9 @@ def main():
         return
     if args.workload == "unet_train_dp":
         run_unet_dp(args)
+        return
+    if args.workload == "sliding_dp":
+        run_sliding_dp(args)
         return
     if args.workload != "conv_sweep":
         run_unet(args)

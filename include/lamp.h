@@ -241,6 +241,21 @@ lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_b
                                    float *grad_w, float *grad_b, float *probs,
                                    void *ws, size_t ws_bytes, void *cuda_stream);
 
+/* The same step for data-parallel training (Sec. 1: replicas that exchange gradients): the caller cuts grad_w into
+ * n_buckets ranges [bucket_start[b], bucket_start[b+1]) (element offsets, ascending, bucket_start[0] = 0, the last
+ * range ends at the weight count) and passes one CUDA event (a cudaEvent_t as void*) per bucket.  bucket_events[b] is
+ * recorded as soon as every gradient of bucket b has been enqueued - the backward pass finishes the layers last to
+ * first, so the buckets become final from the last to the first, the early ones long before the call's work ends -
+ * and a stream that waits on the event may read (e.g. all-reduce) that range while the rest of the backward pass runs.
+ * The events are recorded on a stream of the library; use them only with cudaStreamWaitEvent / cudaEventSynchronize.
+ * grad_b, loss and probs are final when the work of the call on cuda_stream is.  Otherwise as lamp_unet_train_step. */
+lamp_status_t lamp_unet_train_step_buckets(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                           const lamp_tensor_t *x, const uint8_t *labels, float *loss,
+                                           float *grad_w, float *grad_b, float *probs,
+                                           void *ws, size_t ws_bytes, void *cuda_stream,
+                                           const int64_t *bucket_start /* host */, int32_t n_buckets,
+                                           void *const *bucket_events /* host array */);
+
 /* Sliding-window inference (Sec. 3: patches versus the whole image).  Patch origins per axis are
  * 0, s, 2s, ... with s = round(patch * (1 - overlap)) while the patch fits, plus one patch flush
  * with the border if needed; patches are ordered by origin (d, h, w), w fastest; each patch is a
@@ -257,6 +272,23 @@ lamp_status_t lamp_sliding_window_infer(const lamp_unet_t *net, const void *weig
                                         const lamp_tensor_t *volume, const int32_t patch[3], float overlap,
                                         int32_t sw_batch, int32_t window, float *probs_planar, uint8_t *argmax,
                                         void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Sliding-window inference split over replicas by patch index (Sec. 1, data parallelism; Sec. 3, patches).
+ * lamp_sliding_window_num_patches: patches of the grid (0 for invalid arguments).
+ * lamp_sliding_window_partial runs patches first_patch .. first_patch + num_patches - 1 only and writes THEIR blend
+ * un-normalised: sums_planar fp32 [num_classes][d][h][w] = sum_p w p, weight_sums fp32 [d][h][w] = sum_p w (zeros
+ * where none of these patches covers a voxel); both 16-byte aligned.  Workspace as for lamp_sliding_window_infer.
+ * The caller adds the buffers of all replicas (e.g. an all-reduce), then lamp_sliding_window_finish divides in place
+ * (write_probs != 0) and / or takes the arg max (argmax may be NULL if write_probs).  With one replica holding all
+ * patches the two calls give exactly what lamp_sliding_window_infer gives. */
+int32_t lamp_sliding_window_num_patches(int32_t d, int32_t h, int32_t w, const int32_t patch[3], float overlap);
+lamp_status_t lamp_sliding_window_partial(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                          const lamp_tensor_t *volume, const int32_t patch[3], float overlap,
+                                          int32_t sw_batch, int32_t window, int32_t first_patch, int32_t num_patches,
+                                          float *sums_planar, float *weight_sums, void *ws, size_t ws_bytes,
+                                          void *cuda_stream);
+lamp_status_t lamp_sliding_window_finish(float *sums_planar, const float *weight_sums, int32_t k, int64_t voxels,
+                                         int32_t write_probs, uint8_t *argmax, void *cuda_stream);
 
 /* Weighted overlap-add of per-patch probabilities on its own (the aggregation step of
  * lamp_sliding_window_infer).  patch_probs: fp32 [n_patches][pd*ph*pw][k], patches in the order

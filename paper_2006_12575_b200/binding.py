@@ -73,6 +73,11 @@ def lib():
             "lamp_unet_tensor_layout": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, i32, TP, C.POINTER(sz)]),
             "lamp_unet_forward": (C.c_int, [vp, vp, vp, TP, vp, vp, vp, sz, vp]),
             "lamp_unet_train_step": (C.c_int, [vp, vp, vp, TP, vp, vp, vp, vp, vp, vp, sz, vp]),
+            "lamp_unet_train_step_buckets": (C.c_int, [vp, vp, vp, TP, vp, vp, vp, vp, vp, vp, sz, vp,
+                                                       C.POINTER(C.c_int64), i32, C.POINTER(vp)]),
+            "lamp_sliding_window_num_patches": (i32, [i32, i32, i32, I3, f32]),
+            "lamp_sliding_window_partial": (C.c_int, [vp, vp, vp, TP, I3, f32, i32, i32, i32, i32, vp, vp, vp, sz, vp]),
+            "lamp_sliding_window_finish": (C.c_int, [vp, vp, i32, C.c_int64, i32, vp, vp]),
             "lamp_sliding_window_workspace_bytes": (sz, [vp, i32, i32, i32, I3, f32, i32]),
             "lamp_sliding_window_infer": (C.c_int, [vp, vp, vp, TP, I3, f32, i32, i32, vp, vp, vp, sz, vp]),
             "lamp_overlap_add": (C.c_int, [vp, i32, i32, i32, i32, I3, f32, i32, vp, vp, vp]),
@@ -95,6 +100,8 @@ EXPORTS = ["lamp_conv3d_workspace_bytes", "lamp_conv3d_workspace_min_bytes", "la
            "lamp_instnorm_relu_fwd", "lamp_instnorm_relu_bwd", "lamp_unet_create", "lamp_unet_destroy",
            "lamp_unet_num_layers", "lamp_unet_weight_count", "lamp_unet_bias_count", "lamp_unet_param_layout",
            "lamp_unet_workspace_bytes", "lamp_unet_tensor_layout", "lamp_unet_forward", "lamp_unet_train_step",
+           "lamp_unet_train_step_buckets", "lamp_sliding_window_num_patches", "lamp_sliding_window_partial",
+           "lamp_sliding_window_finish",
            "lamp_sliding_window_workspace_bytes", "lamp_sliding_window_infer", "lamp_overlap_add",
            "lamp_rmsprop_step", "lamp_get_async_status", "lamp_selftest_wait_timeout", "lamp_status_string", "lamp_version"]
 
@@ -243,8 +250,40 @@ def lamp_unet_train_step(net, weights, biases, x, labels, loss, grad_w, grad_b, 
            "lamp_unet_train_step")
 
 
+def lamp_unet_train_step_buckets(net, weights, biases, x, labels, loss, grad_w, grad_b, probs, ws, bucket_start, bucket_events):
+    """bucket_start: ascending element offsets into grad_w (first 0); bucket_events: one torch.cuda.Event per bucket,
+    recorded by the library when that range of grad_w is final."""
+    p, nbytes = _ws(ws)
+    n = len(bucket_start)
+    for e in bucket_events:
+        if not e.cuda_event:                 # torch creates the CUDA event lazily, on the first record
+            e.record()
+    starts = (C.c_int64 * n)(*[int(v) for v in bucket_start])
+    events = (C.c_void_p * n)(*[int(e.cuda_event) for e in bucket_events])
+    _check(lib().lamp_unet_train_step_buckets(net, _ptr(weights), _ptr(biases), C.byref(_td(x)), _ptr(labels), _ptr(loss),
+                                              _ptr(grad_w), _ptr(grad_b), _ptr(probs), p, nbytes, _stream(), starts, n, events),
+           "lamp_unet_train_step_buckets")
+
+
 def _i3(v):
     return (C.c_int32 * 3)(*v)
+
+
+def lamp_sliding_window_num_patches(d, h, w, patch, overlap):
+    return lib().lamp_sliding_window_num_patches(d, h, w, _i3(patch), overlap)
+
+
+def lamp_sliding_window_partial(net, weights, biases, volume, patch, overlap, sw_batch, window, first_patch, num_patches,
+                                sums_planar, weight_sums, ws):
+    p, nbytes = _ws(ws)
+    _check(lib().lamp_sliding_window_partial(net, _ptr(weights), _ptr(biases), C.byref(_td(volume)), _i3(patch), overlap,
+                                             sw_batch, window, first_patch, num_patches, _ptr(sums_planar),
+                                             _ptr(weight_sums), p, nbytes, _stream()), "lamp_sliding_window_partial")
+
+
+def lamp_sliding_window_finish(sums_planar, weight_sums, k, voxels, write_probs, argmax):
+    _check(lib().lamp_sliding_window_finish(_ptr(sums_planar), _ptr(weight_sums), k, voxels, 1 if write_probs else 0,
+                                            _ptr(argmax), _stream()), "lamp_sliding_window_finish")
 
 
 def lamp_sliding_window_workspace_bytes(net, d, h, w, patch, overlap, sw_batch):

@@ -223,9 +223,14 @@ lamp_status_t k_rmsprop(int64_t n, const float *g, float *w, float *v, bf16 *wb,
                         cudaStream_t st);
 lamp_status_t k_gather_patches(const TView &vol, const TView &patches, int first_patch, const int32_t nst[3],
                                const int32_t stride[3], cudaStream_t st);
+// p_count < 0: all patches, normalised result (planar may be NULL) and arg max.  Otherwise pp holds the patches
+// p_first .. p_first + p_count - 1 only; with wsum_out the un-normalised sums of those go to planar and their weight
+// totals to wsum_out [d][h][w] (k_overlap_finish divides and takes the arg max once all shares have been added).
 lamp_status_t k_overlap_add(const float *pp, int K, int D, int H, int W, const int32_t patch[3],
                             const int32_t nst[3], const int32_t stride[3], int window, float *planar,
-                            uint8_t *argmax, cudaStream_t st);
+                            uint8_t *argmax, cudaStream_t st, int p_first = 0, int p_count = -1, float *wsum_out = nullptr);
+lamp_status_t k_overlap_finish(float *planar, const float *wsum, int K, int64_t V, int write_probs, uint8_t *argmax,
+                               cudaStream_t st);
 
 // api.cu: shape checks + kernel selection for one conv pass (used by the ABI and by the U-Net executor)
 lamp_status_t conv_geom(const lamp_conv_desc_t *desc, const lamp_tensor_t *in, const lamp_tensor_t *out, ConvGeom *g);

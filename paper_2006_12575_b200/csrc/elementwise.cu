@@ -581,7 +581,8 @@ template <int VEC, int KT>
 __global__ void __launch_bounds__(256)
 overlap_add_kernel(const float *__restrict__ pp, int Krt, int D, int H, int W, int PD, int PH, int PW,
                    int nd, int nh, int nw, int sd, int sh, int sw, int window, int aligned4,
-                   float *__restrict__ planar, uint8_t *__restrict__ amax)
+                   float *__restrict__ planar, uint8_t *__restrict__ amax, int p_first, int p_count,
+                   float *__restrict__ wsum_out)
 {
     pdl_launch_dependents();
     pdl_wait();
@@ -624,7 +625,10 @@ overlap_add_kernel(const float *__restrict__ pp, int Krt, int D, int H, int W, i
             for (int iw = 0; iw < nw; ++iw) {
                 const int ow = patch_origin(iw, nw, sw, W, PW);
                 if (w0 + VEC - 1 < ow || w0 >= ow + PW) continue;
-                const int64_t pi = ((int64_t)id * nh + ih) * nw + iw;
+                // only patches p_first .. p_first + p_count - 1 take part (pp holds those, back to back)
+                const int64_t pg = ((int64_t)id * nh + ih) * nw + iw;
+                if (pg < p_first || pg >= (int64_t)p_first + p_count) continue;
+                const int64_t pi = pg - p_first;
                 const float wdh = td[d - od] * th[h - oh];
                 if (VEC == 4 && KT > 0 && aligned4) {
                     // origins and extents are multiples of 4: the four voxels lie inside the patch together
@@ -666,6 +670,20 @@ overlap_add_kernel(const float *__restrict__ pp, int Krt, int D, int H, int W, i
     }
     const int64_t v0 = ((int64_t)d * H + h) * W + w0;
     const int64_t plane = (int64_t)D * H * W;
+    if (wsum_out) {
+        // partial result of a share of the patches: the weighted sums as they are and the weight totals; the
+        // division and the arg max follow once the shares have been added (overlap_finish_kernel)
+#pragma unroll
+        for (int k = 0; k < KMAX; ++k) {
+            if (k < K) {
+                if (VEC == 4) *reinterpret_cast<float4 *>(planar + k * plane + v0) = make_float4(acc[0][k], acc[1][k], acc[2][k], acc[3][k]);
+                else          planar[k * plane + v0] = acc[0][k];
+            }
+        }
+        if (VEC == 4) *reinterpret_cast<float4 *>(wsum_out + v0) = make_float4(wsum[0], wsum[1], wsum[2], wsum[3]);
+        else          wsum_out[v0] = wsum[0];
+        return;
+    }
     uint8_t am[VEC];
 #pragma unroll
     for (int i = 0; i < VEC; ++i) {
@@ -693,6 +711,27 @@ overlap_add_kernel(const float *__restrict__ pp, int Krt, int D, int H, int W, i
         if (VEC == 4) *reinterpret_cast<uchar4 *>(amax + v0) = make_uchar4(am[0], am[1], am[2], am[3]);
         else          amax[v0] = am[0];
     }
+}
+
+// A[k][v] = acc[k][v] / wsum[v] in place (the same two operations as the one-pass kernel: reciprocal, multiply);
+// arg max over k, lowest index on ties.
+__global__ void __launch_bounds__(256)
+overlap_finish_kernel(float *__restrict__ planar, const float *__restrict__ wsum, int K, int64_t V, int write_probs,
+                      uint8_t *__restrict__ amax)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int64_t v = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (v >= V) return;
+    const float inv = 1.0f / wsum[v];
+    float best = -1.f;
+    int am = 0;
+    for (int k = 0; k < K; ++k) {
+        const float a = planar[k * V + v] * inv;
+        if (write_probs) planar[k * V + v] = a;
+        if (a > best) { best = a; am = k; }
+    }
+    if (amax) amax[v] = (uint8_t)am;
 }
 
 }  // namespace
@@ -883,20 +922,32 @@ lamp_status_t k_gather_patches(const TView &vol, const TView &patches, int first
     return launch_status();
 }
 
-lamp_status_t k_overlap_add(const float *pp, int K, int D, int H, int W, const int32_t patch[3],
-                            const int32_t nst[3], const int32_t stride[3], int window, float *planar,
-                            uint8_t *argmax, cudaStream_t st)
+lamp_status_t k_overlap_finish(float *planar, const float *wsum, int K, int64_t V, int write_probs, uint8_t *argmax,
+                               cudaStream_t st)
 {
     if (K > KMAX || K < 1) return LAMP_ERR_UNSUPPORTED;
+    if (V == 0) return LAMP_OK;
+    (void)launch_pdl(V <= SHORT_ELEMS / 32, overlap_finish_kernel, dim3((unsigned)((V + 255) / 256)), dim3(256), (size_t)0, st,
+                     planar, wsum, K, V, write_probs, argmax);
+    return launch_status();
+}
+
+lamp_status_t k_overlap_add(const float *pp, int K, int D, int H, int W, const int32_t patch[3],
+                            const int32_t nst[3], const int32_t stride[3], int window, float *planar,
+                            uint8_t *argmax, cudaStream_t st, int p_first, int p_count, float *wsum_out)
+{
+    if (K > KMAX || K < 1) return LAMP_ERR_UNSUPPORTED;
+    if (p_count < 0) { p_first = 0; p_count = nst[0] * nst[1] * nst[2]; }
+    if (wsum_out && !planar) return LAMP_ERR_INVALID_ARG;
     if ((int64_t)D * H * W == 0) return LAMP_OK;
     const size_t smem = (size_t)(patch[0] + patch[1] + patch[2]) * sizeof(float);
-    const bool vec = (W % 4 == 0) && ((uintptr_t)planar % 16 == 0) && ((uintptr_t)argmax % 4 == 0);
+    const bool vec = (W % 4 == 0) && ((uintptr_t)planar % 16 == 0) && ((uintptr_t)argmax % 4 == 0) && ((uintptr_t)wsum_out % 16 == 0);
     const int aligned4 = vec && patch[2] % 4 == 0 && (nst[2] == 1 || stride[2] % 4 == 0) && (W - patch[2]) % 4 == 0 &&
                          ((uintptr_t)pp % 16 == 0);
 #define LAMP_OA(VECN, KTN)                                                                                              \
     (void)launch_pdl(total <= SHORT_ELEMS / 32, overlap_add_kernel<VECN, KTN>, dim3((unsigned)((total + 255) / 256)), dim3(256), (size_t)(smem), st,                                 \
         pp, K, D, H, W, patch[0], patch[1], patch[2], nst[0], nst[1], nst[2], stride[0], stride[1], stride[2], window, \
-        aligned4, planar, argmax)
+        aligned4, planar, argmax, p_first, p_count, wsum_out)
     if (vec) {
         const int64_t total = (int64_t)D * H * (W / 4);
         switch (aligned4 ? K : 0) {

@@ -483,13 +483,20 @@ lamp_status_t lamp_unet_forward(const lamp_unet_t *net, const void *weights_bf16
                        (cudaStream_t)cuda_stream);
 }
 
-lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
-                                   const lamp_tensor_t *x, const uint8_t *labels, float *loss,
-                                   float *grad_w, float *grad_b, float *probs,
-                                   void *ws, size_t ws_bytes, void *cuda_stream)
+// bucket_start / bucket_events: see lamp_unet_train_step_buckets (n_buckets = 0: none)
+static lamp_status_t train_step_impl(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                     const lamp_tensor_t *x, const uint8_t *labels, float *loss,
+                                     float *grad_w, float *grad_b, float *probs,
+                                     void *ws, size_t ws_bytes, void *cuda_stream,
+                                     const int64_t *bucket_start, int32_t n_buckets, void *const *bucket_events)
 {
     if (!weights_bf16 || !biases_f32 || !labels || !loss || !grad_w || !grad_b) return LAMP_ERR_INVALID_ARG;
     TRY(check_input(net, x));
+    if (n_buckets < 0 || (n_buckets > 0 && (!bucket_start || !bucket_events))) return LAMP_ERR_INVALID_ARG;
+    for (int b = 0; b < n_buckets; ++b) {
+        if (!bucket_events[b] || bucket_start[b] < 0 || (size_t)bucket_start[b] >= net->n_w) return LAMP_ERR_INVALID_ARG;
+        if (b == 0 ? bucket_start[0] != 0 : bucket_start[b] <= bucket_start[b - 1]) return LAMP_ERR_INVALID_ARG;
+    }
     if (!ws || ((uintptr_t)ws & 255)) return LAMP_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const lamp_unet_spec_t &S = net->spec;
@@ -511,6 +518,23 @@ lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_b
         LAMP_CUDA_OK(cudaStreamWaitEvent(sd, net->ev_fork, 0));
     }
     lamp_status_t rs = LAMP_OK;
+    // Buckets of grad_w whose last contribution has been enqueued get their event recorded: the layers are visited
+    // last to first and their weights lie in layer order, so once the layer at offset `done_from` is enqueued every
+    // bucket that starts at or behind it is final.  The weight gradients run on the side stream (the head's on the
+    // caller's stream: `on_main`), so that is where the events go.
+    int buckets_left = n_buckets;
+    auto mark_final = [&](size_t done_from, bool on_main) -> lamp_status_t {
+        if (buckets_left == 0 || (size_t)bucket_start[buckets_left - 1] < done_from) return LAMP_OK;
+        if (on_main && two) {
+            LAMP_CUDA_OK(cudaEventRecord(net->ev_dy, st));
+            LAMP_CUDA_OK(cudaStreamWaitEvent(sd, net->ev_dy, 0));
+        }
+        while (buckets_left > 0 && (size_t)bucket_start[buckets_left - 1] >= done_from) {
+            LAMP_CUDA_OK(cudaEventRecord((cudaEvent_t)bucket_events[buckets_left - 1], sd));
+            --buckets_left;
+        }
+        return LAMP_OK;
+    };
     auto body = [&]() -> lamp_status_t {
         for (size_t i = 1; i < net->layers.size(); ++i) {
             if (net->layers[i].kind == K_HEAD) continue;
@@ -531,6 +555,7 @@ lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_b
             float *dw = grad_w + Ly.w_off, *db = grad_b + Ly.b_off;
             if (Ly.kind == K_HEAD) {
                 TRY(k_head_bwd(B.in, w, S.num_classes, probs, labels, P.dice, B.din, dw, db, nullptr, P.scratch, P.scratch_bytes, st));
+                TRY(mark_final(Ly.w_off, true));
                 continue;
             }
             if (Ly.kind != K_UP)
@@ -543,6 +568,7 @@ lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_b
                 LAMP_CUDA_OK(cudaStreamWaitEvent(sd, net->ev_dy, 0));
             }
             TRY(conv_wgrad(B.g, B.in, B.dy, dw, Ly.kind == K_UP ? db : nullptr, P.scratch_side, P.scratch_side_bytes, sd));
+            TRY(mark_final(Ly.w_off, false));
             if (i == 0) break;
             TRY(conv_dgrad_run(B.g, B.dy, w, P.wt[i], B.din, P.scratch, P.scratch_bytes, st));
         }
@@ -555,6 +581,25 @@ lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_b
         if (!j && rs == LAMP_OK) rs = LAMP_ERR_CUDA;
     }
     return rs;
+}
+
+lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                   const lamp_tensor_t *x, const uint8_t *labels, float *loss,
+                                   float *grad_w, float *grad_b, float *probs,
+                                   void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    return train_step_impl(net, weights_bf16, biases_f32, x, labels, loss, grad_w, grad_b, probs, ws, ws_bytes, cuda_stream,
+                           nullptr, 0, nullptr);
+}
+
+lamp_status_t lamp_unet_train_step_buckets(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                           const lamp_tensor_t *x, const uint8_t *labels, float *loss,
+                                           float *grad_w, float *grad_b, float *probs,
+                                           void *ws, size_t ws_bytes, void *cuda_stream,
+                                           const int64_t *bucket_start, int32_t n_buckets, void *const *bucket_events)
+{
+    return train_step_impl(net, weights_bf16, biases_f32, x, labels, loss, grad_w, grad_b, probs, ws, ws_bytes, cuda_stream,
+                           bucket_start, n_buckets, bucket_events);
 }
 
 static void window_grid(int len, int patch, float overlap, int32_t *nst, int32_t *stride)
@@ -598,12 +643,16 @@ size_t lamp_sliding_window_workspace_bytes(const lamp_unet_t *net, int32_t d, in
     return total;
 }
 
-lamp_status_t lamp_sliding_window_infer(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+// Patches first_patch .. first_patch + num_patches - 1 of the grid (num_patches < 0: all of them): forward pass of each,
+// then the blend.  wsum == NULL: normalised probabilities and arg max; otherwise the un-normalised sums and weight totals
+// of these patches alone.
+static lamp_status_t sliding_window_run(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
                                         const lamp_tensor_t *volume, const int32_t patch[3], float overlap,
-                                        int32_t sw_batch, int32_t window, float *probs_planar, uint8_t *argmax,
+                                        int32_t sw_batch, int32_t window, int32_t first_patch, int32_t num_patches,
+                                        float *probs_planar, float *wsum, uint8_t *argmax,
                                         void *ws, size_t ws_bytes, void *cuda_stream)
 {
-    if (!weights_bf16 || !biases_f32 || !volume || !volume->ptr || (!argmax && !probs_planar)) return LAMP_ERR_INVALID_ARG;
+    if (!weights_bf16 || !biases_f32 || !volume || !volume->ptr) return LAMP_ERR_INVALID_ARG;
     if (volume->n != 1 || volume->dtype != LAMP_BF16 || volume->c != (net ? net->spec.in_channels : 0)) return LAMP_ERR_INVALID_ARG;
     TRY(sw_check(net, volume->d, volume->h, volume->w, patch, overlap, sw_batch));
     if (!ws || ((uintptr_t)ws & 255)) return LAMP_ERR_WORKSPACE;
@@ -616,6 +665,8 @@ lamp_status_t lamp_sliding_window_infer(const lamp_unet_t *net, const void *weig
     window_grid(volume->h, patch[1], overlap, &nst[1], &str[1]);
     window_grid(volume->w, patch[2], overlap, &nst[2], &str[2]);
     const int np = nst[0] * nst[1] * nst[2];
+    if (num_patches < 0) { first_patch = 0; num_patches = np; }
+    if (first_patch < 0 || first_patch + num_patches > np) return LAMP_ERR_INVALID_ARG;
     const size_t pv = (size_t)patch[0] * patch[1] * patch[2];
     char *p = (char *)ws;
     float *pprobs = (float *)p;
@@ -624,17 +675,60 @@ lamp_status_t lamp_sliding_window_infer(const lamp_unet_t *net, const void *weig
     p += align_up((size_t)sw_batch * pv * S.in_channels * sizeof(bf16), 256);
     void *nws = p;
     TView vol = make_view(volume);
-    for (int first = 0; first < np; first += sw_batch) {
-        const int b = np - first < sw_batch ? np - first : sw_batch;
+    const int end = first_patch + num_patches;
+    for (int first = first_patch; first < end; first += sw_batch) {
+        const int b = end - first < sw_batch ? end - first : sw_batch;
         TView pt = view(pin, b, patch[0], patch[1], patch[2], S.in_channels, S.in_channels, 0);
         TRY(k_gather_patches(vol, pt, first, nst, str, st));
         Plan P;
         make_plan(net, nws, pin, S.in_channels, b, patch[0], patch[1], patch[2], LAMP_MODE_INFER, false, &P);
-        TRY(run_forward(net, P, (const bf16 *)weights_bf16, biases_f32, pprobs + (size_t)first * pv * S.num_classes,
+        TRY(run_forward(net, P, (const bf16 *)weights_bf16, biases_f32, pprobs + (size_t)(first - first_patch) * pv * S.num_classes,
                         nullptr, nullptr, nullptr, st));
     }
     return k_overlap_add(pprobs, S.num_classes, volume->d, volume->h, volume->w, patch, nst, str, window,
-                         probs_planar, argmax, st);
+                         probs_planar, argmax, st, first_patch, num_patches, wsum);
+}
+
+lamp_status_t lamp_sliding_window_infer(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                        const lamp_tensor_t *volume, const int32_t patch[3], float overlap,
+                                        int32_t sw_batch, int32_t window, float *probs_planar, uint8_t *argmax,
+                                        void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!argmax && !probs_planar) return LAMP_ERR_INVALID_ARG;
+    return sliding_window_run(net, weights_bf16, biases_f32, volume, patch, overlap, sw_batch, window, 0, -1, probs_planar,
+                              nullptr, argmax, ws, ws_bytes, cuda_stream);
+}
+
+int32_t lamp_sliding_window_num_patches(int32_t d, int32_t h, int32_t w, const int32_t patch[3], float overlap)
+{
+    if (!patch || !(overlap >= 0.f && overlap < 1.f)) return 0;
+    const int dims[3] = {d, h, w};
+    int n = 1;
+    for (int a = 0; a < 3; ++a) {
+        if (patch[a] <= 0 || patch[a] > dims[a]) return 0;
+        int32_t nst, str;
+        window_grid(dims[a], patch[a], overlap, &nst, &str);
+        n *= nst;
+    }
+    return n;
+}
+
+lamp_status_t lamp_sliding_window_partial(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                          const lamp_tensor_t *volume, const int32_t patch[3], float overlap,
+                                          int32_t sw_batch, int32_t window, int32_t first_patch, int32_t num_patches,
+                                          float *sums_planar, float *weight_sums, void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!sums_planar || !weight_sums || num_patches < 0) return LAMP_ERR_INVALID_ARG;
+    if (((uintptr_t)sums_planar | (uintptr_t)weight_sums) & 15) return LAMP_ERR_INVALID_ARG;
+    return sliding_window_run(net, weights_bf16, biases_f32, volume, patch, overlap, sw_batch, window, first_patch, num_patches,
+                              sums_planar, weight_sums, nullptr, ws, ws_bytes, cuda_stream);
+}
+
+lamp_status_t lamp_sliding_window_finish(float *sums_planar, const float *weight_sums, int32_t k, int64_t voxels,
+                                         int32_t write_probs, uint8_t *argmax, void *cuda_stream)
+{
+    if (!sums_planar || !weight_sums || voxels < 0 || (!write_probs && !argmax)) return LAMP_ERR_INVALID_ARG;
+    return k_overlap_finish(sums_planar, weight_sums, k, voxels, write_probs, argmax, (cudaStream_t)cuda_stream);
 }
 
 lamp_status_t lamp_overlap_add(const float *patch_probs, int32_t k, int32_t d, int32_t h, int32_t w,

@@ -437,3 +437,96 @@ def test_train_step_replayed_from_a_cuda_graph_matches_the_eager_call():
         assert_close(w1[wo:wo + n], w0[wo:wo + n], f"layer {i} dW, graph vs eager", rel=1e-5, mx=1e-4)
     assert np.abs(b1 - b0).max() <= 1e-4 * max(np.abs(b0).max(), 1e-6) + 1e-7
     B.lamp_unet_destroy(net)
+
+
+def test_train_step_with_bucket_events_equals_the_plain_step_and_events_mark_final_ranges():
+    """lamp_unet_train_step_buckets (the data-parallel form): same gradients as lamp_unet_train_step; a stream that
+    waits for bucket b's event and copies that range of grad_w gets its final values although the copy is enqueued
+    before the step has finished; the buckets end on layer boundaries."""
+    from paper_2006_12575_b200 import replicas
+    net, spec, lay, ws, bs, wd, bd, offs = make_net(3, [32, 64, 128], 2, 4, 41)
+    D = H = W = 16
+    x = dev_bf16(synth.bf16_round(synth.blurred_noise((D, H, W), 1.5, 42))[None, ..., None])
+    lab = torch.from_numpy(synth.labels_quartiles((D, H, W), 43, 4)[None]).cuda().reshape(-1)
+    nw, nb = B.lamp_unet_weight_count(net), B.lamp_unet_bias_count(net)
+    wsb = torch.empty(B.lamp_unet_workspace_bytes(net, 1, D, H, W, B.MODE_TRAIN), dtype=torch.uint8, device="cuda")
+    loss0 = torch.zeros(1, dtype=torch.float32, device="cuda")
+    gw0 = torch.full((nw,), 7.0, dtype=torch.float32, device="cuda")
+    gb0 = torch.full((nb,), 7.0, dtype=torch.float32, device="cuda")
+    B.lamp_unet_train_step(net, wd, bd, x, lab, loss0, gw0, gb0, None, wsb)
+    torch.cuda.synchronize()
+    starts = replicas.plan_buckets([o[0] for o in offs], nw, 200000)
+    assert len(starts) >= 3 and set(starts) <= {o[0] for o in offs}
+    ends = starts[1:] + [nw]
+    events = [torch.cuda.Event() for _ in starts]
+    loss1 = torch.zeros(1, dtype=torch.float32, device="cuda")
+    gw1 = torch.full((nw,), float("nan"), dtype=torch.float32, device="cuda")
+    gb1 = torch.full((nb,), 7.0, dtype=torch.float32, device="cuda")
+    copies = [torch.full((e - s,), float("nan"), dtype=torch.float32, device="cuda") for s, e in zip(starts, ends)]
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    B.lamp_unet_train_step_buckets(net, wd, bd, x, lab, loss1, gw1, gb1, None, wsb, starts, events)
+    for b in range(len(starts) - 1, -1, -1):
+        side.wait_event(events[b])
+        with torch.cuda.stream(side):
+            copies[b].copy_(gw1[starts[b]:ends[b]])
+    torch.cuda.synchronize()
+    assert B.lamp_get_async_status() == 0
+    assert abs(float(loss1.item()) - float(loss0.item())) <= 1e-6 * abs(float(loss0.item()))
+    for b, (s, e) in enumerate(zip(starts, ends)):
+        assert torch.equal(copies[b], gw1[s:e]), f"bucket {b} was not final when its event fired"
+    for i, l in enumerate(lay):
+        wo, bo = offs[i]
+        n = ws[i].size
+        assert_close(host_f64(gw1[wo:wo + n]), host_f64(gw0[wo:wo + n]), f"layer {i} dW, bucket form vs plain", rel=1e-5, mx=1e-4)
+    assert np.abs(host_f64(gb1) - host_f64(gb0)).max() <= 1e-4 * max(np.abs(host_f64(gb0)).max(), 1e-6) + 1e-7
+    # the single-replica glue: nothing to exchange, the buffers hold the step's own gradients
+    gw2 = torch.empty_like(gw1)
+    gb2 = torch.empty_like(gb1)
+    replicas.train_step_overlapped(B, net, wd, bd, x, lab, loss1, gw2, gb2, None, wsb, starts, events, torch.cuda.Stream())
+    torch.cuda.synchronize()
+    assert_close(host_f64(gw2), host_f64(gw0), "overlapped step, one replica", rel=1e-5, mx=1e-4)
+    # invalid bucket lists are refused on the host
+    for bad in ([1, 5], [0, 5, 5], [0, nw]):
+        with pytest.raises(B.LampError) as e:
+            B.lamp_unet_train_step_buckets(net, wd, bd, x, lab, loss1, gw1, gb1, None, wsb, bad, events[:len(bad)])
+        assert e.value.status == 1
+    B.lamp_unet_destroy(net)
+
+
+def test_patch_sharded_sliding_window_one_replica_is_bit_identical_and_two_shares_add_up():
+    from paper_2006_12575_b200 import replicas
+    net, spec, lay, ws, bs, wd, bd, _ = make_net(2, [8, 16], 1, 3, seed=9)
+    D, H, W, P, K = 12, 8, 12, (8, 8, 8), 3
+    vol = dev_bf16(synth.bf16_round(synth.ct_volume((D, H, W), 21))[None, ..., None])
+    n_p = B.lamp_sliding_window_num_patches(D, H, W, P, 0.25)
+    assert n_p == len(O.window_starts(D, 8, 0.25)) * len(O.window_starts(H, 8, 0.25)) * len(O.window_starts(W, 8, 0.25)) == 4
+    wsb = torch.empty(B.lamp_sliding_window_workspace_bytes(net, D, H, W, P, 0.25, 3), dtype=torch.uint8, device="cuda")
+    planar = torch.empty((K, D, H, W), dtype=torch.float32, device="cuda")
+    am = torch.empty((D * H * W,), dtype=torch.uint8, device="cuda")
+    B.lamp_sliding_window_infer(net, wd, bd, vol, P, 0.25, 3, 1, planar, am, wsb)
+    # one replica: the sharded path is the same arithmetic
+    sums = torch.empty_like(planar)
+    wsum = torch.empty((D, H, W), dtype=torch.float32, device="cuda")
+    am1 = torch.empty_like(am)
+    replicas.sliding_window_sharded(B, net, wd, bd, vol, P, 0.25, 3, 1, sums, wsum, am1, wsb, write_probs=True)
+    assert torch.equal(sums, planar) and torch.equal(am1, am)
+    # two shares computed one after the other and added, as two replicas' all-reduce would
+    parts = []
+    for r in range(2):
+        mine = replicas.shard_patches(n_p, r, 2)
+        s_r = torch.full_like(planar, float("nan"))
+        w_r = torch.full_like(wsum, float("nan"))
+        B.lamp_sliding_window_partial(net, wd, bd, vol, P, 0.25, 3, 1, mine.start, len(mine), s_r, w_r, wsb)
+        parts.append((s_r, w_r))
+    s2, w2 = parts[0][0] + parts[1][0], parts[0][1] + parts[1][1]
+    assert torch.isfinite(s2).all() and (w2 > 0).all()
+    am2 = torch.empty_like(am)
+    B.lamp_sliding_window_finish(s2, w2, K, D * H * W, True, am2)
+    assert_close(host_f64(s2), host_f64(planar), "two shares vs one pass", rel=1e-6, mx=1e-6)
+    agree, strict, near = tie_aware_agreement(am2.cpu().numpy(), host_f64(planar).reshape(K, -1).T)
+    assert agree == 1.0
+    assert B.lamp_get_async_status() == 0
+    with pytest.raises(B.LampError):
+        B.lamp_sliding_window_partial(net, wd, bd, vol, P, 0.25, 3, 1, 3, 2, s2, w2, wsb)      # range beyond the grid
+    B.lamp_unet_destroy(net)
