@@ -142,6 +142,35 @@ lamp_status_t lamp_conv3d_wgrad(const lamp_conv_desc_t *desc, const lamp_tensor_
                                 float *dw, float *dbias, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /* ------------------------------------------------------------------------
+ * Squeeze-and-excitation residual block: the SEU-Net variant of the network (Sec. 1 and Sec. 3 name a "3D SEU-Net"
+ * after AnatomyNet; Tables 2, 3 and 5 report it; the paper does not define the block).  Reading: at the end of a
+ * level's conv stack, with z = relu((y - mu) * rstd) of the level's LAST conv (y its stored raw output, mu_rstd as
+ * written by lamp_instnorm_relu_fwd) and r = the output of the level's FIRST conv -> InstanceNorm -> ReLU,
+ *     s[n,c] = mean over voxels of z,  h = relu(W1 s + b1),  e = sigmoid(W2 h + b2),  out = r + e[n,c] * z.
+ * W1 fp32 [cr][c], b1 fp32 [cr], W2 fp32 [c][cr], b2 fp32 [c]; e, mean fp32 [n][c]; hidden fp32 [n][cr].
+ * Tensors are bf16 with c a multiple of 8 (c <= 2048), channel slices allowed; z is never stored.
+ * Forward:  lamp_se_squeeze (sums: fp64 [n][c], overwritten with sum_v z) -> lamp_se_excite -> lamp_se_apply_fwd
+ *           (residual may be NULL: out = e * z).
+ * Backward: lamp_se_bwd_reduce (de_sums: fp64 [n][c] = sum_v dout * z) -> lamp_se_excite_bwd (ds_over_v fp32 [n][c],
+ *           and the gradients of W1, b1, W2, b2, summed over the samples) -> lamp_se_apply_bwd (dz = e * dout +
+ *           ds_over_v, bf16: the incoming gradient of the last conv's lamp_instnorm_relu_bwd).  The residual branch's
+ *           gradient is dout itself (the second gradient source of the first conv's lamp_instnorm_relu_bwd).
+ * ---------------------------------------------------------------------- */
+lamp_status_t lamp_se_squeeze(const lamp_tensor_t *y, const float *mu_rstd, double *sums, void *cuda_stream);
+lamp_status_t lamp_se_excite(const double *sums, int64_t voxels_per_sample, int32_t n, int32_t c, int32_t cr,
+                             const float *w1, const float *b1, const float *w2, const float *b2,
+                             float *e, float *hidden, float *mean, void *cuda_stream);
+lamp_status_t lamp_se_apply_fwd(const lamp_tensor_t *y, const float *mu_rstd, const float *e,
+                                const lamp_tensor_t *residual, lamp_tensor_t *out, void *cuda_stream);
+lamp_status_t lamp_se_bwd_reduce(const lamp_tensor_t *dout, const lamp_tensor_t *y, const float *mu_rstd,
+                                 double *de_sums, void *cuda_stream);
+lamp_status_t lamp_se_excite_bwd(const double *de_sums, int64_t voxels_per_sample, int32_t n, int32_t c, int32_t cr,
+                                 const float *e, const float *hidden, const float *mean, const float *w1, const float *w2,
+                                 float *ds_over_v, float *dw1, float *db1, float *dw2, float *db2, void *cuda_stream);
+lamp_status_t lamp_se_apply_bwd(const lamp_tensor_t *dout, const float *e, const float *ds_over_v, lamp_tensor_t *dz,
+                                void *cuda_stream);
+
+/* ------------------------------------------------------------------------
  * Normalisation steps of a block (exported so they can be checked alone).
  * ---------------------------------------------------------------------- */
 

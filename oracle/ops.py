@@ -243,3 +243,49 @@ def dice_loss_grad_logits(p, labels, eps=1e-5):
     Den = (p.sum(axis=ax) + g.sum(axis=ax)).reshape(sh) + eps
     dp = -(2 * g / Den - (2 * I + eps) / Den ** 2) / (N * K)
     return p * (dp - (p * dp).sum(axis=-1, keepdims=True))
+
+
+# ----------------------------------------------------------------------------
+# Squeeze-and-excitation residual block (the SEU-Net of Sec. 1 / Sec. 3, Tables 2, 3, 5)
+# ----------------------------------------------------------------------------
+# The paper names the network ("3D SEU-Net", after AnatomyNet) and never defines the block; the cited paper is not
+# at hand.  Reading used here (stated in full in the design doc): at the end of a level's conv stack, with
+#   r = output of the level's FIRST conv -> InstanceNorm -> ReLU (the residual branch; absent for one conv per level),
+#   z = output of the level's LAST  conv -> InstanceNorm -> ReLU,
+#   s[n,c] = mean over voxels of z                       (squeeze)
+#   h = relu(W1 s + b1),  e = sigmoid(W2 h + b2)         (excitation; W1 [C/ratio, C], W2 [C, C/ratio])
+#   out = r + e[n,c] * z                                 (channel rescale + residual; >= 0, so no further ReLU)
+def se_excite(s, W1, b1, W2, b2):
+    """s [N,C] -> (e [N,C], h [N,Cr])."""
+    s = _f64(s)
+    h = np.maximum(s @ _f64(W1).T + _f64(b1), 0.0)
+    t = h @ _f64(W2).T + _f64(b2)
+    return 1.0 / (1.0 + np.exp(-t)), h
+
+
+def se_block_fwd(z, r, W1, b1, W2, b2):
+    """z, r [N,D,H,W,C] (r may be None).  Returns (out, cache)."""
+    z = _f64(z)
+    s = z.mean(axis=(1, 2, 3))
+    e, h = se_excite(s, W1, b1, W2, b2)
+    out = e[:, None, None, None, :] * z
+    if r is not None:
+        out = out + _f64(r)
+    return out, dict(z=z, s=s, e=e, h=h, W1=_f64(W1), W2=_f64(W2))
+
+
+def se_block_bwd(dout, cache):
+    """Gradient of se_block_fwd.  Returns (dz, dr, dW1, db1, dW2, db2); dr is dout itself."""
+    dout = _f64(dout)
+    z, s, e, h, W1, W2 = (cache[k] for k in ("z", "s", "e", "h", "W1", "W2"))
+    V = z.shape[1] * z.shape[2] * z.shape[3]
+    de = (dout * z).sum(axis=(1, 2, 3))                    # [N,C]
+    dt = de * e * (1.0 - e)                                # through the sigmoid
+    dW2 = dt.T @ h
+    db2 = dt.sum(axis=0)
+    dh = (dt @ W2) * (h > 0)
+    dW1 = dh.T @ s
+    db1 = dh.sum(axis=0)
+    ds = dh @ W1                                           # [N,C], gradient w.r.t. the channel means
+    dz = e[:, None, None, None, :] * dout + (ds / V)[:, None, None, None, :]
+    return dz, dout, dW1, db1, dW2, db2

@@ -63,6 +63,12 @@ def lib():
             "lamp_conv3d_wgrad": (C.c_int, [DP, TP, TP, vp, vp, vp, sz, vp]),
             "lamp_instnorm_relu_fwd": (C.c_int, [TP, vp, f32, vp, TP, vp]),
             "lamp_instnorm_relu_bwd": (C.c_int, [TP, TP, TP, vp, vp, TP, vp]),
+            "lamp_se_squeeze": (C.c_int, [TP, vp, vp, vp]),
+            "lamp_se_excite": (C.c_int, [vp, C.c_int64, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
+            "lamp_se_apply_fwd": (C.c_int, [TP, vp, vp, TP, TP, vp]),
+            "lamp_se_bwd_reduce": (C.c_int, [TP, TP, vp, vp, vp]),
+            "lamp_se_excite_bwd": (C.c_int, [vp, C.c_int64, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
+            "lamp_se_apply_bwd": (C.c_int, [TP, vp, vp, TP, vp]),
             "lamp_unet_create": (C.c_int, [SP, C.POINTER(vp)]),
             "lamp_unet_destroy": (None, [vp]),
             "lamp_unet_num_layers": (i32, [vp]),
@@ -97,7 +103,9 @@ def lib():
 
 EXPORTS = ["lamp_conv3d_workspace_bytes", "lamp_conv3d_workspace_min_bytes", "lamp_conv3d_fwd", "lamp_conv3d_dgrad", "lamp_conv3d_dgrad_static_scratch",
            "lamp_conv3d_wgrad",
-           "lamp_instnorm_relu_fwd", "lamp_instnorm_relu_bwd", "lamp_unet_create", "lamp_unet_destroy",
+           "lamp_instnorm_relu_fwd", "lamp_instnorm_relu_bwd",
+           "lamp_se_squeeze", "lamp_se_excite", "lamp_se_apply_fwd", "lamp_se_bwd_reduce", "lamp_se_excite_bwd", "lamp_se_apply_bwd",
+           "lamp_unet_create", "lamp_unet_destroy",
            "lamp_unet_num_layers", "lamp_unet_weight_count", "lamp_unet_bias_count", "lamp_unet_param_layout",
            "lamp_unet_workspace_bytes", "lamp_unet_tensor_layout", "lamp_unet_forward", "lamp_unet_train_step",
            "lamp_unet_train_step_buckets", "lamp_sliding_window_num_patches", "lamp_sliding_window_partial",
@@ -300,6 +308,35 @@ def lamp_sliding_window_infer(net, weights, biases, volume, patch, overlap, sw_b
 def lamp_overlap_add(patch_probs, k, d, h, w, patch, overlap, window, probs_planar, argmax):
     _check(lib().lamp_overlap_add(_ptr(patch_probs), k, d, h, w, _i3(patch), overlap, window, _ptr(probs_planar),
                                   _ptr(argmax), _stream()), "lamp_overlap_add")
+
+
+def lamp_se_squeeze(y, mu_rstd, sums):
+    _check(lib().lamp_se_squeeze(C.byref(_td(y)), _ptr(mu_rstd), _ptr(sums), _stream()), "lamp_se_squeeze")
+
+
+def lamp_se_excite(sums, voxels_per_sample, n, c, cr, w1, b1, w2, b2, e, hidden, mean):
+    _check(lib().lamp_se_excite(_ptr(sums), voxels_per_sample, n, c, cr, _ptr(w1), _ptr(b1), _ptr(w2), _ptr(b2), _ptr(e),
+                                _ptr(hidden), _ptr(mean), _stream()), "lamp_se_excite")
+
+
+def lamp_se_apply_fwd(y, mu_rstd, e, residual, out):
+    _check(lib().lamp_se_apply_fwd(C.byref(_td(y)), _ptr(mu_rstd), _ptr(e), C.byref(_td(residual)) if residual is not None else None,
+                                   C.byref(_td(out)), _stream()), "lamp_se_apply_fwd")
+
+
+def lamp_se_bwd_reduce(dout, y, mu_rstd, de_sums):
+    _check(lib().lamp_se_bwd_reduce(C.byref(_td(dout)), C.byref(_td(y)), _ptr(mu_rstd), _ptr(de_sums), _stream()),
+           "lamp_se_bwd_reduce")
+
+
+def lamp_se_excite_bwd(de_sums, voxels_per_sample, n, c, cr, e, hidden, mean, w1, w2, ds_over_v, dw1, db1, dw2, db2):
+    _check(lib().lamp_se_excite_bwd(_ptr(de_sums), voxels_per_sample, n, c, cr, _ptr(e), _ptr(hidden), _ptr(mean), _ptr(w1),
+                                    _ptr(w2), _ptr(ds_over_v), _ptr(dw1), _ptr(db1), _ptr(dw2), _ptr(db2), _stream()),
+           "lamp_se_excite_bwd")
+
+
+def lamp_se_apply_bwd(dout, e, ds_over_v, dz):
+    _check(lib().lamp_se_apply_bwd(C.byref(_td(dout)), _ptr(e), _ptr(ds_over_v), C.byref(_td(dz)), _stream()), "lamp_se_apply_bwd")
 
 
 def lamp_rmsprop_step(grad, master, v, param_bf16=None, lr=1e-3, alpha=0.99, eps=1e-8):

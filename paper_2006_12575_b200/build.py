@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblamp.so")
-SOURCES = ["api.cu", "unet.cu", "conv_simt.cu", "conv_umma.cu", "conv_t.cu", "conv_r.cu", "conv_c1_umma.cu", "wgrad_umma.cu", "wgrad_win.cu", "elementwise.cu", "static_scratch.cu"]
+SOURCES = ["api.cu", "unet.cu", "conv_simt.cu", "conv_umma.cu", "conv_t.cu", "conv_r.cu", "conv_c1_umma.cu", "wgrad_umma.cu", "wgrad_win.cu", "elementwise.cu", "se_block.cu", "static_scratch.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC"]
