@@ -267,6 +267,25 @@ def run_gpu(args):
     if status != 0:
         raise SystemExit(f"bench.py: device status {status}")
 
+    # The same passes once more, one channel count at a time (its three passes repeated back to back).  In the step above
+    # the narrow layers' 2 ms follow 15 ms of C = 256 at the power cap and inherit that phase's SM clock; here every
+    # channel count runs at the clock its own load settles at.  Reported beside `passes`, not instead of it.
+    alone_events = []
+    for C in chans:
+        b = devb[C]
+        for it in range(3 + 10):
+            marks = [ev() for _ in range(4)]
+            marks[0].record()
+            B.lamp_conv3d_fwd(b["desc"], b["x"], b["w"], None, b["y"])
+            marks[1].record()
+            B.lamp_conv3d_dgrad(b["desc"], b["dy"], b["w"], b["dx"], b["ws"])
+            marks[2].record()
+            B.lamp_conv3d_wgrad(b["desc"], b["x"], b["dy"], b["dw"], None, b["ws"])
+            marks[3].record()
+            if it >= 3:
+                alone_events.append((C, marks))
+    sync_all()
+
     # end to end through the same calls with host buffers: H2D of x, dy, w and D2H of y, dx, dw every step.
     # Copies run on their own streams so that the transfers of one channel count overlap the kernels of another.
     cur = torch.cuda.current_stream()
@@ -340,6 +359,15 @@ def run_gpu(args):
         tf = pass_flops(C) / (mean * 1e-3) / 1e12
         passes[f"C{C}.{name}"] = dict(ms=round(mean, 4), tflops=round(tf, 1), pct_nominal=round(100 * tf / NOMINAL_BF16_TFLOPS, 1),
                                       pct_measured=round(100 * tf / peaks["bf16"], 1))
+    per_alone = {}
+    for C, m in alone_events:
+        for name, a, b_ in (("fwd", m[0], m[1]), ("dgrad", m[1], m[2]), ("wgrad", m[2], m[3])):
+            per_alone.setdefault((C, name), []).append(a.elapsed_time(b_))
+    passes_alone = {}
+    for (C, name), v in per_alone.items():
+        mean = sum(v) / len(v)
+        tf = pass_flops(C) / (mean * 1e-3) / 1e12
+        passes_alone[f"C{C}.{name}"] = dict(ms=round(mean, 4), tflops=round(tf, 1), pct_nominal=round(100 * tf / NOMINAL_BF16_TFLOPS, 1))
     # kernel families (one CUDA kernel template each); the dgrad pass also holds the tiny weight-transpose launch
     cmax = max(chans)
     # (C >= 128: conv3_t_kernel; C = 64: conv3_r_kernel)
@@ -425,6 +453,7 @@ def run_gpu(args):
                         steps=e2e_steps),
                gpu_launches=args.steps * len(chans) * launches_per_C,
                roofline=roofline, cpu_baseline=cpu, passes=passes,
+               passes_one_channel_count_at_a_time=passes_alone,
                pct_of_nominal_bf16=round(100 * value / world / NOMINAL_BF16_TFLOPS, 2))
     if unet is not None:
         out["unet"] = unet

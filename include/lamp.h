@@ -171,7 +171,9 @@ lamp_status_t lamp_se_apply_bwd(const lamp_tensor_t *dout, const float *e, const
                                 void *cuda_stream);
 
 /* ------------------------------------------------------------------------
- * Normalisation steps of a block (exported so they can be checked alone).
+ * Normalisation steps of a block.  No passage of the paper defines them (it gives the network's
+ * topology only, Sec. 2.2); they are the steps between the convolutions of every block of this
+ * library's U-Net and are exported so that each can be checked against the oracle on its own.
  * ---------------------------------------------------------------------- */
 
 /* z = max(0, (y - mu) * rstd) per (n, c), mu = S1/V, rstd = (S2/V - mu^2 + eps)^-1/2 with
@@ -205,11 +207,18 @@ typedef struct {
     int32_t in_channels;       /* 1, or a multiple of 8                    */
     int32_t num_classes;       /* 2..16                                    */
     float   in_eps;
+    int32_t se_ratio;          /* 0: plain U-Net.  > 0: SEU-Net variant - every level's conv stack ends in the squeeze-and-
+                                  excitation residual step described above (hidden units = width / se_ratio, at least 1);
+                                  needs convs_per_level = 2 (the residual branch is the first conv's output)     */
 } lamp_unet_spec_t;
 
 typedef struct lamp_unet lamp_unet_t;          /* opaque, host-only plan */
 
 lamp_status_t lamp_unet_create(const lamp_unet_spec_t *spec, lamp_unet_t **out);
+/* SEU-Net variant: where the squeeze-and-excitation parameters of `layer` (a level's last conv) sit in the BIAS buffer
+ * (fp32): from *se_off, W1 [cr][c], b1 [cr], W2 [c][cr], b2 [c] back to back, c = the layer's c_out, *cr hidden units;
+ * their gradients sit at the same offsets of grad_b.  *cr = 0 for layers without the step. */
+lamp_status_t lamp_unet_se_layout(const lamp_unet_t *net, int32_t layer, size_t *se_off, int32_t *cr);
 void          lamp_unet_destroy(lamp_unet_t *net);
 int32_t       lamp_unet_num_layers(const lamp_unet_t *net);
 /* Elements of the flat bf16 weight buffer / of the flat fp32 bias buffer. */
@@ -222,7 +231,8 @@ lamp_status_t lamp_unet_param_layout(const lamp_unet_t *net, int32_t layer, size
 enum { LAMP_MODE_INFER = 0, LAMP_MODE_TRAIN = 1 };
 size_t lamp_unet_workspace_bytes(const lamp_unet_t *net, int32_t n, int32_t d, int32_t h, int32_t w, int32_t mode);
 
-/* Where a pass keeps one of its tensors inside the workspace, for inspection after the call.
+/* Where a pass keeps one of its tensors inside the workspace, for inspection after the call
+ * (no passage of the paper: exported so that tests can check every step of a pass on its own).
  * Training mode keeps every tensor listed; inference mode keeps LAMP_T_IN / LAMP_T_OUT only (the
  * raw conv output is a buffer shared by all layers there).  On success *offset is the byte offset
  * from the workspace base to the tensor's first element (the slice's first channel) and *out
@@ -320,7 +330,7 @@ lamp_status_t lamp_sliding_window_finish(float *sums_planar, const float *weight
                                          int32_t write_probs, uint8_t *argmax, void *cuda_stream);
 
 /* Weighted overlap-add of per-patch probabilities on its own (the aggregation step of
- * lamp_sliding_window_infer).  patch_probs: fp32 [n_patches][pd*ph*pw][k], patches in the order
+ * lamp_sliding_window_infer, Sec. 3; no passage of its own: exported for testing).  patch_probs: fp32 [n_patches][pd*ph*pw][k], patches in the order
  * above for a d x h x w volume. */
 lamp_status_t lamp_overlap_add(const float *patch_probs, int32_t k, int32_t d, int32_t h, int32_t w,
                                const int32_t patch[3], float overlap, int32_t window,

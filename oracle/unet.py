@@ -27,6 +27,13 @@ these tensors as bf16, everything else is kept at full precision):
   fp32, and z = relu((y_stored - mu) * rstd) is stored rounded;
   the up-conv output; every activation gradient handed between layers.
 Logits, probabilities, the loss, weight and bias gradients are never rounded.
+
+SEU-Net variant (spec.se_ratio > 0; Sec. 1 and Sec. 3 name it, the block is this build's reading, ops.se_block_fwd):
+the last conv of every level produces z = relu((y_stored - mu) * rstd) WITHOUT storing it, and the level's output is
+out = r + e * z with r the stored output of the level's first conv and e the excitation of the channel means of z;
+out is stored rounded, and in the backward pass dz = e * dout + ds / V is stored rounded before the InstanceNorm
+backward; s, h, e and the squeeze-and-excitation parameters (se[i] = (W1, b1, W2, b2) per such layer) are fp32 values
+held in fp64 here.
 """
 from __future__ import annotations
 
@@ -46,6 +53,7 @@ class UNetSpec:
     in_channels: int = 1
     num_classes: int = 4
     eps: float = 1e-5
+    se_ratio: int = 0      # > 0: SEU-Net variant, hidden units = width // se_ratio (at least 1); needs convs_per_level = 2
 
 
 @dataclass
@@ -57,6 +65,7 @@ class Layer:
     c_out: int
     taps: int
     fan_in: int
+    se_cr: int = 0     # > 0: this conv ends its level's stack with a squeeze-and-excitation residual step (ops.se_block_fwd)
 
 
 def unet_layers(spec: UNetSpec) -> List[Layer]:
@@ -77,6 +86,12 @@ def unet_layers(spec: UNetSpec) -> List[Layer]:
             out.append(Layer(f"dec{l}.conv{j}", "conv", l, c, ch[l], 27, 27 * c))
             c = ch[l]
     out.append(Layer("head", "head", 0, ch[0], spec.num_classes, 1, ch[0]))
+    if spec.se_ratio > 0:
+        if spec.convs_per_level != 2:
+            raise ValueError("the squeeze-and-excitation residual block is defined for two convs per level")
+        for ly in out:
+            if ly.kind == "conv" and ly.name.endswith(".conv1"):
+                ly.se_cr = max(1, ly.c_out // spec.se_ratio)
     return out
 
 
@@ -96,9 +111,9 @@ def _norm_conv_fwd(x, w, b, stride, eps, quantise):
     return z, dict(x=x, ys=ys, mu=mu, rstd=rstd, stride=stride)
 
 
-def forward(spec: UNetSpec, weights, biases, x, quantise=True, want_cache=False):
+def forward(spec: UNetSpec, weights, biases, x, quantise=True, want_cache=False, se=None):
     """x [N,D,H,W,Cin] float64 (bf16-valued when quantise).  Returns probs [N,D,H,W,K]
-    (and the per-layer cache when want_cache)."""
+    (and the per-layer cache when want_cache).  se: per layer (W1, b1, W2, b2) or None (SEU-Net variant)."""
     lay = unet_layers(spec)
     cache = [None] * len(lay)
     skips = {}
@@ -106,7 +121,13 @@ def forward(spec: UNetSpec, weights, biases, x, quantise=True, want_cache=False)
     for i, ly in enumerate(lay):
         w, b = weights[i], biases[i]
         if ly.kind in ("conv", "down"):
+            r = a
             a, cache[i] = _norm_conv_fwd(a, w, b, 2 if ly.kind == "down" else 1, spec.eps, quantise)
+            if ly.se_cr:
+                c = cache[i]
+                z = ops.instnorm_relu_fwd(c["ys"], c["mu"], c["rstd"])          # not stored, hence not rounded
+                out, c["se"] = ops.se_block_fwd(z, r, *se[i])
+                a = _q(out, quantise)
             nxt = lay[i + 1]
             if ly.name.startswith("enc") and nxt.kind == "down":
                 skips[ly.level] = a                     # E_l, used by the down conv and by the skip
@@ -121,10 +142,13 @@ def forward(spec: UNetSpec, weights, biases, x, quantise=True, want_cache=False)
     return (a, cache) if want_cache else a
 
 
-def train_step(spec: UNetSpec, weights, biases, x, labels, quantise=True):
-    """One forward + backward pass.  Returns (loss, dweights, dbiases, probs)."""
+def train_step(spec: UNetSpec, weights, biases, x, labels, quantise=True, se=None):
+    """One forward + backward pass.  Returns (loss, dweights, dbiases, probs), and as a fifth item the gradients of the
+    squeeze-and-excitation parameters per layer when se is given."""
     lay = unet_layers(spec)
-    probs, cache = forward(spec, weights, biases, x, quantise, want_cache=True)
+    probs, cache = forward(spec, weights, biases, x, quantise, want_cache=True, se=se)
+    dSE = [None] * len(lay)
+    res_grad = {}
     loss = ops.dice_loss(probs, labels)
     dW = [None] * len(lay)
     dB = [None] * len(lay)
@@ -139,6 +163,15 @@ def train_step(spec: UNetSpec, weights, biases, x, labels, quantise=True):
         elif ly.kind in ("conv", "down"):
             if ly.name.startswith("enc") and lay[i + 1].kind == "down":
                 g = g + skip_grad.pop(ly.level)         # fan-in at E_l: down-conv path + skip path
+                if ly.se_cr:
+                    g = _q(g, quantise)                 # the summed gradient is stored: three steps read it
+            if ly.se_cr:
+                dz, dr, dW1, db1, dW2, db2 = ops.se_block_bwd(g, c["se"])
+                dSE[i] = (dW1, db1, dW2, db2)
+                res_grad[i - 1] = dr                    # the residual branch: the level's first conv also receives dout
+                g = _q(dz, quantise)
+            if i in res_grad:
+                g = g + res_grad.pop(i)
             dy = _q(ops.instnorm_relu_bwd(g, c["ys"], c["mu"], c["rstd"]), quantise)
             dW[i], dB[i] = ops.conv3d_wgrad(c["x"], dy, 3, c["stride"], 1)
             if i > 0:
@@ -150,6 +183,8 @@ def train_step(spec: UNetSpec, weights, biases, x, labels, quantise=True):
         else:                                           # up conv: no norm, no activation
             dW[i], dB[i] = ops.convT3d_wgrad(c["x"], g, 2, 2)
             g = _q(ops.convT3d_dgrad(g, w, c["x"].shape[1:4], 2, 2), quantise)
+    if se is not None:
+        return loss, dW, dB, probs, dSE
     return loss, dW, dB, probs
 
 

@@ -38,7 +38,7 @@ class ConvDesc(C.Structure):
 
 class UNetSpec(C.Structure):
     _fields_ = [("levels", C.c_int32), ("channels", C.c_int32 * 8), ("convs_per_level", C.c_int32),
-                ("in_channels", C.c_int32), ("num_classes", C.c_int32), ("in_eps", C.c_float)]
+                ("in_channels", C.c_int32), ("num_classes", C.c_int32), ("in_eps", C.c_float), ("se_ratio", C.c_int32)]
 
 
 _lib = None
@@ -70,6 +70,7 @@ def lib():
             "lamp_se_excite_bwd": (C.c_int, [vp, C.c_int64, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
             "lamp_se_apply_bwd": (C.c_int, [TP, vp, vp, TP, vp]),
             "lamp_unet_create": (C.c_int, [SP, C.POINTER(vp)]),
+            "lamp_unet_se_layout": (C.c_int, [vp, i32, C.POINTER(sz), C.POINTER(i32)]),
             "lamp_unet_destroy": (None, [vp]),
             "lamp_unet_num_layers": (i32, [vp]),
             "lamp_unet_weight_count": (sz, [vp]),
@@ -105,7 +106,7 @@ EXPORTS = ["lamp_conv3d_workspace_bytes", "lamp_conv3d_workspace_min_bytes", "la
            "lamp_conv3d_wgrad",
            "lamp_instnorm_relu_fwd", "lamp_instnorm_relu_bwd",
            "lamp_se_squeeze", "lamp_se_excite", "lamp_se_apply_fwd", "lamp_se_bwd_reduce", "lamp_se_excite_bwd", "lamp_se_apply_bwd",
-           "lamp_unet_create", "lamp_unet_destroy",
+           "lamp_unet_create", "lamp_unet_se_layout", "lamp_unet_destroy",
            "lamp_unet_num_layers", "lamp_unet_weight_count", "lamp_unet_bias_count", "lamp_unet_param_layout",
            "lamp_unet_workspace_bytes", "lamp_unet_tensor_layout", "lamp_unet_forward", "lamp_unet_train_step",
            "lamp_unet_train_step_buckets", "lamp_sliding_window_num_patches", "lamp_sliding_window_partial",
@@ -195,9 +196,9 @@ def lamp_instnorm_relu_bwd(dz_a, dz_b, y, mu_rstd, sums, dy):
                                         C.byref(_td(dy)), _stream()), "lamp_instnorm_relu_bwd")
 
 
-def unet_spec(levels, channels, convs_per_level=2, in_channels=1, num_classes=4, eps=1e-5) -> UNetSpec:
+def unet_spec(levels, channels, convs_per_level=2, in_channels=1, num_classes=4, eps=1e-5, se_ratio=0) -> UNetSpec:
     ch = (C.c_int32 * 8)(*(list(channels) + [0] * (8 - len(channels))))
-    return UNetSpec(levels, ch, convs_per_level, in_channels, num_classes, eps)
+    return UNetSpec(levels, ch, convs_per_level, in_channels, num_classes, eps, se_ratio)
 
 
 def lamp_unet_create(spec: UNetSpec):
@@ -226,6 +227,12 @@ def lamp_unet_param_layout(net, layer):
     wo, bo, d = C.c_size_t(), C.c_size_t(), ConvDesc()
     _check(lib().lamp_unet_param_layout(net, layer, C.byref(wo), C.byref(bo), C.byref(d)), "lamp_unet_param_layout")
     return wo.value, bo.value, d
+
+
+def lamp_unet_se_layout(net, layer):
+    off, cr = C.c_size_t(), C.c_int32()
+    _check(lib().lamp_unet_se_layout(net, layer, C.byref(off), C.byref(cr)), "lamp_unet_se_layout")
+    return off.value, cr.value
 
 
 def lamp_unet_workspace_bytes(net, n, d, h, w, mode):

@@ -232,6 +232,16 @@ lamp_status_t k_overlap_add(const float *pp, int K, int D, int H, int W, const i
 lamp_status_t k_overlap_finish(float *planar, const float *wsum, int K, int64_t V, int write_probs, uint8_t *argmax,
                                cudaStream_t st);
 
+// se_block.cu: the squeeze-and-excitation residual block's steps for the U-Net executor (params: W1 [cr][c], b1 [cr],
+// W2 [c][cr], b2 [c] back to back in fp32, dparams likewise), mu / rstd from the InstanceNorm sums, out = a + b
+lamp_status_t k_mu_rstd(const double *stats, int64_t Vn, float eps, float *mr, int nc, cudaStream_t st);
+lamp_status_t k_add2(const TView &a, const TView &b, const TView &out, cudaStream_t st);
+lamp_status_t k_se_fwd(const TView &y, const float *mr, const float *params, int cr, double *sums, float *e, float *hid,
+                       float *mean, const TView *res, const TView &out, cudaStream_t st);
+lamp_status_t k_se_bwd(const TView &dout, const TView &y, const float *mr, const float *params, int cr, const float *e,
+                       const float *hid, const float *mean, double *de, float *dsv, float *dparams, const TView &dz,
+                       cudaStream_t st);
+
 // api.cu: shape checks + kernel selection for one conv pass (used by the ABI and by the U-Net executor)
 lamp_status_t conv_geom(const lamp_conv_desc_t *desc, const lamp_tensor_t *in, const lamp_tensor_t *out, ConvGeom *g);
 size_t        conv_ws_bytes(const ConvGeom &g, int pass);       // scratch with which the pass runs fastest

@@ -195,6 +195,41 @@ se_excite_bwd_kernel(const double *__restrict__ de_sums, double inv_v, int N, in
     }
 }
 
+// mu = S1 / V, rstd = (S2 / V - mu^2 + eps)^-1/2 from the fp64 sums, as the normalise kernel derives them
+__global__ void __launch_bounds__(SE_THREADS)
+mu_rstd_kernel(const double *__restrict__ stats, double inv_v, float eps, float *__restrict__ mr, int nc)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int i = blockIdx.x * SE_THREADS + threadIdx.x;
+    if (i >= nc) return;
+    const double m = stats[2 * i] * inv_v;
+    double var = stats[2 * i + 1] * inv_v - m * m;
+    if (var < 0.0) var = 0.0;
+    mr[2 * i] = (float)m;
+    mr[2 * i + 1] = __frsqrt_rn((float)var + eps);
+}
+
+// out = a + b (bf16, fp32 add)
+__global__ void __launch_bounds__(SE_THREADS)
+add2_kernel(const bf16 *__restrict__ a, int64_t ap, const bf16 *__restrict__ b, int64_t bp, bf16 *__restrict__ o, int64_t op,
+            int C, int64_t total)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int G = C >> 3;
+    const int64_t t = (int64_t)blockIdx.x * SE_THREADS + threadIdx.x;
+    if (t >= total) return;
+    const int cg = (int)(t % G);
+    const int64_t vox = t / G;
+    float fa[8], fb[8];
+    unpack8(__ldg(reinterpret_cast<const uint4 *>(a + vox * ap) + cg), fa);
+    unpack8(__ldg(reinterpret_cast<const uint4 *>(b + vox * bp) + cg), fb);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) fa[i] += fb[i];
+    reinterpret_cast<uint4 *>(o + vox * op)[cg] = pack8(fa);
+}
+
 bool se_tensor_ok(const lamp_tensor_t *t)
 {
     return t && t->ptr && t->dtype == LAMP_BF16 && t->c > 0 && t->c % 8 == 0 && t->c_pitch % 8 == 0 && t->c_offset % 8 == 0 &&
@@ -234,7 +269,69 @@ lamp_status_t se_reduce(int mode, const lamp_tensor_t *y, const lamp_tensor_t *g
     return launch_status();
 }
 
+lamp_tensor_t as_tensor(const TView &v)
+{
+    lamp_tensor_t t;
+    t.ptr = v.p; t.dtype = LAMP_BF16; t.n = v.n; t.d = v.d; t.h = v.h; t.w = v.w; t.c = v.c; t.c_pitch = v.pitch; t.c_offset = 0;
+    return t;
+}
+
 }  // namespace
+
+lamp_status_t k_mu_rstd(const double *stats, int64_t Vn, float eps, float *mr, int nc, cudaStream_t st)
+{
+    if (nc <= 0 || Vn <= 0) return LAMP_OK;
+    (void)launch_pdl(true, mu_rstd_kernel, dim3((nc + SE_THREADS - 1) / SE_THREADS), dim3(SE_THREADS), (size_t)0, st, stats,
+                     1.0 / (double)Vn, eps, mr, nc);
+    return launch_status();
+}
+
+lamp_status_t k_add2(const TView &a, const TView &b, const TView &out, cudaStream_t st)
+{
+    const int64_t total = (int64_t)a.n * a.d * a.h * a.w * (a.c / 8);
+    if (total == 0) return LAMP_OK;
+    if (a.c % 8 || a.pitch % 8 || b.pitch % 8 || out.pitch % 8) return LAMP_ERR_UNSUPPORTED;
+    (void)launch_pdl(false, add2_kernel, dim3((unsigned)((total + SE_THREADS - 1) / SE_THREADS)), dim3(SE_THREADS), (size_t)0, st,
+                     (const bf16 *)a.p, a.pitch, (const bf16 *)b.p, b.pitch, (bf16 *)out.p, out.pitch, a.c, total);
+    return launch_status();
+}
+
+// params: W1 [cr][c], b1 [cr], W2 [c][cr], b2 [c] back to back (fp32); dparams likewise
+lamp_status_t k_se_fwd(const TView &y, const float *mr, const float *params, int cr, double *sums, float *e, float *hid,
+                       float *mean, const TView *res, const TView &out, cudaStream_t st)
+{
+    const lamp_tensor_t ty = as_tensor(y), to = as_tensor(out);
+    lamp_tensor_t tr{};
+    if (res) tr = as_tensor(*res);
+    const int c = y.c;
+    const int64_t Vn = (int64_t)y.d * y.h * y.w;
+    if (Vn == 0 || y.n == 0) return LAMP_OK;
+    const float *w1 = params, *b1 = w1 + (size_t)cr * c, *w2 = b1 + cr, *b2 = w2 + (size_t)c * cr;
+    lamp_status_t s = lamp_se_squeeze(&ty, mr, sums, st);
+    if (s != LAMP_OK) return s;
+    s = lamp_se_excite(sums, Vn, y.n, c, cr, w1, b1, w2, b2, e, hid, mean, st);
+    if (s != LAMP_OK) return s;
+    lamp_tensor_t tout = to;
+    return lamp_se_apply_fwd(&ty, mr, e, res ? &tr : nullptr, &tout, st);
+}
+
+lamp_status_t k_se_bwd(const TView &dout, const TView &y, const float *mr, const float *params, int cr, const float *e,
+                       const float *hid, const float *mean, double *de, float *dsv, float *dparams, const TView &dz,
+                       cudaStream_t st)
+{
+    const lamp_tensor_t tg = as_tensor(dout), ty = as_tensor(y);
+    lamp_tensor_t tz = as_tensor(dz);
+    const int c = y.c;
+    const int64_t Vn = (int64_t)y.d * y.h * y.w;
+    if (Vn == 0 || y.n == 0) return LAMP_OK;
+    const float *w1 = params, *w2 = params + (size_t)cr * c + cr;
+    float *dw1 = dparams, *db1 = dw1 + (size_t)cr * c, *dw2 = db1 + cr, *db2 = dw2 + (size_t)c * cr;
+    lamp_status_t s = lamp_se_bwd_reduce(&tg, &ty, mr, de, st);
+    if (s != LAMP_OK) return s;
+    s = lamp_se_excite_bwd(de, Vn, y.n, c, cr, e, hid, mean, w1, w2, dsv, dw1, db1, dw2, db2, st);
+    if (s != LAMP_OK) return s;
+    return lamp_se_apply_bwd(&tg, e, dsv, &tz, st);
+}
 
 }  // namespace lamp
 

@@ -20,6 +20,13 @@ struct Layer {
     size_t w_off, b_off;
     bool to_cat;                // output is E_l, written to the concat buffer slice [0, C_l)
     bool from_cat;              // input is the full concat buffer (2 C_l channels)
+    // SEU-Net variant: the level's last conv ends in a squeeze-and-excitation residual step, out = r + e * z with
+    // r = this conv's input (the output of the level's first conv).  se_cr > 0: hidden units; its fp32 parameters
+    // W1 [cr][c], b1 [cr], W2 [c][cr], b2 [c] sit in the bias buffer from se_off.  The level's first conv then gets the
+    // block output's gradient as a second gradient source (res_from = index of that last conv, else -1).
+    int se_cr = 0;
+    size_t se_off = 0;
+    int res_from = -1;
 };
 
 struct lamp_unet {
@@ -61,6 +68,10 @@ struct LayerBuf {
     TView dout, dout2;          // gradient w.r.t. the layer's output: main source and skip source (may be empty)
     ConvGeom g;
     lamp_conv_desc_t desc;
+    // squeeze-and-excitation step of a level's last conv (SEU-Net variant)
+    double *se_sums, *se_de;    // [n][c] fp64: sum_v z, sum_v dout * z
+    float *se_e, *se_mean, *se_hid, *se_dsv;
+    TView dsum, dz;             // train mode: dout + dout2 where the block output has two consumers; e * dout + ds / V
 };
 
 struct Plan {
@@ -170,6 +181,15 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
             B.stats = P->stats_pool ? (double *)((char *)P->stats_pool + stats_off) : nullptr;
             stats_off += align_up((size_t)n * Ly.c_out * 2 * sizeof(double), 256);
             B.mr = (float *)A.take((size_t)n * Ly.c_out * 2 * sizeof(float));
+            B.se_sums = nullptr; B.se_de = nullptr; B.se_e = nullptr; B.se_mean = nullptr; B.se_hid = nullptr; B.se_dsv = nullptr;
+            if (Ly.se_cr) {
+                B.se_sums = (double *)A.take((size_t)n * Ly.c_out * sizeof(double));
+                B.se_de = (double *)A.take((size_t)n * Ly.c_out * sizeof(double));
+                B.se_e = (float *)A.take((size_t)n * Ly.c_out * sizeof(float));
+                B.se_mean = (float *)A.take((size_t)n * Ly.c_out * sizeof(float));
+                B.se_dsv = (float *)A.take((size_t)n * Ly.c_out * sizeof(float));
+                B.se_hid = (float *)A.take((size_t)n * Ly.se_cr * sizeof(float));
+            }
             if (Ly.to_cat) {
                 B.out = P->cat[l];
                 B.out.c = Ly.c_out;                      // slice [0, C_l)
@@ -195,7 +215,7 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
     P->wt.assign(net->layers.size(), nullptr);
     P->wt_bytes.assign(net->layers.size(), 0);
     for (LayerBuf &B : P->lb) {
-        B.dy = TView{}; B.din = TView{}; B.dout = TView{}; B.dout2 = TView{};
+        B.dy = TView{}; B.din = TView{}; B.dout = TView{}; B.dout2 = TView{}; B.dsum = TView{}; B.dz = TView{};
         B.bsums = nullptr; B.db_acc = nullptr; B.db_count = nullptr;
     }
     if (mode == LAMP_MODE_TRAIN) {
@@ -237,6 +257,14 @@ void make_plan(const lamp_unet *net, void *base, const void *x_ptr, int64_t x_pi
                 if (Ly.to_cat) {                        // E_l also fed the skip: slice [0, C_l) of dcat_l
                     B.dout2 = P->dcat[Ly.level];
                     B.dout2.c = Ly.c_out;
+                }
+                if (Ly.se_cr) {
+                    void *pz = A.take(vox(Ly.level) * Ly.c_out * sizeof(bf16));
+                    B.dz = view(pz, n, dd(Ly.level), hh(Ly.level), ww(Ly.level), Ly.c_out, Ly.c_out, 0);
+                    if (Ly.to_cat) {
+                        void *ps = A.take(vox(Ly.level) * Ly.c_out * sizeof(bf16));
+                        B.dsum = view(ps, n, dd(Ly.level), hh(Ly.level), ww(Ly.level), Ly.c_out, Ly.c_out, 0);
+                    }
                 }
             } else if (Ly.kind == K_UP) {
                 B.dy = g;                               // no norm / activation after the up conv
@@ -304,7 +332,12 @@ lamp_status_t run_forward(const lamp_unet *net, const Plan &P, const bf16 *W, co
         const LayerBuf &B = P.lb[i];
         const bf16 *w = W + Ly.w_off;
         const float *b = Bv + Ly.b_off;
-        if (Ly.kind == K_CONV || Ly.kind == K_DOWN) {
+        if (Ly.se_cr) {
+            // last conv of a level in the SEU-Net variant: out = r + e * relu(norm(y)), r = this conv's input
+            TRY(conv_fwd(B.g, B.in, w, b, B.y, B.stats, P.scratch, P.scratch_bytes, st));
+            TRY(k_mu_rstd(B.stats, (int64_t)B.y.d * B.y.h * B.y.w, S.in_eps, B.mr, B.y.n * Ly.c_out, st));
+            TRY(k_se_fwd(B.y, B.mr, Bv + Ly.se_off, Ly.se_cr, B.se_sums, B.se_e, B.se_hid, B.se_mean, &B.in, B.out, st));
+        } else if (Ly.kind == K_CONV || Ly.kind == K_DOWN) {
             TRY(conv_fwd(B.g, B.in, w, b, B.y, B.stats, P.scratch, P.scratch_bytes, st));
             TRY(k_instnorm_relu_fwd(B.y, B.stats, S.in_eps, B.mr, B.out, st));
         } else if (Ly.kind == K_UP) {
@@ -364,23 +397,32 @@ lamp_status_t lamp_unet_create(const lamp_unet_spec_t *spec, lamp_unet_t **out)
         if (spec->channels[l] <= 0 || spec->channels[l] % 8 || spec->channels[l] > 2048) return LAMP_ERR_UNSUPPORTED;
     if (spec->channels[0] > 128) return LAMP_ERR_UNSUPPORTED;          // the head's backward kernel keeps 256 voxels x channels[0] in shared memory
     if (!(spec->in_eps > 0.f)) return LAMP_ERR_INVALID_ARG;
+    if (spec->se_ratio < 0) return LAMP_ERR_INVALID_ARG;
+    // the residual branch of the squeeze-and-excitation block is the input of the level's last conv: two convs per level
+    if (spec->se_ratio > 0 && spec->convs_per_level != 2) return LAMP_ERR_UNSUPPORTED;
     lamp_unet *net = new (std::nothrow) lamp_unet;
     if (!net) return LAMP_ERR_INVALID_ARG;
     net->spec = *spec;
     const int L = spec->levels;
     const int32_t *ch = spec->channels;
     size_t wo = 0, bo = 0;
-    auto add = [&](int kind, int level, int ci, int co, int taps, bool to_cat, bool from_cat) {
+    auto add = [&](int kind, int level, int ci, int co, int taps, bool to_cat, bool from_cat, bool se_last = false) {
         Layer y{kind, level, ci, co, taps, wo, bo, to_cat, from_cat};
-        net->layers.push_back(y);
         wo += (size_t)taps * ci * co;
         wo = (wo + 7) / 8 * 8;                  // keep every layer's weights 16-byte aligned
         bo += (size_t)co;
+        if (se_last && spec->se_ratio > 0) {
+            y.se_cr = co / spec->se_ratio > 0 ? co / spec->se_ratio : 1;
+            y.se_off = bo;
+            bo += (size_t)2 * co * y.se_cr + co + y.se_cr;
+            net->layers.back().res_from = (int)net->layers.size();      // the conv in front is the level's first conv
+        }
+        net->layers.push_back(y);
     };
     int c = spec->in_channels;
     for (int l = 0; l < L; ++l) {
         for (int j = 0; j < spec->convs_per_level; ++j) {
-            add(K_CONV, l, c, ch[l], 27, j == spec->convs_per_level - 1 && l < L - 1, false);
+            add(K_CONV, l, c, ch[l], 27, j == spec->convs_per_level - 1 && l < L - 1, false, j == spec->convs_per_level - 1);
             c = ch[l];
         }
         if (l < L - 1) { add(K_DOWN, l + 1, ch[l], ch[l + 1], 27, false, false); c = ch[l + 1]; }
@@ -388,7 +430,7 @@ lamp_status_t lamp_unet_create(const lamp_unet_spec_t *spec, lamp_unet_t **out)
     for (int l = L - 2; l >= 0; --l) {
         add(K_UP, l, ch[l + 1], ch[l], 8, false, false);
         c = 2 * ch[l];
-        for (int j = 0; j < spec->convs_per_level; ++j) { add(K_CONV, l, c, ch[l], 27, false, j == 0); c = ch[l]; }
+        for (int j = 0; j < spec->convs_per_level; ++j) { add(K_CONV, l, c, ch[l], 27, false, j == 0, j == spec->convs_per_level - 1); c = ch[l]; }
     }
     add(K_HEAD, 0, ch[0], spec->num_classes, 1, false, false);
     net->n_w = wo;
@@ -406,6 +448,14 @@ void lamp_unet_destroy(lamp_unet_t *net)
 int32_t lamp_unet_num_layers(const lamp_unet_t *net) { return net ? (int32_t)net->layers.size() : 0; }
 size_t lamp_unet_weight_count(const lamp_unet_t *net) { return net ? net->n_w : 0; }
 size_t lamp_unet_bias_count(const lamp_unet_t *net) { return net ? net->n_b : 0; }
+
+lamp_status_t lamp_unet_se_layout(const lamp_unet_t *net, int32_t layer, size_t *se_off, int32_t *cr)
+{
+    if (!net || layer < 0 || layer >= (int32_t)net->layers.size() || !se_off || !cr) return LAMP_ERR_INVALID_ARG;
+    *se_off = net->layers[layer].se_off;
+    *cr = net->layers[layer].se_cr;
+    return LAMP_OK;
+}
 
 lamp_status_t lamp_unet_param_layout(const lamp_unet_t *net, int32_t layer, size_t *w_off, size_t *b_off,
                                      lamp_conv_desc_t *desc)
@@ -558,9 +608,23 @@ static lamp_status_t train_step_impl(const lamp_unet_t *net, const void *weights
                 TRY(mark_final(Ly.w_off, true));
                 continue;
             }
-            if (Ly.kind != K_UP)
-                TRY(k_instnorm_relu_bwd(B.dout, Ly.to_cat ? &B.dout2 : nullptr, B.y, B.mr, B.bsums, true, B.dy, B.db_acc,
-                                        B.db_count, db, st));
+            if (Ly.se_cr) {
+                // gradient of the block output (both consumers where it also fed the skip), through the
+                // squeeze-and-excitation step to dz, then the InstanceNorm backward of this conv
+                const TView *src = &B.dout;
+                if (Ly.to_cat) { TRY(k_add2(B.dout, B.dout2, B.dsum, st)); src = &B.dsum; }
+                TRY(k_se_bwd(*src, B.y, B.mr, biases_f32 + Ly.se_off, Ly.se_cr, B.se_e, B.se_hid, B.se_mean, B.se_de, B.se_dsv,
+                             grad_b + Ly.se_off, B.dz, st));
+                TRY(k_instnorm_relu_bwd(B.dz, nullptr, B.y, B.mr, B.bsums, true, B.dy, B.db_acc, B.db_count, db, st));
+            } else if (Ly.kind != K_UP) {
+                // (the first conv of a squeeze-and-excitation level also receives the block output's gradient: the residual)
+                const TView *second = Ly.to_cat ? &B.dout2 : nullptr;
+                if (Ly.res_from >= 0) {
+                    const LayerBuf &R = P.lb[Ly.res_from];
+                    second = net->layers[Ly.res_from].to_cat ? &R.dsum : &R.dout;
+                }
+                TRY(k_instnorm_relu_bwd(B.dout, second, B.y, B.mr, B.bsums, true, B.dy, B.db_acc, B.db_count, db, st));
+            }
             // dy is complete on the caller's stream: the weight gradient starts from here on the side stream (the
             // bias gradient of a normalised layer came out of the InstanceNorm backward kernel above)
             if (two) {

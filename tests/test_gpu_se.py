@@ -170,3 +170,82 @@ def test_se_residual_block_forward_backward_composed_from_the_library_calls():
     assert_close(host_f64(dya), dya_o, "block dy of the first conv", rel=1e-2, mx=1e-1)
     assert_close(host_f64(dwa), dwa_o, "block dW of the first conv", rel=1e-2, mx=1e-1)
     assert_close(host_f64(dx), dx_o, "block dx", rel=1e-2, mx=1e-1)
+
+
+def test_seunet_train_step_matches_the_mirrored_oracle_within_the_storage_budget():
+    """The SEU-Net variant through lamp_unet_create(se_ratio) / lamp_unet_train_step / lamp_unet_forward: probabilities,
+    loss and every gradient (conv weights, biases, squeeze-and-excitation parameters) against the oracle that mirrors
+    the bf16 storage points, held to the arithmetic's own budget (mirrored oracle against unrounded oracle) as the
+    plain network is; the steps of the block themselves are checked one by one above."""
+    from oracle import unet as O
+    levels, ch, K, ratio = 2, [32, 64], 5, 4
+    D, H, W = 8, 12, 20
+    net = B.lamp_unet_create(B.unet_spec(levels, ch, 2, 1, K, se_ratio=ratio))
+    spec = O.UNetSpec(levels, list(ch), 2, 1, K, se_ratio=ratio)
+    lay = O.unet_layers(spec)
+    ws = synth.kaiming_for_layers([(l.taps, l.c_out, l.c_in, l.fan_in) for l in lay], 61)
+    rs = synth.rng(62)
+    bs = [0.1 * rs.standard_normal(l.c_out).astype(np.float32) for l in lay]
+    se = [None] * len(lay)
+    wflat = np.zeros(B.lamp_unet_weight_count(net), dtype=np.float32)
+    bflat = np.zeros(B.lamp_unet_bias_count(net), dtype=np.float32)
+    offs = []
+    for i, l in enumerate(lay):
+        wo, bo, _ = B.lamp_unet_param_layout(net, i)
+        so, cr = B.lamp_unet_se_layout(net, i)
+        assert cr == l.se_cr
+        wflat[wo:wo + ws[i].size] = ws[i].ravel()
+        bflat[bo:bo + l.c_out] = bs[i]
+        if cr:
+            c = l.c_out
+            W1, b1, W2, b2 = _params(c, cr, 70 + i)
+            se[i] = (W1, b1, W2, b2)
+            bflat[so:so + 2 * c * cr + c + cr] = np.concatenate([W1.ravel(), b1, W2.ravel(), b2])
+        offs.append((wo, bo, so, cr))
+    assert sum(1 for l in lay if l.se_cr) == 3
+    x = synth.bf16_round(np.stack([synth.blurred_noise((D, H, W), 1.5, s) for s in (63, 64)]))[..., None]
+    lab = np.stack([synth.labels_blobs((D, H, W), 65 + s, K, 1.5) for s in (0, 1)])
+    V = 2 * D * H * W
+    wd, bd = dev_bf16(wflat), f32(bflat)
+    loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+    gw = torch.full((wflat.size,), float("nan"), dtype=torch.float32, device="cuda")
+    gb = torch.full((bflat.size,), float("nan"), dtype=torch.float32, device="cuda")
+    probs = torch.empty((V, K), dtype=torch.float32, device="cuda")
+    wsb = torch.empty(B.lamp_unet_workspace_bytes(net, 2, D, H, W, B.MODE_TRAIN), dtype=torch.uint8, device="cuda")
+    B.lamp_unet_train_step(net, wd, bd, dev_bf16(x), torch.from_numpy(lab).cuda().reshape(-1), loss, gw, gb, probs, wsb)
+    assert B.lamp_get_async_status() == 0
+    ws64 = [a.astype(np.float64) for a in ws]
+    bs64 = [a.astype(np.float64) for a in bs]
+    se64 = [None if t is None else tuple(a.astype(np.float64) for a in t) for t in se]
+    l_q, dWq, dBq, p_q, dSq = O.train_step(spec, ws64, bs64, x.astype(np.float64), lab, quantise=True, se=se64)
+    l_f, dWf, dBf, p_f, dSf = O.train_step(spec, ws64, bs64, x.astype(np.float64), lab, quantise=False, se=se64)
+    relerr = lambda a, b: np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300)
+    p_gpu = host_f64(probs).reshape(p_q.shape)
+    budget = relerr(p_q, p_f)
+    assert relerr(p_gpu, p_q) <= max(1e-3, 2 * budget), (relerr(p_gpu, p_q), budget)
+    assert np.abs(p_gpu - p_q).max() <= max(1e-2 * np.abs(p_q).max(), 2 * np.abs(p_q - p_f).max())
+    assert abs(float(loss.item()) - l_q) <= max(1e-3, 2 * abs(l_q - l_f) / abs(l_f)) * abs(l_q)
+    gw_h, gb_h = host_f64(gw), host_f64(gb)
+    assert np.isfinite(gw_h).all() and np.isfinite(gb_h).all()
+    for i, l in enumerate(lay):
+        wo, bo, so, cr = offs[i]
+        got = gw_h[wo:wo + ws[i].size].reshape(ws[i].shape)
+        assert relerr(got, dWq[i]) <= max(1e-3, 2 * relerr(dWq[i], dWf[i])), (l.name, relerr(got, dWq[i]), relerr(dWq[i], dWf[i]))
+        if cr:
+            c = l.c_out
+            blk = gb_h[so:so + 2 * c * cr + c + cr]
+            got_se = (blk[:cr * c].reshape(cr, c), blk[cr * c:cr * c + cr], blk[cr * c + cr:cr * c + cr + c * cr].reshape(c, cr),
+                      blk[cr * c + cr + c * cr:])
+            for k in range(4):
+                bud = relerr(dSq[i][k], dSf[i][k])
+                assert relerr(got_se[k], dSq[i][k]) <= max(2e-3, 2 * bud), (l.name, k, relerr(got_se[k], dSq[i][k]), bud)
+    # the forward pass alone gives the same probabilities as the training step
+    p2 = torch.empty_like(probs)
+    wsf = torch.empty(B.lamp_unet_workspace_bytes(net, 2, D, H, W, B.MODE_INFER), dtype=torch.uint8, device="cuda")
+    B.lamp_unet_forward(net, wd, bd, dev_bf16(x), p2, None, wsf)
+    assert torch.equal(p2, probs)
+    B.lamp_unet_destroy(net)
+    # three convs per level have no defined residual branch: refused
+    with pytest.raises(B.LampError) as e:
+        B.lamp_unet_create(B.unet_spec(2, [32, 64], 3, 1, K, se_ratio=4))
+    assert e.value.status == 2

@@ -74,3 +74,62 @@ def test_block_backward_matches_central_finite_differences():
     # the gradient w.r.t. z has two parts: the rescaled upstream gradient and, through the squeeze, a constant per (n, c)
     part = dz - cache["e"][:, None, None, None, :] * g
     assert np.allclose(part, part[:, :1, :1, :1, :], rtol=0, atol=1e-14)
+
+
+def _se_net(seed):
+    from oracle import unet
+    from paper_2006_12575_b200 import synth
+    spec = unet.UNetSpec(2, [4, 8], 2, 1, 3, se_ratio=2)
+    lay = unet.unet_layers(spec)
+    ws = [w.astype(np.float64) for w in synth.kaiming_for_layers([(l.taps, l.c_out, l.c_in, l.fan_in) for l in lay], seed)]
+    rs = np.random.default_rng(seed)
+    bs = [0.1 * rs.standard_normal(l.c_out) for l in lay]
+    se = [None] * len(lay)
+    for i, l in enumerate(lay):
+        if l.se_cr:
+            se[i] = (rs.standard_normal((l.se_cr, l.c_out)) * 0.6, rs.standard_normal(l.se_cr) * 0.2 + 0.4,
+                     rs.standard_normal((l.c_out, l.se_cr)) * 0.6, rs.standard_normal(l.c_out) * 0.2)
+    x = rs.standard_normal((1, 4, 4, 4, 1))
+    lab = rs.integers(0, 3, (1, 4, 4, 4))
+    return unet, spec, lay, ws, bs, se, x, lab
+
+
+def test_seunet_layers_and_gradients_by_finite_differences():
+    """The SEU-Net variant of the oracle's network: which layers end in the block, the excitation-one identity, and the
+    whole network's gradient (conv weights in front of, inside and behind the blocks, and the blocks' own parameters)."""
+    unet, spec, lay, ws, bs, se, x, lab = _se_net(4)
+    assert [l.name for l in lay if l.se_cr] == ["enc0.conv1", "enc1.conv1", "dec0.conv1"]
+    assert [l.se_cr for l in lay if l.se_cr] == [2, 4, 2]
+    loss, dW, dB, probs, dSE = unet.train_step(spec, ws, bs, x, lab, quantise=False, se=se)
+    assert probs.shape == (1, 4, 4, 4, 3) and np.allclose(probs.sum(-1), 1)
+    f = lambda: unet.train_step(spec, ws, bs, x, lab, quantise=False, se=se)[0]
+    rs = np.random.default_rng(9)
+    h = 1e-6
+    for i, l in enumerate(lay):
+        for _ in range(3):
+            idx = tuple(rs.integers(0, n) for n in ws[i].shape)
+            old = ws[i][idx]
+            ws[i][idx] = old + h
+            lp = f()
+            ws[i][idx] = old - h
+            lm = f()
+            ws[i][idx] = old
+            fd = (lp - lm) / (2 * h)
+            assert abs(fd - dW[i][idx]) <= 2e-6 * max(1.0, abs(fd) * 1e3), (l.name, fd, dW[i][idx])
+        if l.se_cr:
+            for k in range(4):
+                a = se[i][k]
+                idx = tuple(rs.integers(0, n) for n in a.shape)
+                old = a[idx]
+                a[idx] = old + h
+                lp = f()
+                a[idx] = old - h
+                lm = f()
+                a[idx] = old
+                fd = (lp - lm) / (2 * h)
+                assert abs(fd - dSE[i][k][idx]) <= 2e-6 * max(1.0, abs(fd) * 1e3), (l.name, k, fd, dSE[i][k][idx])
+    # the plain network is the variant without the blocks: different function, same layer list and shapes
+    plain = unet.UNetSpec(2, [4, 8], 2, 1, 3)
+    assert [l.name for l in unet.unet_layers(plain)] == [l.name for l in lay]
+    p_plain = unet.forward(plain, ws, bs, x, quantise=False)
+    assert np.abs(p_plain - probs).max() > 1e-3
