@@ -27,17 +27,16 @@
 //    tile, which halves the L2 -> SM weight traffic per MMA (the tiles are streamed: 27 * c_in * c_out * 2 bytes
 //    do not fit beside the planes).  The nine in-plane taps are shifted windows of the halo box (descriptor
 //    start (kh * 10 + kw) rows in, 10 rows between 8-voxel groups; the swizzle is a function of the address).
-//  * Every weight tile is used by window 0, then by window 1; window 0's slot hand-over (TMEM -> registers, zero
-//    store, barrier) after the last tile of an input plane runs behind window 1's MMAs of that tile.  (Issuing the
-//    last two and first two tiles of a plane window by window, to give the hand-over twice that time, measured 9 %
-//    slower.)
+//  * Each window has its own MMA-issuing thread; both walk the same plane and weight stages, which are released once
+//    both have committed them.  A window's slot hand-over (TMEM -> registers, zero store, barrier) after the last tile
+//    of an input plane runs behind the other window's MMAs.
 //  * A CTA owns a contiguous run of (window column, output plane) units; a run that starts or ends inside a
 //    column costs one extra input plane each (the halo along d), columns that end at the volume border none.
 //  * Epilogue: one voxel per thread with all its channels: bias, InstanceNorm sums (a transposing shuffle
 //    butterfly per 32 columns), conversion and 32-byte stores of the voxel's channel run at the output's pitch.
 //
-// Warps: 0 = activation-plane TMA producer, 1 = MMA issuer (+ TMEM owner), 2 = weight-tile TMA producer,
-// 4..7 / 8..11 = epilogue of window 0 / 1.  All waits are bounded (LAMP_ERR_TIMEOUT on expiry).
+// Warps: 0 = activation-plane TMA producer, 1 / 3 = MMA issuer of window 0 / 1 (warp 1 also owns the TMEM allocation),
+// 2 = weight-tile TMA producer, 4..7 / 8..11 = epilogue of window 0 / 1.  All waits are bounded (LAMP_ERR_TIMEOUT on expiry).
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include "common.cuh"
@@ -141,8 +140,9 @@ conv3_r_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
-        for (int s = 0; s < MAX_NP; ++s) { mbar_init(pfull0 + 8 * s, 1); mbar_init(pempty0 + 8 * s, 1); }
-        for (int s = 0; s < MAX_NW; ++s) { mbar_init(wfull0 + 8 * s, 1); mbar_init(wempty0 + 8 * s, 1); }
+        // (a plane or weight stage is free again once BOTH windows' issuers have committed it)
+        for (int s = 0; s < MAX_NP; ++s) { mbar_init(pfull0 + 8 * s, 1); mbar_init(pempty0 + 8 * s, 2); }
+        for (int s = 0; s < MAX_NW; ++s) { mbar_init(wfull0 + 8 * s, 1); mbar_init(wempty0 + 8 * s, 2); }
         for (int s = 0; s < 2; ++s) { mbar_init(done0 + 8 * s, 1); mbar_init(free0 + 8 * s, 4); }
         *abort_flag = 0;
         mbar_init_fence();
@@ -221,9 +221,15 @@ conv3_r_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || warp == 3) {
         if (lane == 0) {
-            // ---------------------------------------------------------------- MMA issuer
+            // ---------------------------------------------------------------- MMA issuers: warp 1 -> window 0, warp 3 -> window 1
+            // One thread issuing both windows' MMAs spent 115-118 cycles per N = 192 instruction (barrier round trips,
+            // descriptors and commits included) where the pipe needs 96: the tensor pipe idled a third of the time
+            // waiting for its next instruction.  Each window therefore has its own issuing thread; the two share the
+            // stages (every stage barrier expects both commits) and nothing else.
+            const int j = warp == 1 ? 0 : 1;
+            const uint32_t d_tmem = tmem_base + j * WIN_COLS;
             int ps = 0, ws = 0;
             uint32_t pph = 0, wph = 0, gs = 0;                  // gs: input planes issued so far (barrier phases)
             bool ok = true;
@@ -236,31 +242,26 @@ conv3_r_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     for (int c = 0; c < P.chunks && ok; ++c) {
                         if (!mbar_wait(pfull0 + 8 * ps, pph, abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        const uint32_t plane = smem_u32(p_base + (size_t)ps * P.plane_bytes);
+                        // window j: 16 groups of 8 voxels along w, J halo rows apart, from halo row hs + 16 J j
+                        const uint32_t win = smem_u32(p_base + (size_t)ps * P.plane_bytes) + (16 * J * j) * HALO_W * ROWB;
+                        if (c == 0) {
+                            // the slot that input plane p starts afresh has been zeroed
+                            if (!mbar_wait(free0 + 8 * j, gs & 1, abort_flag)) { ok = false; break; }
+                            tc_fence_after();
+                        }
                         for (int t0 = 0; t0 < NT && ok; t0 += TPS) {
                             if (!mbar_wait(wfull0 + 8 * ws, wph, abort_flag)) { ok = false; break; }
                             tc_fence_after();
+                            const uint32_t wst = smem_u32(w_base + (size_t)ws * WST_BYTES);
 #pragma unroll
                             for (int ti = 0; ti < TPS; ++ti) {
                                 const int tt = t0 + ti, hs = tt / 3, kw = tt - hs * 3;
-                                const bool first = c == 0 && tt == 0, last = c == P.chunks - 1 && tt == NT - 1;
-                                const uint64_t db = make_desc(smem_u32(w_base + (size_t)ws * WST_BYTES) + ti * TILE_BYTES, 0, 8 * ROWB, SWZ);
+                                const uint64_t db = make_desc(wst + ti * TILE_BYTES, 0, 8 * ROWB, SWZ);
+                                const uint64_t da = make_desc(win + (hs * HALO_W + kw) * ROWB, 0, J * HALO_W * ROWB, SWZ);
 #pragma unroll
-                                for (int j = 0; j < 2; ++j) {
-                                    if (first) {
-                                        // the slot that input plane p starts afresh has been zeroed
-                                        if (!mbar_wait(free0 + 8 * j, gs & 1, abort_flag)) { ok = false; break; }
-                                        tc_fence_after();
-                                    }
-                                    // window j: 16 groups of 8 voxels along w, J halo rows apart, from halo row hs + 16 J j
-                                    const uint64_t da = make_desc(plane + ((hs + 16 * J * j) * HALO_W + kw) * ROWB, 0, J * HALO_W * ROWB, SWZ);
-#pragma unroll
-                                    for (int k = 0; k < KC / 16; ++k) umma_bf16(tmem_base + j * WIN_COLS, da + 2 * k, db + 2 * k, IDESC, 1u);
-                                    if (last) umma_commit(done0 + 8 * j);
-                                }
-                                if (!ok) break;
+                                for (int k = 0; k < KC / 16; ++k) umma_bf16(d_tmem, da + 2 * k, db + 2 * k, IDESC, 1u);
                             }
-                            if (!ok) break;
+                            if (c == P.chunks - 1 && t0 + TPS >= NT) umma_commit(done0 + 8 * j);
                             umma_commit(wempty0 + 8 * ws);
                             if (++ws == P.nw) { ws = 0; wph ^= 1; }
                         }
