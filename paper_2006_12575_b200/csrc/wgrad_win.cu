@@ -13,7 +13,7 @@
 // conv's zero padding).  The swizzle is a function of the shared-memory address bits, so windows that
 // start off the swizzle-atom boundary read exactly what TMA wrote.
 //
-// A CTA keeps two accumulators (128 x 192 fp32 each) in TMEM while it sweeps its share of the
+// A CTA keeps two accumulators (128 x 192 fp32 each, one MMA-issuing thread each) in TMEM while it sweeps its share of the
 // 8 x 16-voxel tiles (split-K over CTAs); partial sums go to scratch and are added in a fixed order.
 #include <cuda.h>
 #include <cudaTypedefs.h>
@@ -26,7 +26,7 @@ namespace {
 
 using namespace ptx;
 
-constexpr int WW_THREADS = 192;
+constexpr int WW_THREADS = 224;
 constexpr int TWW = 8, THH = 16;                   // tile: 8 (w) x 16 (h) voxels of one plane = K = 128
 constexpr int XW = TWW + 2;                        // x box: w halo only
 constexpr int DYH = THH + 2;                       // dy box: h halo only
@@ -95,8 +95,9 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
-        for (int s = 0; s < MAX_ST; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-        mbar_init(done_bar, 1);
+        // (each of the two accumulators has its own issuing thread: a stage is free, and a unit done, after both)
+        for (int s = 0; s < MAX_ST; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 2); }
+        mbar_init(done_bar, 2);
         mbar_init(drained_bar, 4);
         *abort_flag = 0;
         mbar_init_fence();
@@ -142,9 +143,13 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || warp == 6) {
         if (lane == 0) {
-            // ---------------------------------------------------------------- MMA issuer
+            // ---------------------------------------------------------------- MMA issuers: warp 1 -> accumulator 0, warp 6 -> 1
+            // One thread cannot issue faster than about one tcgen05.mma per 60-100 cycles (waits, descriptors and
+            // commits included); with N = 96 (32 input channels) the pipe needs an instruction every 48 cycles, and a
+            // single issuer left it idle more than half of the time.  Two threads, one accumulator each.
+            const int q = warp == 1 ? 0 : 1;
             int st = 0;
             uint32_t ph = 0, uph = 0;
             bool ok = true;
@@ -159,10 +164,9 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     if (!mbar_wait(full0 + 8 * st, ph, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sb = smem_u32(smem + (size_t)st * P.stage_bytes);
-#pragma unroll
-                    for (int q = 0; q < 2; ++q) {
+                    {
                         const Acc &a = q ? a1 : a0;
-                        if (!a.live) continue;
+                        if (!a.live) { mbar_arrive(empty0 + 8 * st); if (++st == P.nst) { st = 0; ph ^= 1; } accumulate = 1; continue; }
                         const uint32_t dyb = sb + ((q && two_dy) ? P.dy_bytes : 0) + a.ls0 * LINE_A;
                         const uint32_t xb = sb + P.ndy * P.dy_bytes + ((q && P.pair_cx) ? P.x_bytes : 0);
                         // A: blocks of 64 (32) rows = c_out channels of one window; next block = next 64 channels of
@@ -181,7 +185,7 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     accumulate = 1;
                 }
                 if (!ok) break;
-                umma_commit(done_bar);
+                if ((q ? a1 : a0).live) umma_commit(done_bar); else mbar_arrive(done_bar);
                 uph ^= 1;
             }
         }
