@@ -42,6 +42,7 @@ struct WwParams {
     int32_t ncx;             // c_in chunks (of 64, or one of 32)
     int32_t pair_cx;         // 1: a set = one M block x two c_in chunks; 0: a set = two M blocks x the one chunk
     int32_t nsets, nsplit, nunits;
+    int32_t nsplit_last;     // CTAs that share the LAST set (fewer where that set has one live accumulator: half the work per tile)
     int32_t nst;             // pipeline stages
     int32_t ndy;             // dy buffers per stage (2 where the two accumulators of a set can need different planes)
     int32_t dy_bytes, x_bytes, stage_bytes;
@@ -117,12 +118,14 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             uint32_t ph = 0;
             bool ok = true;
             for (int unit = blockIdx.x; unit < P.nunits && ok; unit += gridDim.x) {
-                const int set = unit / P.nsplit, split = unit - set * P.nsplit;
+                const int full = (P.nsets - 1) * P.nsplit;
+                const int set = unit < full ? unit / P.nsplit : P.nsets - 1, split = unit < full ? unit % P.nsplit : unit - full;
+                const int stride = unit < full ? P.nsplit : P.nsplit_last;
                 const Acc a0 = decode_acc(P, set, 0), a1 = decode_acc(P, set, 1);
                 const bool two_dy = P.ndy == 2 && (a1.kd != a0.kd || a1.cc != a0.cc);
                 const bool two_x = P.pair_cx;
                 const uint32_t bytes = (two_dy ? 2 : 1) * aboxes * DYBOX + (two_x ? 2 : 1) * XBOX;
-                for (int tile = split; tile < P.ntiles && ok; tile += P.nsplit) {
+                for (int tile = split; tile < P.ntiles && ok; tile += stride) {
                     int t = tile;
                     const int w0 = (t % P.nwt) * TWW; t /= P.nwt;
                     const int h0 = (t % P.nht) * THH; t /= P.nht;
@@ -154,13 +157,15 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             uint32_t ph = 0, uph = 0;
             bool ok = true;
             for (int unit = blockIdx.x; unit < P.nunits && ok; unit += gridDim.x) {
-                const int set = unit / P.nsplit, split = unit - set * P.nsplit;
+                const int full = (P.nsets - 1) * P.nsplit;
+                const int set = unit < full ? unit / P.nsplit : P.nsets - 1, split = unit < full ? unit % P.nsplit : unit - full;
+                const int stride = unit < full ? P.nsplit : P.nsplit_last;
                 const Acc a0 = decode_acc(P, set, 0), a1 = decode_acc(P, set, 1);
                 const bool two_dy = P.ndy == 2 && (a1.kd != a0.kd || a1.cc != a0.cc);
                 if (!mbar_wait(drained_bar, uph ^ 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 uint32_t accumulate = 0;
-                for (int tile = split; tile < P.ntiles && ok; tile += P.nsplit) {
+                for (int tile = split; tile < P.ntiles && ok; tile += stride) {
                     if (!mbar_wait(full0 + 8 * st, ph, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sb = smem_u32(smem + (size_t)st * P.stage_bytes);
@@ -195,7 +200,8 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         uint32_t uph = 0;
         bool ok = true;
         for (int unit = blockIdx.x; unit < P.nunits && ok; unit += gridDim.x) {
-            const int set = unit / P.nsplit, split = unit - set * P.nsplit;
+            const int full = (P.nsets - 1) * P.nsplit;
+            const int set = unit < full ? unit / P.nsplit : P.nsets - 1, split = unit < full ? unit % P.nsplit : unit - full;
             ok = __all_sync(0xffffffffu, mbar_wait(done_bar, uph, abort_flag));
             if (!ok) break;
             tc_fence_after();
@@ -305,7 +311,14 @@ bool make_ww_plan(const ConvGeom &g, WwPlan *out)
     if (nsplit < 1) nsplit = 1;
     if (nsplit > P.ntiles) nsplit = P.ntiles;
     P.nsplit = nsplit;
-    P.nunits = P.nsets * nsplit;
+    P.nsplit_last = nsplit;
+    // 32 output channels: three M blocks (kd = 0, 1, 2) in two sets, the second with ONE live accumulator, i.e. half the
+    // MMAs per tile.  Its share of the CTAs is halved accordingly (2 : 1), so that all CTAs finish together.
+    if (P.cob == 32 && P.nsets == 2 && !P.pair_cx && sms >= 3 && P.ntiles >= sms) {
+        P.nsplit = sms * 2 / 3;
+        P.nsplit_last = sms - P.nsplit;
+    }
+    P.nunits = (P.nsets - 1) * P.nsplit + P.nsplit_last;
     P.entries = (int64_t)27 * g.co * g.ci;
     out->CBA = CBA; out->CBB = CBB;
     out->smem = 1024 + (size_t)nst * P.stage_bytes + 1024;
@@ -351,6 +364,13 @@ lamp_status_t win_wgrad(const ConvGeom &g, const TView &x, const TView &dy, floa
     if (!encode) return LAMP_ERR_CUDA;
     const bool direct = pl.P.nsplit == 1;
     pl.P.part = direct ? dw : (float *)ws;
+    if (pl.P.nsplit_last < pl.P.nsplit) {
+        // the last set (taps kd = 2: entries [18, 27) x c_out x c_in) writes fewer partial slices than the reduction adds:
+        // the slices it does not write are zero
+        const size_t tap_bytes = (size_t)g.co * g.ci * sizeof(float);
+        LAMP_CUDA_OK(cudaMemset2DAsync((char *)pl.P.part + (size_t)pl.P.nsplit_last * pl.P.entries * sizeof(float) + 18 * tap_bytes,
+                                       (size_t)pl.P.entries * sizeof(float), 0, 9 * tap_bytes, (size_t)(pl.P.nsplit - pl.P.nsplit_last), st));
+    }
     pl.P.status = status_word_ptr();
     CUtensorMap mx, mdy;
     if (!encode_box(encode, &mx, x, pl.CBB, XW, THH)) return LAMP_ERR_CUDA;
