@@ -8,8 +8,10 @@
 // voxels, MN-major) read through a descriptor whose three 64-channel blocks are the windows starting
 // 0, 1 and 2 rows in (leading-dimension offset = one row, 8-voxel groups 10 rows apart).  N = 192 costs
 // 96 cycles: the full rate.  The A operand is a window of a dy halo box (8 (w) x 18 (h) voxels of plane
-// d + 1 - kd): it starts (2 - kh) lines in; for c_out = 64 (32) the 128 rows hold two (four) windows one
-// line apart, i.e. two (three) kh taps per MMA.  Out-of-volume voxels are zero-filled by TMA (the
+// d + 1 - kd): it starts (2 - kh) lines in.  For c_out = 32 the 128 rows hold four windows one line apart (three kh
+// taps per MMA).  For c_out = 64 they hold ANY two of the nine (kd, kh) taps: the second 64-row block is reached
+// through the descriptor's block stride, which may lead into the dy box of the neighbouring plane (both boxes sit
+// in the same stage), so nine taps take five M blocks instead of six.  Out-of-volume voxels are zero-filled by TMA (the
 // conv's zero padding).  The swizzle is a function of the shared-memory address bits, so windows that
 // start off the swizzle-atom boundary read exactly what TMA wrote.
 //
@@ -51,7 +53,10 @@ struct WwParams {
     int    *status;
 };
 
-struct Acc { int kd, ls0, nvalid, cc, cx; bool live; };
+// kd, ls0: plane tap and first line of the M block's first window.  c_out = 64 pairs any two of the nine (kd, kh)
+// taps on the 128 rows: the second 64-row block is the window (kdB, lineB), which may lie in ANOTHER plane's dy box
+// (reached through the descriptor's block stride); validB says whether it carries a tap at all.
+struct Acc { int kd, ls0, nvalid, cc, cx; bool live; int kdB, lineB, validB; };
 
 // accumulator a (0 or 1) of a set
 __device__ __forceinline__ Acc decode_acc(const WwParams &P, int set, int a)
@@ -63,6 +68,14 @@ __device__ __forceinline__ Acc decode_acc(const WwParams &P, int set, int a)
     r.live = mb < P.nmb;
     if (!r.live) mb = P.nmb - 1;
     r.cx = cx;
+    r.kdB = 0; r.lineB = 0; r.validB = 0;
+    if (P.cob == 64) {
+        // five M blocks for nine taps (line = 2 - kh): (kd0: kh1, kh0) (kd0 kh2 | kd1 kh0) (kd1: kh2, kh1) (kd2: kh1, kh0) (kd2 kh2 | -)
+        const int kdA[5] = {0, 0, 1, 2, 2}, lnA[5] = {1, 0, 0, 1, 0}, kdB[5] = {0, 1, 1, 2, 2}, lnB[5] = {2, 2, 1, 2, 1};
+        r.cc = 0; r.kd = kdA[mb]; r.ls0 = lnA[mb]; r.kdB = kdB[mb]; r.lineB = lnB[mb]; r.validB = mb != 4;
+        r.nvalid = r.validB ? 2 : 1;
+        return r;
+    }
     r.kd = mb / P.mb_per_kd;
     const int j = mb % P.mb_per_kd;
     if (P.cob >= 128)     { const int kh = j % 3; r.cc = j / 3; r.ls0 = 2 - kh; r.nvalid = 1; }
@@ -122,7 +135,14 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const int set = unit < full ? unit / P.nsplit : P.nsets - 1, split = unit < full ? unit % P.nsplit : unit - full;
                 const int stride = unit < full ? P.nsplit : P.nsplit_last;
                 const Acc a0 = decode_acc(P, set, 0), a1 = decode_acc(P, set, 1);
-                const bool two_dy = P.ndy == 2 && (a1.kd != a0.kd || a1.cc != a0.cc);
+                // c_out = 64: the set's dy planes: the first block's plane of accumulator 0, and the one other plane any of
+                // the set's blocks uses (at most one)
+                int kd_other = -1;
+                if (P.cob == 64) {
+                    const int cand[3] = {a0.validB ? a0.kdB : a0.kd, a1.live ? a1.kd : a0.kd, (a1.live && a1.validB) ? a1.kdB : a0.kd};
+                    for (int i = 0; i < 3; ++i) if (cand[i] != a0.kd) kd_other = cand[i];
+                }
+                const bool two_dy = P.cob == 64 ? kd_other >= 0 : (P.ndy == 2 && (a1.kd != a0.kd || a1.cc != a0.cc));
                 const bool two_x = P.pair_cx;
                 const uint32_t bytes = (two_dy ? 2 : 1) * aboxes * DYBOX + (two_x ? 2 : 1) * XBOX;
                 for (int tile = split; tile < P.ntiles && ok; tile += stride) {
@@ -136,9 +156,10 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     const uint32_t sb = smem_u32(smem + (size_t)st * P.stage_bytes);
                     for (int q = 0; q < (two_dy ? 2 : 1); ++q) {
                         const Acc &a = q ? a1 : a0;
+                        const int kd = P.cob == 64 ? (q ? kd_other : a0.kd) : a.kd;
                         for (int b = 0; b < aboxes; ++b)
                             tma_load_5d(sb + q * P.dy_bytes + b * DYBOX, &map_dy, full0 + 8 * st, a.cc * 128 + b * 64, w0, h0 - 1,
-                                        d + 1 - a.kd, n);
+                                        d + 1 - kd, n);
                     }
                     for (int q = 0; q < (two_x ? 2 : 1); ++q)
                         tma_load_5d(sb + P.ndy * P.dy_bytes + q * P.x_bytes, &map_x, full0 + 8 * st, (q ? a1.cx : a0.cx) * CBB, w0 - 1, h0, d, n);
@@ -161,7 +182,7 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const int set = unit < full ? unit / P.nsplit : P.nsets - 1, split = unit < full ? unit % P.nsplit : unit - full;
                 const int stride = unit < full ? P.nsplit : P.nsplit_last;
                 const Acc a0 = decode_acc(P, set, 0), a1 = decode_acc(P, set, 1);
-                const bool two_dy = P.ndy == 2 && (a1.kd != a0.kd || a1.cc != a0.cc);
+                const bool two_dy = P.ndy == 2 && (a1.kd != a0.kd || a1.cc != a0.cc);      // (c_out = 64 has its own buffer rule below)
                 if (!mbar_wait(drained_bar, uph ^ 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 uint32_t accumulate = 0;
@@ -172,11 +193,15 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     {
                         const Acc &a = q ? a1 : a0;
                         if (!a.live) { mbar_arrive(empty0 + 8 * st); if (++st == P.nst) { st = 0; ph ^= 1; } accumulate = 1; continue; }
-                        const uint32_t dyb = sb + ((q && two_dy) ? P.dy_bytes : 0) + a.ls0 * LINE_A;
+                        // c_out = 64: plane buffer 0 holds accumulator 0's first plane, buffer 1 the set's other plane
+                        const int bufA = (P.cob == 64) ? (a.kd != a0.kd) : ((q && two_dy) ? 1 : 0);
+                        const int bufB = (P.cob == 64) ? (a.kdB != a0.kd) : bufA;
+                        const uint32_t dyb = sb + bufA * P.dy_bytes + a.ls0 * LINE_A;
+                        const uint32_t lbo64 = (uint32_t)((bufB - bufA) * P.dy_bytes + (a.lineB - a.ls0) * (int)LINE_A);
                         const uint32_t xb = sb + P.ndy * P.dy_bytes + ((q && P.pair_cx) ? P.x_bytes : 0);
                         // A: blocks of 64 (32) rows = c_out channels of one window; next block = next 64 channels of
                         // the same window (cob = 128: next box) or the window one line further down (cob < 128)
-                        const uint64_t da = make_desc(dyb, P.cob >= 128 ? DYBOX : LINE_A, LINE_A, SWA);
+                        const uint64_t da = make_desc(dyb, P.cob >= 128 ? DYBOX : (P.cob == 64 ? lbo64 : LINE_A), LINE_A, SWA);
                         // B: three blocks = the windows kw = 0, 1, 2 (one row apart); 8-voxel groups 10 rows apart
                         const uint64_t db = make_desc(xb, ROWB, XW * ROWB, SWB);
                         const uint32_t d_tmem = tmem_base + q * ACC_COLS;
@@ -211,7 +236,8 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const Acc a = decode_acc(P, set, q);
                 const int rows_per_win = P.cob >= 128 ? 128 : P.cob;
                 const int b = m / rows_per_win;                     // window index inside the M block
-                const int kh = 2 - (a.ls0 + b);
+                const int kh = P.cob == 64 ? (b ? 2 - a.lineB : 2 - a.ls0) : 2 - (a.ls0 + b);
+                const int kd_row = (P.cob == 64 && b) ? a.kdB : a.kd;
                 const bool row_ok = a.live && b < a.nvalid;
                 const int co = a.cc * 128 + m % rows_per_win;
                 const uint32_t trow = tmem_base + ((uint32_t)(q4 * 32) << 16) + q * ACC_COLS;
@@ -222,7 +248,7 @@ wgrad_win_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     tmem_ld_wait();
                     if (row_ok) {
                         const int kw = c0 / CBB, ci = a.cx * CBB + c0 % CBB;
-                        const int tap = (a.kd * 3 + kh) * 3 + kw;
+                        const int tap = (kd_row * 3 + kh) * 3 + kw;
                         float4 *d4 = reinterpret_cast<float4 *>(P.part + (int64_t)split * P.entries +
                                                                 ((int64_t)tap * P.co + co) * P.ci + ci);
 #pragma unroll
@@ -290,7 +316,7 @@ bool make_ww_plan(const ConvGeom &g, WwPlan *out)
     P.co = g.co; P.ci = g.ci;
     P.cob = g.co < 128 ? g.co : 128;
     P.mb_per_kd = P.cob >= 128 ? 3 * (g.co / 128) : (P.cob == 64 ? 2 : 1);
-    P.nmb = 3 * P.mb_per_kd;
+    P.nmb = P.cob == 64 ? 5 : 3 * P.mb_per_kd;       // c_out = 64: nine taps in five blocks of two (decode_acc)
     P.ncx = ncx;
     P.pair_cx = ncx >= 2;
     P.nsets = P.pair_cx ? P.nmb * (ncx / 2) : (P.nmb + 1) / 2;
@@ -299,7 +325,7 @@ bool make_ww_plan(const ConvGeom &g, WwPlan *out)
     // one extra h-line behind the dy box: the fourth (unused) window of a 32-channel block reads it
     P.dy_bytes = (int)align_up((size_t)aboxes * TWW * DYH * CBA * 2 + TWW * CBA * 2, 1024);
     P.x_bytes = (int)align_up((size_t)XW * THH * CBB * 2, 1024);
-    P.ndy = (P.pair_cx || P.mb_per_kd % 2 == 0) ? 1 : 2;
+    P.ndy = P.cob == 64 ? 2 : ((P.pair_cx || P.mb_per_kd % 2 == 0) ? 1 : 2);
     P.stage_bytes = P.ndy * P.dy_bytes + (P.pair_cx ? 2 : 1) * P.x_bytes;
     const int budget = 227 * 1024 - 1024 - 1024;
     int nst = budget / P.stage_bytes;
@@ -312,11 +338,13 @@ bool make_ww_plan(const ConvGeom &g, WwPlan *out)
     if (nsplit > P.ntiles) nsplit = P.ntiles;
     P.nsplit = nsplit;
     P.nsplit_last = nsplit;
-    // 32 output channels: three M blocks (kd = 0, 1, 2) in two sets, the second with ONE live accumulator, i.e. half the
-    // MMAs per tile.  Its share of the CTAs is halved accordingly (2 : 1), so that all CTAs finish together.
-    if (P.cob == 32 && P.nsets == 2 && !P.pair_cx && sms >= 3 && P.ntiles >= sms) {
-        P.nsplit = sms * 2 / 3;
-        P.nsplit_last = sms - P.nsplit;
+    // (32 output channels: three M blocks in two sets, the second with one live accumulator.  Giving that set a third
+    // instead of half of the CTAs made the pass SLOWER, 782 -> 628 TFLOP/s: at this width a tile's time is set by its
+    // loads and barrier round trips, not by its MMAs, so both kinds of set take the same time per tile.)
+    // 64 output channels, one c_in chunk: five M blocks in three sets, the last with one live accumulator (2 : 2 : 1)
+    if (P.cob == 64 && P.nsets == 3 && !P.pair_cx && sms >= 5 && P.ntiles >= sms) {
+        P.nsplit = sms * 2 / 5;
+        P.nsplit_last = sms - 2 * P.nsplit;
     }
     P.nunits = (P.nsets - 1) * P.nsplit + P.nsplit_last;
     P.entries = (int64_t)27 * g.co * g.ci;
@@ -365,11 +393,13 @@ lamp_status_t win_wgrad(const ConvGeom &g, const TView &x, const TView &dy, floa
     const bool direct = pl.P.nsplit == 1;
     pl.P.part = direct ? dw : (float *)ws;
     if (pl.P.nsplit_last < pl.P.nsplit) {
-        // the last set (taps kd = 2: entries [18, 27) x c_out x c_in) writes fewer partial slices than the reduction adds:
-        // the slices it does not write are zero
+        // the last set (c_out = 64: tap (kd 2, kh 2), entries [24, 27) x c_out x c_in) writes fewer partial slices than the
+        // reduction adds: the slices it does not write are zero
         const size_t tap_bytes = (size_t)g.co * g.ci * sizeof(float);
-        LAMP_CUDA_OK(cudaMemset2DAsync((char *)pl.P.part + (size_t)pl.P.nsplit_last * pl.P.entries * sizeof(float) + 18 * tap_bytes,
-                                       (size_t)pl.P.entries * sizeof(float), 0, 9 * tap_bytes, (size_t)(pl.P.nsplit - pl.P.nsplit_last), st));
+        const int first_tap = 24;
+        LAMP_CUDA_OK(cudaMemset2DAsync((char *)pl.P.part + (size_t)pl.P.nsplit_last * pl.P.entries * sizeof(float) + first_tap * tap_bytes,
+                                       (size_t)pl.P.entries * sizeof(float), 0, (27 - first_tap) * tap_bytes,
+                                       (size_t)(pl.P.nsplit - pl.P.nsplit_last), st));
     }
     pl.P.status = status_word_ptr();
     CUtensorMap mx, mdy;
