@@ -550,18 +550,19 @@ def unet_floor_ms(cfg, train, peaks, vol=None):
     return total * 1e3
 
 
-def measure_unet(workload, cfg_id, steps, warmup, sw_batch=32, graph=True):
+def measure_unet(workload, cfg_id, steps, warmup, sw_batch=32, graph=True, se_ratio=0):
     """Times one U-Net workload on cuda:0 through the C ABI; returns the fields of its JSON line."""
     import torch
     from paper_2006_12575_b200 import binding as B
     from paper_2006_12575_b200 import synth
     cfg = UNET_CFGS[cfg_id]
     args = argparse.Namespace(cfg=cfg_id, workload=workload, steps=steps, warmup=warmup, sw_batch=sw_batch,
-                              no_graph=not graph)
+                              no_graph=not graph, se_ratio=se_ratio)
     peaks = measured_peaks()
     D, H, W = cfg["vol"]
     V = D * H * W
-    net = B.lamp_unet_create(B.unet_spec(cfg["levels"], cfg["ch"], cfg["cpl"], 1, cfg["K"]))
+    # se_ratio > 0: the SEU-Net variant (every level's conv stack ends in a squeeze-and-excitation residual step)
+    net = B.lamp_unet_create(B.unet_spec(cfg["levels"], cfg["ch"], cfg["cpl"], 1, cfg["K"], se_ratio=args.se_ratio))
     nl = B.lamp_unet_num_layers(net)
     g = torch.Generator().manual_seed(10 * args.cfg + 1)
     wflat = torch.zeros(B.lamp_unet_weight_count(net), dtype=torch.float32)
@@ -572,7 +573,13 @@ def measure_unet(workload, cfg_id, steps, warmup, sw_batch=32, graph=True):
         n = taps * d.c_in * d.c_out
         wflat[wo:wo + n] = torch.randn(n, generator=g) * (2.0 / fan) ** 0.5
     wd = wflat.cuda().to(torch.bfloat16)
-    bd = torch.zeros(B.lamp_unet_bias_count(net), dtype=torch.float32, device="cuda")
+    bflat = torch.zeros(B.lamp_unet_bias_count(net), dtype=torch.float32)
+    for i in range(nl):
+        so, cr = B.lamp_unet_se_layout(net, i)
+        if cr:                                   # squeeze-and-excitation parameters: small random values
+            c = B.lamp_unet_param_layout(net, i)[2].c_out
+            bflat[so:so + 2 * c * cr + c + cr] = torch.randn(2 * c * cr + c + cr, generator=g) * 0.3
+    bd = bflat.cuda()
     if args.cfg == 4:
         vol = synth.ct_volume((D, H, W), 40)
     else:
@@ -582,6 +589,8 @@ def measure_unet(workload, cfg_id, steps, warmup, sw_batch=32, graph=True):
     ev = lambda: torch.cuda.Event(enable_timing=True)
     out = dict(n_gpus=1, steps=args.steps, warmup=args.warmup, higher_is_better=True, scaling="weak", vs_baseline=None,
                dtype="bf16", data="synthetic", unit="voxels/s")
+    if args.se_ratio:
+        out["variant"] = f"SEU-Net, reduction ratio {args.se_ratio} (the roofline floor below is the plain network's)"
     if args.workload == "unet_train":
         lab = torch.from_numpy(synth.labels_quartiles((D, H, W), 10 * args.cfg + 2, cfg["K"], 4.0)).reshape(-1).cuda()
         loss = torch.zeros(1, dtype=torch.float32, device="cuda")
@@ -675,7 +684,8 @@ def run_unet(args):
     from paper_2006_12575_b200 import build as lamp_build
     lamp_build.build()
     torch.cuda.set_device(0)
-    print(json.dumps(measure_unet(args.workload, args.cfg, args.steps, args.warmup, args.sw_batch, not args.no_graph)), flush=True)
+    print(json.dumps(measure_unet(args.workload, args.cfg, args.steps, args.warmup, args.sw_batch, not args.no_graph,
+                                  args.se_ratio)), flush=True)
 
 
 def run_unet_dp(args):
@@ -951,6 +961,7 @@ def main():
     ap.add_argument("--cfg", type=int, default=2)
     ap.add_argument("--sw-batch", type=int, default=32)
     ap.add_argument("--no-graph", action="store_true", help="U-Net workloads: skip the CUDA-graph replay timing")
+    ap.add_argument("--se-ratio", type=int, default=0, help="U-Net workloads: SEU-Net variant with this reduction ratio (0: plain)")
     ap.add_argument("--no-unet", action="store_true", help="conv sweep: leave out the U-Net workloads that follow it")
     args = ap.parse_args()
     if args.workload == "hbm":

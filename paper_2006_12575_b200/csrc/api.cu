@@ -1,4 +1,8 @@
 // C ABI (include/lamp.h): argument checks, kernel selection, status word.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <mutex>
+#include <string.h>
 #include "common.cuh"
 #include "umma_ptx.cuh"
 
@@ -13,6 +17,52 @@ int *status_word_ptr()
     return p;
 }
 
+// cuTensorMapEncodeTiled with a small cache in front.  A training step encodes two tensor maps per tensor-core launch
+// (about 460 per step), always from the same few hundred argument sets: the encoded map depends on nothing but the
+// arguments, so a hit returns the stored 128 bytes.  Direct-mapped, 1024 entries, one mutex (calls come from the host
+// threads that enqueue work; an entry is compared in full before it is used).
+namespace {
+
+struct MapKey {
+    uint64_t addr, gdim[5], gstride[4];
+    uint32_t box[5], es[5], rank, dt, il, sw, l2, oob;
+};
+struct MapEntry { bool valid; MapKey key; CUtensorMap map; };
+constexpr int MAP_CACHE_SLOTS = 1024;
+MapEntry g_map_cache[MAP_CACHE_SLOTS];
+std::mutex g_map_mutex;
+PFN_cuTensorMapEncodeTiled_v12000 g_real_encode = nullptr;
+
+CUresult CUDAAPI encode_tiled_cached(CUtensorMap *out, CUtensorMapDataType dt, cuuint32_t rank, void *addr, const cuuint64_t *gdim,
+                                     const cuuint64_t *gstride, const cuuint32_t *box, const cuuint32_t *es,
+                                     CUtensorMapInterleave il, CUtensorMapSwizzle sw, CUtensorMapL2promotion l2,
+                                     CUtensorMapFloatOOBfill oob)
+{
+    if (rank < 1 || rank > 5) return g_real_encode(out, dt, rank, addr, gdim, gstride, box, es, il, sw, l2, oob);
+    MapKey k;
+    memset(&k, 0, sizeof(k));
+    k.addr = (uint64_t)(uintptr_t)addr; k.rank = rank; k.dt = (uint32_t)dt; k.il = (uint32_t)il; k.sw = (uint32_t)sw;
+    k.l2 = (uint32_t)l2; k.oob = (uint32_t)oob;
+    for (cuuint32_t i = 0; i < rank; ++i) { k.gdim[i] = gdim[i]; k.box[i] = box[i]; k.es[i] = es[i]; }
+    for (cuuint32_t i = 0; i + 1 < rank; ++i) k.gstride[i] = gstride[i];
+    uint64_t h = 1469598103934665603ull;
+    const unsigned char *b = (const unsigned char *)&k;
+    for (size_t i = 0; i < sizeof(k); ++i) h = (h ^ b[i]) * 1099511628211ull;
+    MapEntry &e = g_map_cache[h % MAP_CACHE_SLOTS];
+    {
+        std::lock_guard<std::mutex> lock(g_map_mutex);
+        if (e.valid && memcmp(&e.key, &k, sizeof(k)) == 0) { *out = e.map; return CUDA_SUCCESS; }
+    }
+    const CUresult r = g_real_encode(out, dt, rank, addr, gdim, gstride, box, es, il, sw, l2, oob);
+    if (r == CUDA_SUCCESS) {
+        std::lock_guard<std::mutex> lock(g_map_mutex);
+        e.key = k; e.map = *out; e.valid = true;
+    }
+    return r;
+}
+
+}  // namespace
+
 void *tensor_map_encoder()
 {
     // resolved once per process; the entry point does not depend on the device
@@ -22,7 +72,8 @@ void *tensor_map_encoder()
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
             qres != cudaDriverEntryPointSuccess)
             p = nullptr;
-        return p;
+        g_real_encode = (PFN_cuTensorMapEncodeTiled_v12000)p;
+        return p ? (void *)&encode_tiled_cached : nullptr;
     }();
     return fn;
 }

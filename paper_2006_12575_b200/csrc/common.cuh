@@ -74,8 +74,9 @@ static inline lamp_status_t launch_status()
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// api.cu.  The driver's cuTensorMapEncodeTiled, resolved once through the runtime (NULL if unavailable); declared
-// as void* so that this header needs no driver types.
+// api.cu.  The driver's cuTensorMapEncodeTiled (a function of that signature with a small cache in front: the same
+// arguments give the stored map), resolved once through the runtime (NULL if unavailable); declared as void* so that
+// this header needs no driver types.
 void *tensor_map_encoder();
 // api.cu.  Number of SMs of the current device.
 int sm_count();
