@@ -64,6 +64,8 @@ CASES = [
     ("r_c64_to_32_ragged", 1, 44, 90, 140, 64, 32, 3, 1, 1, 0),
     ("r_c32_batch_odd_rows", 2, 29, 75, 100, 32, 32, 3, 1, 1, 0),
     ("r_c32_to_64", 1, 30, 128, 104, 32, 64, 3, 1, 1, 0),
+    ("r_c64_single_plane", 1, 1, 352, 288, 64, 64, 3, 1, 1, 0),
+    ("r_c32_two_planes", 1, 2, 384, 288, 32, 32, 3, 1, 1, 0),
     ("deep_512_cube8", 1, 8, 8, 8, 512, 512, 3, 1, 1, 0),
     ("deep_512_to_256_ragged", 2, 3, 5, 7, 512, 256, 3, 1, 1, 0),
     ("deep_down_256_512", 1, 8, 8, 8, 256, 512, 3, 2, 1, 0),
