@@ -249,7 +249,7 @@ def dice_loss_grad_logits(p, labels, eps=1e-5):
 # Squeeze-and-excitation residual block (the SEU-Net of Sec. 1 / Sec. 3, Tables 2, 3, 5)
 # ----------------------------------------------------------------------------
 # The paper names the network ("3D SEU-Net", after AnatomyNet) and never defines the block; the cited paper is not
-# at hand.  Reading used here (stated in full in the design doc): at the end of a level's conv stack, with
+# at hand.  Reading used here: at the end of a level's conv stack, with
 #   r = output of the level's FIRST conv -> InstanceNorm -> ReLU (the residual branch; absent for one conv per level),
 #   z = output of the level's LAST  conv -> InstanceNorm -> ReLU,
 #   s[n,c] = mean over voxels of z                       (squeeze)
