@@ -209,7 +209,7 @@ typedef struct {
     float   in_eps;
     int32_t se_ratio;          /* 0: plain U-Net.  > 0: SEU-Net variant - every level's conv stack ends in the squeeze-and-
                                   excitation residual step described above (hidden units = width / se_ratio, at least 1);
-                                  needs convs_per_level = 2 (the residual branch is the first conv's output)     */
+                                  needs convs_per_level >= 2 (the residual branch is the first conv's output)    */
 } lamp_unet_spec_t;
 
 typedef struct lamp_unet lamp_unet_t;          /* opaque, host-only plan */

@@ -53,7 +53,7 @@ class UNetSpec:
     in_channels: int = 1
     num_classes: int = 4
     eps: float = 1e-5
-    se_ratio: int = 0      # > 0: SEU-Net variant, hidden units = width // se_ratio (at least 1); needs convs_per_level = 2
+    se_ratio: int = 0      # > 0: SEU-Net variant, hidden units = width // se_ratio (at least 1); needs convs_per_level >= 2
 
 
 @dataclass
@@ -87,10 +87,10 @@ def unet_layers(spec: UNetSpec) -> List[Layer]:
             c = ch[l]
     out.append(Layer("head", "head", 0, ch[0], spec.num_classes, 1, ch[0]))
     if spec.se_ratio > 0:
-        if spec.convs_per_level != 2:
-            raise ValueError("the squeeze-and-excitation residual block is defined for two convs per level")
+        if spec.convs_per_level < 2:
+            raise ValueError("the squeeze-and-excitation residual block needs at least two convs per level")
         for ly in out:
-            if ly.kind == "conv" and ly.name.endswith(".conv1"):
+            if ly.kind == "conv" and ly.name.endswith(f".conv{spec.convs_per_level - 1}"):
                 ly.se_cr = max(1, ly.c_out // spec.se_ratio)
     return out
 
@@ -121,12 +121,14 @@ def forward(spec: UNetSpec, weights, biases, x, quantise=True, want_cache=False,
     for i, ly in enumerate(lay):
         w, b = weights[i], biases[i]
         if ly.kind in ("conv", "down"):
-            r = a
             a, cache[i] = _norm_conv_fwd(a, w, b, 2 if ly.kind == "down" else 1, spec.eps, quantise)
+            if ly.kind == "conv" and ly.name.endswith(".conv0"):
+                first_out, first_idx = a, i                                     # the residual branch of this level
             if ly.se_cr:
                 c = cache[i]
                 z = ops.instnorm_relu_fwd(c["ys"], c["mu"], c["rstd"])          # not stored, hence not rounded
-                out, c["se"] = ops.se_block_fwd(z, r, *se[i])
+                out, c["se"] = ops.se_block_fwd(z, first_out, *se[i])
+                c["res_idx"] = first_idx
                 a = _q(out, quantise)
             nxt = lay[i + 1]
             if ly.name.startswith("enc") and nxt.kind == "down":
@@ -168,7 +170,7 @@ def train_step(spec: UNetSpec, weights, biases, x, labels, quantise=True, se=Non
             if ly.se_cr:
                 dz, dr, dW1, db1, dW2, db2 = ops.se_block_bwd(g, c["se"])
                 dSE[i] = (dW1, db1, dW2, db2)
-                res_grad[i - 1] = dr                    # the residual branch: the level's first conv also receives dout
+                res_grad[c["res_idx"]] = dr             # the residual branch: the level's first conv also receives dout
                 g = _q(dz, quantise)
             if i in res_grad:
                 g = g + res_grad.pop(i)

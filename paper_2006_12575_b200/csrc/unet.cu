@@ -21,11 +21,12 @@ struct Layer {
     bool to_cat;                // output is E_l, written to the concat buffer slice [0, C_l)
     bool from_cat;              // input is the full concat buffer (2 C_l channels)
     // SEU-Net variant: the level's last conv ends in a squeeze-and-excitation residual step, out = r + e * z with
-    // r = this conv's input (the output of the level's first conv).  se_cr > 0: hidden units; its fp32 parameters
+    // r = the output of the level's first conv (layer res_of).  se_cr > 0: hidden units; its fp32 parameters
     // W1 [cr][c], b1 [cr], W2 [c][cr], b2 [c] sit in the bias buffer from se_off.  The level's first conv then gets the
     // block output's gradient as a second gradient source (res_from = index of that last conv, else -1).
     int se_cr = 0;
     size_t se_off = 0;
+    int res_of = -1;
     int res_from = -1;
 };
 
@@ -333,10 +334,10 @@ lamp_status_t run_forward(const lamp_unet *net, const Plan &P, const bf16 *W, co
         const bf16 *w = W + Ly.w_off;
         const float *b = Bv + Ly.b_off;
         if (Ly.se_cr) {
-            // last conv of a level in the SEU-Net variant: out = r + e * relu(norm(y)), r = this conv's input
+            // last conv of a level in the SEU-Net variant: out = r + e * relu(norm(y)), r = the output of the level's first conv
             TRY(conv_fwd(B.g, B.in, w, b, B.y, B.stats, P.scratch, P.scratch_bytes, st));
             TRY(k_mu_rstd(B.stats, (int64_t)B.y.d * B.y.h * B.y.w, S.in_eps, B.mr, B.y.n * Ly.c_out, st));
-            TRY(k_se_fwd(B.y, B.mr, Bv + Ly.se_off, Ly.se_cr, B.se_sums, B.se_e, B.se_hid, B.se_mean, &B.in, B.out, st));
+            TRY(k_se_fwd(B.y, B.mr, Bv + Ly.se_off, Ly.se_cr, B.se_sums, B.se_e, B.se_hid, B.se_mean, &P.lb[Ly.res_of].out, B.out, st));
         } else if (Ly.kind == K_CONV || Ly.kind == K_DOWN) {
             TRY(conv_fwd(B.g, B.in, w, b, B.y, B.stats, P.scratch, P.scratch_bytes, st));
             TRY(k_instnorm_relu_fwd(B.y, B.stats, S.in_eps, B.mr, B.out, st));
@@ -398,8 +399,8 @@ lamp_status_t lamp_unet_create(const lamp_unet_spec_t *spec, lamp_unet_t **out)
     if (spec->channels[0] > 128) return LAMP_ERR_UNSUPPORTED;          // the head's backward kernel keeps 256 voxels x channels[0] in shared memory
     if (!(spec->in_eps > 0.f)) return LAMP_ERR_INVALID_ARG;
     if (spec->se_ratio < 0) return LAMP_ERR_INVALID_ARG;
-    // the residual branch of the squeeze-and-excitation block is the input of the level's last conv: two convs per level
-    if (spec->se_ratio > 0 && spec->convs_per_level != 2) return LAMP_ERR_UNSUPPORTED;
+    // the residual branch of the squeeze-and-excitation block is the output of the level's first conv
+    if (spec->se_ratio > 0 && spec->convs_per_level < 2) return LAMP_ERR_UNSUPPORTED;
     lamp_unet *net = new (std::nothrow) lamp_unet;
     if (!net) return LAMP_ERR_INVALID_ARG;
     net->spec = *spec;
@@ -415,7 +416,8 @@ lamp_status_t lamp_unet_create(const lamp_unet_spec_t *spec, lamp_unet_t **out)
             y.se_cr = co / spec->se_ratio > 0 ? co / spec->se_ratio : 1;
             y.se_off = bo;
             bo += (size_t)2 * co * y.se_cr + co + y.se_cr;
-            net->layers.back().res_from = (int)net->layers.size();      // the conv in front is the level's first conv
+            y.res_of = (int)net->layers.size() - (spec->convs_per_level - 1);      // the level's first conv
+            net->layers[y.res_of].res_from = (int)net->layers.size();
         }
         net->layers.push_back(y);
     };

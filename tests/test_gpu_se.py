@@ -172,7 +172,8 @@ def test_se_residual_block_forward_backward_composed_from_the_library_calls():
     assert_close(host_f64(dx), dx_o, "block dx", rel=1e-2, mx=1e-1)
 
 
-def test_seunet_train_step_matches_the_mirrored_oracle_within_the_storage_budget():
+@pytest.mark.parametrize("cpl", [2, 3])
+def test_seunet_train_step_matches_the_mirrored_oracle_within_the_storage_budget(cpl):
     """The SEU-Net variant through lamp_unet_create(se_ratio) / lamp_unet_train_step / lamp_unet_forward: probabilities,
     loss and every gradient (conv weights, biases, squeeze-and-excitation parameters) against the oracle that mirrors
     the bf16 storage points, held to the arithmetic's own budget (mirrored oracle against unrounded oracle) as the
@@ -180,8 +181,8 @@ def test_seunet_train_step_matches_the_mirrored_oracle_within_the_storage_budget
     from oracle import unet as O
     levels, ch, K, ratio = 2, [32, 64], 5, 4
     D, H, W = 8, 12, 20
-    net = B.lamp_unet_create(B.unet_spec(levels, ch, 2, 1, K, se_ratio=ratio))
-    spec = O.UNetSpec(levels, list(ch), 2, 1, K, se_ratio=ratio)
+    net = B.lamp_unet_create(B.unet_spec(levels, ch, cpl, 1, K, se_ratio=ratio))
+    spec = O.UNetSpec(levels, list(ch), cpl, 1, K, se_ratio=ratio)
     lay = O.unet_layers(spec)
     ws = synth.kaiming_for_layers([(l.taps, l.c_out, l.c_in, l.fan_in) for l in lay], 61)
     rs = synth.rng(62)
@@ -245,7 +246,7 @@ def test_seunet_train_step_matches_the_mirrored_oracle_within_the_storage_budget
     B.lamp_unet_forward(net, wd, bd, dev_bf16(x), p2, None, wsf)
     assert torch.equal(p2, probs)
     B.lamp_unet_destroy(net)
-    # three convs per level have no defined residual branch: refused
+    # one conv per level has no residual branch: refused
     with pytest.raises(B.LampError) as e:
-        B.lamp_unet_create(B.unet_spec(2, [32, 64], 3, 1, K, se_ratio=4))
+        B.lamp_unet_create(B.unet_spec(2, [32, 64], 1, 1, K, se_ratio=4))
     assert e.value.status == 2

@@ -76,10 +76,10 @@ def test_block_backward_matches_central_finite_differences():
     assert np.allclose(part, part[:, :1, :1, :1, :], rtol=0, atol=1e-14)
 
 
-def _se_net(seed):
+def _se_net(seed, cpl=2):
     from oracle import unet
     from paper_2006_12575_b200 import synth
-    spec = unet.UNetSpec(2, [4, 8], 2, 1, 3, se_ratio=2)
+    spec = unet.UNetSpec(2, [4, 8], cpl, 1, 3, se_ratio=2)
     lay = unet.unet_layers(spec)
     ws = [w.astype(np.float64) for w in synth.kaiming_for_layers([(l.taps, l.c_out, l.c_in, l.fan_in) for l in lay], seed)]
     rs = np.random.default_rng(seed)
@@ -92,6 +92,29 @@ def _se_net(seed):
     x = rs.standard_normal((1, 4, 4, 4, 1))
     lab = rs.integers(0, 3, (1, 4, 4, 4))
     return unet, spec, lay, ws, bs, se, x, lab
+
+
+def test_seunet_with_three_convs_per_level_takes_the_first_conv_as_residual_branch():
+    unet, spec, lay, ws, bs, se, x, lab = _se_net(6, cpl=3)
+    assert [l.name for l in lay if l.se_cr] == ["enc0.conv2", "enc1.conv2", "dec0.conv2"]
+    loss, dW, dB, probs, dSE = unet.train_step(spec, ws, bs, x, lab, quantise=False, se=se)
+    f = lambda: unet.train_step(spec, ws, bs, x, lab, quantise=False, se=se)[0]
+    names = [l.name for l in lay]
+    rs = np.random.default_rng(2)
+    h = 1e-6
+    # the first conv of a level feeds the second conv AND the residual branch; the middle conv only the last conv
+    for name in ("enc0.conv0", "enc0.conv1", "enc1.conv0", "dec0.conv0", "dec0.conv2"):
+        i = names.index(name)
+        for _ in range(4):
+            idx = tuple(rs.integers(0, n) for n in ws[i].shape)
+            old = ws[i][idx]
+            ws[i][idx] = old + h
+            lp = f()
+            ws[i][idx] = old - h
+            lm = f()
+            ws[i][idx] = old
+            fd = (lp - lm) / (2 * h)
+            assert abs(fd - dW[i][idx]) <= 2e-6 * max(1.0, abs(fd) * 1e3), (name, fd, dW[i][idx])
 
 
 def test_seunet_layers_and_gradients_by_finite_differences():
