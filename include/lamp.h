@@ -264,6 +264,19 @@ lamp_status_t lamp_unet_forward(const lamp_unet_t *net, const void *weights_bf16
                                 const lamp_tensor_t *x, float *probs, uint8_t *argmax,
                                 void *ws, size_t ws_bytes, void *cuda_stream);
 
+/* Layers [first_layer, last_layer) of the forward pass only: one partition F_k of the sequentialised network (Sec. 2.1,
+ * Eq. 1; Sec. 2.2, Eq. 3).  The partition reads what earlier layers left in the workspace - the activation that enters
+ * first_layer and, for every skip that crosses the cut, the kept encoder output e_{i,1} (LAMP_T_OUT of that encoder
+ * layer, in inference mode) - and leaves its own outputs there; lamp_unet_tensor_layout says where each of them
+ * lives, so a pipeline copies exactly those tensors from the previous partition's workspace (on another device: into
+ * this device's own memory first) and calls this.  x must describe the network input in every partition (its shape
+ * fixes the layout; its data is read only when first_layer = 0).  probs / argmax are written only by the partition
+ * that contains the head.  Running the partitions of any cut one after the other on one workspace, or on several with
+ * the boundary tensors copied, gives exactly lamp_unet_forward's result. */
+lamp_status_t lamp_unet_forward_layers(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                       const lamp_tensor_t *x, int32_t first_layer, int32_t last_layer,
+                                       float *probs, uint8_t *argmax, void *ws, size_t ws_bytes, void *cuda_stream);
+
 /* One forward + backward pass with the softmax-Dice loss
  *   L = mean_n [ 1 - (1/K) sum_k (2 I_k + e)/(P_k + G_k + e) ],  I = sum p g, P = sum p, G = sum g, e = 1e-5.
  * labels: uint8 [n*d*h*w], values < num_classes.  loss: fp32 device scalar.

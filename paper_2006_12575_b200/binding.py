@@ -79,6 +79,7 @@ def lib():
             "lamp_unet_workspace_bytes": (sz, [vp, i32, i32, i32, i32, i32]),
             "lamp_unet_tensor_layout": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, i32, TP, C.POINTER(sz)]),
             "lamp_unet_forward": (C.c_int, [vp, vp, vp, TP, vp, vp, vp, sz, vp]),
+            "lamp_unet_forward_layers": (C.c_int, [vp, vp, vp, TP, i32, i32, vp, vp, vp, sz, vp]),
             "lamp_unet_train_step": (C.c_int, [vp, vp, vp, TP, vp, vp, vp, vp, vp, vp, sz, vp]),
             "lamp_unet_train_step_buckets": (C.c_int, [vp, vp, vp, TP, vp, vp, vp, vp, vp, vp, sz, vp,
                                                        C.POINTER(C.c_int64), i32, C.POINTER(vp)]),
@@ -108,7 +109,7 @@ EXPORTS = ["lamp_conv3d_workspace_bytes", "lamp_conv3d_workspace_min_bytes", "la
            "lamp_se_squeeze", "lamp_se_excite", "lamp_se_apply_fwd", "lamp_se_bwd_reduce", "lamp_se_excite_bwd", "lamp_se_apply_bwd",
            "lamp_unet_create", "lamp_unet_se_layout", "lamp_unet_destroy",
            "lamp_unet_num_layers", "lamp_unet_weight_count", "lamp_unet_bias_count", "lamp_unet_param_layout",
-           "lamp_unet_workspace_bytes", "lamp_unet_tensor_layout", "lamp_unet_forward", "lamp_unet_train_step",
+           "lamp_unet_workspace_bytes", "lamp_unet_tensor_layout", "lamp_unet_forward", "lamp_unet_forward_layers", "lamp_unet_train_step",
            "lamp_unet_train_step_buckets", "lamp_sliding_window_num_patches", "lamp_sliding_window_partial",
            "lamp_sliding_window_finish",
            "lamp_sliding_window_workspace_bytes", "lamp_sliding_window_infer", "lamp_overlap_add",
@@ -256,6 +257,12 @@ def lamp_unet_forward(net, weights, biases, x, probs, argmax, ws):
     p, nbytes = _ws(ws)
     _check(lib().lamp_unet_forward(net, _ptr(weights), _ptr(biases), C.byref(_td(x)), _ptr(probs), _ptr(argmax),
                                    p, nbytes, _stream()), "lamp_unet_forward")
+
+
+def lamp_unet_forward_layers(net, weights, biases, x, first_layer, last_layer, probs, argmax, ws):
+    p, nbytes = _ws(ws)
+    _check(lib().lamp_unet_forward_layers(net, _ptr(weights), _ptr(biases), C.byref(_td(x)), first_layer, last_layer,
+                                          _ptr(probs), _ptr(argmax), p, nbytes, _stream()), "lamp_unet_forward_layers")
 
 
 def lamp_unet_train_step(net, weights, biases, x, labels, loss, grad_w, grad_b, probs, ws):

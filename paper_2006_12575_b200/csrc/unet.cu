@@ -322,13 +322,16 @@ lamp_status_t check_input(const lamp_unet *net, const lamp_tensor_t *x)
         if (s__ != LAMP_OK) return s__;             \
     } while (0)
 
+// layers [first, last) of the forward pass (the whole network by default)
 lamp_status_t run_forward(const lamp_unet *net, const Plan &P, const bf16 *W, const float *Bv, float *probs,
-                          uint8_t *argmax, const uint8_t *labels, double *dice, cudaStream_t st)
+                          uint8_t *argmax, const uint8_t *labels, double *dice, cudaStream_t st, size_t first = 0,
+                          size_t last = (size_t)-1)
 {
     const lamp_unet_spec_t &S = net->spec;
+    if (last > net->layers.size()) last = net->layers.size();
     // the InstanceNorm sums of all layers sit in one pool: one memset clears them
     if (P.stats_pool_bytes) LAMP_CUDA_OK(cudaMemsetAsync(P.stats_pool, 0, P.stats_pool_bytes, st));
-    for (size_t i = 0; i < net->layers.size(); ++i) {
+    for (size_t i = first; i < last; ++i) {
         const Layer &Ly = net->layers[i];
         const LayerBuf &B = P.lb[i];
         const bf16 *w = W + Ly.w_off;
@@ -647,6 +650,21 @@ static lamp_status_t train_step_impl(const lamp_unet_t *net, const void *weights
         if (!j && rs == LAMP_OK) rs = LAMP_ERR_CUDA;
     }
     return rs;
+}
+
+lamp_status_t lamp_unet_forward_layers(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,
+                                       const lamp_tensor_t *x, int32_t first_layer, int32_t last_layer,
+                                       float *probs, uint8_t *argmax, void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!weights_bf16 || !biases_f32) return LAMP_ERR_INVALID_ARG;
+    TRY(check_input(net, x));
+    if (first_layer < 0 || last_layer <= first_layer || last_layer > (int32_t)net->layers.size()) return LAMP_ERR_INVALID_ARG;
+    if (!ws || ((uintptr_t)ws & 255)) return LAMP_ERR_WORKSPACE;
+    Plan P;
+    make_plan(net, ws, x->ptr, x->c_pitch, x->n, x->d, x->h, x->w, LAMP_MODE_INFER, false, &P);
+    if (P.total > ws_bytes) return LAMP_ERR_WORKSPACE;
+    return run_forward(net, P, (const bf16 *)weights_bf16, biases_f32, probs, argmax, nullptr, nullptr,
+                       (cudaStream_t)cuda_stream, (size_t)first_layer, (size_t)last_layer);
 }
 
 lamp_status_t lamp_unet_train_step(const lamp_unet_t *net, const void *weights_bf16, const float *biases_f32,

@@ -2,7 +2,8 @@
 pipeline (Sec. 2.1, Eq. 1; Sec. 2.2, Eq. 3).
 
 On one B200 every listed network fits unsplit, so the library itself runs no pipeline; what is here is the logic a
-multi-GPU pipeline needs on the host, testable with CPU ranks:
+multi-GPU pipeline needs on the host, testable with CPU ranks, and (at the end) partitions of whole-volume inference
+that run the library's kernels:
 
 * sequential_unet_stages: the U-Net as a plain sequence of steps acting on a state (activation, stack of skips).
   Eq. 3 duplicates every encoder output as e_{i,0} (fed to the next block) and e_{i,1} (kept for the skip); carrying
@@ -101,6 +102,11 @@ def gpipe_schedule(K: int, M: int):
     return ticks
 
 
+def forward_schedule(K: int, M: int):
+    """The forward half alone (pipelined inference of M volumes over K partitions): M + K - 1 ticks."""
+    return gpipe_schedule(K, M)[:M + K - 1]
+
+
 def bubble_fraction(K: int, M: int) -> float:
     """Share of partition-ticks in which a partition idles: (K - 1) / (M + K - 1)."""
     return (K - 1) / (M + K - 1)
@@ -139,14 +145,14 @@ class PipelineStage:
         raise NotImplementedError
 
 
-def run_pipeline(stage: PipelineStage, micro_batches: Sequence, M: int, group=None):
-    """Runs gpipe_schedule(world, M) with one partition per rank of `group`: every rank executes its own entries of
-    every tick in order.  Boundary states and their gradients travel by send / recv between neighbouring ranks: the
+def run_pipeline(stage: PipelineStage, micro_batches: Sequence, M: int, group=None, forward_only: bool = False):
+    """Runs gpipe_schedule(world, M) (forward_only: forward_schedule) with one partition per rank of `group`: every rank
+    executes its own entries of every tick in order.  Boundary states and their gradients travel by send / recv between neighbouring ranks: the
     receiver owns the memory they land in.  Returns the last partition's forward outputs (other ranks: [])."""
     world = dist.get_world_size(group)
     rank = dist.get_rank(group)
     outs = []
-    for tick in gpipe_schedule(world, M):
+    for tick in (forward_schedule(world, M) if forward_only else gpipe_schedule(world, M)):
         for (k, m, direction) in tick:
             if k != rank:
                 continue
@@ -174,3 +180,109 @@ def run_pipeline(stage: PipelineStage, micro_batches: Sequence, M: int, group=No
                     for t in gin:
                         dist.send(t.contiguous(), dst=rank - 1, group=group)
     return outs
+
+
+# ------------------------------------------------------------------------------------------------------
+# Partitions that run the library's kernels: whole-volume inference cut into F_1 ... F_K (Eq. 1), every partition a
+# range of layers executed by lamp_unet_forward_layers in its own workspace.  What crosses a cut is exactly the
+# state of the sequential U-Net (Eq. 3): the activation entering the first layer of the partition and every kept
+# encoder output e_{i,1} whose skip crosses the cut (plus, in the SEU-Net variant, the first conv's output of a
+# level whose stack is cut in the middle).
+# ------------------------------------------------------------------------------------------------------
+def library_layers(binding, net):
+    """Kinds and sizes of the library's layers, derived from lamp_unet_param_layout / lamp_unet_se_layout."""
+    out = []
+    for i in range(binding.lamp_unet_num_layers(net)):
+        _, _, d = binding.lamp_unet_param_layout(net, i)
+        kind = "up" if d.transposed else "head" if d.ksize == 1 else "down" if d.stride == 2 else "conv"
+        _, cr = binding.lamp_unet_se_layout(net, i)
+        out.append(dict(kind=kind, c_in=d.c_in, c_out=d.c_out, se=cr > 0))
+    return out
+
+
+def boundary_tensors(layers, cut, convs_per_level):
+    """What the partition that starts at layer `cut` needs from earlier layers: a list of (layer, 'in' | 'out')."""
+    need = [(cut, "in")]
+    # skips: the last conv of encoder level l (followed by a down conv) is read again by the conv behind up conv l;
+    # encoder levels are entered in order, decoder levels left in reverse order
+    enc_last = [i for i, ly in enumerate(layers[:-1]) if ly["kind"] == "conv" and layers[i + 1]["kind"] == "down"]
+    ups = [i for i, ly in enumerate(layers) if ly["kind"] == "up"]
+    for l, i in enumerate(enc_last):
+        consumer = ups[len(ups) - 1 - l] + 1
+        if i < cut <= consumer and (i, "out") not in need:
+            need.append((i, "out"))
+    for j, ly in enumerate(layers):
+        first = j - (convs_per_level - 1)
+        if ly["se"] and j >= cut > first:
+            need.append((first, "out"))
+    return need
+
+
+def _tensor_view(binding, net, shape, ws, layer, which):
+    import torch as _t
+    n, d, h, w = shape
+    t, off = binding.lamp_unet_tensor_layout(net, n, d, h, w, binding.MODE_INFER, layer, binding.T_IN if which == "in" else binding.T_OUT)
+    V = t.n * t.d * t.h * t.w
+    flat = ws[off:off + ((V - 1) * t.c_pitch + t.c) * 2].view(_t.bfloat16)
+    return _t.as_strided(flat, (V, t.c), (t.c_pitch, 1))
+
+
+def copy_boundary(binding, net, shape, need, ws_src, ws_dst):
+    """Copies the boundary tensors from one partition's workspace into the next one's (same layout in both)."""
+    for layer, which in need:
+        _tensor_view(binding, net, shape, ws_dst, layer, which).copy_(_tensor_view(binding, net, shape, ws_src, layer, which))
+
+
+def partitioned_forward(binding, net, weights, biases, x, cuts, workspaces, probs, argmax, convs_per_level=2):
+    """Whole-volume inference as K partitions run one after the other, partition k in workspaces[k] (on one device
+    this is the pipeline's arithmetic without its overlap; over several devices every rank runs its own partition and
+    the boundary tensors travel by send / recv into the receiver's workspace).  cuts: ascending first layers of
+    partitions 1 .. K-1."""
+    layers = library_layers(binding, net)
+    n, d, h, w = x.shape[0], x.shape[1], x.shape[2], x.shape[3]
+    bounds = [0] + list(cuts) + [len(layers)]
+    for k in range(len(bounds) - 1):
+        if k > 0:
+            copy_boundary(binding, net, (n, d, h, w), boundary_tensors(layers, bounds[k], convs_per_level), workspaces[k - 1], workspaces[k])
+        last = k == len(bounds) - 2
+        binding.lamp_unet_forward_layers(net, weights, biases, x, bounds[k], bounds[k + 1], probs if last else None,
+                                         argmax if last else None, workspaces[k])
+
+
+class LibraryPartition(PipelineStage):
+    """One partition of pipelined whole-volume inference on this rank's GPU: layers [first, last) through
+    lamp_unet_forward_layers in this rank's own workspace.  forward() takes the boundary state as contiguous tensors
+    (as received from the previous rank), copies it to where the layers expect it, runs the layers and returns the
+    state for the next rank (the last partition returns clones of probs and argmax)."""
+
+    def __init__(self, binding, net, weights, biases, shape, first, last, workspace, x_like, convs_per_level=2,
+                 probs=None, argmax=None):
+        self.b, self.net, self.w, self.bias = binding, net, weights, biases
+        self.shape, self.first, self.last, self.ws, self.x_like = tuple(shape), first, last, workspace, x_like
+        self.probs, self.argmax = probs, argmax
+        self.layers = library_layers(binding, net)
+        self.need_in = boundary_tensors(self.layers, first, convs_per_level) if first > 0 else []
+        self.need_out = boundary_tensors(self.layers, last, convs_per_level) if last < len(self.layers) else []
+
+    def _views(self, need):
+        return [_tensor_view(self.b, self.net, self.shape, self.ws, layer, which) for layer, which in need]
+
+    def incoming(self, m):
+        return [torch.empty(v.shape, dtype=v.dtype, device=v.device) for v in self._views(self.need_in)]
+
+    def outgoing(self, m):
+        return [torch.empty(v.shape, dtype=v.dtype, device=v.device) for v in self._views(self.need_out)]
+
+    def forward(self, m, state):
+        x = self.x_like
+        if self.first == 0:
+            x = state[0]
+        else:
+            for dst, src in zip(self._views(self.need_in), state):
+                dst.copy_(src)
+        is_last = self.last == len(self.layers)
+        self.b.lamp_unet_forward_layers(self.net, self.w, self.bias, x, self.first, self.last, self.probs if is_last else None,
+                                        self.argmax if is_last else None, self.ws)
+        if is_last:
+            return [t.clone() for t in (self.probs, self.argmax) if t is not None]
+        return [v.contiguous() for v in self._views(self.need_out)]

@@ -530,3 +530,91 @@ def test_patch_sharded_sliding_window_one_replica_is_bit_identical_and_two_share
     with pytest.raises(B.LampError):
         B.lamp_sliding_window_partial(net, wd, bd, vol, P, 0.25, 3, 1, 3, 2, s2, w2, wsb)      # range beyond the grid
     B.lamp_unet_destroy(net)
+
+
+@pytest.mark.parametrize("se_ratio", [0, 4])
+def test_forward_pass_cut_into_partitions_equals_the_unsplit_pass(se_ratio):
+    """lamp_unet_forward_layers (Sec. 2.1 Eq. 1, Sec. 2.2 Eq. 3): the network cut at ANY layer into two partitions, and by
+    the balanced partitioner into three, each partition in its own workspace that starts out as garbage and receives
+    only the boundary state of the sequential U-Net (entering activation + the kept encoder outputs whose skip crosses
+    the cut): probabilities and arg max are bit-identical to the unsplit forward pass."""
+    from paper_2006_12575_b200 import pipeline as PL
+    levels, ch, cpl, K = 3, [32, 64, 128], 2, 4
+    net = B.lamp_unet_create(B.unet_spec(levels, ch, cpl, 1, K, se_ratio=se_ratio))
+    nl = B.lamp_unet_num_layers(net)
+    g = torch.Generator().manual_seed(77)
+    wflat = torch.zeros(B.lamp_unet_weight_count(net), dtype=torch.float32)
+    for i in range(nl):
+        wo, bo, d = B.lamp_unet_param_layout(net, i)
+        n = d.ksize ** 3 * d.c_in * d.c_out
+        wflat[wo:wo + n] = torch.randn(n, generator=g) * (2.0 / ((1 if d.transposed else d.ksize ** 3) * d.c_in)) ** 0.5
+    wd = wflat.cuda().to(torch.bfloat16)
+    bd = (torch.randn(B.lamp_unet_bias_count(net), generator=g) * 0.2).cuda()
+    D, H, W = 16, 16, 32
+    V = D * H * W
+    x = dev_bf16(synth.bf16_round(synth.blurred_noise((D, H, W), 1.5, 78))[None, ..., None])
+    nbytes = B.lamp_unet_workspace_bytes(net, 1, D, H, W, B.MODE_INFER)
+    ws0 = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    p_ref = torch.empty((V, K), dtype=torch.float32, device="cuda")
+    a_ref = torch.empty((V,), dtype=torch.uint8, device="cuda")
+    B.lamp_unet_forward(net, wd, bd, x, p_ref, a_ref, ws0)
+    layers = PL.library_layers(B, net)
+    assert [l["kind"] for l in layers] == ["conv", "conv", "down", "conv", "conv", "down", "conv", "conv", "up", "conv", "conv",
+                                          "up", "conv", "conv", "head"]
+    # the skip of level 0 crosses every cut between its producer (layer 1) and its consumer (layer 12)
+    assert (1, "out") in PL.boundary_tensors(layers, 7, cpl) and (4, "out") in PL.boundary_tensors(layers, 7, cpl)
+    assert PL.boundary_tensors(layers, 13, cpl) == [(13, "in")] + ([(12, "out")] if se_ratio else [])
+    fresh = lambda: torch.full((nbytes,), 0xFF, dtype=torch.uint8, device="cuda")
+    costs = [2.0 * (27 if l["kind"] in ("conv", "down") else 1) * l["c_in"] * l["c_out"] for l in layers]
+    three = [s for s, e in PL.partition_balanced(costs, 3)][1:]
+    for cuts in [[c] for c in range(1, nl)] + [three]:
+        probs = torch.full((V, K), float("nan"), dtype=torch.float32, device="cuda")
+        am = torch.full((V,), 255, dtype=torch.uint8, device="cuda")
+        PL.partitioned_forward(B, net, wd, bd, x, cuts, [fresh() for _ in range(len(cuts) + 1)], probs, am, cpl)
+        assert B.lamp_get_async_status() == 0
+        assert torch.equal(probs, p_ref), f"cuts {cuts}"
+        assert torch.equal(am, a_ref), f"cuts {cuts}"
+    with pytest.raises(B.LampError):
+        B.lamp_unet_forward_layers(net, wd, bd, x, 3, 3, None, None, ws0)
+    B.lamp_unet_destroy(net)
+
+
+def test_pipelined_inference_of_two_volumes_over_three_library_partitions():
+    """pipeline.LibraryPartition: three partitions, each with its own workspace, run two volumes in the order of the
+    forward schedule; the state handed from partition to partition is what a rank would send to the next (here passed
+    on directly: one GPU, so the partitions' kernels simply follow one another).  Every volume's result equals the
+    unsplit forward pass."""
+    from paper_2006_12575_b200 import pipeline as PL
+    net, spec, lay, ws, bs, wd, bd, _ = make_net(3, [32, 64, 128], 2, 4, seed=81)
+    D, H, W, K = 16, 16, 16, 4
+    V = D * H * W
+    vols = [dev_bf16(synth.bf16_round(synth.blurred_noise((D, H, W), 1.5, 82 + i))[None, ..., None]) for i in range(2)]
+    nbytes = B.lamp_unet_workspace_bytes(net, 1, D, H, W, B.MODE_INFER)
+    refs = []
+    for v in vols:
+        p = torch.empty((V, K), dtype=torch.float32, device="cuda")
+        a = torch.empty((V,), dtype=torch.uint8, device="cuda")
+        B.lamp_unet_forward(net, wd, bd, v, p, a, torch.empty(nbytes, dtype=torch.uint8, device="cuda"))
+        refs.append((p, a))
+    layers = PL.library_layers(B, net)
+    costs = [2.0 * (27 if l["kind"] in ("conv", "down") else 1) * l["c_in"] * l["c_out"] for l in layers]
+    parts = PL.partition_balanced(costs, 3)
+    probs = torch.empty((V, K), dtype=torch.float32, device="cuda")
+    am = torch.empty((V,), dtype=torch.uint8, device="cuda")
+    stages = [PL.LibraryPartition(B, net, wd, bd, (1, D, H, W), s, e, torch.full((nbytes,), 0xFF, dtype=torch.uint8, device="cuda"),
+                                  vols[0], 2, probs, am) for s, e in parts]
+    in_flight, outs = {}, {}
+    for tick in PL.forward_schedule(3, 2):
+        for (k, m, _) in tick:
+            state = [vols[m]] if k == 0 else in_flight.pop((k, m))
+            if k > 0:
+                assert [tuple(t.shape) for t in state] == [tuple(t.shape) for t in stages[k].incoming(m)]
+            res = stages[k].forward(m, state)
+            if k == 2:
+                outs[m] = res
+            else:
+                in_flight[(k + 1, m)] = res
+    assert B.lamp_get_async_status() == 0
+    for m in range(2):
+        assert torch.equal(outs[m][0], refs[m][0]) and torch.equal(outs[m][1], refs[m][1])
+    B.lamp_unet_destroy(net)

@@ -164,3 +164,9 @@ def test_two_rank_pipeline_accumulates_the_same_gradients_as_one_device():
         assert torch.allclose(got, ref.grad, rtol=1e-10, atol=1e-14)
     for got, ref in zip(out[1][1], s1.params):
         assert torch.allclose(got, ref.grad, rtol=1e-10, atol=1e-14)
+
+
+def test_forward_only_schedule_is_the_first_half():
+    assert PL.forward_schedule(3, 4) == PL.gpipe_schedule(3, 4)[:6]
+    assert sum(len(t) for t in PL.forward_schedule(3, 4)) == 12
+    assert all(d == "F" for t in PL.forward_schedule(2, 5) for (_, _, d) in t)
