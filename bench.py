@@ -497,7 +497,7 @@ def unet_fwd_flops(cfg):
     return fl + 2.0 * ch[0] * cfg["K"] * vox[0]
 
 
-def unet_floor_ms(cfg, train, peaks, vol=None):
+def unet_floor_ms(cfg, train, peaks, vol=None, probs_out=True):
     """Roofline floor of one U-Net pass: the sum over its steps of max(FLOPs / tensor peak, algorithmic bytes /
     HBM peak), with the measured peaks.  Bytes per step: a conv reads its input and writes its output once
     (bf16) and reads its weights; normalise + ReLU moves 4 B per element; its backward 10 B per element; a data
@@ -547,7 +547,7 @@ def unet_floor_ms(cfg, train, peaks, vol=None):
         for _ in range(cfg["cpl"]):
             conv(c, ch[l], vox[l], vox[l], 27, True)
             c = ch[l]
-    step(2.0 * ch[0] * K * vox[0], vox[0] * (2.0 * ch[0] + 4.0 * K + 1))
+    step(2.0 * ch[0] * K * vox[0], vox[0] * (2.0 * ch[0] + (4.0 * K if probs_out else 0.0) + 1))
     if train:
         step(4.0 * ch[0] * K * vox[0], vox[0] * (4.0 * ch[0] + 4.0 * K + 1))
     return total * 1e3
@@ -607,15 +607,16 @@ def measure_unet(workload, cfg_id, steps, warmup, sw_batch=32, graph=True, se_ra
         out.update(metric="unet_train_step_voxels_per_s", config=dict(workload=f"configs[{args.cfg}] U-Net forward+backward",
                                                                          workspace_bytes=nbytes))
     elif args.workload == "unet_infer":
-        probs = torch.empty((V, cfg["K"]), dtype=torch.float32, device="cuda")
+        # the output of both inference modes is the segmentation (arg-max) map; the sliding window writes no
+        # probabilities either
         seg = torch.empty(V, dtype=torch.uint8, device="cuda")
         nbytes = B.lamp_unet_workspace_bytes(net, 1, D, H, W, B.MODE_INFER)
         ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
-        fn = lambda: B.lamp_unet_forward(net, wd, bd, x, probs, seg, ws)
+        fn = lambda: B.lamp_unet_forward(net, wd, bd, x, None, seg, ws)
         flops = unet_fwd_flops(cfg)
-        floor_ms = unet_floor_ms(cfg, False, peaks)
+        floor_ms = unet_floor_ms(cfg, False, peaks, probs_out=False)
         out.update(metric="unet_whole_volume_infer_voxels_per_s",
-                   config=dict(workload=f"configs[{args.cfg}] whole-volume forward", workspace_bytes=nbytes))
+                   config=dict(workload=f"configs[{args.cfg}] whole-volume forward, output: arg-max map", workspace_bytes=nbytes))
     else:
         patch = (64, 64, 64)
         seg = torch.empty(V, dtype=torch.uint8, device="cuda")

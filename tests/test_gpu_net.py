@@ -269,6 +269,10 @@ def test_unet_forward_head_argmax_matches_oracle_on_stored_input():
     agree, strict, near = tie_aware_agreement(seg.cpu().numpy(), p_ref)
     assert agree >= 0.9999, (agree, strict, near)
     assert (seg.cpu().numpy() == np.argmax(host_f64(probs), -1)).all()
+    # the arg-max map alone (no probabilities written) is the same map
+    seg_only = torch.full((V,), 255, dtype=torch.uint8, device="cuda")
+    B.lamp_unet_forward(net, wd, bd, dev_bf16(x), None, seg_only, wsb)
+    assert torch.equal(seg_only, seg)
     # inference and training forward passes give the same probabilities
     loss = torch.zeros((1,), dtype=torch.float32, device="cuda")
     gw = torch.empty((B.lamp_unet_weight_count(net),), dtype=torch.float32, device="cuda")
