@@ -1,9 +1,9 @@
 // 3x3x3 stride-1 pad-1 convolution of narrow layers (c_out = 64 or 32): "voxels x (kd, channels)" implicit
 // GEMM whose accumulators rotate through three TMEM column slots.
 //
-// Why this shape.  One tcgen05.mma (M = 128, K = 16, bf16) holds the tensor pipe for max(76, N/2) cycles
-// (measured), so c_out = 64 alone on N runs at 42 % of the full rate, and stacking the weights of two output
-// planes on M (conv_t.cu) still spends a quarter of the MMAs on zero blocks.  Here the M rows are 128 OUTPUT
+// Why this shape.  One tcgen05.mma (M = 128, K = 16, bf16) holds the tensor pipe for N/2 cycles and one thread
+// issues at most one every 60-100 cycles (measured), so c_out = 64 alone on N runs far below the full rate, and
+// stacking the weights of two output planes on M (conv_t.cu) still spends a quarter of the MMAs on zero blocks.  Here the M rows are 128 OUTPUT
 // VOXELS of one plane (8 (w) x 16 (h)) and the N columns are the THREE kd TAPS side by side:
 //
 //      D_p[voxel, (kd, co)] += X_p[voxel + (kh-1, kw-1), ci] * W[kd, kh, kw][co, ci]        (input plane p)
@@ -15,7 +15,7 @@
 // of a tile accordingly.  After input plane p the slot of output plane p - 1 is complete: the epilogue moves it
 // to registers, stores zeros in its place (it becomes the fresh slot of plane p + 2) and hands it back.
 //
-//  * c_out = 32 (J = 2).  Three kd blocks of 32 channels would leave N = 96, which costs 76 cycles instead of 48.  So a
+//  * c_out = 32 (J = 2).  Three kd blocks of 32 channels would leave N = 96: 48 cycles, less than a thread's issue interval.  So a
 //    slot holds TWO output rows side by side: the 128 M rows are the voxels of every second h row (8 (w) x 16 rows, the
 //    descriptor steps two halo rows between 8-voxel groups), and column block (kd, jj) belongs to output row h + jj.
 //    A window that starts hs rows into the halo box is tap kh = hs - jj of block jj: four window shifts hs = 0..3 x three

@@ -1,8 +1,8 @@
 // 3x3x3 stride-1 pad-1 convolution, c_out in blocks of at most 128 channels: "weights x voxels"
 // implicit GEMM with the activation planes resident in shared memory.
 //
-// Why this shape.  One tcgen05.mma (M = 128, K = 16, bf16) occupies the tensor pipe for max(76, N/2)
-// cycles (measured): only N = 256 reaches the full rate.  With output channels on N, a 64-channel layer
+// Why this shape.  One tcgen05.mma (M = 128, K = 16, bf16) occupies the tensor pipe for N/2 cycles and a
+// thread issues at most one every 60-100 cycles (measured): N = 256 keeps one issuing thread ahead of the pipe.  With output channels on N, a 64-channel layer
 // would run at 42 % of it.  So here the OUTPUT CHANNELS are the M rows (A operand = weight tile
 // [128 x 64], K-major) and 256 OUTPUT VOXELS are the N columns (B operand = an 8 (w) x 32 (h) window of
 // an activation plane, K-major): D^T[co, voxel] += W[co, ci] * X[voxel + tap, ci].
