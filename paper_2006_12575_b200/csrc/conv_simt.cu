@@ -529,7 +529,7 @@ lamp_status_t simt_conv_fwd(const ConvGeom &g, const TView &x, const bf16 *w, co
     if (g.ci == 1 && g.k == 3 && g.s == 1 && g.p == 1 && !g.transposed && (g.co == 32 || g.co == 64) &&
         ((uintptr_t)y.p & 15) == 0 && (y.f32 ? y.pitch % 4 == 0 : y.pitch % 8 == 0)) {
         int blocks = (int)((Vn + 127) / 128);
-        const int cap = 148 * 16 / (g.n > 0 ? g.n : 1) + 1;
+        const int cap = sm_count() * 16 / (g.n > 0 ? g.n : 1) + 1;
         if (blocks > cap) blocks = cap;
         dim3 grid(blocks, g.n);
         if (g.co == 32)
@@ -635,7 +635,7 @@ static void c1_wgrad_plan(const ConvGeom &g, int *blocks, int64_t *vpb)
 {
     const int64_t V = (int64_t)g.n * g.d * g.h * g.w;
     int b = (int)((V + 2047) / 2048);
-    if (b > 148 * 8) b = 148 * 8;
+    if (b > sm_count() * 8) b = sm_count() * 8;
     if (b < 1) b = 1;
     *blocks = b;
     *vpb = (V + b - 1) / b;

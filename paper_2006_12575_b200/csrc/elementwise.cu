@@ -746,7 +746,7 @@ lamp_status_t k_instnorm_relu_fwd(const TView &y, const double *stats, float eps
     if (Vn == 0 || y.n == 0) return LAMP_OK;
     if (y.c / 8 > 256) return LAMP_ERR_UNSUPPORTED;
     const int64_t rb = 256 / (y.c / 8);
-    int64_t vpb = (Vn / (148 * 16) + rb - 1) / rb * rb;
+    int64_t vpb = (Vn / ((int64_t)sm_count() * 16) + rb - 1) / rb * rb;
     if (vpb < rb * 8) vpb = rb * 8;
     dim3 grid((unsigned)((Vn + vpb - 1) / vpb), y.n);
     (void)launch_pdl((int64_t)y.n * Vn * y.c <= SHORT_ELEMS, instnorm_relu_fwd_kernel, grid, dim3(256), (size_t)(0), st, (const bf16 *)y.p, y.pitch, stats, 1.0 / (double)Vn, eps, mu_rstd,
@@ -769,7 +769,7 @@ lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TVie
     const int RB = 256 / G;
     // pass 1: at most 8 blocks per SM, and at least 16 voxels per thread: every block ends with 2 C fp64 atomics, which
     // dominate when a small tensor is cut into many blocks
-    int64_t blocks = (148 * 8 + y.n - 1) / y.n;
+    int64_t blocks = ((int64_t)sm_count() * 8 + y.n - 1) / y.n;
     const int64_t max_blocks = (Vn + RB * 16 - 1) / (RB * 16);
     if (blocks > max_blocks) blocks = max_blocks;
     const int64_t vpb = (Vn + blocks - 1) / blocks;
@@ -785,7 +785,7 @@ lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TVie
     else
         (void)launch_pdl(early, instnorm_bwd_sums_kernel<false, 4>, sgrid, dim3(256), smem, st, pa, dza.pitch, pb, bpitch, py, y.pitch,
                          mu_rstd, sums, Vn, C, vpb);
-    int64_t vpa = (Vn / (148 * 16) + RB - 1) / RB * RB;
+    int64_t vpa = (Vn / ((int64_t)sm_count() * 16) + RB - 1) / RB * RB;
     if (vpa < (int64_t)RB * 8) vpa = (int64_t)RB * 8;
     dim3 grid((unsigned)((Vn + vpa - 1) / vpa), y.n);
     const size_t dsmem = db ? (size_t)RB * C * sizeof(float) : 0;
@@ -801,7 +801,7 @@ lamp_status_t k_instnorm_relu_bwd(const TView &dza, const TView *dzb, const TVie
 
 static void head_grid(int64_t Vn, int n, int64_t &blocks, int64_t &vpb)
 {
-    blocks = (148 * 8 + n - 1) / n;
+    blocks = ((int64_t)sm_count() * 8 + n - 1) / n;
     const int64_t max_blocks = (Vn + 255) / 256;
     if (blocks > max_blocks) blocks = max_blocks;
     if (blocks < 1) blocks = 1;
