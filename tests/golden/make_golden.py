@@ -47,6 +47,26 @@ def entries():
         out.append((f"tiny unet dW[{i}] sumsq", float((g * g).sum())))
     out.append(("window starts 512/64/0.25 count", float(len(O.window_starts(512, 64, 0.25)))))
     out.append(("gaussian window 8 min", float(O.gaussian_window((8, 8, 8)).min())))
+    out.append(("gaussian window 8 [2,3,4]", float(O.gaussian_window((8, 8, 8))[2, 3, 4])))
+    # squeeze-and-excitation residual block (the SEU-Net variant named in Sec. 1 / Sec. 3; the block is this build's reading)
+    g = synth.rng(18)
+    zz = np.maximum(g.standard_normal((2, 3, 4, 5, 8)), 0.0)
+    rr = np.maximum(g.standard_normal((2, 3, 4, 5, 8)), 0.0)
+    W1, b1, W2, b2 = g.standard_normal((2, 8)) * 0.5, g.standard_normal(2) * 0.2 + 0.3, g.standard_normal((8, 2)) * 0.5, g.standard_normal(8) * 0.2
+    o, cache = ops.se_block_fwd(zz, rr, W1, b1, W2, b2)
+    dz, dr, dW1, db1, dW2, db2 = ops.se_block_bwd(g.standard_normal(zz.shape), cache)
+    out += [("se block out sumsq", float((o * o).sum())), ("se block excitation sum", float(cache["e"].sum())),
+            ("se block dz sumsq", float((dz * dz).sum())), ("se block dW1 sumsq", float((dW1 * dW1).sum())),
+            ("se block dW2 sumsq", float((dW2 * dW2).sum())), ("se block db2 sum", float(db2.sum()))]
+    sspec = O.UNetSpec(2, [8, 16], 2, 1, 3, se_ratio=4)
+    slay = O.unet_layers(sspec)
+    sws = [a.astype(np.float64) for a in synth.kaiming_for_layers([(l.taps, l.c_out, l.c_in, l.fan_in) for l in slay], 19)]
+    sbs = [np.zeros(l.c_out) for l in slay]
+    sse = [None if not l.se_cr else (g.standard_normal((l.se_cr, l.c_out)) * 0.4, np.full(l.se_cr, 0.2),
+                                     g.standard_normal((l.c_out, l.se_cr)) * 0.4, np.zeros(l.c_out)) for l in slay]
+    sloss, sdW, sdB, sp, sdS = O.train_step(sspec, sws, sbs, vol, lab, se=sse)
+    out += [("tiny seunet loss", float(sloss)), ("tiny seunet probs sumsq", float((sp * sp).sum())),
+            ("tiny seunet dW[0] sumsq", float((sdW[0] * sdW[0]).sum()))]
     return out
 
 
