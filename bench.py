@@ -553,6 +553,9 @@ def unet_floor_ms(cfg, train, peaks, vol=None, probs_out=True):
     return total * 1e3
 
 
+_VOLUMES = {}
+
+
 def measure_unet(workload, cfg_id, steps, warmup, sw_batch=32, graph=True, se_ratio=0):
     """Times one U-Net workload on cuda:0 through the C ABI; returns the fields of its JSON line."""
     import torch
@@ -583,10 +586,10 @@ def measure_unet(workload, cfg_id, steps, warmup, sw_batch=32, graph=True, se_ra
             c = B.lamp_unet_param_layout(net, i)[2].c_out
             bflat[so:so + 2 * c * cr + c + cr] = torch.randn(2 * c * cr + c + cr, generator=g) * 0.3
     bd = bflat.cuda()
-    if args.cfg == 4:
-        vol = synth.ct_volume((D, H, W), 40)
-    else:
-        vol = synth.blurred_noise((D, H, W), 2.0, 10 * args.cfg)
+    key = (args.cfg, D, H, W)
+    if key not in _VOLUMES:                      # the 512 x 512 x 128 volume takes 15 s to draw: once per process
+        _VOLUMES[key] = synth.ct_volume((D, H, W), 40) if args.cfg == 4 else synth.blurred_noise((D, H, W), 2.0, 10 * args.cfg)
+    vol = _VOLUMES[key]
     hx = torch.from_numpy(vol).to(torch.bfloat16).reshape(1, D, H, W, 1).pin_memory()
     x = hx.cuda()
     ev = lambda: torch.cuda.Event(enable_timing=True)
